@@ -1,0 +1,304 @@
+"""CPU oracle for FastVAR's cached token pruning (test infrastructure, NOT a product path).
+
+A plain, slow, double-precision restatement of what the pruned next-scale-prediction step
+computes, written from the paper: Pivotal Token Selection (Eq. 4, Eq. 5, Algorithm 1, first
+routine), Cached Token Restoration (Eq. 6, Algorithm 1, second routine), the rule that the pair
+wraps every attention and FFN layer at the pruned steps (Sec. 3.3 "Implementation", Fig. 3b),
+the cache written at step K-N (Sec. 3.3 "Overview") and the reduced KV cache (Sec. 3.3, end of
+the PTS paragraph).  Only tests, the smoke check and the benchmark's CPU-baseline leg may import
+this file; it shares no code with the CUDA path and imports nothing from it.
+
+Everything is numpy float64.  There is no blocking, fusion or reordering: each function is the
+definition written out, with numpy's matmul / sort as library steps.
+
+Readings taken where the paper is silent or inconsistent (each is also listed in the design notes):
+  * score = SUM of squared deviations (Algorithm 1), not its square root (Eq. 5): same ranking.
+  * the scored tensor is the residual stream entering the sublayer, before normalisation.
+  * kept count k = ceil(keep_ratio * h*w) (keep ratio = 1 - the paper's pruning ratio).
+  * ties in the score go to the LOWEST token index; the kept set is emitted in ascending index
+    order (the set, not the order, is what the method defines: no later step depends on order).
+  * interpolate(.) of Eq. 6 = nearest neighbour, src = floor(dst * in / out) per axis.
+  * the cache holds the sublayer's branch output before gate and residual, one per wrapped sublayer,
+    taken at the last unpruned step and never refreshed.
+  * at a pruned step only the kept rows' K/V are appended to the KV cache.
+  * the transformer block (not specified by the paper): pre-LayerNorm without affine (eps 1e-6),
+    AdaLN modulation a = LN(x)*(1+sigma)+beta and gate x += gamma*y, tanh-GELU MLP, softmax scale
+    1/sqrt(head_dim), biases on qkv / out / fc1 / fc2, optional cross-attention to text with plain
+    LN, no biases and no gate.
+
+Parity pins: every function here is pinned by tests/test_oracle_pins.py (closed forms, brute force,
+invariants, library special cases).  The end-to-end activation values of a whole step have no
+printed example in the paper: "parity unpinned" for `VarOracle.var_step` as a whole beyond the
+invariants tested there (keep_ratio = 1 equals the unpruned forward, token-count invariance,
+restore equals the cache outside the pivot slots, KV length bookkeeping).
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+F64 = np.float64
+
+
+# ----------------------------------------------------------------------------------------------
+# Pivotal Token Selection  (Sec. 3.3, Eq. 4-5, Algorithm 1 first routine)
+# ----------------------------------------------------------------------------------------------
+
+def kept_count(keep_ratio: float, h: int, w: int) -> int:
+    """k = ceil(keep_ratio * h * w), clamped to [1, h*w].  The small epsilon keeps products
+    that are integers in exact arithmetic (0.6 * 1600 = 960) from rounding up."""
+    n = h * w
+    k = int(math.ceil(float(keep_ratio) * n - 1e-9))
+    return min(n, max(1, k))
+
+
+def pts_mean(x: np.ndarray) -> np.ndarray:
+    """Eq. 4: global average pool over the h*w tokens of each image.  x [B,n,C] -> [B,C]."""
+    x = np.asarray(x, dtype=F64)
+    return x.sum(axis=1) / x.shape[1]
+
+
+def pts_score(x: np.ndarray) -> np.ndarray:
+    """Eq. 5 in the squared form of Algorithm 1: s[b,n] = sum_c (x[b,n,c] - mean[b,c])^2."""
+    x = np.asarray(x, dtype=F64)
+    d = x - pts_mean(x)[:, None, :]
+    return (d * d).sum(axis=2)
+
+
+def pts_topk(score: np.ndarray, k: int) -> np.ndarray:
+    """Index set I: the k largest scores per image (stable descending sort, so equal scores keep
+    the lower index first), then emitted in ascending index order.  score [B,n] -> int64 [B,k]."""
+    score = np.asarray(score)
+    B, n = score.shape
+    out = np.empty((B, k), dtype=np.int64)
+    for b in range(B):
+        order = np.argsort(-score[b], kind="stable")   # stable: ties -> lowest index first
+        out[b] = np.sort(order[:k])
+    return out
+
+
+def inverse_map(idx: np.ndarray, n: int) -> np.ndarray:
+    """inv[b,t] = position j with idx[b,j] == t, or -1 when token t was pruned."""
+    B, k = idx.shape
+    inv = np.full((B, n), -1, dtype=np.int64)
+    for b in range(B):
+        inv[b, idx[b]] = np.arange(k)
+    return inv
+
+
+def pts_gather(x: np.ndarray, idx: np.ndarray) -> np.ndarray:
+    """x[b, I[b], :]  ->  [B,k,C]."""
+    return np.stack([x[b, idx[b]] for b in range(x.shape[0])], axis=0)
+
+
+def pivotal_token_selection(x: np.ndarray, h: int, w: int, keep_ratio: float):
+    """Algorithm 1, first routine.  Returns (idx [B,k] ascending, score [B,n], kept rows [B,k,C])."""
+    assert x.shape[1] == h * w
+    k = kept_count(keep_ratio, h, w)
+    s = pts_score(x)
+    idx = pts_topk(s, k)
+    return idx, s, pts_gather(np.asarray(x, dtype=F64), idx)
+
+
+# ----------------------------------------------------------------------------------------------
+# Cached Token Restoration  (Sec. 3.3, Eq. 6, Algorithm 1 second routine)
+# ----------------------------------------------------------------------------------------------
+
+def nearest_source(h: int, w: int, hc: int, wc: int) -> np.ndarray:
+    """Nearest-neighbour source token of every destination token when a (hc,wc) map is
+    interpolated to (h,w): sy = floor(y*hc/h), sx = floor(x*wc/w), row-major token order."""
+    src = np.empty(h * w, dtype=np.int64)
+    for y in range(h):
+        sy = (y * hc) // h
+        for xx in range(w):
+            sx = (xx * wc) // w
+            src[y * w + xx] = sy * wc + sx
+    return src
+
+
+def ctr_upsample(cache: np.ndarray, hc: int, wc: int, h: int, w: int) -> np.ndarray:
+    """Eq. 6: y_cache_k = interpolate(y_{K-N}, (h_k, w_k)).  cache [B,hc*wc,C] -> [B,h*w,C]."""
+    assert cache.shape[1] == hc * wc
+    return cache[:, nearest_source(h, w, hc, wc), :]
+
+
+def cached_token_restoration(pivots: np.ndarray, idx: np.ndarray, cache: np.ndarray,
+                             hc: int, wc: int, h: int, w: int) -> np.ndarray:
+    """Algorithm 1, second routine: upsample the cache to the current scale, then write the
+    forwarded rows into their slots.  pivots [B,k,C], idx [B,k] -> [B,h*w,C]."""
+    out = np.array(ctr_upsample(np.asarray(cache, dtype=F64), hc, wc, h, w), dtype=F64, copy=True)
+    for b in range(out.shape[0]):
+        out[b, idx[b], :] = pivots[b]
+    return out
+
+
+# ----------------------------------------------------------------------------------------------
+# Transformer sublayer pieces (standard definitions; the paper only names "Attention & FFN layer")
+# ----------------------------------------------------------------------------------------------
+
+def layernorm(x: np.ndarray, eps: float = 1e-6) -> np.ndarray:
+    """Per-row LayerNorm over the last axis, biased variance, no affine."""
+    x = np.asarray(x, dtype=F64)
+    mu = x.mean(axis=-1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (x - mu) / np.sqrt(var + eps)
+
+
+def modulate(a: np.ndarray, sigma: np.ndarray, beta: np.ndarray) -> np.ndarray:
+    """AdaLN: a*(1+sigma)+beta with per-image vectors.  a [B,k,C]; sigma, beta [B,C]."""
+    return a * (1.0 + sigma[:, None, :]) + beta[:, None, :]
+
+
+def gelu_tanh(x: np.ndarray) -> np.ndarray:
+    x = np.asarray(x, dtype=F64)
+    return 0.5 * x * (1.0 + np.tanh(math.sqrt(2.0 / math.pi) * (x + 0.044715 * x ** 3)))
+
+
+def linear(a: np.ndarray, W: np.ndarray, b: Optional[np.ndarray] = None) -> np.ndarray:
+    """y = a @ W^T + b with W stored [out, in]."""
+    y = np.asarray(a, dtype=F64) @ np.asarray(W, dtype=F64).T
+    if b is not None:
+        y = y + np.asarray(b, dtype=F64)
+    return y
+
+
+def softmax_rows(s: np.ndarray) -> np.ndarray:
+    s = s - s.max(axis=-1, keepdims=True)
+    e = np.exp(s)
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, H: int) -> np.ndarray:
+    """Multi-head softmax(q K^T / sqrt(hd)) V with a materialised attention matrix, no mask.
+    q [k,C], K [Lkv,C], V [Lkv,C]; head h owns channels [h*hd, (h+1)*hd)."""
+    k, C = q.shape
+    hd = C // H
+    out = np.empty((k, C), dtype=F64)
+    for h in range(H):
+        sl = slice(h * hd, (h + 1) * hd)
+        p = softmax_rows((q[:, sl] @ K[:, sl].T) / math.sqrt(hd))
+        out[:, sl] = p @ V[:, sl]
+    return out
+
+
+# ----------------------------------------------------------------------------------------------
+# The pruned scale step
+# ----------------------------------------------------------------------------------------------
+
+SUBLAYERS_SELF = ("attn", "ffn")
+SUBLAYERS_CROSS = ("attn", "xattn", "ffn")
+
+
+class VarOracle:
+    """State (KV cache per block and image, sublayer caches) plus `var_step`.
+
+    weights: dict of lists indexed by block, float arrays already widened from bf16:
+      w_qkv [3C,C], b_qkv [3C], w_o [C,C], b_o [C], w_fc1 [F,C], b_fc1 [F], w_fc2 [C,F], b_fc2 [C],
+      optional w_q_x [C,C], w_kv_x [2C,C] (K rows then V rows), w_o_x [C,C];
+      'mod' [L,B,6,C] = (sigma1, beta1, gamma1, sigma2, beta2, gamma2); 'text' [B,T,C] or None.
+    """
+
+    def __init__(self, L: int, C: int, H: int, sides_hw: Sequence[Sequence[int]], cache_step: int,
+                 weights: Dict, B: int, cross_len: int = 0):
+        self.L, self.C, self.H, self.B = L, C, H, B
+        self.hw = [tuple(s) for s in sides_hw]
+        self.cache_step = cache_step
+        self.cross_len = cross_len
+        self.w = weights
+        self.subs = SUBLAYERS_CROSS if cross_len else SUBLAYERS_SELF
+        self.reset()
+
+    def reset(self) -> None:
+        self.kv_len = 0
+        self.step = 0
+        self.Kc = [[np.zeros((0, self.C)) for _ in range(self.B)] for _ in range(self.L)]
+        self.Vc = [[np.zeros((0, self.C)) for _ in range(self.B)] for _ in range(self.L)]
+        self.cache: List[Dict[str, np.ndarray]] = [dict() for _ in range(self.L)]
+
+    # -- one wrapped sublayer on compact rows ---------------------------------------------------
+    def _branch(self, l: int, sub: str, xp: np.ndarray) -> np.ndarray:
+        """Sublayer branch output y for the compact rows xp [B,k,C] (before gate and residual)."""
+        w, mod = self.w, np.asarray(self.w["mod"][l], dtype=F64)      # mod [B,6,C]
+        B = xp.shape[0]
+        a = layernorm(xp)
+        if sub == "attn":
+            a = modulate(a, mod[:, 0], mod[:, 1])
+            qkv = linear(a, w["w_qkv"][l], w["b_qkv"][l])
+            q, kk, vv = qkv[..., :self.C], qkv[..., self.C:2 * self.C], qkv[..., 2 * self.C:]
+            y = np.empty_like(xp)
+            for b in range(B):
+                # KV cache: all earlier (possibly pruned) scales plus the rows forwarded now
+                self.Kc[l][b] = np.concatenate([self.Kc[l][b][:self.kv_len], kk[b]], axis=0)
+                self.Vc[l][b] = np.concatenate([self.Vc[l][b][:self.kv_len], vv[b]], axis=0)
+                o = attention(q[b], self.Kc[l][b], self.Vc[l][b], self.H)
+                y[b] = linear(o, w["w_o"][l], w["b_o"][l])
+            return y
+        if sub == "xattn":
+            q = linear(a, w["w_q_x"][l])
+            y = np.empty_like(xp)
+            for b in range(B):
+                kv = linear(np.asarray(w["text"][b], dtype=F64), w["w_kv_x"][l])
+                o = attention(q[b], kv[:, :self.C], kv[:, self.C:], self.H)
+                y[b] = linear(o, w["w_o_x"][l])
+            return y
+        if sub == "ffn":
+            a = modulate(a, mod[:, 3], mod[:, 4])
+            hmid = gelu_tanh(linear(a, w["w_fc1"][l], w["b_fc1"][l]))
+            return linear(hmid, w["w_fc2"][l], w["b_fc2"][l])
+        raise ValueError(sub)
+
+    def var_step(self, x: np.ndarray, scale_idx: int, keep_ratio: float,
+                 forced_idx: Optional[Dict] = None, trace: Optional[Dict] = None) -> np.ndarray:
+        """One scale step over all L blocks.  x [B,n,C] is the residual stream entering block 0.
+
+        For each block and each wrapped sublayer: PTS (when keep_ratio < 1) -> branch on kept rows
+        -> cache write (at the caching step) -> CTR (when keep_ratio < 1) -> gate and residual add.
+        `forced_idx[(l,sub)]` overrides the selection; `trace[(l,sub)]` receives idx / score / y."""
+        assert scale_idx == self.step, "steps must be taken in order"
+        x = np.array(x, dtype=F64, copy=True)
+        B, n, C = x.shape
+        h, w_ = self.hw[scale_idx]
+        assert n == h * w_ and B == self.B and C == self.C
+        pruned = keep_ratio < 1.0
+        k = kept_count(keep_ratio, h, w_) if pruned else n
+        for l in range(self.L):
+            mod = np.asarray(self.w["mod"][l], dtype=F64)
+            for sub in self.subs:
+                score = None
+                if pruned:
+                    score = pts_score(x)
+                    if forced_idx is not None:
+                        idx = np.asarray(forced_idx[(l, sub)], dtype=np.int64)
+                    else:
+                        idx = pts_topk(score, k)
+                    xp = pts_gather(x, idx)
+                else:
+                    idx = None
+                    xp = x
+                y = self._branch(l, sub, xp)
+                if scale_idx == self.cache_step:
+                    assert not pruned, "the caching step is the last unpruned step"
+                    self.cache[l][sub] = y.copy()
+                if pruned:
+                    hc, wc = self.hw[self.cache_step]
+                    yfull = cached_token_restoration(y, idx, self.cache[l][sub], hc, wc, h, w_)
+                else:
+                    yfull = y
+                if trace is not None:
+                    trace[(l, sub)] = {"idx": idx, "score": score, "y": y}
+                if sub == "attn":
+                    x = x + mod[:, 2][:, None, :] * yfull
+                elif sub == "ffn":
+                    x = x + mod[:, 5][:, None, :] * yfull
+                else:
+                    x = x + yfull
+        self.kv_len += k
+        self.step += 1
+        return x
+
+    def run_schedule(self, inputs: Sequence[np.ndarray], keep: Sequence[float]) -> List[np.ndarray]:
+        """All steps 0..K-1 in order; inputs[k] is the token map entering step k."""
+        self.reset()
+        return [self.var_step(inputs[i], i, keep[i]) for i in range(len(inputs))]
