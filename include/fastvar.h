@@ -1,0 +1,212 @@
+/* fastvar.h -- C ABI of the B200 (sm_100a) hot path of FastVAR's cached token pruning:
+ * the pruned large-scale next-scale-prediction step of a VAR transformer.
+ *
+ * Conventions (all entry points)
+ *   - Pointers named *_dev are DEVICE pointers, *_host are HOST pointers.  Every device buffer is
+ *     allocated and owned by the caller; the library allocates no device memory, keeps no copy of
+ *     weights and only borrows the pointers it is given (they must stay valid while used).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All device
+ *     work is enqueued on it; no entry point synchronises with the device unless it says so.
+ *   - bf16 = bfloat16, row-major.  "Token map" layout is [B, h*w, C], tokens row-major over (y, x).
+ *   - Linear weights are stored [out_features, in_features] (y = a * W^T + b).
+ *   - Every call returns fv_status; argument and state errors are detected on the host BEFORE any
+ *     launch.  Device-side trouble (a bounded wait that expired) is recorded in a status word in the
+ *     workspace and reported by fv_device_status(); kernels never trap and never wait unboundedly.
+ *   - Results are deterministic: the same inputs give bit-identical outputs run to run.
+ */
+#ifndef FASTVAR_H_
+#define FASTVAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fv_ctx fv_ctx; /* opaque; host-side metadata only */
+
+typedef enum {
+  FV_OK = 0,
+  FV_ERR_INVALID_ARG = 1, /* NULL pointer, non-positive size, ratio outside (0,1], bad alignment   */
+  FV_ERR_BAD_STATE = 2,   /* scale step taken out of order, missing cache, ...                       */
+  FV_ERR_CAPACITY = 3,    /* KV cache or workspace too small for this call                           */
+  FV_ERR_UNSUPPORTED = 4, /* shape outside what the kernels cover (stated per call)                  */
+  FV_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed (launch error, descriptor encoding) */
+  FV_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (see fv_device_status)               */
+} fv_status;
+
+const char *fv_status_string(fv_status s);
+
+/* Kept-token count of Pivotal Token Selection (Sec. 3.3): k = ceil(keep_ratio * h * w), clamped to
+ * [1, h*w]; keep_ratio = 1 - the paper's pruning ratio (Sec. 4.1).  Pure host function. */
+int32_t fv_k_for(double keep_ratio, int32_t h, int32_t w);
+
+/* ------------------------------------------------------------------------------------------------
+ * (1) Pivotal Token Selection -- Sec. 3.3 "Pivotal Token Selection", Eq. 4-5, Algorithm 1 (first
+ *     routine).  Per image: mean token over the h*w tokens (Eq. 4), score of every token = sum over
+ *     channels of the squared deviation from that mean (Algorithm 1; the square of Eq. 5's norm, same
+ *     ranking), exact top-k with ties going to the LOWEST token index, kept indices emitted in
+ *     ASCENDING order.
+ *   x_dev        [B, h*w, C] fp32 token map (the residual stream entering a sublayer).  C % 4 == 0.
+ *   keep_ratio   in (0, 1]; k = fv_k_for(keep_ratio, h, w) is also written to *k_out_host if non-NULL.
+ *   idx_out_dev  [B, k] int32, ascending per image.
+ *   inv_out_dev  [B, h*w] int32 or NULL: position j of token t in idx, or -1 if pruned.
+ *   score_out_dev[B, h*w] fp32 or NULL: the scores.
+ *   near_tie_dev [B] int32 or NULL: number of tokens whose score is within 1e-5 (relative) of the
+ *                k-th largest score (>= 1; values > 1 mean the kept set is decided by a near-tie).
+ *   workspace_dev scratch of at least fv_prune_select_workspace_bytes(B, h*w, C) bytes, 16-byte aligned.
+ * Errors: INVALID_ARG (NULLs, sizes, ratio, alignment), CAPACITY (workspace too small),
+ *         UNSUPPORTED (h*w > 49152), CUDA (launch failed).  */
+size_t fv_prune_select_workspace_bytes(int32_t B, int32_t n_tokens, int32_t C);
+fv_status fv_prune_select(const float *x_dev, int32_t B, int32_t h, int32_t w, int32_t C,
+                          double keep_ratio, int32_t *idx_out_dev, int32_t *inv_out_dev,
+                          float *score_out_dev, int32_t *near_tie_dev, int32_t *k_out_host,
+                          void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * (3) Cached Token Restoration -- Sec. 3.3 "Cached Token Restoration", Eq. 6, Algorithm 1 (second
+ *     routine).  out[b,t,:] = pivots[b,j,:] if t == idx[b,j], else cache_prev[b, src(t), :] where
+ *     src is the nearest-neighbour source of token t when the (hc,wc) map is interpolated to (h,w):
+ *     src = floor(y*hc/h)*wc + floor(x*wc/w).  Exact (a copy): bit-identical to the inputs.
+ *   cache_prev_dev [B, hc*wc, C] bf16 : the cached sublayer output y_{K-N}.
+ *   pivots_dev     [B, k, C] bf16     : the forwarded rows.
+ *   idx_dev        [B, k] int32       : their token indices (any order, no duplicates, in [0,h*w)).
+ *   out_dev        [B, h*w, C] bf16.   C % 8 == 0.
+ *   inv_scratch_dev[B, h*w] int32 scratch (overwritten).
+ * Errors: INVALID_ARG, CUDA. */
+fv_status fv_restore(const void *cache_prev_dev, int32_t hc, int32_t wc, const void *pivots_dev,
+                     const int32_t *idx_dev, int32_t B, int32_t k, int32_t h, int32_t w, int32_t C,
+                     void *out_dev, int32_t *inv_scratch_dev, void *stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * (2) The pruned scale step -- Sec. 3.3 "Overview" and "Implementation", Fig. 3: at the pruned steps
+ *     PTS runs before and CTR after EVERY attention and FFN layer; the per-layer outputs of the last
+ *     unpruned step (K-N) are the cache; only the kept rows' K/V enter the KV cache.
+ *
+ * Model (the paper leaves the backbone block open; this is the block both this library and its CPU
+ * oracle define): per block, for sublayer in (self-attention, [cross-attention], FFN):
+ *     I = PTS(x)  (keep_ratio < 1)             a = LayerNorm(x[I]) (eps 1e-6, no affine)
+ *     self-attn : a = a*(1+sigma1)+beta1; [q,k,v] = a*Wqkv^T+b; append k,v to the KV cache;
+ *                 o = softmax(q K^T / sqrt(hd)) V over all cached keys + the rows just appended;
+ *                 y = o*Wo^T+bo;  x += gamma1 * CTR(y)
+ *     cross-attn: q = a*Wq^T; K,V = text*Wkv^T; y = softmax(q K^T/sqrt(hd)) V * Wo^T;  x += CTR(y)
+ *     FFN       : a = a*(1+sigma2)+beta2; y = gelu_tanh(a*W1^T+b1)*W2^T+b2;  x += gamma2 * CTR(y)
+ * At scale step `cache_step` (unpruned) every sublayer's y is stored (bf16) as that sublayer's cache.
+ */
+typedef struct {
+  int32_t L;          /* transformer blocks                                                        */
+  int32_t C;          /* width; C % 64 == 0                                                        */
+  int32_t H;          /* heads; C / H must be 64 or 128                                            */
+  int32_t mlp_ratio;  /* hidden = mlp_ratio * C                                                    */
+  int32_t cross_len;  /* text tokens T (0 = no cross-attention sublayer); T % 8 == 0                */
+  int32_t B_max;      /* largest batch any call will use                                           */
+  int32_t n_steps;    /* number of scale steps K                                                   */
+  const int32_t *h;   /* HOST arrays [n_steps]: token-map height / width per step (copied)         */
+  const int32_t *w;
+  int32_t cache_step; /* 0-based index of step K-N, the last unpruned step; -1 = never cache       */
+  int32_t kv_capacity;/* KV rows per image per block the caller provides room for; % 8 == 0        */
+} fv_config;
+
+typedef struct { /* HOST arrays of length L holding DEVICE pointers; bf16 unless noted; borrowed   */
+  const void *const *w_qkv;  /* [3C, C]  rows: Q then K then V; head h owns channels [h*hd,(h+1)*hd) */
+  const void *const *b_qkv;  /* [3C]                                                               */
+  const void *const *w_o;    /* [C, C]                                                             */
+  const void *const *b_o;    /* [C]                                                                */
+  const void *const *w_fc1;  /* [mlp_ratio*C, C]                                                   */
+  const void *const *b_fc1;  /* [mlp_ratio*C]                                                      */
+  const void *const *w_fc2;  /* [C, mlp_ratio*C]                                                   */
+  const void *const *b_fc2;  /* [C]                                                                */
+  const void *const *w_q_x;  /* [C, C]   cross-attention (arrays may be NULL when cross_len == 0)  */
+  const void *const *w_kv_x; /* [2C, C]  rows: K then V                                            */
+  const void *const *w_o_x;  /* [C, C]                                                             */
+  const float *mod_dev;      /* [L, B_max, 6, C] fp32: sigma1, beta1, gamma1, sigma2, beta2, gamma2 */
+  const void *text_dev;      /* [B_max, cross_len, C] bf16 or NULL                                 */
+} fv_weights;
+
+size_t fv_workspace_bytes(const fv_config *cfg); /* scratch for fv_var_step                         */
+size_t fv_kv_bytes(const fv_config *cfg);        /* KV cache of all blocks (+ text K/V)             */
+size_t fv_cache_bytes(const fv_config *cfg);     /* sublayer caches y_{K-N} of all blocks           */
+
+/* Builds a context over caller-owned buffers (sizes from the three queries above, 1024-byte aligned).
+ * Clears the KV buffer once (synchronously) so that never-written rows hold zeros.
+ * Errors: INVALID_ARG, UNSUPPORTED (head dim not 64/128, C > 2048, ...), CUDA. */
+fv_status fv_create(const fv_config *cfg, const fv_weights *weights, void *kv_dev, void *cache_dev,
+                    void *workspace_dev, fv_ctx **out);
+void fv_destroy(fv_ctx *ctx);
+/* Rewinds to the start of a schedule: next step 0, empty KV cache. No device work. */
+fv_status fv_reset(fv_ctx *ctx);
+/* Resume support: read / set (next scale step, KV rows already held per image).  Setting a state
+ * past `cache_step` asserts that the caller has filled the sublayer caches and KV prefix itself. */
+fv_status fv_get_state(const fv_ctx *ctx, int32_t *next_step_host, int32_t *kv_len_host);
+fv_status fv_set_state(fv_ctx *ctx, int32_t next_step, int32_t kv_len);
+/* Device addresses inside the caller's buffers (for tests / resume): K rows [B_max, kv_capacity, C]
+ * and V^T [B_max, C, kv_capacity] of one block; the cache [B_max, n_cache, C] of (block, sublayer). */
+fv_status fv_kv_pointers(const fv_ctx *ctx, int32_t block, void **k_dev, void **vt_dev);
+fv_status fv_cache_pointer(const fv_ctx *ctx, int32_t block, int32_t sublayer, void **cache_dev);
+/* Projects the text tokens to per-block K / V^T for cross-attention (step-invariant).  Called by
+ * fv_var_step at scale step 0; call it yourself after fv_set_state on a fresh context. */
+fv_status fv_prepare_text(fv_ctx *ctx, int32_t B, void *stream);
+/* Synchronises `stream` and returns FV_OK, or FV_ERR_TIMEOUT (code in *code_host) if a kernel's bounded
+ * wait expired since the last call; clears the word. */
+fv_status fv_device_status(fv_ctx *ctx, int32_t *code_host, void *stream);
+
+/* One scale step over all L blocks.
+ *   tokens_dev  [B, h*w, C] fp32: residual stream entering block 0 at this scale.
+ *   out_dev     [B, h*w, C] fp32: residual stream after block L-1 (may alias tokens_dev).
+ *   scale_idx   must equal the context's next step (steps are taken in order).
+ *   keep_ratio  1.0 = unpruned path (no select / gather / restore work at all); < 1 = FastVAR.
+ *   forced_idx_dev NULL, or int32 [L, n_sub, B, k]: use these kept indices (ascending per image)
+ *               instead of selecting -- separates index parity from floating-point parity in tests.
+ *   idx_trace_dev  NULL, or int32 [L, n_sub, B, k]: receives the kept indices of every sublayer.
+ * n_sub = 3 with cross-attention else 2; sublayer order: self-attention, [cross-attention], FFN.
+ * Errors: INVALID_ARG, BAD_STATE (wrong scale_idx; pruned step before the cache step),
+ *         CAPACITY (kv_len + k > kv_capacity), CUDA. */
+fv_status fv_var_step(fv_ctx *ctx, const float *tokens_dev, int32_t B, int32_t scale_idx,
+                      double keep_ratio, float *out_dev, const int32_t *forced_idx_dev,
+                      int32_t *idx_trace_dev, void *stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Building blocks of the step, exported for kernel-level parity tests and profiling.            */
+
+/* Gather + LayerNorm + AdaLN modulate (the compaction of Algorithm 1's gather fused with the block's
+ * pre-norm): a[b,j,:] = LN(x[b, idx[b,j], :]) * (1 + sigma[b,:]) + beta[b,:]  -> bf16.
+ *   idx_dev NULL = all rows (k = n_tokens);  sigma_dev / beta_dev NULL = plain LayerNorm;
+ *   their per-image stride is mod_stride floats.  C % 4 == 0, C <= 2048. */
+fv_status fv_gather_ln(const float *x_dev, const int32_t *idx_dev, int32_t B, int32_t n_tokens,
+                       int32_t k, int32_t C, const float *sigma_dev, const float *beta_dev,
+                       int32_t mod_stride, void *a_out_dev, void *stream);
+
+/* Restore fused with gate and residual (Eq. 6 + the block's x += gamma * y):
+ *   x[b,t,:] += gamma[b,:] * (inv[b,t] >= 0 ? y[b, inv[b,t], :] : cache[b, src(t), :]).
+ * gamma_dev NULL = 1.  y, cache bf16; x fp32 in place.  C % 8 == 0. */
+fv_status fv_restore_residual(float *x_dev, const void *y_dev, const void *cache_dev,
+                              const int32_t *inv_dev, const float *gamma_dev, int32_t mod_stride,
+                              int32_t B, int32_t k, int32_t h, int32_t w, int32_t hc, int32_t wc,
+                              int32_t C, void *stream);
+
+/* tcgen05 GEMM  out = epilogue(A[M,K] * W[N,K]^T + bias), bf16 operands, fp32 accumulation in TMEM.
+ *   epilogue 0: bf16 store to out [M, N].          1: tanh-GELU then bf16 store.
+ *   epilogue 2: fp32 residual: out[m,n] += gamma[m / rows_per_image, n] * (acc + bias)  (out fp32;
+ *               gamma NULL = 1; if aux_dev != NULL the bf16 value of acc+bias is also stored there).
+ *   K % 8 == 0, N % 8 == 0, all pointers 16-byte aligned.  bias_dev may be NULL.
+ *   status_dev: int32 device word that receives a non-zero code if a bounded wait expires (or NULL). */
+fv_status fv_gemm_bf16(const void *a_dev, const void *w_dev, const void *bias_dev, int32_t M,
+                       int32_t N, int32_t K, int32_t epilogue, void *out_dev, void *aux_dev,
+                       const float *gamma_dev, int32_t mod_stride, int32_t rows_per_image,
+                       int32_t *status_dev, void *stream);
+
+/* Flash-style attention over a KV cache (Sec. 3.1 KV cache; Sec. 3.3: pivotal queries attend to the
+ * cached keys of all earlier scales plus the current pivotal keys; no mask inside a step).
+ *   q_dev  [B*rows, C] bf16 (image b owns rows [b*rows, (b+1)*rows)); head h = channels [h*hd, ..).
+ *   k_dev  [B, kv_capacity, C] bf16;  vt_dev [B, C, kv_capacity] bf16 (V transposed).
+ *   kv_len keys are attended (rows [0, kv_len) of every image).  out_dev [B*rows, C] bf16.
+ *   hd = C / H in {64, 128}; kv_capacity % 8 == 0. */
+fv_status fv_attention(const void *q_dev, const void *k_dev, const void *vt_dev, int32_t B,
+                       int32_t rows, int32_t H, int32_t C, int32_t kv_len, int32_t kv_capacity,
+                       void *out_dev, int32_t *status_dev, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FASTVAR_H_ */

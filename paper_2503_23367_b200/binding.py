@@ -1,0 +1,299 @@
+"""ctypes binding of libfastvar.so: same names as the C ABI, argument marshalling only.
+
+Every step of the pruned VAR scale step runs in the CUDA kernels behind the C ABI; torch is used here
+for device buffers and streams.  There is no CPU fallback: loading fails loudly when the library has
+not been built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfastvar.so")
+
+FV_OK = 0
+STATUS_NAMES = {0: "FV_OK", 1: "FV_ERR_INVALID_ARG", 2: "FV_ERR_BAD_STATE", 3: "FV_ERR_CAPACITY",
+                4: "FV_ERR_UNSUPPORTED", 5: "FV_ERR_CUDA", 6: "FV_ERR_TIMEOUT"}
+
+EXPORTS = ["fv_status_string", "fv_k_for", "fv_prune_select_workspace_bytes", "fv_prune_select", "fv_restore",
+           "fv_workspace_bytes", "fv_kv_bytes", "fv_cache_bytes", "fv_create", "fv_destroy", "fv_reset",
+           "fv_get_state", "fv_set_state", "fv_kv_pointers", "fv_cache_pointer", "fv_prepare_text",
+           "fv_device_status", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_gemm_bf16", "fv_attention"]
+
+
+class FvError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__(f"{where}: {STATUS_NAMES.get(code, code)}")
+        self.code = code
+
+
+class fv_config(C.Structure):
+    _fields_ = [("L", C.c_int32), ("C", C.c_int32), ("H", C.c_int32), ("mlp_ratio", C.c_int32),
+                ("cross_len", C.c_int32), ("B_max", C.c_int32), ("n_steps", C.c_int32),
+                ("h", C.POINTER(C.c_int32)), ("w", C.POINTER(C.c_int32)),
+                ("cache_step", C.c_int32), ("kv_capacity", C.c_int32)]
+
+
+class fv_weights(C.Structure):
+    _fields_ = [(n, C.POINTER(C.c_void_p)) for n in
+                ("w_qkv", "b_qkv", "w_o", "b_o", "w_fc1", "b_fc1", "w_fc2", "b_fc2", "w_q_x", "w_kv_x", "w_o_x")] + \
+               [("mod_dev", C.c_void_p), ("text_dev", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libfastvar.so (once).  Raises if it has not been built: there is no fallback path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2503_23367_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, sz, dbl = C.c_void_p, C.c_int32, C.c_size_t, C.c_double
+        L.fv_status_string.restype = C.c_char_p; L.fv_status_string.argtypes = [C.c_int]
+        L.fv_k_for.restype = i32; L.fv_k_for.argtypes = [dbl, i32, i32]
+        L.fv_prune_select_workspace_bytes.restype = sz; L.fv_prune_select_workspace_bytes.argtypes = [i32, i32, i32]
+        L.fv_prune_select.restype = C.c_int
+        L.fv_prune_select.argtypes = [vp, i32, i32, i32, i32, dbl, vp, vp, vp, vp, C.POINTER(i32), vp, sz, vp]
+        L.fv_restore.restype = C.c_int
+        L.fv_restore.argtypes = [vp, i32, i32, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]
+        for f in ("fv_workspace_bytes", "fv_kv_bytes", "fv_cache_bytes"):
+            getattr(L, f).restype = sz; getattr(L, f).argtypes = [C.POINTER(fv_config)]
+        L.fv_create.restype = C.c_int
+        L.fv_create.argtypes = [C.POINTER(fv_config), C.POINTER(fv_weights), vp, vp, vp, C.POINTER(vp)]
+        L.fv_destroy.restype = None; L.fv_destroy.argtypes = [vp]
+        L.fv_reset.restype = C.c_int; L.fv_reset.argtypes = [vp]
+        L.fv_get_state.restype = C.c_int; L.fv_get_state.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
+        L.fv_set_state.restype = C.c_int; L.fv_set_state.argtypes = [vp, i32, i32]
+        L.fv_kv_pointers.restype = C.c_int; L.fv_kv_pointers.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp)]
+        L.fv_cache_pointer.restype = C.c_int; L.fv_cache_pointer.argtypes = [vp, i32, i32, C.POINTER(vp)]
+        L.fv_prepare_text.restype = C.c_int; L.fv_prepare_text.argtypes = [vp, i32, vp]
+        L.fv_device_status.restype = C.c_int; L.fv_device_status.argtypes = [vp, C.POINTER(i32), vp]
+        L.fv_var_step.restype = C.c_int; L.fv_var_step.argtypes = [vp, vp, i32, i32, dbl, vp, vp, vp, vp]
+        L.fv_gather_ln.restype = C.c_int; L.fv_gather_ln.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, i32, vp, vp]
+        L.fv_restore_residual.restype = C.c_int
+        L.fv_restore_residual.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp]
+        L.fv_gemm_bf16.restype = C.c_int
+        L.fv_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp]
+        L.fv_attention.restype = C.c_int
+        L.fv_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None or isinstance(t, int):
+        return t                      # None, or a raw device address (sub-tensor with its own stride)
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(code: int, where: str) -> None:
+    if code != FV_OK:
+        raise FvError(code, where)
+
+
+def fv_k_for(keep_ratio: float, h: int, w: int) -> int:
+    return lib().fv_k_for(float(keep_ratio), h, w)
+
+
+def fv_prune_select(x: torch.Tensor, h: int, w: int, keep_ratio: float, want_inv=True, want_score=False,
+                    want_near_tie=False, workspace: Optional[torch.Tensor] = None):
+    """x fp32 [B, h*w, C] -> dict(idx int32 [B,k], inv, score, near_tie, k)."""
+    B, n, Cw = x.shape
+    assert x.dtype == torch.float32 and n == h * w
+    k = fv_k_for(keep_ratio, h, w)
+    dev = x.device
+    idx = torch.empty((B, k), dtype=torch.int32, device=dev)
+    inv = torch.empty((B, n), dtype=torch.int32, device=dev) if want_inv else None
+    score = torch.empty((B, n), dtype=torch.float32, device=dev) if want_score else None
+    near = torch.empty((B,), dtype=torch.int32, device=dev) if want_near_tie else None
+    need = lib().fv_prune_select_workspace_bytes(B, n, Cw)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    k_out = C.c_int32(0)
+    _check(lib().fv_prune_select(_ptr(x), B, h, w, Cw, float(keep_ratio), _ptr(idx), _ptr(inv), _ptr(score), _ptr(near),
+                                 C.byref(k_out), _ptr(workspace), workspace.numel(), _stream()), "fv_prune_select")
+    assert k_out.value == k
+    return {"idx": idx, "inv": inv, "score": score, "near_tie": near, "k": k}
+
+
+def fv_restore(cache_prev: torch.Tensor, hc: int, wc: int, pivots: torch.Tensor, idx: torch.Tensor, h: int, w: int,
+               out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """cache_prev bf16 [B,hc*wc,C], pivots bf16 [B,k,C], idx int32 [B,k] -> bf16 [B,h*w,C]."""
+    B, k, Cw = pivots.shape
+    if out is None:
+        out = torch.empty((B, h * w, Cw), dtype=torch.bfloat16, device=pivots.device)
+    inv = torch.empty((B, h * w), dtype=torch.int32, device=pivots.device)
+    _check(lib().fv_restore(_ptr(cache_prev), hc, wc, _ptr(pivots), _ptr(idx), B, k, h, w, Cw, _ptr(out), _ptr(inv),
+                            _stream()), "fv_restore")
+    return out
+
+
+def fv_gather_ln(x: torch.Tensor, idx: Optional[torch.Tensor], sigma: Optional[torch.Tensor],
+                 beta: Optional[torch.Tensor], mod_stride: int = 0) -> torch.Tensor:
+    B, n, Cw = x.shape
+    k = n if idx is None else idx.shape[1]
+    out = torch.empty((B, k, Cw), dtype=torch.bfloat16, device=x.device)
+    _check(lib().fv_gather_ln(_ptr(x), _ptr(idx), B, n, k, Cw, _ptr(sigma), _ptr(beta), mod_stride, _ptr(out), _stream()),
+           "fv_gather_ln")
+    return out
+
+
+def fv_restore_residual(x: torch.Tensor, y: torch.Tensor, cache: torch.Tensor, inv: torch.Tensor,
+                        gamma: Optional[torch.Tensor], mod_stride: int, h: int, w: int, hc: int, wc: int) -> None:
+    B, n, Cw = x.shape
+    k = y.shape[1]
+    _check(lib().fv_restore_residual(_ptr(x), _ptr(y), _ptr(cache), _ptr(inv), _ptr(gamma), mod_stride, B, k, h, w, hc, wc,
+                                     Cw, _stream()), "fv_restore_residual")
+
+
+def fv_gemm_bf16(a: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor], epilogue: int = 0,
+                 out: Optional[torch.Tensor] = None, aux: Optional[torch.Tensor] = None,
+                 gamma: Optional[torch.Tensor] = None, mod_stride: int = 0, rows_per_image: int = 0,
+                 status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    M, K = a.shape
+    N = w.shape[0]
+    assert w.shape[1] == K and a.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
+    if out is None:
+        assert epilogue in (0, 1)
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=a.device)
+    _check(lib().fv_gemm_bf16(_ptr(a), _ptr(w), _ptr(bias), M, N, K, epilogue, _ptr(out), _ptr(aux), _ptr(gamma),
+                              mod_stride, rows_per_image, _ptr(status), _stream()), "fv_gemm_bf16")
+    return out
+
+
+def fv_attention(q: torch.Tensor, k_cache: torch.Tensor, vt_cache: torch.Tensor, B: int, rows: int, H: int, kv_len: int,
+                 status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """q bf16 [B*rows, C]; k_cache bf16 [B, cap, C]; vt_cache bf16 [B, C, cap] -> bf16 [B*rows, C]."""
+    Cw = q.shape[1]
+    cap = k_cache.shape[1]
+    out = torch.empty_like(q)
+    _check(lib().fv_attention(_ptr(q), _ptr(k_cache), _ptr(vt_cache), B, rows, H, Cw, kv_len, cap, _ptr(out), _ptr(status),
+                              _stream()), "fv_attention")
+    return out
+
+
+class FvContext:
+    """Owns the device buffers a context borrows (weights, KV cache, sublayer caches, workspace) and
+    forwards to fv_create / fv_var_step / ...  Weights are given as numpy bf16 bit patterns
+    (`inputs.ModelTensors`) or as torch bf16 CUDA tensors with the same field names."""
+
+    def __init__(self, L: int, Cw: int, H: int, sides_hw: Sequence[Sequence[int]], cache_step: int, B_max: int,
+                 kv_capacity: int, tensors, cross_len: int = 0, mlp_ratio: int = 4, device="cuda:0"):
+        self.dev = torch.device(device)
+        self.L, self.C, self.H, self.B_max, self.cross_len = L, Cw, H, B_max, cross_len
+        self.n_sub = 3 if cross_len else 2
+        self.hw = [tuple(s) for s in sides_hw]
+        self.kv_capacity = (kv_capacity + 7) // 8 * 8
+        self._h = (C.c_int32 * len(self.hw))(*[s[0] for s in self.hw])
+        self._w = (C.c_int32 * len(self.hw))(*[s[1] for s in self.hw])
+        self.cfg = fv_config(L, Cw, H, mlp_ratio, cross_len, B_max, len(self.hw), self._h, self._w, cache_step,
+                             self.kv_capacity)
+        self._keep: List[torch.Tensor] = []
+
+        def dev_bf16(a):
+            if isinstance(a, torch.Tensor):
+                t = a.to(self.dev).contiguous()
+            else:
+                t = torch.from_numpy(a.view("int16")).to(self.dev).view(torch.bfloat16).contiguous()
+            self._keep.append(t)
+            return t
+
+        self._arrays = {}
+        W = fv_weights()
+        for name in ("w_qkv", "b_qkv", "w_o", "b_o", "w_fc1", "b_fc1", "w_fc2", "b_fc2", "w_q_x", "w_kv_x", "w_o_x"):
+            lst = getattr(tensors, name)
+            if not lst:
+                setattr(W, name, None)
+                continue
+            ts = [dev_bf16(a) for a in lst]
+            arr = (C.c_void_p * L)(*[t.data_ptr() for t in ts])
+            self._arrays[name] = arr
+            setattr(W, name, C.cast(arr, C.POINTER(C.c_void_p)))
+        mod = tensors.mod
+        self.mod = (mod if isinstance(mod, torch.Tensor) else torch.from_numpy(mod)).to(self.dev, torch.float32).contiguous()
+        assert tuple(self.mod.shape) == (L, B_max, 6, Cw)
+        W.mod_dev = self.mod.data_ptr()
+        self.text = dev_bf16(tensors.text) if cross_len else None
+        W.text_dev = self.text.data_ptr() if cross_len else None
+        self.weights = W
+        Lb = lib()
+        self.kv = torch.empty(Lb.fv_kv_bytes(C.byref(self.cfg)) + 1024, dtype=torch.uint8, device=self.dev)
+        self.cache = torch.empty(Lb.fv_cache_bytes(C.byref(self.cfg)) + 1024, dtype=torch.uint8, device=self.dev)
+        self.ws = torch.empty(Lb.fv_workspace_bytes(C.byref(self.cfg)) + 1024, dtype=torch.uint8, device=self.dev)
+        al = lambda t: (t.data_ptr() + 1023) // 1024 * 1024
+        self.ctx = C.c_void_p()
+        torch.cuda.synchronize(self.dev)
+        _check(Lb.fv_create(C.byref(self.cfg), C.byref(W), al(self.kv), al(self.cache) if cache_step >= 0 else None,
+                            al(self.ws), C.byref(self.ctx)), "fv_create")
+
+    def close(self):
+        if self.ctx:
+            lib().fv_destroy(self.ctx)
+            self.ctx = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def reset(self):
+        _check(lib().fv_reset(self.ctx), "fv_reset")
+
+    def state(self):
+        a, b = C.c_int32(), C.c_int32()
+        _check(lib().fv_get_state(self.ctx, C.byref(a), C.byref(b)), "fv_get_state")
+        return a.value, b.value
+
+    def set_state(self, next_step: int, kv_len: int):
+        _check(lib().fv_set_state(self.ctx, next_step, kv_len), "fv_set_state")
+
+    def prepare_text(self, B: int):
+        _check(lib().fv_prepare_text(self.ctx, B, _stream()), "fv_prepare_text")
+
+    def device_status(self) -> int:
+        code = C.c_int32()
+        rc = lib().fv_device_status(self.ctx, C.byref(code), _stream())
+        if rc not in (0, 6):
+            raise FvError(rc, "fv_device_status")
+        return code.value
+
+    def kv_views(self, block: int):
+        """(K [B_max, cap, C], V^T [B_max, C, cap]) bf16 views of one block's KV cache."""
+        kp, vp = C.c_void_p(), C.c_void_p()
+        _check(lib().fv_kv_pointers(self.ctx, block, C.byref(kp), C.byref(vp)), "fv_kv_pointers")
+        base = self.kv.data_ptr()
+        nel = self.B_max * self.kv_capacity * self.C
+        kview = self.kv[kp.value - base: kp.value - base + 2 * nel].view(torch.bfloat16).view(self.B_max, self.kv_capacity, self.C)
+        vview = self.kv[vp.value - base: vp.value - base + 2 * nel].view(torch.bfloat16).view(self.B_max, self.C, self.kv_capacity)
+        return kview, vview
+
+    def cache_view(self, block: int, sublayer: int, B: Optional[int] = None):
+        p = C.c_void_p()
+        _check(lib().fv_cache_pointer(self.ctx, block, sublayer, C.byref(p)), "fv_cache_pointer")
+        hc, wc = self.hw[self.cfg.cache_step]
+        B = B or self.B_max
+        nel = B * hc * wc * self.C
+        off = p.value - self.cache.data_ptr()
+        return self.cache[off: off + 2 * nel].view(torch.bfloat16).view(B, hc * wc, self.C)
+
+    def var_step(self, tokens: torch.Tensor, scale_idx: int, keep_ratio: float, out: Optional[torch.Tensor] = None,
+                 forced_idx: Optional[torch.Tensor] = None, idx_trace: Optional[torch.Tensor] = None) -> torch.Tensor:
+        assert tokens.dtype == torch.float32
+        B = tokens.shape[0]
+        if out is None:
+            out = torch.empty_like(tokens)
+        _check(lib().fv_var_step(self.ctx, _ptr(tokens), B, scale_idx, float(keep_ratio), _ptr(out), _ptr(forced_idx),
+                                 _ptr(idx_trace), _stream()), "fv_var_step")
+        return out

@@ -1,0 +1,458 @@
+// C ABI of libfastvar: argument checking, the context (host metadata only), and the per-step
+// orchestration of the pruned scale step (Sec. 3.3 "Overview" / "Implementation", Fig. 3).
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "internal.h"
+
+using namespace fv;
+
+struct fv_ctx {
+  fv_config cfg;
+  std::vector<int32_t> h, w;
+  // borrowed device pointers, per block
+  std::vector<const void*> w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2, w_q_x, w_kv_x, w_o_x;
+  const float* mod = nullptr;
+  const void* text = nullptr;
+  char* kv = nullptr;
+  char* cache = nullptr;
+  char* ws = nullptr;
+  int n_sub = 2, n_cache = 0, n_max = 0;
+  int next_step = 0, kv_len = 0;
+  bool text_ready = false;
+  // workspace carve-up
+  int32_t* status = nullptr;
+  char *a_buf = nullptr, *q_buf = nullptr, *o_buf = nullptr, *y_buf = nullptr, *h_buf = nullptr;
+  int32_t *idx = nullptr, *inv = nullptr;
+  void* sel_ws = nullptr;
+  size_t kv_block_bytes = 0, k_bytes = 0, text_k_bytes = 0, text_block_bytes = 0, cache_sub_bytes = 0;
+};
+
+namespace {
+
+std::once_flag g_init_once;
+cudaError_t g_init_err = cudaSuccess;
+
+cudaError_t ensure_init() {
+  std::call_once(g_init_once, [] {
+    g_init_err = select_init();
+    if (g_init_err == cudaSuccess) g_init_err = gemm_init();
+    if (g_init_err == cudaSuccess) g_init_err = attention_init();
+  });
+  return g_init_err;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Layout {
+  size_t status, a, q, o, y, hbuf, idx, inv, sel, total;
+};
+
+int max_tokens(const fv_config* c) {
+  int n = 0;
+  for (int i = 0; i < c->n_steps; ++i) n = std::max(n, c->h[i] * c->w[i]);
+  return n;
+}
+
+bool config_ok(const fv_config* c) {
+  if (!c || c->L <= 0 || c->C <= 0 || c->H <= 0 || c->mlp_ratio <= 0 || c->B_max <= 0 || c->n_steps <= 0) return false;
+  if (!c->h || !c->w || c->cross_len < 0 || c->kv_capacity <= 0) return false;
+  for (int i = 0; i < c->n_steps; ++i)
+    if (c->h[i] <= 0 || c->w[i] <= 0) return false;
+  if (c->cache_step >= c->n_steps) return false;
+  return true;
+}
+
+Layout workspace_layout(const fv_config* c) {
+  Layout l;
+  const size_t M = (size_t)c->B_max * max_tokens(c);
+  const size_t C = c->C, F = (size_t)c->C * c->mlp_ratio;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 1024); return o; };
+  l.status = take(256);
+  l.a = take(M * C * 2);
+  l.q = take(M * C * 2);
+  l.o = take(M * C * 2);
+  l.y = take(M * C * 2);
+  l.hbuf = take(M * F * 2);
+  l.idx = take(M * 4);
+  l.inv = take(M * 4);
+  l.sel = take(select_workspace_bytes(c->B_max, max_tokens(c), c->C));
+  l.total = off;
+  return l;
+}
+
+fv_status cuda_status(cudaError_t e) { return e == cudaSuccess ? FV_OK : FV_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+const char* fv_status_string(fv_status s) {
+  switch (s) {
+    case FV_OK: return "ok";
+    case FV_ERR_INVALID_ARG: return "invalid argument";
+    case FV_ERR_BAD_STATE: return "bad state";
+    case FV_ERR_CAPACITY: return "capacity exceeded";
+    case FV_ERR_UNSUPPORTED: return "unsupported shape";
+    case FV_ERR_CUDA: return "CUDA error";
+    case FV_ERR_TIMEOUT: return "device-side wait expired";
+  }
+  return "unknown";
+}
+
+int32_t fv_k_for(double keep_ratio, int32_t h, int32_t w) {
+  const long n = (long)h * w;
+  long k = (long)std::ceil(keep_ratio * (double)n - 1e-9);
+  if (k < 1) k = 1;
+  if (k > n) k = n;
+  return (int32_t)k;
+}
+
+size_t fv_prune_select_workspace_bytes(int32_t B, int32_t n_tokens, int32_t C) {
+  if (B <= 0 || n_tokens <= 0 || C <= 0) return 0;
+  return select_workspace_bytes(B, n_tokens, C);
+}
+
+fv_status fv_prune_select(const float* x_dev, int32_t B, int32_t h, int32_t w, int32_t C, double keep_ratio,
+                          int32_t* idx_out_dev, int32_t* inv_out_dev, float* score_out_dev, int32_t* near_tie_dev,
+                          int32_t* k_out_host, void* workspace_dev, size_t workspace_bytes, void* stream) {
+  if (!x_dev || !idx_out_dev || !workspace_dev || B <= 0 || h <= 0 || w <= 0 || C <= 0) return FV_ERR_INVALID_ARG;
+  if (!(keep_ratio > 0.0) || keep_ratio > 1.0 || (C % 4) || !aligned16(x_dev) || !aligned16(workspace_dev)) return FV_ERR_INVALID_ARG;
+  const long n = (long)h * w;
+  if (n > kTopkMaxTokens) return FV_ERR_UNSUPPORTED;
+  if (workspace_bytes < select_workspace_bytes(B, (int)n, C)) return FV_ERR_CAPACITY;
+  if (ensure_init() != cudaSuccess) return FV_ERR_CUDA;
+  const int k = fv_k_for(keep_ratio, h, w);
+  if (k_out_host) *k_out_host = k;
+  return cuda_status(launch_select(x_dev, B, (int)n, C, k, idx_out_dev, inv_out_dev, score_out_dev, near_tie_dev,
+                                   workspace_dev, static_cast<cudaStream_t>(stream)));
+}
+
+fv_status fv_restore(const void* cache_prev_dev, int32_t hc, int32_t wc, const void* pivots_dev, const int32_t* idx_dev,
+                     int32_t B, int32_t k, int32_t h, int32_t w, int32_t C, void* out_dev, int32_t* inv_scratch_dev,
+                     void* stream) {
+  if (!cache_prev_dev || !pivots_dev || !idx_dev || !out_dev || !inv_scratch_dev) return FV_ERR_INVALID_ARG;
+  if (B <= 0 || k <= 0 || h <= 0 || w <= 0 || hc <= 0 || wc <= 0 || C <= 0 || (C % 8) || k > h * w) return FV_ERR_INVALID_ARG;
+  if (!aligned16(cache_prev_dev) || !aligned16(pivots_dev) || !aligned16(out_dev)) return FV_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = launch_inv_from_idx(idx_dev, B, k, h * w, inv_scratch_dev, st);
+  if (e != cudaSuccess) return FV_ERR_CUDA;
+  return cuda_status(launch_restore_bf16(cache_prev_dev, hc, wc, pivots_dev, inv_scratch_dev, B, k, h, w, C, out_dev, st));
+}
+
+fv_status fv_gather_ln(const float* x_dev, const int32_t* idx_dev, int32_t B, int32_t n_tokens, int32_t k, int32_t C,
+                       const float* sigma_dev, const float* beta_dev, int32_t mod_stride, void* a_out_dev, void* stream) {
+  if (!x_dev || !a_out_dev || B <= 0 || n_tokens <= 0 || k <= 0 || k > n_tokens || C <= 0 || (C % 4)) return FV_ERR_INVALID_ARG;
+  if ((sigma_dev == nullptr) != (beta_dev == nullptr)) return FV_ERR_INVALID_ARG;
+  if (C > 2048) return FV_ERR_UNSUPPORTED;
+  if (!idx_dev && k != n_tokens) return FV_ERR_INVALID_ARG;
+  return cuda_status(launch_gather_ln(x_dev, idx_dev, B, n_tokens, k, C, sigma_dev, beta_dev, mod_stride, a_out_dev,
+                                      static_cast<cudaStream_t>(stream)));
+}
+
+fv_status fv_restore_residual(float* x_dev, const void* y_dev, const void* cache_dev, const int32_t* inv_dev,
+                              const float* gamma_dev, int32_t mod_stride, int32_t B, int32_t k, int32_t h, int32_t w,
+                              int32_t hc, int32_t wc, int32_t C, void* stream) {
+  if (!x_dev || !y_dev || !cache_dev || !inv_dev || B <= 0 || k <= 0 || h <= 0 || w <= 0 || hc <= 0 || wc <= 0) return FV_ERR_INVALID_ARG;
+  if (C <= 0 || (C % 8)) return FV_ERR_INVALID_ARG;
+  return cuda_status(launch_restore_residual(x_dev, y_dev, cache_dev, inv_dev, gamma_dev, mod_stride, B, k, h, w, hc, wc, C,
+                                             static_cast<cudaStream_t>(stream)));
+}
+
+fv_status fv_gemm_bf16(const void* a_dev, const void* w_dev, const void* bias_dev, int32_t M, int32_t N, int32_t K,
+                       int32_t epilogue, void* out_dev, void* aux_dev, const float* gamma_dev, int32_t mod_stride,
+                       int32_t rows_per_image, int32_t* status_dev, void* stream) {
+  if (!a_dev || !w_dev || !out_dev || epilogue < 0 || epilogue > 2) return FV_ERR_INVALID_ARG;
+  if (!aligned16(a_dev) || !aligned16(w_dev) || !aligned16(out_dev) || (bias_dev && !aligned16(bias_dev))) return FV_ERR_INVALID_ARG;
+  if (ensure_init() != cudaSuccess) return FV_ERR_CUDA;
+  GemmArgs g{};
+  g.a = a_dev; g.w = w_dev; g.bias = bias_dev; g.M = M; g.N = N; g.K = K; g.epilogue = epilogue; g.out = out_dev;
+  g.aux = aux_dev; g.gamma = gamma_dev; g.mod_stride = mod_stride; g.rows_per_image = rows_per_image > 0 ? rows_per_image : M;
+  g.status = status_dev;
+  return launch_gemm(g, static_cast<cudaStream_t>(stream));
+}
+
+fv_status fv_attention(const void* q_dev, const void* k_dev, const void* vt_dev, int32_t B, int32_t rows, int32_t H,
+                       int32_t C, int32_t kv_len, int32_t kv_capacity, void* out_dev, int32_t* status_dev, void* stream) {
+  if (ensure_init() != cudaSuccess) return FV_ERR_CUDA;
+  if (!aligned16(q_dev) || !aligned16(k_dev) || !aligned16(vt_dev) || !aligned16(out_dev)) return FV_ERR_INVALID_ARG;
+  AttnArgs a{};
+  a.q = q_dev; a.k = k_dev; a.vt = vt_dev; a.out = out_dev; a.B = B; a.rows = rows; a.H = H; a.C = C; a.kv_len = kv_len;
+  a.kv_capacity = kv_capacity; a.status = status_dev;
+  return launch_attention(a, static_cast<cudaStream_t>(stream));
+}
+
+// ------------------------------------------------------------------------------------------------ context
+
+size_t fv_workspace_bytes(const fv_config* cfg) { return config_ok(cfg) ? workspace_layout(cfg).total : 0; }
+
+size_t fv_kv_bytes(const fv_config* cfg) {
+  if (!config_ok(cfg)) return 0;
+  const size_t per_block = 2 * align_up((size_t)cfg->B_max * cfg->kv_capacity * cfg->C * 2, 1024);
+  const size_t text_block = 2 * align_up((size_t)cfg->B_max * cfg->cross_len * cfg->C * 2, 1024);
+  return (size_t)cfg->L * (per_block + text_block);
+}
+
+size_t fv_cache_bytes(const fv_config* cfg) {
+  if (!config_ok(cfg) || cfg->cache_step < 0) return 0;
+  const size_t n_cache = (size_t)cfg->h[cfg->cache_step] * cfg->w[cfg->cache_step];
+  const int n_sub = cfg->cross_len ? 3 : 2;
+  return (size_t)cfg->L * n_sub * align_up((size_t)cfg->B_max * n_cache * cfg->C * 2, 1024);
+}
+
+fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, void* cache_dev, void* workspace_dev,
+                    fv_ctx** out) {
+  if (!out) return FV_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!config_ok(cfg) || !wts || !kv_dev || !workspace_dev) return FV_ERR_INVALID_ARG;
+  if (cfg->cache_step >= 0 && !cache_dev) return FV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(kv_dev) | reinterpret_cast<uintptr_t>(workspace_dev) | reinterpret_cast<uintptr_t>(cache_dev)) & 1023u)
+    return FV_ERR_INVALID_ARG;
+  if (cfg->C % cfg->H || cfg->kv_capacity % 8 || cfg->cross_len % 8) return FV_ERR_INVALID_ARG;
+  const int hd = cfg->C / cfg->H;
+  if ((hd != 64 && hd != 128) || cfg->C > 2048 || cfg->C % 128) return FV_ERR_UNSUPPORTED;
+  if (max_tokens(cfg) > kTopkMaxTokens) return FV_ERR_UNSUPPORTED;
+  if (!wts->w_qkv || !wts->b_qkv || !wts->w_o || !wts->b_o || !wts->w_fc1 || !wts->b_fc1 || !wts->w_fc2 || !wts->b_fc2 || !wts->mod_dev)
+    return FV_ERR_INVALID_ARG;
+  if (cfg->cross_len && (!wts->w_q_x || !wts->w_kv_x || !wts->w_o_x || !wts->text_dev)) return FV_ERR_INVALID_ARG;
+  if (ensure_init() != cudaSuccess) return FV_ERR_CUDA;
+
+  fv_ctx* c = new (std::nothrow) fv_ctx();
+  if (!c) return FV_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->h.assign(cfg->h, cfg->h + cfg->n_steps);
+  c->w.assign(cfg->w, cfg->w + cfg->n_steps);
+  c->cfg.h = c->h.data();
+  c->cfg.w = c->w.data();
+  auto copy = [&](std::vector<const void*>& dst, const void* const* src) { if (src) dst.assign(src, src + cfg->L); };
+  copy(c->w_qkv, wts->w_qkv); copy(c->b_qkv, wts->b_qkv); copy(c->w_o, wts->w_o); copy(c->b_o, wts->b_o);
+  copy(c->w_fc1, wts->w_fc1); copy(c->b_fc1, wts->b_fc1); copy(c->w_fc2, wts->w_fc2); copy(c->b_fc2, wts->b_fc2);
+  if (cfg->cross_len) { copy(c->w_q_x, wts->w_q_x); copy(c->w_kv_x, wts->w_kv_x); copy(c->w_o_x, wts->w_o_x); }
+  for (int l = 0; l < cfg->L; ++l) {
+    const void* must[] = {c->w_qkv[l], c->b_qkv[l], c->w_o[l], c->b_o[l], c->w_fc1[l], c->b_fc1[l], c->w_fc2[l], c->b_fc2[l]};
+    for (const void* p : must)
+      if (!p || !aligned16(p)) { delete c; return FV_ERR_INVALID_ARG; }
+    if (cfg->cross_len && (!c->w_q_x[l] || !c->w_kv_x[l] || !c->w_o_x[l])) { delete c; return FV_ERR_INVALID_ARG; }
+  }
+  c->mod = wts->mod_dev;
+  c->text = wts->text_dev;
+  c->kv = static_cast<char*>(kv_dev);
+  c->cache = static_cast<char*>(cache_dev);
+  c->ws = static_cast<char*>(workspace_dev);
+  c->n_sub = cfg->cross_len ? 3 : 2;
+  c->n_max = max_tokens(cfg);
+  c->n_cache = cfg->cache_step >= 0 ? cfg->h[cfg->cache_step] * cfg->w[cfg->cache_step] : 0;
+  c->k_bytes = align_up((size_t)cfg->B_max * cfg->kv_capacity * cfg->C * 2, 1024);
+  c->kv_block_bytes = 2 * c->k_bytes;
+  c->text_k_bytes = align_up((size_t)cfg->B_max * cfg->cross_len * cfg->C * 2, 1024);
+  c->text_block_bytes = 2 * c->text_k_bytes;
+  c->cache_sub_bytes = align_up((size_t)cfg->B_max * c->n_cache * cfg->C * 2, 1024);
+  const Layout lay = workspace_layout(cfg);
+  c->status = reinterpret_cast<int32_t*>(c->ws + lay.status);
+  c->a_buf = c->ws + lay.a; c->q_buf = c->ws + lay.q; c->o_buf = c->ws + lay.o; c->y_buf = c->ws + lay.y;
+  c->h_buf = c->ws + lay.hbuf;
+  c->idx = reinterpret_cast<int32_t*>(c->ws + lay.idx);
+  c->inv = reinterpret_cast<int32_t*>(c->ws + lay.inv);
+  c->sel_ws = c->ws + lay.sel;
+  // Never-written KV rows must read as zeros (they meet zero probabilities in P*V).
+  if (cudaMemset(kv_dev, 0, fv_kv_bytes(cfg)) != cudaSuccess || cudaMemset(c->status, 0, 256) != cudaSuccess ||
+      cudaDeviceSynchronize() != cudaSuccess) {
+    delete c;
+    return FV_ERR_CUDA;
+  }
+  *out = c;
+  return FV_OK;
+}
+
+void fv_destroy(fv_ctx* ctx) { delete ctx; }
+
+fv_status fv_reset(fv_ctx* ctx) {
+  if (!ctx) return FV_ERR_INVALID_ARG;
+  ctx->next_step = 0;
+  ctx->kv_len = 0;
+  return FV_OK;
+}
+
+fv_status fv_get_state(const fv_ctx* ctx, int32_t* next_step_host, int32_t* kv_len_host) {
+  if (!ctx) return FV_ERR_INVALID_ARG;
+  if (next_step_host) *next_step_host = ctx->next_step;
+  if (kv_len_host) *kv_len_host = ctx->kv_len;
+  return FV_OK;
+}
+
+fv_status fv_set_state(fv_ctx* ctx, int32_t next_step, int32_t kv_len) {
+  if (!ctx || next_step < 0 || next_step > ctx->cfg.n_steps || kv_len < 0 || kv_len > ctx->cfg.kv_capacity) return FV_ERR_INVALID_ARG;
+  ctx->next_step = next_step;
+  ctx->kv_len = kv_len;
+  return FV_OK;
+}
+
+fv_status fv_kv_pointers(const fv_ctx* ctx, int32_t block, void** k_dev, void** vt_dev) {
+  if (!ctx || block < 0 || block >= ctx->cfg.L) return FV_ERR_INVALID_ARG;
+  char* base = ctx->kv + (size_t)block * ctx->kv_block_bytes;
+  if (k_dev) *k_dev = base;
+  if (vt_dev) *vt_dev = base + ctx->k_bytes;
+  return FV_OK;
+}
+
+fv_status fv_cache_pointer(const fv_ctx* ctx, int32_t block, int32_t sublayer, void** cache_dev) {
+  if (!ctx || !cache_dev || block < 0 || block >= ctx->cfg.L || sublayer < 0 || sublayer >= ctx->n_sub || !ctx->cache) return FV_ERR_INVALID_ARG;
+  *cache_dev = ctx->cache + ((size_t)block * ctx->n_sub + sublayer) * ctx->cache_sub_bytes;
+  return FV_OK;
+}
+
+static char* text_k(const fv_ctx* c, int l) { return c->kv + (size_t)c->cfg.L * c->kv_block_bytes + (size_t)l * c->text_block_bytes; }
+
+fv_status fv_prepare_text(fv_ctx* ctx, int32_t B, void* stream) {
+  if (!ctx || B <= 0 || B > ctx->cfg.B_max) return FV_ERR_INVALID_ARG;
+  if (!ctx->cfg.cross_len) return FV_OK;
+  const fv_config& c = ctx->cfg;
+  for (int l = 0; l < c.L; ++l) {
+    GemmArgs g{};
+    g.a = ctx->text; g.w = ctx->w_kv_x[l]; g.bias = nullptr; g.M = B * c.cross_len; g.N = 2 * c.C; g.K = c.C;
+    g.epilogue = EPI_QKV_SPLIT; g.out = nullptr; g.q_cols = 0; g.C = c.C; g.rows_per_image = c.cross_len;
+    g.k_cache = text_k(ctx, l); g.vt_cache = text_k(ctx, l) + ctx->text_k_bytes; g.kv_capacity = c.cross_len; g.kv_offset = 0;
+    g.status = ctx->status;
+    fv_status s = launch_gemm(g, static_cast<cudaStream_t>(stream));
+    if (s != FV_OK) return s;
+  }
+  ctx->text_ready = true;
+  return FV_OK;
+}
+
+fv_status fv_device_status(fv_ctx* ctx, int32_t* code_host, void* stream) {
+  if (!ctx) return FV_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t code = 0;
+  if (cudaMemcpyAsync(&code, ctx->status, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FV_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return FV_ERR_CUDA;
+  if (code_host) *code_host = code;
+  if (code != 0) {
+    cudaMemsetAsync(ctx->status, 0, 4, st);
+    cudaStreamSynchronize(st);
+    return FV_ERR_TIMEOUT;
+  }
+  return FV_OK;
+}
+
+fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t scale_idx, double keep_ratio, float* out_dev,
+                      const int32_t* forced_idx_dev, int32_t* idx_trace_dev, void* stream) {
+  if (!ctx || !tokens_dev || !out_dev || B <= 0 || B > ctx->cfg.B_max) return FV_ERR_INVALID_ARG;
+  if (!(keep_ratio > 0.0) || keep_ratio > 1.0 || !aligned16(tokens_dev) || !aligned16(out_dev)) return FV_ERR_INVALID_ARG;
+  const fv_config& c = ctx->cfg;
+  if (scale_idx < 0 || scale_idx >= c.n_steps) return FV_ERR_INVALID_ARG;
+  if (scale_idx != ctx->next_step) return FV_ERR_BAD_STATE;
+  const bool pruned = keep_ratio < 1.0;
+  if (pruned && (c.cache_step < 0 || scale_idx <= c.cache_step)) return FV_ERR_BAD_STATE;
+  if (!pruned && (forced_idx_dev || idx_trace_dev)) return FV_ERR_INVALID_ARG;
+  const int h = c.h[scale_idx], w = c.w[scale_idx], n = h * w, C = c.C, F = c.C * c.mlp_ratio;
+  const int k = pruned ? fv_k_for(keep_ratio, h, w) : n;
+  const int M = B * k;
+  if (ctx->kv_len + k > c.kv_capacity) return FV_ERR_CAPACITY;
+  if (c.cross_len && scale_idx > 0 && !ctx->text_ready) return FV_ERR_BAD_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* x = out_dev;
+  if (out_dev != tokens_dev &&
+      cudaMemcpyAsync(out_dev, tokens_dev, (size_t)B * n * C * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return FV_ERR_CUDA;
+  if (c.cross_len && scale_idx == 0) {
+    fv_status s = fv_prepare_text(ctx, B, stream);
+    if (s != FV_OK) return s;
+  }
+  const bool write_cache = (scale_idx == c.cache_step);
+  const int hc = c.cache_step >= 0 ? c.h[c.cache_step] : 1, wc = c.cache_step >= 0 ? c.w[c.cache_step] : 1;
+  const int mod_stride = 6 * C;
+  fv_status s = FV_OK;
+  cudaError_t e = cudaSuccess;
+
+  for (int l = 0; l < c.L && s == FV_OK; ++l) {
+    const float* mod = ctx->mod + (size_t)l * c.B_max * 6 * C;
+    char* kbase = ctx->kv + (size_t)l * ctx->kv_block_bytes;
+    for (int sub = 0; sub < ctx->n_sub && s == FV_OK; ++sub) {
+      const int kind = (ctx->n_sub == 3) ? sub : (sub == 0 ? 0 : 2);  // 0 self-attention, 1 cross-attention, 2 FFN
+      char* cache_sub = ctx->cache ? ctx->cache + ((size_t)l * ctx->n_sub + sub) * ctx->cache_sub_bytes : nullptr;
+      const size_t trace_off = ((size_t)l * ctx->n_sub + sub) * (size_t)B * k;
+      // ---- Pivotal Token Selection
+      const int32_t* idx = nullptr;
+      if (pruned) {
+        if (forced_idx_dev) {
+          idx = forced_idx_dev + trace_off;
+          e = launch_inv_from_idx(idx, B, k, n, ctx->inv, st);
+        } else {
+          idx = ctx->idx;
+          e = launch_select(x, B, n, C, k, ctx->idx, ctx->inv, nullptr, nullptr, ctx->sel_ws, st);
+        }
+        if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
+        if (idx_trace_dev && cudaMemcpyAsync(idx_trace_dev + trace_off, idx, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+          s = FV_ERR_CUDA; break;
+        }
+      }
+      // ---- gather + LayerNorm (+ AdaLN modulation)
+      const float* sigma = kind == 0 ? mod : (kind == 2 ? mod + 3 * C : nullptr);
+      const float* beta = kind == 0 ? mod + C : (kind == 2 ? mod + 4 * C : nullptr);
+      const float* gamma = kind == 0 ? mod + 2 * C : (kind == 2 ? mod + 5 * C : nullptr);
+      e = launch_gather_ln(x, idx, B, n, k, C, sigma, beta, mod_stride, ctx->a_buf, st);
+      if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
+      // ---- branch on the compact rows
+      GemmArgs g{};
+      g.status = ctx->status; g.rows_per_image = k; g.mod_stride = mod_stride;
+      const void* last_in = nullptr; const void* last_w = nullptr; const void* last_b = nullptr; int last_K = C;
+      if (kind == 0) {
+        g.a = ctx->a_buf; g.w = ctx->w_qkv[l]; g.bias = ctx->b_qkv[l]; g.M = M; g.N = 3 * C; g.K = C;
+        g.epilogue = EPI_QKV_SPLIT; g.out = ctx->q_buf; g.q_cols = C; g.C = C;
+        g.k_cache = kbase; g.vt_cache = kbase + ctx->k_bytes; g.kv_capacity = c.kv_capacity; g.kv_offset = ctx->kv_len;
+        s = launch_gemm(g, st);
+        if (s != FV_OK) break;
+        AttnArgs a{};
+        a.q = ctx->q_buf; a.k = kbase; a.vt = kbase + ctx->k_bytes; a.out = ctx->o_buf; a.B = B; a.rows = k; a.H = c.H; a.C = C;
+        a.kv_len = ctx->kv_len + k; a.kv_capacity = c.kv_capacity; a.status = ctx->status;
+        s = launch_attention(a, st);
+        if (s != FV_OK) break;
+        last_in = ctx->o_buf; last_w = ctx->w_o[l]; last_b = ctx->b_o[l];
+      } else if (kind == 1) {
+        g.a = ctx->a_buf; g.w = ctx->w_q_x[l]; g.bias = nullptr; g.M = M; g.N = C; g.K = C; g.epilogue = EPI_BF16; g.out = ctx->q_buf;
+        s = launch_gemm(g, st);
+        if (s != FV_OK) break;
+        AttnArgs a{};
+        a.q = ctx->q_buf; a.k = text_k(ctx, l); a.vt = text_k(ctx, l) + ctx->text_k_bytes; a.out = ctx->o_buf; a.B = B; a.rows = k;
+        a.H = c.H; a.C = C; a.kv_len = c.cross_len; a.kv_capacity = c.cross_len; a.status = ctx->status;
+        s = launch_attention(a, st);
+        if (s != FV_OK) break;
+        last_in = ctx->o_buf; last_w = ctx->w_o_x[l]; last_b = nullptr;
+      } else {
+        g.a = ctx->a_buf; g.w = ctx->w_fc1[l]; g.bias = ctx->b_fc1[l]; g.M = M; g.N = F; g.K = C; g.epilogue = EPI_GELU_BF16;
+        g.out = ctx->h_buf;
+        s = launch_gemm(g, st);
+        if (s != FV_OK) break;
+        last_in = ctx->h_buf; last_w = ctx->w_fc2[l]; last_b = ctx->b_fc2[l]; last_K = F;
+      }
+      // ---- last projection, then Cached Token Restoration + gate + residual
+      GemmArgs o{};
+      o.status = ctx->status; o.rows_per_image = k; o.mod_stride = mod_stride;
+      o.a = last_in; o.w = last_w; o.bias = last_b; o.M = M; o.N = C; o.K = last_K;
+      if (pruned) {
+        o.epilogue = EPI_BF16; o.out = ctx->y_buf;
+        s = launch_gemm(o, st);
+        if (s != FV_OK) break;
+        e = launch_restore_residual(x, ctx->y_buf, cache_sub, ctx->inv, gamma, mod_stride, B, k, h, w, hc, wc, C, st);
+        if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
+      } else {
+        o.epilogue = EPI_RESIDUAL; o.out = x; o.gamma = gamma; o.aux = write_cache ? cache_sub : nullptr;
+        s = launch_gemm(o, st);
+        if (s != FV_OK) break;
+      }
+    }
+  }
+  if (s != FV_OK) return s;
+  ctx->kv_len += k;
+  ctx->next_step += 1;
+  return FV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,71 @@
+// Host-side launch functions shared between the translation units of libfastvar.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/fastvar.h"
+
+namespace fv {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---- select.cu : Pivotal Token Selection (Eq. 4-5, Algorithm 1) ---------------------------------
+constexpr int kColsumRows = 32;        // token rows folded by one CTA of the column-sum kernel
+constexpr int kTopkMaxTokens = 49152;  // scores of one image must fit the top-k CTA's shared memory
+size_t select_workspace_bytes(int B, int n, int C);
+// Scores [B,n] (fp32), then exact per-image top-k -> idx [B,k] ascending, inv [B,n].
+cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* idx, int32_t* inv, float* score,
+                          int32_t* near_tie, void* workspace, cudaStream_t st);
+cudaError_t launch_inv_from_idx(const int32_t* idx, int B, int k, int n, int32_t* inv, cudaStream_t st);
+cudaError_t select_init();  // one-time function attributes
+
+// ---- rows.cu : gather + LayerNorm + modulate, restore (+ gate and residual) ----------------------
+cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
+                             const float* beta, int mod_stride, void* a_out, cudaStream_t st);
+cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv,
+                                    const float* gamma, int mod_stride, int B, int k, int h, int w, int hc, int wc,
+                                    int C, cudaStream_t st);
+cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* pivots, const int32_t* inv, int B,
+                                int k, int h, int w, int C, void* out, cudaStream_t st);
+
+// ---- gemm.cu : tcgen05 GEMM with fused epilogues -----------------------------------------------
+enum GemmEpilogue : int { EPI_BF16 = 0, EPI_GELU_BF16 = 1, EPI_RESIDUAL = 2, EPI_QKV_SPLIT = 3 };
+struct GemmArgs {
+  const void* a;     // [M,K] bf16
+  const void* w;     // [N,K] bf16
+  const void* bias;  // [N] bf16 or null
+  int M, N, K;
+  int epilogue;
+  void* out;           // EPI_BF16/GELU: bf16 [M,N]; EPI_RESIDUAL: fp32 [M,N] in place; EPI_QKV_SPLIT: Q bf16 [M,q_cols]
+  void* aux;           // EPI_RESIDUAL: optional bf16 [M,N] copy of acc+bias
+  const float* gamma;  // EPI_RESIDUAL: per-image gate or null
+  int mod_stride;      // floats between images in gamma
+  int rows_per_image;  // rows of A that belong to one image
+  // EPI_QKV_SPLIT: columns [0,q_cols) -> out; [q_cols, q_cols+C) -> K rows; the rest -> V^T.
+  int q_cols, C;
+  void* k_cache;       // [B, kv_capacity, C] bf16
+  void* vt_cache;      // [B, C, kv_capacity] bf16
+  int kv_capacity, kv_offset;
+  int32_t* status;     // device status word or null
+};
+cudaError_t gemm_init();
+fv_status launch_gemm(const GemmArgs& g, cudaStream_t st);
+
+// ---- attention.cu : flash-style attention over the KV cache ------------------------------------
+struct AttnArgs {
+  const void* q;   // [B*rows, C] bf16
+  const void* k;   // [B, kv_capacity, C] bf16
+  const void* vt;  // [B, C, kv_capacity] bf16
+  void* out;       // [B*rows, C] bf16
+  int B, rows, H, C, kv_len, kv_capacity;
+  int32_t* status;
+};
+cudaError_t attention_init();
+fv_status launch_attention(const AttnArgs& a, cudaStream_t st);
+
+// ---- tensor maps (gemm.cu) ------------------------------------------------------------------------
+// 2-D bf16 row-major tensor [rows, cols] -> TMA descriptor with a (box_rows x 64) box and 128-byte swizzle.
+bool make_tmap_bf16_2d(void* tmap_out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+
+}  // namespace fv

@@ -1,0 +1,166 @@
+"""Whole-step parity: fv_var_step through the C ABI against the CPU oracle on the same seeded inputs.
+
+Forced-index mode (the oracle's kept indices are fed to the GPU) isolates floating-point parity:
+every token must be within max-abs 3e-2 and cosine >= 0.999 of the fp64 oracle.  Free-running mode
+checks the integer side: the first pruned sublayer sees identical inputs on both sides, so its kept
+set must match the oracle's (up to near-ties at the threshold)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fastvar_oracle as O
+from paper_2503_23367_b200 import binding as fv
+from paper_2503_23367_b200 import inputs as I
+from tests.helpers import SUB_NAMES, make_oracle, per_token_errors, run_oracle, trace_to_index_tensor
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+MAX_ABS, MIN_COS = 3e-2, 0.999
+
+
+def make_ctx(wl: I.Workload, mt: I.ModelTensors, unpruned=False) -> fv.FvContext:
+    cap = sum(wl.tokens(i) if (unpruned or wl.keep[i] >= 1.0) else O.kept_count(wl.keep[i], wl.sides[i], wl.sides[i])
+              for i in range(len(wl.sides)))
+    return fv.FvContext(wl.L, wl.C, wl.H, [(s, s) for s in wl.sides], wl.cache_step, wl.B, cap, mt,
+                        cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio, device=DEV)
+
+
+def gpu_schedule(ctx, wl, xs, forced=None, trace=False):
+    outs, traces = [], []
+    ctx.reset()
+    for i, x in enumerate(xs):
+        xd = torch.from_numpy(x).to(DEV)
+        f = t = None
+        if wl.keep[i] < 1.0:
+            k = O.kept_count(wl.keep[i], wl.sides[i], wl.sides[i])
+            if forced is not None:
+                f = torch.from_numpy(forced[i]).to(DEV)
+            if trace:
+                t = torch.zeros((wl.L, wl.n_sub, wl.B, k), dtype=torch.int32, device=DEV)
+        outs.append(ctx.var_step(xd, i, wl.keep[i], forced_idx=f, idx_trace=t).cpu().numpy())
+        traces.append(None if t is None else t.cpu().numpy())
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    return outs, traces
+
+
+def check_forced(wl, kind="iid"):
+    mt = I.model_tensors(wl)
+    xs = [I.step_input(wl, i, kind) for i in range(len(wl.sides))]
+    orc, ref, tr = run_oracle(wl, mt, xs)
+    forced = [trace_to_index_tensor(wl, tr[i]) if wl.keep[i] < 1.0 else None for i in range(len(xs))]
+    ctx = make_ctx(wl, mt)
+    got, _ = gpu_schedule(ctx, wl, xs, forced=forced)
+    worst = (0.0, 1.0)
+    for i in range(len(xs)):
+        err, cos = per_token_errors(got[i], ref[i])
+        worst = (max(worst[0], err), min(worst[1], cos))
+        assert err <= MAX_ABS and cos >= MIN_COS, f"step {i} side {wl.sides[i]}: max-abs {err:.4g}, cos {cos:.6f}"
+    assert ctx.state() == (len(xs), orc.kv_len)
+    ctx.close()
+    return worst
+
+
+def test_tiny_full_schedule_forced_indices():
+    check_forced(I.WORKLOADS["tiny"])
+
+
+def test_tiny_full_schedule_structured_maps():
+    check_forced(I.WORKLOADS["tiny"], kind="structured")
+
+
+def test_var_d16_shape_two_blocks_forced_indices():
+    wl = I.WORKLOADS["var_d16_256"].with_depth(2)
+    wl = I.Workload(wl.name, L=2, C=wl.C, H=wl.H, B=2, sides=wl.sides, keep=wl.keep, seed=wl.seed)
+    check_forced(wl)
+
+
+def test_var_d30_shape_one_block_forced_indices():
+    base = I.WORKLOADS["var_d30_512"]
+    sides = (1, 2, 4, 9, 13, 18, 24)
+    wl = I.Workload("d30-short", L=1, C=base.C, H=base.H, B=2, sides=sides,
+                    keep=(1.0, 1.0, 1.0, 1.0, 1.0, 0.75, 0.5), seed=base.seed)
+    check_forced(wl)
+
+
+def test_infinity_shape_cross_attention_forced_indices():
+    base = I.WORKLOADS["infinity_2b_1k"]
+    sides = (1, 2, 4, 8, 12, 16, 24)
+    wl = I.Workload("inf-short", L=1, C=base.C, H=base.H, B=2, sides=sides,
+                    keep=(1.0, 1.0, 1.0, 1.0, 1.0, 0.6, 0.4), cross_len=64, seed=base.seed)
+    check_forced(wl)
+
+
+def test_free_running_selection_matches_oracle_on_identical_input():
+    wl = I.WORKLOADS["tiny"]
+    mt = I.model_tensors(wl)
+    xs = [I.step_input(wl, i) for i in range(len(wl.sides))]
+    orc, ref, tr = run_oracle(wl, mt, xs)
+    ctx = make_ctx(wl, mt)
+    got, traces = gpu_schedule(ctx, wl, xs, trace=True)
+    first = wl.cache_step + 1
+    names = SUB_NAMES[wl.n_sub]
+    # block 0 / self-attention of every pruned step scores the step input itself: identical on both sides
+    for i in range(first, len(xs)):
+        idx_o = tr[i][(0, "attn")]["idx"]
+        s_o = tr[i][(0, "attn")]["score"]
+        idx_g = traces[i][0, 0].astype(np.int64)
+        for b in range(wl.B):
+            assert np.all(np.diff(idx_g[b]) > 0)                         # ascending, no duplicates
+            diff = np.setxor1d(idx_g[b], idx_o[b])
+            if len(diff):
+                tau = np.sort(s_o[b])[::-1][idx_o.shape[1] - 1]
+                assert np.all(np.abs(s_o[b, diff] - tau) <= 1e-5 * tau)
+    # deeper sublayers see inputs that differ by bf16 rounding, so sets may differ near the threshold;
+    # they must still be valid index sets and agree with the oracle on the bulk of the tokens
+    agree = []
+    for i in range(first, len(xs)):
+        for l in range(wl.L):
+            for si, name in enumerate(names):
+                g, o = traces[i][l, si], tr[i][(l, name)]["idx"]
+                for b in range(wl.B):
+                    assert np.all(np.diff(g[b]) > 0) and g[b].min() >= 0 and g[b].max() < wl.tokens(i)
+                    agree.append(len(np.intersect1d(g[b], o[b])) / o.shape[1])
+    assert min(agree) >= 0.9
+    ctx.close()
+
+
+def test_keep_ratio_one_is_the_unpruned_path_and_is_deterministic():
+    wl = I.WORKLOADS["tiny"]
+    mt = I.model_tensors(wl)
+    xs = [I.step_input(wl, i) for i in range(len(wl.sides))]
+    wl_full = I.Workload("tiny-full", L=wl.L, C=wl.C, H=wl.H, B=wl.B, sides=wl.sides, keep=(1.0,) * len(wl.sides), seed=wl.seed)
+    _, ref, _ = run_oracle(wl_full, mt, xs)
+    ctx = make_ctx(wl, mt, unpruned=True)
+    a, _ = gpu_schedule(ctx, wl_full, xs)
+    b, _ = gpu_schedule(ctx, wl_full, xs)
+    for i in range(len(xs)):
+        assert np.array_equal(a[i], b[i])                                # bit-identical run to run
+        err, cos = per_token_errors(a[i], ref[i])
+        assert err <= MAX_ABS and cos >= MIN_COS
+    ctx.close()
+
+
+def test_state_and_argument_errors():
+    wl = I.WORKLOADS["tiny"]
+    mt = I.model_tensors(wl)
+    ctx = make_ctx(wl, mt)
+    x0 = torch.from_numpy(I.step_input(wl, 0)).to(DEV)
+    x1 = torch.from_numpy(I.step_input(wl, 1)).to(DEV)
+    with pytest.raises(fv.FvError) as e:
+        ctx.var_step(x1, 1, 1.0)                                         # out of order
+    assert e.value.code == 2
+    with pytest.raises(fv.FvError) as e:
+        ctx.var_step(x0, 0, 0.5)                                         # pruned before the cache step
+    assert e.value.code == 2
+    with pytest.raises(fv.FvError) as e:
+        ctx.var_step(x0, 0, 0.0)
+    assert e.value.code == 1
+    ctx.var_step(x0, 0, 1.0)
+    assert ctx.state() == (1, 1)
+    ctx.set_state(9, ctx.kv_capacity)                                    # cache full: the next step cannot fit
+    x9 = torch.from_numpy(I.step_input(wl, 9)).to(DEV)
+    with pytest.raises(fv.FvError) as e:
+        ctx.var_step(x9, 9, 0.5)
+    assert e.value.code == 3
+    ctx.close()
