@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Benchmark of the pruned VAR scale step (FastVAR cached token pruning) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" = one pass of the whole hot path over one batch of synthetic input: the full scale
+schedule of the workload (unpruned steps, the caching step, the pruned steps with select -> gather ->
+sublayers -> restore around every attention / FFN layer).  The headline metric is forwarded (kept)
+tokens per second over the pruned scale steps; ms per image is printed beside it.  Rank 0 prints ONE
+JSON line.  With N > 1 every rank runs its own batch of images (replicas, no collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2503_23367_b200 import inputs as I  # noqa: E402
+
+METRIC = "forwarded_tokens_per_s_over_pruned_scale_steps"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def kept(wl: I.Workload, i: int, pruned: bool = True) -> int:
+    n = wl.tokens(i)
+    if not pruned or wl.keep[i] >= 1.0:
+        return n
+    import math
+    return min(n, max(1, int(math.ceil(wl.keep[i] * n - 1e-9))))
+
+
+# ------------------------------------------------------------------------------------------------ reference arm
+def oracle_sample(wl: I.Workload):
+    """Bounded sample of the workload for the CPU oracle: ONE transformer block of every pruned scale
+    step, entered with a synthetic KV prefix and synthetic sublayer caches of the right sizes.
+    Returns a callable that runs the sample and the kept tokens it forwards."""
+    from oracle import fastvar_oracle as O
+    wl1 = wl.with_depth(1)
+    mt = I.model_tensors(wl1)
+    widen = lambda lst: [I.bf16_bits_to_f32(a).astype(np.float64) for a in lst]
+    w = {k: widen(getattr(mt, k)) for k in ("w_qkv", "b_qkv", "w_o", "b_o", "w_fc1", "b_fc1", "w_fc2", "b_fc2",
+                                              "w_q_x", "w_kv_x", "w_o_x")}
+    w["mod"] = mt.mod.astype(np.float64)
+    w["text"] = None if mt.text is None else I.bf16_bits_to_f32(mt.text).astype(np.float64)
+    steps = [i for i in range(len(wl.sides)) if wl.keep[i] < 1.0]
+    n_c = wl.tokens(wl.cache_step)
+    subs = ("attn", "xattn", "ffn") if wl.cross_len else ("attn", "ffn")
+    xs = {i: I.step_input(wl, i) for i in steps}
+    kv_before = {i: sum(kept(wl, j) for j in range(i)) for i in steps}
+    kvmax = max(kv_before.values())
+    kpre = [I.normal(wl.seed + 900 + b, (kvmax, wl.C)).astype(np.float64) for b in range(wl.B)]
+    vpre = [I.normal(wl.seed + 950 + b, (kvmax, wl.C)).astype(np.float64) for b in range(wl.B)]
+    caches = {s: I.normal(wl.seed + 990 + j, (wl.B, n_c, wl.C), 0.5).astype(np.float64) for j, s in enumerate(subs)}
+
+    def run():
+        for i in steps:
+            orc = O.VarOracle(1, wl.C, wl.H, [(s, s) for s in wl.sides], cache_step=wl.cache_step, weights=w,
+                              B=wl.B, cross_len=wl.cross_len)
+            orc.step, orc.kv_len = i, kv_before[i]
+            orc.Kc[0] = [kpre[b][:kv_before[i]] for b in range(wl.B)]
+            orc.Vc[0] = [vpre[b][:kv_before[i]] for b in range(wl.B)]
+            orc.cache[0] = dict(caches)
+            orc.var_step(xs[i], i, wl.keep[i])
+
+    tokens = sum(wl.B * kept(wl, i) for i in steps)
+    desc = (f"one transformer block (of {wl.L}) of each pruned scale step (sides "
+            f"{[wl.sides[i] for i in steps]}), synthetic KV prefix and caches; time x{wl.L} extrapolates to full depth")
+    return run, tokens, desc
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(wl, reps: int, warmup: int):
+    run, tokens, desc = oracle_sample(wl)
+    for _ in range(warmup):
+        run()
+    ts = []
+    for _ in range(reps):
+        t0 = time.perf_counter(); run(); ts.append(time.perf_counter() - t0)
+    t = statistics.mean(ts)
+    return {"value": tokens / (t * wl.L), "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": desc,
+            "sample_seconds": t}
+
+
+def reference_arm(args, wl):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    cb = time_oracle(wl, max(1, args.steps), max(0, args.warmup))
+    ms_step = cb["sample_seconds"] * wl.L * 1e3
+    line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "note": "CPU oracle, pruned scale steps only, depth-extrapolated"},
+            "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ our arm
+class GpuTensors:
+    """Random bf16 weights of the workload's shapes, drawn on the device (seeded)."""
+
+    def __init__(self, wl: I.Workload, dev, seed: int):
+        g = torch.Generator(device=dev); g.manual_seed(seed)
+        C, F, L = wl.C, wl.C * wl.mlp_ratio, wl.L
+        r = lambda *s, std=0.02: (torch.randn(*s, generator=g, device=dev, dtype=torch.float32) * std).to(torch.bfloat16)
+        self.w_qkv = [r(3 * C, C) for _ in range(L)]; self.b_qkv = [r(3 * C) for _ in range(L)]
+        self.w_o = [r(C, C) for _ in range(L)]; self.b_o = [r(C) for _ in range(L)]
+        self.w_fc1 = [r(F, C) for _ in range(L)]; self.b_fc1 = [r(F) for _ in range(L)]
+        self.w_fc2 = [r(C, F) for _ in range(L)]; self.b_fc2 = [r(C) for _ in range(L)]
+        x = wl.cross_len > 0
+        self.w_q_x = [r(C, C) for _ in range(L)] if x else []
+        self.w_kv_x = [r(2 * C, C) for _ in range(L)] if x else []
+        self.w_o_x = [r(C, C) for _ in range(L)] if x else []
+        self.mod = torch.randn(L, wl.B, 6, C, generator=g, device=dev, dtype=torch.float32) * 0.3
+        self.text = r(wl.B, wl.cross_len, C, std=1.0) if x else None
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.p = None
+
+    def stop(self) -> dict:
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            out, _ = self.p.communicate(timeout=5)
+        except Exception:
+            self.p.kill(); out = ""
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for nme, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nme)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [s for s in sm if s > 0.5 * max(sm)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def ours(args, wl):
+    from paper_2503_23367_b200 import binding as fv
+    from paper_2503_23367_b200 import build as fv_build
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the pruned VAR step has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        fv_build.build()
+    if world > 1:
+        dist.barrier()
+    fv.lib()
+
+    S = len(wl.sides)
+    pruned_steps = [i for i in range(S) if wl.keep[i] < 1.0]
+    gt = GpuTensors(wl, dev, seed=wl.seed + rank)
+    cap = sum(kept(wl, i) for i in range(S))
+    hw = [(s, s) for s in wl.sides]
+    ctx = fv.FvContext(wl.L, wl.C, wl.H, hw, wl.cache_step, wl.B, cap, gt, cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio, device=dev)
+    g = torch.Generator(device=dev); g.manual_seed(wl.seed + 77 + rank)
+    xs = [torch.randn(wl.B, wl.tokens(i), wl.C, generator=g, device=dev, dtype=torch.float32) for i in range(S)]
+    outs = [torch.empty_like(x) for x in xs]
+
+    def schedule(c, keep, events=None):
+        c.reset()
+        for i in range(S):
+            if events is not None:
+                events[i].record()
+            c.var_step(xs[i], i, keep[i], out=outs[i])
+        if events is not None:
+            events[S].record()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def max_over_ranks(v: float) -> float:
+        if world == 1:
+            return v
+        t = torch.tensor([v], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    for _ in range(args.warmup):
+        schedule(ctx, wl.keep)
+    barrier()
+    fv.fv_profile_read()                                   # zero the launch counters
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(S + 1)] for _ in range(args.steps)]
+    sampler = ClockSampler(local) if rank == 0 else None
+    t_wall = time.perf_counter()
+    for k in range(args.steps):
+        schedule(ctx, wl.keep, evs[k])
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    clocks = sampler.stop() if sampler else None
+    launches = fv.fv_profile_read()
+    gpu_launches = sum(v["launches"] for v in launches.values())
+    if ctx.device_status() != 0:
+        raise SystemExit("a kernel reported an expired wait")
+    total_ms = sum(evs[k][0].elapsed_time(evs[k][S]) for k in range(args.steps))
+    step_ms = [statistics.mean(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) for i in range(S)]
+    total_ms = max_over_ranks(total_ms)
+    pruned_ms = max_over_ranks(sum(step_ms[i] for i in pruned_steps))
+    ms_per_step = total_ms / args.steps
+    fwd_tokens = sum(wl.B * kept(wl, i) for i in pruned_steps)
+    value = world * fwd_tokens / (pruned_ms * 1e-3)
+
+    # ---- end to end through the public API with HOST buffers (pinned), copies inside the timed region
+    hx = [torch.randn(x.shape, dtype=torch.float32).pin_memory() for x in xs]
+    ho = [torch.empty(x.shape, dtype=torch.float32).pin_memory() for x in xs]
+    e2e_steps = 0 if args.skip_e2e else max(2, min(args.steps, 5))
+
+    def schedule_e2e(events=None):
+        ctx.reset()
+        for i in range(S):
+            if events is not None:
+                events[i].record()
+            xs[i].copy_(hx[i], non_blocking=True)
+            ctx.var_step(xs[i], i, wl.keep[i], out=outs[i])
+            ho[i].copy_(outs[i], non_blocking=True)
+        if events is not None:
+            events[S].record()
+
+    e2e = None
+    if e2e_steps:
+      schedule_e2e()
+      barrier()
+      ev2 = [[torch.cuda.Event(enable_timing=True) for _ in range(S + 1)] for _ in range(e2e_steps)]
+      for k in range(e2e_steps):
+          schedule_e2e(ev2[k])
+      barrier()
+      e2e_pruned_ms = max_over_ranks(sum(statistics.mean(ev2[k][i].elapsed_time(ev2[k][i + 1]) for k in range(e2e_steps))
+                                       for i in pruned_steps))
+      e2e_total_ms = max_over_ranks(statistics.mean(ev2[k][0].elapsed_time(ev2[k][S]) for k in range(e2e_steps)))
+      bytes_io = sum(x.numel() * 4 for x in xs)
+      e2e = {"value": world * fwd_tokens / (e2e_pruned_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": bytes_io,
+             "d2h_bytes_per_step": bytes_io, "ms_per_step": e2e_total_ms, "ms_per_image": e2e_total_ms / wl.B}
+
+    # ---- per-kernel-class device time: CUDA events around every launch, in passes of their own (the
+    # event pairs serialise the launches a little, so the timed region above runs without them)
+    peaks = measured_peaks()
+
+    def class_table(only_pruned: bool, reps: int = 2):
+        fv.fv_profile_read()                               # clear counters
+        for _ in range(reps):
+            ctx.reset()
+            for i in range(S):
+                fv.fv_profile_enable((not only_pruned) or (i in pruned_steps))
+                ctx.var_step(xs[i], i, wl.keep[i], out=outs[i])
+        raw = fv.fv_profile_read() if not only_pruned else None
+        fv.fv_profile_enable(False)
+        return raw, reps
+
+    def summarise(raw, reps):
+        table = {}
+        for name, v in raw.items():
+            if v["launches"] == 0 or v["ms"] <= 0:
+                continue
+            ms = v["ms"] / reps
+            tensor = name in ("gemm", "attention")
+            ach = (v["work"] / reps) / (ms * 1e-3) / (1e12 if tensor else 1e9)
+            peak = peaks["bf16_tflops_sustained"] if tensor else peaks["hbm_gbs"]
+            table[name] = {"ms_per_step": ms, "launches_per_step": v["launches"] // reps, "bound": "tensor" if tensor else "hbm",
+                           "achieved": ach, "unit": "TFLOP/s" if tensor else "GB/s", "peak": peak, "frac": ach / peak}
+        return table
+
+    kernels, kernels_pruned, roofline = {}, {}, None
+    if not args.skip_profile:
+        kernels = summarise(*class_table(False))
+        # pruned scale steps only: launches and work are counted always, time only while enabled, so
+        # count work with the counters cleared around exactly those steps
+        reps = 2
+        acc = None
+        for _ in range(reps):
+            ctx.reset()
+            for i in range(S):
+                if i in pruned_steps:
+                    fv.fv_profile_read(); fv.fv_profile_enable(True)
+                ctx.var_step(xs[i], i, wl.keep[i], out=outs[i])
+                if i in pruned_steps:
+                    r = fv.fv_profile_read(); fv.fv_profile_enable(False)
+                    if acc is None:
+                        acc = r
+                    else:
+                        for n_, v_ in r.items():
+                            for f_ in ("ms", "launches", "work"):
+                                acc[n_][f_] += v_[f_]
+        kernels_pruned = summarise(acc, reps)
+        dom = max(kernels_pruned, key=lambda n: kernels_pruned[n]["ms_per_step"])
+        d = kernels_pruned[dom]
+        roofline = {"kernel": dom, "region": "pruned scale steps", "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"],
+                    "unit": d["unit"], "frac": d["frac"], "traffic": None,
+                    "peak_source": f"of {peaks['source']} ({'sustained bf16 matmul' if d['bound'] == 'tensor' else 'copy bandwidth'})",
+                    "avg_launch_ms": d["ms_per_step"] / max(1, d["launches_per_step"])}
+
+    # ---- the unpruned GPU step beside it (same kernels, keep_ratio = 1 everywhere)
+    unpruned = None
+    if not args.skip_unpruned:
+        ctx.close()
+        del ctx
+        torch.cuda.empty_cache()
+        cap_full = sum(wl.tokens(i) for i in range(S))
+        ctx_full = fv.FvContext(wl.L, wl.C, wl.H, hw, wl.cache_step, wl.B, cap_full, gt, cross_len=wl.cross_len,
+                                mlp_ratio=wl.mlp_ratio, device=dev)
+        keep1 = (1.0,) * S
+        schedule(ctx_full, keep1)
+        barrier()
+        evu = [[torch.cuda.Event(enable_timing=True) for _ in range(S + 1)] for _ in range(2)]
+        for k in range(2):
+            schedule(ctx_full, keep1, evu[k])
+        barrier()
+        u_total = statistics.mean(evu[k][0].elapsed_time(evu[k][S]) for k in range(2))
+        u_pruned = sum(statistics.mean(evu[k][i].elapsed_time(evu[k][i + 1]) for k in range(2)) for i in pruned_steps)
+        unpruned = {"ms_per_image": u_total / wl.B, "ms_same_scale_steps": u_pruned, "speedup_whole_schedule": u_total / ms_per_step,
+                    "speedup_pruned_steps": u_pruned / pruned_ms}
+        ctx_full.close()
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        cb = time_oracle(wl, reps=1, warmup=0)
+        cpu_baseline = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": wl.name, "B_per_gpu": wl.B, "L": wl.L, "C": wl.C, "H": wl.H, "cross_len": wl.cross_len,
+                       "sides": list(wl.sides), "keep": list(wl.keep), "parallelism": f"replicas x{world} (images sharded, no collective)",
+                       "cache_hygiene": "inputs larger than L2 (weights + KV + token maps of one pass >> 126 MB)",
+                       "step": "one full scale schedule for one batch"},
+            "ms_per_image": ms_per_step / wl.B, "ms_per_image_pruned_steps": pruned_ms / wl.B,
+            "scale_step_ms": [round(t, 4) for t in step_ms], "wall_ms_per_step": t_wall * 1e3 / args.steps,
+            "roofline": roofline, "kernels": kernels, "kernels_pruned_steps": kernels_pruned, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": gpu_launches,
+            "clocks": clocks, "unpruned_gpu": unpruned, "peaks": peaks}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="infinity_2b_1k", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--skip-cpu", action="store_true", help="omit the CPU-oracle leg")
+    ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer end-to-end leg")
+    ap.add_argument("--skip-profile", action="store_true", help="omit the per-kernel-class timing passes")
+    ap.add_argument("--skip-unpruned", action="store_true", help="omit the unpruned GPU comparison")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    wl = I.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        reference_arm(args, wl)
+    else:
+        ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

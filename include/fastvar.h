@@ -206,6 +206,19 @@ fv_status fv_attention(const void *q_dev, const void *k_dev, const void *vt_dev,
                        int32_t rows, int32_t H, int32_t C, int32_t kv_len, int32_t kv_capacity,
                        void *out_dev, int32_t *status_dev, void *stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * Measurement support (no counterpart in the paper; Appendix "efficiency profiling" motivates the
+ * per-module breakdown).  Kernel classes, in array order: 0 select (column mean + score + top-k),
+ * 1 gather+LayerNorm, 2 GEMM, 3 attention, 4 restore.
+ *   fv_kernel_launches : kernels this library has launched since the last fv_profile_read.
+ *   fv_profile_enable  : when on, every launch is bracketed by CUDA events on its stream.
+ *   fv_profile_read    : synchronises the device; fills (each [5], HOST, may be NULL) the summed device
+ *                        milliseconds per class (0 unless timing was on), launches per class and the
+ *                        algorithmic work per class (bytes for classes 0,1,4; flops for 2,3), then clears. */
+uint64_t fv_kernel_launches(void);
+fv_status fv_profile_enable(int32_t on);
+fv_status fv_profile_read(double *ms_host, uint64_t *launches_host, double *work_host);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "FV_OK", 1: "FV_ERR_INVALID_ARG", 2: "FV_ERR_BAD_STATE", 3: "
 EXPORTS = ["fv_status_string", "fv_k_for", "fv_prune_select_workspace_bytes", "fv_prune_select", "fv_restore",
            "fv_workspace_bytes", "fv_kv_bytes", "fv_cache_bytes", "fv_create", "fv_destroy", "fv_reset",
            "fv_get_state", "fv_set_state", "fv_kv_pointers", "fv_cache_pointer", "fv_prepare_text",
-           "fv_device_status", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_gemm_bf16", "fv_attention"]
+           "fv_device_status", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_gemm_bf16", "fv_attention",
+           "fv_kernel_launches", "fv_profile_enable", "fv_profile_read"]
 
 
 class FvError(RuntimeError):
@@ -82,6 +83,10 @@ def lib() -> C.CDLL:
         L.fv_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp]
         L.fv_attention.restype = C.c_int
         L.fv_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp]
+        L.fv_kernel_launches.restype = C.c_uint64; L.fv_kernel_launches.argtypes = []
+        L.fv_profile_enable.restype = C.c_int; L.fv_profile_enable.argtypes = [i32]
+        L.fv_profile_read.restype = C.c_int
+        L.fv_profile_read.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_double)]
         _lib = L
     return _lib
 
@@ -100,6 +105,24 @@ def _stream() -> int:
 def _check(code: int, where: str) -> None:
     if code != FV_OK:
         raise FvError(code, where)
+
+
+KERNEL_CLASSES = ("select", "gather_ln", "gemm", "attention", "restore")
+
+
+def fv_kernel_launches() -> int:
+    return int(lib().fv_kernel_launches())
+
+
+def fv_profile_enable(on: bool) -> None:
+    _check(lib().fv_profile_enable(1 if on else 0), "fv_profile_enable")
+
+
+def fv_profile_read() -> dict:
+    """{class: {"ms", "launches", "work"}}; work = algorithmic bytes (select, gather_ln, restore) or flops."""
+    ms, ln, wk = (C.c_double * 5)(), (C.c_uint64 * 5)(), (C.c_double * 5)()
+    _check(lib().fv_profile_read(ms, ln, wk), "fv_profile_read")
+    return {n: {"ms": ms[i], "launches": int(ln[i]), "work": wk[i]} for i, n in enumerate(KERNEL_CLASSES)}
 
 
 def fv_k_for(keep_ratio: float, h: int, w: int) -> int:

@@ -274,6 +274,7 @@ template <int HD> fv_status launch_hd(const AttnArgs& a, cudaStream_t st) {
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   p.status = a.status;
   dim3 grid((a.rows + QT - 1) / QT, a.H, a.B);
+  LaunchScope scope(KC_ATTENTION, 1, 4.0 * a.B * (double)a.rows * a.kv_len * a.C, st);
   attention_kernel<HD><<<grid, kAttnThreads, AttnCfg<HD>::kSmemBytes, st>>>(tmQ, tmK, tmV, p);
   return cudaGetLastError() == cudaSuccess ? FV_OK : FV_ERR_CUDA;
 }

@@ -294,6 +294,7 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   p.mod_stride = g.mod_stride; p.rows_per_image = g.rows_per_image; p.q_cols = g.q_cols; p.C = g.C;
   p.k_cache = static_cast<__nv_bfloat16*>(g.k_cache); p.vt_cache = static_cast<__nv_bfloat16*>(g.vt_cache);
   p.kv_capacity = g.kv_capacity; p.kv_offset = g.kv_offset; p.status = g.status;
+  LaunchScope scope(KC_GEMM, 1, 2.0 * g.M * (double)g.N * g.K, st);
   if (wide) {
     dim3 grid(g.N / 256, tiles_m);
     gemm_bf16_kernel<256><<<grid, kGemmThreads, GemmCfg<256>::kSmemBytes, st>>>(tmA, tmB, p);

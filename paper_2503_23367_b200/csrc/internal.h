@@ -10,6 +10,18 @@ namespace fv {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// ---- prof.cu : launch counting and optional per-kernel-class timing (CUDA events on the stream) ---
+enum KernelClass : int { KC_SELECT = 0, KC_GATHER_LN = 1, KC_GEMM = 2, KC_ATTENTION = 3, KC_RESTORE = 4, KC_COUNT = 5 };
+// Brackets the launches of one kernel class: counts `kernels` launches, adds `work` (algorithmic bytes
+// for the HBM-bound classes, flops for GEMM / attention) and, when timing is enabled, records an event
+// pair around them on `st`.
+struct LaunchScope {
+  LaunchScope(KernelClass c, int kernels, double work, cudaStream_t st);
+  ~LaunchScope();
+  int slot;
+  cudaStream_t st;
+};
+
 // ---- select.cu : Pivotal Token Selection (Eq. 4-5, Algorithm 1) ---------------------------------
 constexpr int kColsumRows = 32;        // token rows folded by one CTA of the column-sum kernel
 constexpr int kTopkMaxTokens = 49152;  // scores of one image must fit the top-k CTA's shared memory

@@ -139,6 +139,7 @@ cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, i
                              const float* beta, int mod_stride, void* a_out, cudaStream_t st) {
   const int rows = B * k;
   const int blocks = (rows + 7) / 8;
+  LaunchScope scope(KC_GATHER_LN, 1, (double)rows * C * 6.0, st);
   gather_ln_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(x), idx, n, k, C / 4, sigma, beta, mod_stride,
                                            reinterpret_cast<uint2*>(a_out), rows);
   return cudaGetLastError();
@@ -147,6 +148,7 @@ cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, i
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv, const float* gamma,
                                     int mod_stride, int B, int k, int h, int w, int hc, int wc, int C, cudaStream_t st) {
   const int rows = B * h * w;
+  LaunchScope scope(KC_RESTORE, 1, (double)B * C * (8.0 * h * w + 2.0 * k + 2.0 * hc * wc), st);
   restore_residual_kernel<<<(rows + 7) / 8, 256, 0, st>>>(reinterpret_cast<float4*>(x), reinterpret_cast<const uint4*>(y),
                                                           reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride,
                                                           h * w, k, h, w, hc, wc, C / 8, rows);
@@ -156,6 +158,7 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
 cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* pivots, const int32_t* inv, int B, int k,
                                 int h, int w, int C, void* out, cudaStream_t st) {
   const int rows = B * h * w;
+  LaunchScope scope(KC_RESTORE, 1, (double)B * C * (2.0 * h * w + 2.0 * k + 2.0 * hc * wc), st);
   restore_bf16_kernel<<<(rows + 7) / 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(cache), hc, wc,
                                                       reinterpret_cast<const uint4*>(pivots), inv, h * w, k, h, w, C / 8,
                                                       reinterpret_cast<uint4*>(out), rows);

@@ -233,7 +233,7 @@ cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* i
   float* mean = reinterpret_cast<float*>(ws);
   ws += align_up((size_t)B * C * sizeof(float), 256);
   float* sc = score ? score : reinterpret_cast<float*>(ws);
-
+  LaunchScope scope(KC_SELECT, 4, (double)B * n * C * 4.0 + 4.0 * B * n + 4.0 * B * ((double)k + n), st);
   const int cs_threads = C4 >= 512 ? 512 : ((C4 + 31) / 32 * 32);
   colsum_partial_kernel<<<dim3(nchunks, B), cs_threads, 0, st>>>(reinterpret_cast<const float4*>(x), n, C4, nchunks,
                                                                  reinterpret_cast<float4*>(partial));
@@ -246,6 +246,7 @@ cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* i
 
 cudaError_t launch_inv_from_idx(const int32_t* idx, int B, int k, int n, int32_t* inv, cudaStream_t st) {
   const size_t total = (size_t)B * n;
+  LaunchScope scope(KC_SELECT, 2, 4.0 * B * ((double)k + n), st);
   inv_fill_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(inv, total);
   inv_scatter_kernel<<<(B * k + 255) / 256, 256, 0, st>>>(idx, B, k, n, inv);
   return cudaGetLastError();

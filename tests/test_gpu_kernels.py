@@ -33,6 +33,7 @@ SELECT_CASES = [  # B, h, w, C, keep, kind
     (1, 13, 13, 256, 0.5, "iid"), (8, 16, 16, 1024, 0.5, "iid"), (4, 18, 18, 1920, 0.75, "iid"),
     (2, 64, 64, 2048, 0.2, "structured"), (1, 1, 1, 256, 0.5, "iid"), (3, 5, 7, 260, 0.3, "iid"),
     (2, 40, 40, 2048, 0.6, "structured"), (1, 3, 2, 8, 1.0, "iid"), (2, 33, 31, 128, 0.01, "iid"),
+    (1, 128, 128, 2048, 0.2, "iid"),        # 2K zero-shot step: 16384 tokens, map larger than L2
 ]
 
 
