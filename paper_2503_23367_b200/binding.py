@@ -23,7 +23,8 @@ EXPORTS = ["fv_status_string", "fv_k_for", "fv_prune_select_workspace_bytes", "f
            "fv_workspace_bytes", "fv_kv_bytes", "fv_cache_bytes", "fv_create", "fv_destroy", "fv_reset",
            "fv_get_state", "fv_set_state", "fv_kv_pointers", "fv_cache_pointer", "fv_prepare_text",
            "fv_device_status", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_gemm_bf16", "fv_attention",
-           "fv_kernel_launches", "fv_profile_enable", "fv_profile_read"]
+           "fv_kernel_launches", "fv_profile_enable", "fv_profile_read",
+           "fv_prune_select_static", "fv_prune_select_static_capacity"]
 
 
 class FvError(RuntimeError):
@@ -83,6 +84,9 @@ def lib() -> C.CDLL:
         L.fv_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp]
         L.fv_attention.restype = C.c_int
         L.fv_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp]
+        L.fv_prune_select_static_capacity.restype = sz; L.fv_prune_select_static_capacity.argtypes = []
+        L.fv_prune_select_static.restype = C.c_int
+        L.fv_prune_select_static.argtypes = [vp, i32, i32, i32, i32, dbl, vp, vp, vp, vp, C.POINTER(i32), vp]
         L.fv_kernel_launches.restype = C.c_uint64; L.fv_kernel_launches.argtypes = []
         L.fv_profile_enable.restype = C.c_int; L.fv_profile_enable.argtypes = [i32]
         L.fv_profile_read.restype = C.c_int
@@ -148,6 +152,19 @@ def fv_prune_select(x: torch.Tensor, h: int, w: int, keep_ratio: float, want_inv
                                  C.byref(k_out), _ptr(workspace), workspace.numel(), _stream()), "fv_prune_select")
     assert k_out.value == k
     return {"idx": idx, "inv": inv, "score": score, "near_tie": near, "k": k}
+
+
+def fv_prune_select_static(x: torch.Tensor, h: int, w: int, keep_ratio: float, out: dict) -> int:
+    """Selection without a caller workspace, for hosts that cannot allocate: the scratch is a fixed array
+    inside the library (see fv_prune_select_static_capacity).  `out` holds the caller's own pre-made
+    output tensors: "idx" int32 [B,k] (required), optional "inv" int32 [B,n], "score" fp32 [B,n],
+    "near_tie" int32 [B].  Nothing is allocated here or in the library.  Returns k."""
+    B, n, Cw = x.shape
+    k_out = C.c_int32(0)
+    _check(lib().fv_prune_select_static(_ptr(x), B, h, w, Cw, float(keep_ratio), _ptr(out["idx"]), _ptr(out.get("inv")),
+                                        _ptr(out.get("score")), _ptr(out.get("near_tie")), C.byref(k_out), _stream()),
+           "fv_prune_select_static")
+    return k_out.value
 
 
 def fv_restore(cache_prev: torch.Tensor, hc: int, wc: int, pivots: torch.Tensor, idx: torch.Tensor, h: int, w: int,
