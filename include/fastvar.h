@@ -79,7 +79,8 @@ fv_status fv_prune_select(const float *x_dev, int32_t B, int32_t h, int32_t w, i
  *   - The first call on each device looks up the array's device address (with that device current);
  *     make that first call outside any stream capture.
  *   - All calls on a device share the one array and it keeps the previous call's contents; every
- *     word read is written earlier in the same call, so nothing needs clearing, but two calls whose
+ *     call first clears the few counters that must start at zero (every other word it reads it has
+ *     written itself), so leftovers are harmless, but two calls whose
  *     kernels overlap on the GPU (different streams, no ordering between them) race on it: order them.
  * Errors: INVALID_ARG, UNSUPPORTED (h*w > 49152), CAPACITY, CUDA. */
 size_t fv_prune_select_static_capacity(void);

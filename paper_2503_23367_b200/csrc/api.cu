@@ -125,13 +125,16 @@ fv_status fv_prune_select(const float* x_dev, int32_t B, int32_t h, int32_t w, i
   if (!x_dev || !idx_out_dev || !workspace_dev || B <= 0 || h <= 0 || w <= 0 || C <= 0) return FV_ERR_INVALID_ARG;
   if (!(keep_ratio > 0.0) || keep_ratio > 1.0 || (C % 4) || !aligned16(x_dev) || !aligned16(workspace_dev)) return FV_ERR_INVALID_ARG;
   const long n = (long)h * w;
-  if (n > kTopkMaxTokens) return FV_ERR_UNSUPPORTED;
+  if (n > kTopkMaxTokens || C > kTopkMaxTokens) return FV_ERR_UNSUPPORTED;
   if (workspace_bytes < select_workspace_bytes(B, (int)n, C)) return FV_ERR_CAPACITY;
   if (ensure_init() != cudaSuccess) return FV_ERR_CUDA;
   const int k = fv_k_for(keep_ratio, h, w);
   if (k_out_host) *k_out_host = k;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the arrival counters at the head of the workspace must start at zero
+  if (cudaMemsetAsync(workspace_dev, 0, select_ticket_bytes(B), st) != cudaSuccess) return FV_ERR_CUDA;
   return cuda_status(launch_select(x_dev, B, (int)n, C, k, idx_out_dev, inv_out_dev, score_out_dev, near_tie_dev,
-                                   workspace_dev, static_cast<cudaStream_t>(stream)));
+                                   workspace_dev, false, st));
 }
 
 fv_status fv_restore(const void* cache_prev_dev, int32_t hc, int32_t wc, const void* pivots_dev, const int32_t* idx_dev,
@@ -162,7 +165,7 @@ fv_status fv_restore_residual(float* x_dev, const void* y_dev, const void* cache
   if (!x_dev || !y_dev || !cache_dev || !inv_dev || B <= 0 || k <= 0 || h <= 0 || w <= 0 || hc <= 0 || wc <= 0) return FV_ERR_INVALID_ARG;
   if (C <= 0 || (C % 8)) return FV_ERR_INVALID_ARG;
   return cuda_status(launch_restore_residual(x_dev, y_dev, cache_dev, inv_dev, gamma_dev, mod_stride, B, k, h, w, hc, wc, C,
-                                             static_cast<cudaStream_t>(stream)));
+                                             nullptr, static_cast<cudaStream_t>(stream)));
 }
 
 fv_status fv_gemm_bf16(const void* a_dev, const void* w_dev, const void* bias_dev, int32_t M, int32_t N, int32_t K,
@@ -262,6 +265,7 @@ fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, v
   c->sel_ws = c->ws + lay.sel;
   // Never-written KV rows must read as zeros (they meet zero probabilities in P*V).
   if (cudaMemset(kv_dev, 0, fv_kv_bytes(cfg)) != cudaSuccess || cudaMemset(c->status, 0, 256) != cudaSuccess ||
+      cudaMemset(c->sel_ws, 0, select_ticket_bytes(cfg->B_max)) != cudaSuccess ||
       cudaDeviceSynchronize() != cudaSuccess) {
     delete c;
     return FV_ERR_CUDA;
@@ -370,6 +374,11 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   const int mod_stride = 6 * C;
   fv_status s = FV_OK;
   cudaError_t e = cudaSuccess;
+  // Column sums of x (Eq. 4) for the next selection are left in the selection scratch by the restore
+  // kernel of the sublayer before it; only the first sublayer of a step has to sum the map itself.
+  bool have_partials = false;
+  const bool selecting = pruned && !forced_idx_dev;
+  if (selecting && cudaMemsetAsync(ctx->sel_ws, 0, select_ticket_bytes(B), st) != cudaSuccess) return FV_ERR_CUDA;
 
   for (int l = 0; l < c.L && s == FV_OK; ++l) {
     const float* mod = ctx->mod + (size_t)l * c.B_max * 6 * C;
@@ -386,7 +395,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
           e = launch_inv_from_idx(idx, B, k, n, ctx->inv, st);
         } else {
           idx = ctx->idx;
-          e = launch_select(x, B, n, C, k, ctx->idx, ctx->inv, nullptr, nullptr, ctx->sel_ws, st);
+          e = launch_select(x, B, n, C, k, ctx->idx, ctx->inv, nullptr, nullptr, ctx->sel_ws, have_partials, st);
         }
         if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
         if (idx_trace_dev && cudaMemcpyAsync(idx_trace_dev + trace_off, idx, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
@@ -440,8 +449,11 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         o.epilogue = EPI_BF16; o.out = ctx->y_buf;
         s = launch_gemm(o, st);
         if (s != FV_OK) break;
-        e = launch_restore_residual(x, ctx->y_buf, cache_sub, ctx->inv, gamma, mod_stride, B, k, h, w, hc, wc, C, st);
+        const bool more = selecting && !(l == c.L - 1 && sub == ctx->n_sub - 1);
+        e = launch_restore_residual(x, ctx->y_buf, cache_sub, ctx->inv, gamma, mod_stride, B, k, h, w, hc, wc, C,
+                                    more ? ctx->sel_ws : nullptr, st);
         if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
+        have_partials = more;
       } else {
         o.epilogue = EPI_RESIDUAL; o.out = x; o.gamma = gamma; o.aux = write_cache ? cache_sub : nullptr;
         s = launch_gemm(o, st);

@@ -23,21 +23,37 @@ struct LaunchScope {
 };
 
 // ---- select.cu : Pivotal Token Selection (Eq. 4-5, Algorithm 1) ---------------------------------
-constexpr int kColsumRows = 32;        // token rows folded by one CTA of the column-sum kernel
+constexpr int kColsumRows = 32;        // token rows folded into one chunk partial of the column sums
+constexpr int kMaxGroups = 8;          // chunk partials are folded again into at most this many group partials
 constexpr int kTopkMaxTokens = 49152;  // scores of one image must fit the top-k CTA's shared memory
+// Scratch of the selection, carved out of one caller buffer.  Column sums of the token map are kept at
+// two levels: one partial per chunk of kColsumRows tokens, folded (by the last CTA of each group to
+// finish) into <= kMaxGroups group partials per image, which the scoring kernel adds up itself.
+struct SelectWs {
+  unsigned int* tickets;  // [B, kMaxGroups] group arrival counters, then [B] image counters; zero between launches
+  float* chunk_partial;   // [B, nchunks, C]
+  float* group_partial;   // [B, ngroups, C]
+  float* score;           // [B, n]
+  int nchunks, group, ngroups;
+};
 size_t select_workspace_bytes(int B, int n, int C);
-// Scores [B,n] (fp32), then exact per-image top-k -> idx [B,k] ascending, inv [B,n].
+size_t select_ticket_bytes(int B);  // leading bytes of the workspace that must be zero before first use
+SelectWs select_ws_carve(void* workspace, int B, int n, int C);
+// Scores [B,n] (fp32), then exact per-image top-k -> idx [B,k] ascending, inv [B,n].  have_partials:
+// the group partials in the workspace already hold the column sums of x (left there by
+// launch_restore_residual), so the column-sum pass is skipped.
 cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* idx, int32_t* inv, float* score,
-                          int32_t* near_tie, void* workspace, cudaStream_t st);
+                          int32_t* near_tie, void* workspace, bool have_partials, cudaStream_t st);
 cudaError_t launch_inv_from_idx(const int32_t* idx, int B, int k, int n, int32_t* inv, cudaStream_t st);
 cudaError_t select_init();  // one-time function attributes
 
 // ---- rows.cu : gather + LayerNorm + modulate, restore (+ gate and residual) ----------------------
 cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
                              const float* beta, int mod_stride, void* a_out, cudaStream_t st);
+// colsum_ws: null, or the selection workspace that receives the column sums of the updated x.
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv,
                                     const float* gamma, int mod_stride, int B, int k, int h, int w, int hc, int wc,
-                                    int C, cudaStream_t st);
+                                    int C, void* colsum_ws, cudaStream_t st);
 cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* pivots, const int32_t* inv, int B,
                                 int k, int h, int w, int C, void* out, cudaStream_t st);
 

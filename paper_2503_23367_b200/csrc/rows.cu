@@ -5,10 +5,12 @@
 //                      gather through the inverse index map (no scatter, so no write races), fused
 //                      with the gate and the residual add.
 //   restore_bf16     : the plain restoration, bf16 in / bf16 out, bit-exact copy.
-// One warp owns one token row; every global access is a 128-bit vector, consecutive lanes touching
-// consecutive 16-byte words.
+// Every global access is a 128-bit vector, consecutive lanes touching consecutive 16-byte words.  The
+// kernels are short, so they are arranged to keep the chain of dependent global accesses short (index
+// -> row -> store) with everything else (modulation vectors, the residual rows) fetched beside it.
 #include <cuda_bf16.h>
 
+#include "colsum_fold.cuh"
 #include "internal.h"
 
 namespace fv {
@@ -17,25 +19,39 @@ namespace {
 
 constexpr int kMaxVec = 16;  // float4 per lane -> C <= 2048
 
+// grid (ceil(k / 8), B): one warp per kept row; sigma / beta of the image staged in shared memory while
+// the row index and the row itself are in flight.
 __global__ void __launch_bounds__(256) gather_ln_kernel(const float4* __restrict__ x, const int32_t* __restrict__ idx, int n,
                                                         int k, int C4, const float* __restrict__ sigma,
                                                         const float* __restrict__ beta, int mod_stride,
-                                                        uint2* __restrict__ a_out, int total_rows) {
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (warp >= total_rows) return;
-  const int b = warp / k, j = warp - b * k;
-  const int t = idx ? idx[warp] : j;
+                                                        uint2* __restrict__ a_out) {
+  extern __shared__ float4 s_mod[];  // sigma [C4] then beta [C4]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.y, j = blockIdx.x * 8 + warp;
+  const bool live = j < k;
+  const int t = live ? (idx ? __ldg(idx + (size_t)b * k + j) : j) : 0;
+  if (sigma) {
+    const float4* sg = reinterpret_cast<const float4*>(sigma + (size_t)b * mod_stride);
+    const float4* bt = reinterpret_cast<const float4*>(beta + (size_t)b * mod_stride);
+    for (int i = threadIdx.x; i < C4; i += 256) { s_mod[i] = __ldg(sg + i); s_mod[C4 + i] = __ldg(bt + i); }
+  }
   const float4* row = x + ((size_t)b * n + t) * C4;
   float4 v[kMaxVec];
   float sum = 0.f;
+  if (live) {
 #pragma unroll
-  for (int i = 0; i < kMaxVec; ++i) {
-    const int c4 = lane + 32 * i;
-    if (c4 < C4) {
-      v[i] = __ldg(row + c4);
-      sum += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+    for (int i = 0; i < kMaxVec; ++i) {
+      const int c4 = lane + 32 * i;
+      if (c4 < C4) v[i] = __ldg(row + c4);
+    }
+#pragma unroll
+    for (int i = 0; i < kMaxVec; ++i) {
+      const int c4 = lane + 32 * i;
+      if (c4 < C4) sum += (v[i].x + v[i].y) + (v[i].z + v[i].w);
     }
   }
+  __syncthreads();
+  if (!live) return;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
   const float inv_c = 1.0f / (float)(C4 * 4);
@@ -52,19 +68,17 @@ __global__ void __launch_bounds__(256) gather_ln_kernel(const float4* __restrict
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) var += __shfl_xor_sync(0xffffffffu, var, o);
   const float rstd = rsqrtf(var * inv_c + 1e-6f);
-  const float4* sg = sigma ? reinterpret_cast<const float4*>(sigma + (size_t)b * mod_stride) : nullptr;
-  const float4* bt = beta ? reinterpret_cast<const float4*>(beta + (size_t)b * mod_stride) : nullptr;
-  uint2* dst = a_out + (size_t)warp * C4;
+  uint2* dst = a_out + ((size_t)b * k + j) * C4;
 #pragma unroll
   for (int i = 0; i < kMaxVec; ++i) {
     const int c4 = lane + 32 * i;
     if (c4 < C4) {
       float4 a;
       a.x = (v[i].x - mu) * rstd; a.y = (v[i].y - mu) * rstd; a.z = (v[i].z - mu) * rstd; a.w = (v[i].w - mu) * rstd;
-      if (sg) {
-        float4 s = __ldg(sg + c4), bb = __ldg(bt + c4);
-        a.x = fmaf(a.x, 1.f + s.x, bb.x); a.y = fmaf(a.y, 1.f + s.y, bb.y);
-        a.z = fmaf(a.z, 1.f + s.z, bb.z); a.w = fmaf(a.w, 1.f + s.w, bb.w);
+      if (sigma) {
+        const float4 sg = s_mod[c4], bb = s_mod[C4 + c4];
+        a.x = fmaf(a.x, 1.f + sg.x, bb.x); a.y = fmaf(a.y, 1.f + sg.y, bb.y);
+        a.z = fmaf(a.z, 1.f + sg.z, bb.z); a.w = fmaf(a.w, 1.f + sg.w, bb.w);
       }
       __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
       uint2 o;
@@ -90,33 +104,72 @@ __device__ __forceinline__ void bf16x8_to_float(const uint4& p, float (&f)[8]) {
 }
 
 // x[b,t,:] += gamma[b,:] * (inv[b,t] >= 0 ? y[b*k + inv[b,t], :] : cache[b, src(t), :])
+// grid (chunks of 32 tokens, B), 256 threads; a thread owns 8 channels (one 16-byte bf16 word of the
+// source, two float4 of x) for all rows of the chunk, so the column sums of the updated rows -- the
+// next sublayer's Eq. 4 -- fall out of the same registers with no cross-thread reduction.  The source
+// row of every token is resolved once into shared memory; the x rows do not wait for it.
 __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restrict__ x, const uint4* __restrict__ y,
                                                                const uint4* __restrict__ cache, const int32_t* __restrict__ inv,
                                                                const float* __restrict__ gamma, int mod_stride, int n, int k,
-                                                               int h, int w, int hc, int wc, int C8, int total_rows) {
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (warp >= total_rows) return;
-  const int b = warp / n, t = warp - b * n;
-  const int j = inv[warp];
-  const uint4* src = (j >= 0) ? y + ((size_t)b * k + j) * C8
-                              : cache + ((size_t)b * hc * wc + nearest_src(t, h, w, hc, wc)) * C8;
-  float4* xr = x + (size_t)warp * C8 * 2;
-  const float4* g = gamma ? reinterpret_cast<const float4*>(gamma + (size_t)b * mod_stride) : nullptr;
-  for (int c8 = lane; c8 < C8; c8 += 32) {
-    float f[8];
-    bf16x8_to_float(__ldg(src + c8), f);
-    float4 x0 = xr[2 * c8], x1 = xr[2 * c8 + 1];
-    if (g) {
-      float4 g0 = __ldg(g + 2 * c8), g1 = __ldg(g + 2 * c8 + 1);
-      x0.x = fmaf(g0.x, f[0], x0.x); x0.y = fmaf(g0.y, f[1], x0.y); x0.z = fmaf(g0.z, f[2], x0.z); x0.w = fmaf(g0.w, f[3], x0.w);
-      x1.x = fmaf(g1.x, f[4], x1.x); x1.y = fmaf(g1.y, f[5], x1.y); x1.z = fmaf(g1.z, f[6], x1.z); x1.w = fmaf(g1.w, f[7], x1.w);
-    } else {
-      x0.x += f[0]; x0.y += f[1]; x0.z += f[2]; x0.w += f[3];
-      x1.x += f[4]; x1.y += f[5]; x1.z += f[6]; x1.w += f[7];
-    }
-    xr[2 * c8] = x0;
-    xr[2 * c8 + 1] = x1;
+                                                               int h, int w, int hc, int wc, int C8, int nchunks, int group,
+                                                               int ngroups, float4* __restrict__ chunk_partial,
+                                                               float4* __restrict__ group_partial, unsigned int* tickets) {
+  __shared__ const uint4* s_src[kColsumRows];
+  const int b = blockIdx.y, chunk = blockIdx.x;
+  const int t0 = chunk * kColsumRows;
+  const int rows = min(kColsumRows, n - t0);
+  if (threadIdx.x < rows) {
+    const int t = t0 + threadIdx.x;
+    const int j = __ldg(inv + (size_t)b * n + t);
+    s_src[threadIdx.x] = (j >= 0) ? y + ((size_t)b * k + j) * C8
+                                  : cache + ((size_t)b * hc * wc + nearest_src(t, h, w, hc, wc)) * C8;
   }
+  __syncthreads();
+  float4* xbase = x + ((size_t)b * n + t0) * C8 * 2;
+  for (int c8 = threadIdx.x; c8 < C8; c8 += 256) {
+    float4 g0 = make_float4(1.f, 1.f, 1.f, 1.f), g1 = g0;
+    if (gamma) {
+      const float4* g = reinterpret_cast<const float4*>(gamma + (size_t)b * mod_stride);
+      g0 = __ldg(g + 2 * c8); g1 = __ldg(g + 2 * c8 + 1);
+    }
+    float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+    for (int r = 0; r < rows; r += 4) {
+      uint4 p[4];
+      float4 x0[4], x1[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (r + i < rows) {
+          float4* xr = xbase + (size_t)(r + i) * C8 * 2 + 2 * c8;
+          x0[i] = xr[0]; x1[i] = xr[1];
+          p[i] = __ldg(s_src[r + i] + c8);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (r + i < rows) {
+          float f[8];
+          bf16x8_to_float(p[i], f);
+          float4 u0 = x0[i], u1 = x1[i];
+          if (gamma) {
+            u0.x = fmaf(g0.x, f[0], u0.x); u0.y = fmaf(g0.y, f[1], u0.y); u0.z = fmaf(g0.z, f[2], u0.z); u0.w = fmaf(g0.w, f[3], u0.w);
+            u1.x = fmaf(g1.x, f[4], u1.x); u1.y = fmaf(g1.y, f[5], u1.y); u1.z = fmaf(g1.z, f[6], u1.z); u1.w = fmaf(g1.w, f[7], u1.w);
+          } else {
+            u0.x += f[0]; u0.y += f[1]; u0.z += f[2]; u0.w += f[3];
+            u1.x += f[4]; u1.y += f[5]; u1.z += f[6]; u1.w += f[7];
+          }
+          float4* xr = xbase + (size_t)(r + i) * C8 * 2 + 2 * c8;
+          xr[0] = u0; xr[1] = u1;
+          a0.x += u0.x; a0.y += u0.y; a0.z += u0.z; a0.w += u0.w;
+          a1.x += u1.x; a1.y += u1.y; a1.z += u1.z; a1.w += u1.w;
+        }
+      }
+    }
+    if (chunk_partial) {
+      float4* cp = chunk_partial + ((size_t)b * nchunks + chunk) * C8 * 2 + 2 * c8;
+      cp[0] = a0; cp[1] = a1;
+    }
+  }
+  if (chunk_partial) fold_group_partials(b, chunk, nchunks, group, ngroups, C8 * 2, chunk_partial, group_partial, tickets);
 }
 
 __global__ void __launch_bounds__(256) restore_bf16_kernel(const uint4* __restrict__ cache, int hc, int wc,
@@ -138,20 +191,26 @@ __global__ void __launch_bounds__(256) restore_bf16_kernel(const uint4* __restri
 cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
                              const float* beta, int mod_stride, void* a_out, cudaStream_t st) {
   const int rows = B * k;
-  const int blocks = (rows + 7) / 8;
   LaunchScope scope(KC_GATHER_LN, 1, (double)rows * C * 6.0, st);
-  gather_ln_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(x), idx, n, k, C / 4, sigma, beta, mod_stride,
-                                           reinterpret_cast<uint2*>(a_out), rows);
+  gather_ln_kernel<<<dim3((k + 7) / 8, B), 256, sigma ? (size_t)C * 8 : 0, st>>>(reinterpret_cast<const float4*>(x), idx, n, k, C / 4,
+                                                                                sigma, beta, mod_stride,
+                                                                                reinterpret_cast<uint2*>(a_out));
   return cudaGetLastError();
 }
 
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv, const float* gamma,
-                                    int mod_stride, int B, int k, int h, int w, int hc, int wc, int C, cudaStream_t st) {
-  const int rows = B * h * w;
-  LaunchScope scope(KC_RESTORE, 1, (double)B * C * (8.0 * h * w + 2.0 * k + 2.0 * hc * wc), st);
-  restore_residual_kernel<<<(rows + 7) / 8, 256, 0, st>>>(reinterpret_cast<float4*>(x), reinterpret_cast<const uint4*>(y),
-                                                          reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride,
-                                                          h * w, k, h, w, hc, wc, C / 8, rows);
+                                    int mod_stride, int B, int k, int h, int w, int hc, int wc, int C, void* colsum_ws,
+                                    cudaStream_t st) {
+  const int n = h * w;
+  SelectWs ws{};
+  if (colsum_ws) ws = select_ws_carve(colsum_ws, B, n, C);
+  const int nchunks = (n + kColsumRows - 1) / kColsumRows;
+  LaunchScope scope(KC_RESTORE, 1, (double)B * C * (8.0 * n + 2.0 * k + 2.0 * hc * wc), st);
+  restore_residual_kernel<<<dim3(nchunks, B), 256, 0, st>>>(reinterpret_cast<float4*>(x), reinterpret_cast<const uint4*>(y),
+                                                            reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k,
+                                                            h, w, hc, wc, C / 8, nchunks, ws.group, ws.ngroups,
+                                                            reinterpret_cast<float4*>(ws.chunk_partial),
+                                                            reinterpret_cast<float4*>(ws.group_partial), ws.tickets);
   return cudaGetLastError();
 }
 

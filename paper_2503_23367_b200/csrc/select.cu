@@ -1,22 +1,33 @@
 // Pivotal Token Selection (Sec. 3.3, Eq. 4-5, Algorithm 1 first routine) on sm_100a.
 //
-//   colsum_partial -> mean_finalize : Eq. 4, the per-image mean token (deterministic two-stage sum)
-//   score_rows                      : s[b,t] = sum_c (x[b,t,c] - mean[b,c])^2   (one warp per token)
-//   topk_select                     : exact k largest per image, ties to the lowest index, ascending
-//                                     output, inverse map (one CTA per image, radix select on the
-//                                     fp32 bit patterns, which order like the values for s >= 0)
-// All HBM access is 128-bit and coalesced; no float atomics anywhere (bit-reproducible).
+//   colsum_chunk_kernel : Eq. 4's sum over tokens, one partial per chunk of 32 tokens, folded into at most
+//                         8 group partials per image by the last CTA of each group (fixed order).  Skipped
+//                         when the previous restore kernel has already left the partials of its output.
+//   score_topk_kernel   : s[b,t] = sum_c (x[b,t,c] - mean[b,c])^2, one warp per token, the mean token
+//                         rebuilt from the group partials in shared memory; the last CTA of each image to
+//                         finish then runs the exact top-k of that image: radix select on the fp32 bit
+//                         patterns (which order like the values for s >= 0), ties to the lowest index,
+//                         ascending output, inverse map.
+// Few launches and short chains of dependent loads matter more here than peak bandwidth: the maps are
+// tens of MB, and every dependent global access costs about a microsecond.  All HBM access is 128-bit
+// and coalesced; no float atomics anywhere (bit-reproducible).
+#include "colsum_fold.cuh"
 #include "internal.h"
 
 namespace fv {
 
 namespace {
 
-constexpr int kScoreRowsPerCta = 32;
-constexpr int kTopkThreads = 1024;
+constexpr int kTopkThreads = 512;
+constexpr int kTopkWarps = kTopkThreads / 32;
+// Keys sit in shared memory with one pad word per 32, so that both access patterns of the top-k are
+// free of bank conflicts: consecutive lanes on consecutive tokens, and each lane on its own contiguous run.
+__device__ __forceinline__ int KI(int i) { return i + (i >> 5); }
+constexpr size_t kTopkMaxSmem = ((size_t)kTopkMaxTokens + kTopkMaxTokens / 32) * 4;
 
-__global__ void __launch_bounds__(512) colsum_partial_kernel(const float4* __restrict__ x, int n, int C4, int nchunks,
-                                                             float4* __restrict__ partial) {
+__global__ void __launch_bounds__(256) colsum_chunk_kernel(const float4* __restrict__ x, int n, int C4, int nchunks, int group,
+                                                           int ngroups, float4* __restrict__ chunk_partial,
+                                                           float4* __restrict__ group_partial, unsigned int* tickets) {
   const int b = blockIdx.y, chunk = blockIdx.x;
   const int r0 = chunk * kColsumRows;
   const int r1 = min(n, r0 + kColsumRows);
@@ -24,60 +35,23 @@ __global__ void __launch_bounds__(512) colsum_partial_kernel(const float4* __res
   for (int c4 = threadIdx.x; c4 < C4; c4 += blockDim.x) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     int r = r0;
-    for (; r + 4 <= r1; r += 4) {
-      float4 v0 = __ldg(base + (size_t)(r + 0) * C4 + c4);
-      float4 v1 = __ldg(base + (size_t)(r + 1) * C4 + c4);
-      float4 v2 = __ldg(base + (size_t)(r + 2) * C4 + c4);
-      float4 v3 = __ldg(base + (size_t)(r + 3) * C4 + c4);
-      acc.x += v0.x; acc.y += v0.y; acc.z += v0.z; acc.w += v0.w;
-      acc.x += v1.x; acc.y += v1.y; acc.z += v1.z; acc.w += v1.w;
-      acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w;
-      acc.x += v3.x; acc.y += v3.y; acc.z += v3.z; acc.w += v3.w;
+    for (; r + 8 <= r1; r += 8) {
+      float4 v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = __ldg(base + (size_t)(r + i) * C4 + c4);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w; }
     }
     for (; r < r1; ++r) {
-      float4 v = __ldg(base + (size_t)r * C4 + c4);
+      const float4 v = __ldg(base + (size_t)r * C4 + c4);
       acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
     }
-    partial[((size_t)b * nchunks + chunk) * C4 + c4] = acc;
+    chunk_partial[((size_t)b * nchunks + chunk) * C4 + c4] = acc;
   }
+  fold_group_partials(b, chunk, nchunks, group, ngroups, C4, chunk_partial, group_partial, tickets);
 }
 
-__global__ void mean_finalize_kernel(const float* __restrict__ partial, int nchunks, int C, int n, float* __restrict__ mean) {
-  const int b = blockIdx.y;
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= C) return;
-  const float* p = partial + (size_t)b * nchunks * C + c;
-  float acc = 0.f;
-  for (int i = 0; i < nchunks; ++i) acc += p[(size_t)i * C];
-  mean[(size_t)b * C + c] = acc / (float)n;
-}
-
-__global__ void __launch_bounds__(256) score_rows_kernel(const float4* __restrict__ x, const float4* __restrict__ mean, int n,
-                                                         int C4, float* __restrict__ score) {
-  extern __shared__ float4 s_mean[];
-  const int b = blockIdx.y;
-  for (int i = threadIdx.x; i < C4; i += blockDim.x) s_mean[i] = mean[(size_t)b * C4 + i];
-  __syncthreads();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r0 = blockIdx.x * kScoreRowsPerCta;
-  for (int rr = warp; rr < kScoreRowsPerCta; rr += 8) {
-    const int r = r0 + rr;
-    if (r >= n) break;
-    const float4* row = x + ((size_t)b * n + r) * C4;
-    float acc = 0.f;
-    for (int c4 = lane; c4 < C4; c4 += 32) {
-      float4 v = __ldg(row + c4);
-      float4 m = s_mean[c4];
-      float dx = v.x - m.x, dy = v.y - m.y, dz = v.z - m.z, dw = v.w - m.w;
-      acc += dx * dx; acc += dy * dy; acc += dz * dz; acc += dw * dw;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) score[(size_t)b * n + r] = acc;
-  }
-}
-
-// Exclusive prefix sum of one value per thread over the whole CTA (1024 threads); returns the
+// Exclusive prefix sum of one value per thread over the whole CTA (kTopkThreads threads); returns the
 // exclusive prefix and, through `total`, the CTA-wide sum.  s_warp is 32 words of scratch.
 __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s_warp, uint32_t* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -90,7 +64,7 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
   __syncthreads();  // s_warp may still be read from a previous scan
   if (lane == 31) s_warp[warp] = inc;
   __syncthreads();
-  uint32_t wv = s_warp[lane];  // blockDim.x == 1024 -> 32 warps
+  uint32_t wv = lane < kTopkWarps ? s_warp[lane] : 0u;
   uint32_t winc = wv;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -102,29 +76,110 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
   return warp_excl + inc - v;
 }
 
-__global__ void __launch_bounds__(kTopkThreads) topk_select_kernel(const float* __restrict__ score, int n, int k,
-                                                                   int32_t* __restrict__ idx, int32_t* __restrict__ inv,
-                                                                   int32_t* __restrict__ near_tie) {
-  extern __shared__ uint32_t s_keys[];  // n keys
+// grid (CTAs per image, B), 512 threads, sized to be resident all at once (two CTAs per SM); the warps of
+// an image stride over its token rows.  Dynamic shared memory max(C, n + n/32) * 4 bytes (mean token, then keys).
+__global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float4* __restrict__ x,
+                                                                  const float4* __restrict__ group_partial, int ngroups, int n,
+                                                                  int C4, int k, float* __restrict__ score,
+                                                                  unsigned int* img_tickets, int32_t* __restrict__ idx,
+                                                                  int32_t* __restrict__ inv, int32_t* __restrict__ near_tie) {
+  extern __shared__ float4 s_dyn[];
+  float4* s_mean = s_dyn;
+  uint32_t* s_keys = reinterpret_cast<uint32_t*>(s_dyn);  // reused once the scores are out
   __shared__ uint32_t s_hist[256];
   __shared__ uint32_t s_warp[32];
   __shared__ uint32_t s_prefix, s_remaining, s_near;
-  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
-  const float* sc = score + (size_t)b * n;
-  for (int i = tid; i < n; i += kTopkThreads) s_keys[i] = __float_as_uint(sc[i]) & 0x7FFFFFFFu;  // s >= 0; drops the sign of -0
-  if (tid == 0) { s_prefix = 0u; s_remaining = (uint32_t)k; s_near = 0u; }
+  __shared__ int s_last;
+  const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  // ---- Eq. 4: the mean token of image b from the group partials (fixed order)
+  {
+    const float4* gp = group_partial + (size_t)b * ngroups * C4;
+    const float fn = (float)n;
+    for (int c4 = tid; c4 < C4; c4 += kTopkThreads) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int g = 0; g < ngroups; ++g) {
+        const float4 v = __ldcg(gp + (size_t)g * C4 + c4);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+      s_mean[c4] = make_float4(acc.x / fn, acc.y / fn, acc.z / fn, acc.w / fn);
+    }
+  }
   __syncthreads();
 
-  // Radix select, most significant byte first: after 4 passes s_prefix is the k-th largest key and
+  // ---- Eq. 5 / Algorithm 1: squared deviation from the mean, one warp per token row
+  for (int r = blockIdx.x * kTopkWarps + warp; r < n; r += gridDim.x * kTopkWarps) {
+    const float4* row = x + ((size_t)b * n + r) * C4;
+    float acc = 0.f;
+    int c4 = lane;
+    for (; c4 + 32 * 7 < C4; c4 += 32 * 8) {
+      float4 v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = __ldg(row + c4 + 32 * i);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float4 m = s_mean[c4 + 32 * i];
+        const float dx = v[i].x - m.x, dy = v[i].y - m.y, dz = v[i].z - m.z, dw = v[i].w - m.w;
+        acc += dx * dx; acc += dy * dy; acc += dz * dz; acc += dw * dw;
+      }
+    }
+    for (; c4 < C4; c4 += 32) {
+      const float4 v = __ldg(row + c4);
+      const float4 m = s_mean[c4];
+      const float dx = v.x - m.x, dy = v.y - m.y, dz = v.z - m.z, dw = v.w - m.w;
+      acc += dx * dx; acc += dy * dy; acc += dz * dz; acc += dw * dw;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) score[(size_t)b * n + r] = acc;
+  }
+  __threadfence();  // this thread's scores are visible device-wide before the CTA takes its ticket
+
+  // ---- the last CTA of this image to get here ranks the image
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned int prev = atomicAdd(img_tickets + b, 1u);
+    s_last = (prev == gridDim.x - 1);
+    if (s_last) img_tickets[b] = 0u;
+    s_prefix = 0u; s_remaining = (uint32_t)k; s_near = 0u;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+
+  // Keys = fp32 bit patterns of the scores (s >= 0, so they order like the values) taken relative to the
+  // smallest key of the image: the scores of one map share their leading bits, and ranking only the
+  // bits that differ both skips passes and spreads the keys over the histogram bins.
+  const float* sc = score + (size_t)b * n;
+  uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+  for (int i = tid; i < n; i += kTopkThreads) {
+    const uint32_t key = __float_as_uint(__ldcg(sc + i)) & 0x7FFFFFFFu;  // drops the sign of -0
+    s_keys[KI(i)] = key;
+    kmin = min(kmin, key); kmax = max(kmax, key);
+  }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) { s_warp[warp] = kmin; s_hist[warp] = kmax; }
+  __syncthreads();
+  kmin = s_warp[lane < kTopkWarps ? lane : 0];
+  kmax = s_hist[lane < kTopkWarps ? lane : 0];
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  __syncthreads();
+  for (int i = tid; i < n; i += kTopkThreads) s_keys[KI(i)] -= kmin;  // each thread rewrites its own keys
+  const uint32_t range = kmax - kmin;
+  const int npass = range ? (32 - __clz(range) + 7) / 8 : 0;
+
+  // Radix select, most significant byte first: after the passes s_prefix is the k-th largest key and
   // s_remaining how many keys equal to it belong to the kept set.
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    const uint32_t hi_mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+  for (int pass = 0; pass < npass; ++pass) {
+    const int shift = 8 * (npass - 1 - pass);
+    const uint32_t hi_mask = shift + 8 >= 32 ? 0u : (0xFFFFFFFFu << (shift + 8));
     if (tid < 256) s_hist[tid] = 0u;
     __syncthreads();
     const uint32_t prefix = s_prefix;
     for (int i = tid; i < n; i += kTopkThreads) {
-      uint32_t key = s_keys[i];
+      const uint32_t key = s_keys[KI(i)];
       if ((key & hi_mask) == prefix) atomicAdd(&s_hist[(key >> shift) & 255u], 1u);
     }
     __syncthreads();
@@ -158,35 +213,35 @@ __global__ void __launch_bounds__(kTopkThreads) topk_select_kernel(const float* 
     }
     __syncthreads();
   }
-  const uint32_t tau = s_prefix;
+  const uint32_t tau = s_prefix;  // relative to kmin
   const uint32_t need_eq = s_remaining;
 
   // Ordered compaction: thread t owns the contiguous tokens [t*per, (t+1)*per).
   const int per = (n + kTopkThreads - 1) / kTopkThreads;
   const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
   uint32_t eq = 0;
-  for (int i = i0; i < i1; ++i) eq += (s_keys[i] == tau);
+  for (int i = i0; i < i1; ++i) eq += (s_keys[KI(i)] == tau);
   uint32_t tot;
   uint32_t eq_before = block_exclusive_scan(eq, s_warp, &tot);
   uint32_t kept = 0, e = eq_before;
   for (int i = i0; i < i1; ++i) {
-    uint32_t key = s_keys[i];
+    uint32_t key = s_keys[KI(i)];
     if (key > tau) ++kept;
     else if (key == tau) { kept += (e < need_eq); ++e; }
   }
   uint32_t pos = block_exclusive_scan(kept, s_warp, &tot);
   e = eq_before;
-  const float tau_f = __uint_as_float(tau);
+  const float tau_f = __uint_as_float(tau + kmin);
   const float band = 1e-5f * tau_f;
   uint32_t near = 0;
   for (int i = i0; i < i1; ++i) {
-    uint32_t key = s_keys[i];
+    uint32_t key = s_keys[KI(i)];
     bool take = key > tau;
     if (key == tau) { take = (e < need_eq); ++e; }
     if (take) idx[(size_t)b * k + pos] = i;
     if (inv) inv[(size_t)b * n + i] = take ? (int32_t)pos : -1;
     pos += take;
-    near += (fabsf(__uint_as_float(key) - tau_f) <= band);
+    near += (fabsf(__uint_as_float(key + kmin) - tau_f) <= band);
   }
   if (near_tie) {
 #pragma unroll
@@ -196,7 +251,6 @@ __global__ void __launch_bounds__(kTopkThreads) topk_select_kernel(const float* 
     if (tid == 0) near_tie[b] = (int32_t)s_near;
   }
 }
-
 __global__ void inv_fill_kernel(int32_t* inv, size_t total) {
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < total) inv[i] = -1;
@@ -211,36 +265,68 @@ __global__ void inv_scatter_kernel(const int32_t* __restrict__ idx, int B, int k
 
 }  // namespace
 
+size_t select_ticket_bytes(int B) { return align_up((size_t)B * (kMaxGroups + 1) * sizeof(unsigned int), 256); }
+
+static void chunking(int n, int* nchunks, int* group, int* ngroups) {
+  *nchunks = (n + kColsumRows - 1) / kColsumRows;
+  *group = (*nchunks + kMaxGroups - 1) / kMaxGroups;
+  *ngroups = (*nchunks + *group - 1) / *group;
+}
+
 size_t select_workspace_bytes(int B, int n, int C) {
-  const size_t nchunks = (n + kColsumRows - 1) / kColsumRows;
-  size_t bytes = align_up((size_t)B * nchunks * C * sizeof(float), 256);  // partial column sums
-  bytes += align_up((size_t)B * C * sizeof(float), 256);                   // mean token
-  bytes += align_up((size_t)B * n * sizeof(float), 256);                   // scores
+  int nchunks, group, ngroups;
+  chunking(n, &nchunks, &group, &ngroups);
+  size_t bytes = select_ticket_bytes(B);
+  bytes += align_up((size_t)B * nchunks * C * sizeof(float), 256);  // chunk partials of the column sums
+  bytes += align_up((size_t)B * ngroups * C * sizeof(float), 256);  // group partials
+  bytes += align_up((size_t)B * n * sizeof(float), 256);            // scores
   return bytes;
 }
 
+SelectWs select_ws_carve(void* workspace, int B, int n, int C) {
+  SelectWs w;
+  chunking(n, &w.nchunks, &w.group, &w.ngroups);
+  char* p = static_cast<char*>(workspace);
+  w.tickets = reinterpret_cast<unsigned int*>(p);
+  p += select_ticket_bytes(B);
+  w.chunk_partial = reinterpret_cast<float*>(p);
+  p += align_up((size_t)B * w.nchunks * C * sizeof(float), 256);
+  w.group_partial = reinterpret_cast<float*>(p);
+  p += align_up((size_t)B * w.ngroups * C * sizeof(float), 256);
+  w.score = reinterpret_cast<float*>(p);
+  return w;
+}
+
+static int g_num_sms = 148;
+
 cudaError_t select_init() {
-  return cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkMaxTokens * 4);
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(score_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkMaxSmem);
 }
 
 cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* idx, int32_t* inv, float* score,
-                          int32_t* near_tie, void* workspace, cudaStream_t st) {
-  const int nchunks = (n + kColsumRows - 1) / kColsumRows;
+                          int32_t* near_tie, void* workspace, bool have_partials, cudaStream_t st) {
   const int C4 = C / 4;
-  char* ws = static_cast<char*>(workspace);
-  float* partial = reinterpret_cast<float*>(ws);
-  ws += align_up((size_t)B * nchunks * C * sizeof(float), 256);
-  float* mean = reinterpret_cast<float*>(ws);
-  ws += align_up((size_t)B * C * sizeof(float), 256);
-  float* sc = score ? score : reinterpret_cast<float*>(ws);
-  LaunchScope scope(KC_SELECT, 4, (double)B * n * C * 4.0 + 4.0 * B * n + 4.0 * B * ((double)k + n), st);
-  const int cs_threads = C4 >= 512 ? 512 : ((C4 + 31) / 32 * 32);
-  colsum_partial_kernel<<<dim3(nchunks, B), cs_threads, 0, st>>>(reinterpret_cast<const float4*>(x), n, C4, nchunks,
-                                                                 reinterpret_cast<float4*>(partial));
-  mean_finalize_kernel<<<dim3((C + 255) / 256, B), 256, 0, st>>>(partial, nchunks, C, n, mean);
-  score_rows_kernel<<<dim3((n + kScoreRowsPerCta - 1) / kScoreRowsPerCta, B), 256, C * sizeof(float), st>>>(
-      reinterpret_cast<const float4*>(x), reinterpret_cast<const float4*>(mean), n, C4, sc);
-  topk_select_kernel<<<B, kTopkThreads, (size_t)n * 4, st>>>(sc, n, k, idx, inv, near_tie);
+  const SelectWs w = select_ws_carve(workspace, B, n, C);
+  float* sc = score ? score : w.score;
+  LaunchScope scope(KC_SELECT, have_partials ? 1 : 2, (double)B * n * C * 4.0 + 4.0 * B * n + 4.0 * B * ((double)k + n), st);
+  if (!have_partials)
+    colsum_chunk_kernel<<<dim3(w.nchunks, B), 256, 0, st>>>(reinterpret_cast<const float4*>(x), n, C4, w.nchunks, w.group, w.ngroups,
+                                                            reinterpret_cast<float4*>(w.chunk_partial),
+                                                            reinterpret_cast<float4*>(w.group_partial), w.tickets);
+  const size_t keys_smem = ((size_t)n + n / 32 + 1) * 4;
+  const size_t smem = keys_smem > (size_t)C * 4 ? keys_smem : (size_t)C * 4;
+  // all CTAs resident at once: two per SM over the B images, never more than one warp per token row
+  int per_image = (2 * g_num_sms + B - 1) / B;
+  const int need = (n + kTopkWarps - 1) / kTopkWarps;
+  if (per_image > need) per_image = need;
+  if (per_image < 1) per_image = 1;
+  score_topk_kernel<<<dim3(per_image, B), kTopkThreads, smem, st>>>(
+      reinterpret_cast<const float4*>(x), reinterpret_cast<const float4*>(w.group_partial), w.ngroups, n, C4, k, sc,
+      w.tickets + (size_t)B * kMaxGroups, idx, inv, near_tie);
   return cudaGetLastError();
 }
 

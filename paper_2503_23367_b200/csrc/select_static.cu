@@ -55,7 +55,7 @@ fv_status fv_prune_select_static(const float* x_dev, int32_t B, int32_t h, int32
   if (!x_dev || !idx_out_dev || B <= 0 || h <= 0 || w <= 0 || C <= 0) return FV_ERR_INVALID_ARG;
   if (!(keep_ratio > 0.0) || keep_ratio > 1.0 || (C % 4) || (reinterpret_cast<uintptr_t>(x_dev) & 15u)) return FV_ERR_INVALID_ARG;
   const long n = (long)h * w;
-  if (n > fv::kTopkMaxTokens) return FV_ERR_UNSUPPORTED;
+  if (n > fv::kTopkMaxTokens || C > fv::kTopkMaxTokens) return FV_ERR_UNSUPPORTED;
   // The shape must fit the fixed scratch: this entry point never allocates, so it refuses instead.
   if (fv::select_workspace_bytes(B, (int)n, C) > kStaticScratchBytes) return FV_ERR_CAPACITY;
   if (fv::select_init() != cudaSuccess) return FV_ERR_CUDA;
@@ -63,10 +63,13 @@ fv_status fv_prune_select_static(const float* x_dev, int32_t B, int32_t h, int32
   if (scratch_address(&scratch) != cudaSuccess) return FV_ERR_CUDA;
   const int k = fv_k_for(keep_ratio, h, w);
   if (k_out_host) *k_out_host = k;
-  // Nothing in the scratch has to start at zero: every word the kernels read (partial sums, mean,
-  // scores) is written earlier in the same call, so the previous call's leftovers are harmless.
+  // Of the scratch only the arrival counters at its head have to start at zero; they are cleared here on
+  // every call (a memset node on the stream, no allocation).  Every other word the kernels read
+  // (partial sums, scores) is written earlier in the same call, so the previous call's leftovers are harmless.
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(scratch, 0, fv::select_ticket_bytes(B), st) != cudaSuccess) return FV_ERR_CUDA;
   cudaError_t e = fv::launch_select(x_dev, B, (int)n, C, k, idx_out_dev, inv_out_dev, score_out_dev, near_tie_dev, scratch,
-                                    static_cast<cudaStream_t>(stream));
+                                    false, st);
   return e == cudaSuccess ? FV_OK : FV_ERR_CUDA;
 }
 
