@@ -3,15 +3,19 @@
 // the attention map, so a fused kernel applies).  Within a scale step there is no mask: a query sees
 // every cached key of the earlier scales and all keys appended by its own step.
 //
-// One CTA = 128 queries of one head of one image.  Keys are consumed in tiles of 128:
-//   warp 0   : TMA producer (Q once; K tiles [128 keys x hd]; V^T tiles [hd x 128 keys]).
-//   warp 1   : one lane issues tcgen05.mma:  S = Q K^T into one of two TMEM score buffers, and
-//              O += P V with P read from shared memory; S of tile j+1 is issued before P V of tile j
-//              so the tensor core works while the softmax warps handle tile j.
-//   warps 2-5: online softmax, thread = query row: tcgen05.ld the 128 scores, running max / sum in
-//              fp32 (base-2 exponent), bf16 probabilities written to shared memory in the 128-byte
-//              swizzled K-major layout the MMA reads; the O accumulator in TMEM is rescaled in place
-//              when the running max moves; final O / l is written as bf16.
+// One CTA = 256 queries (two tiles of 128) of one head of one image; keys are consumed in tiles of 128.
+// The two query tiles take turns on the tensor core: while the softmax warps of one tile work on its
+// scores, the MMAs of the other tile run.
+//   warp 0   : TMA producer (both Q tiles once; K tiles [128 keys x hd]; V^T tiles [hd x 128 keys]).
+//   warp 1   : one lane issues tcgen05.mma.  Per key tile j and query tile t:  O_t += P_t V_j  with P_t
+//              read from TENSOR MEMORY (it overwrites the first 64 columns of S_t), then
+//              S_t = Q_t K_{j+1}^T.  MMAs of one thread execute in issue order, which is what makes
+//              the P_t / S_t aliasing safe.
+//   warps 2-5, 6-9: online softmax of tile 0 / tile 1, thread = query row.  Pass 1 reads the 128 scores
+//              from TMEM for the row maximum, pass 2 reads them again, exponentiates (base 2), sums,
+//              and writes bf16 probabilities back to TMEM.  The running maximum is only raised when
+//              it would grow by more than 2^8, so the O accumulator (TMEM) is rescaled in place only
+//              on the rare tiles where that happens; the final O / l is written as bf16.
 // V is read transposed ([channel, key], keys contiguous), which makes it a K-major B operand.
 // Every wait is bounded (status word + normal unwind on expiry).
 #include <cuda.h>
@@ -24,18 +28,18 @@ namespace fv {
 
 namespace {
 
-constexpr int QT = 128;  // queries per CTA
-constexpr int KT = 128;  // keys per tile
-constexpr int kAttnThreads = 192;
+constexpr int QT = 128;   // queries per tile (two tiles per CTA)
+constexpr int KT = 128;   // keys per tile
+constexpr int kAttnThreads = 320;
+constexpr float kRescaleThreshold = 8.f;  // log2 units
 
 template <int HD> struct AttnCfg {
-  static constexpr int kStages = (HD == 128) ? 2 : 3;
-  static constexpr int kQBytes = QT * HD * 2;
+  static constexpr int kStages = (HD == 128) ? 2 : 4;
+  static constexpr int kQBytes = QT * HD * 2;   // one query tile
   static constexpr int kKBytes = KT * HD * 2;
   static constexpr int kVBytes = HD * KT * 2;
-  static constexpr int kPBytes = QT * KT * 2;
-  static constexpr int kSmemBytes = kQBytes + kStages * (kKBytes + kVBytes) + kPBytes + 1024 + 256;
-  static constexpr int kTmemCols = 512;  // S0 [0,128) S1 [128,256) O [256, 256+HD)
+  static constexpr int kSmemBytes = 2 * kQBytes + kStages * (kKBytes + kVBytes) + 1024 + 256;
+  static constexpr int kTmemCols = 512;  // S0 [0,128) S1 [128,256) O0 [256,256+HD) O1 [384,384+HD)
 };
 
 struct AttnDev {
@@ -55,6 +59,56 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// Row maximum over one 128-key score tile held in TMEM (lanes = rows).  MASK: keys >= valid are ignored.
+template <bool MASK>
+__device__ __forceinline__ float tile_row_max(uint32_t s_addr, int valid) {
+  float mx = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < KT / 64; ++c) {
+    uint32_t a[32], b[32];
+    tmem_ld32(s_addr + c * 64, a);
+    tmem_ld32(s_addr + c * 64 + 32, b);
+    tmem_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      float va = __uint_as_float(a[i]), vb = __uint_as_float(b[i]);
+      if (MASK) {
+        if (c * 64 + i >= valid) va = -INFINITY;
+        if (c * 64 + 32 + i >= valid) vb = -INFINITY;
+      }
+      mx = fmaxf(mx, fmaxf(va, vb));
+    }
+  }
+  return mx;
+}
+
+// p = 2^(s * scale - m) for the 128 scores of a row; bf16 pairs written to TMEM columns [p_addr, +64);
+// returns the row sum of the UNROUNDED probabilities.
+template <bool MASK>
+__device__ __forceinline__ float tile_exp_store(uint32_t s_addr, uint32_t p_addr, float scale, float m, int valid) {
+  float rs = 0.f;
+#pragma unroll
+  for (int c = 0; c < KT / 32; ++c) {
+    uint32_t a[32];
+    tmem_ld32(s_addr + c * 32, a);
+    tmem_wait_ld();
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      float p0 = fast_exp2(fmaf(__uint_as_float(a[2 * i]), scale, -m));
+      float p1 = fast_exp2(fmaf(__uint_as_float(a[2 * i + 1]), scale, -m));
+      if (MASK) {
+        if (c * 32 + 2 * i >= valid) p0 = 0.f;
+        if (c * 32 + 2 * i + 1 >= valid) p1 = 0.f;
+      }
+      rs += p0 + p1;
+      pk[i] = pack_bf16x2(p0, p1);
+    }
+    tmem_st16(p_addr + c * 16, pk);
+  }
+  return rs;
+}
+
 template <int HD>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -63,32 +117,29 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   constexpr int NS = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* q_s = smem;
-  uint8_t* k_s = q_s + Cfg::kQBytes;
+  uint8_t* q_s = smem;                          // two query tiles
+  uint8_t* k_s = q_s + 2 * Cfg::kQBytes;
   uint8_t* v_s = k_s + NS * Cfg::kKBytes;
-  uint8_t* p_s = v_s + NS * Cfg::kVBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(p_s + Cfg::kPBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(v_s + NS * Cfg::kVBytes);
   uint64_t* q_full = bars;
   uint64_t* k_full = bars + 1;
   uint64_t* k_empty = k_full + NS;
   uint64_t* v_full = k_empty + NS;
   uint64_t* v_empty = v_full + NS;
-  uint64_t* s_full = v_empty + NS;   // [2]
-  uint64_t* s_free = s_full + 2;     // [2]
-  uint64_t* p_full = s_free + 2;
-  uint64_t* p_free = p_full + 1;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(p_free + 1);
+  uint64_t* s_full = v_empty + NS;   // [2] scores of query tile t are in TMEM
+  uint64_t* p_full = s_full + 2;     // [2] probabilities of query tile t are in TMEM (128 arrivals)
+  uint64_t* o_done = p_full + 2;     // [2] the latest P V of query tile t has completed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_done + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int q0 = blockIdx.x * QT, head = blockIdx.y, img = blockIdx.z;
+  const int q0 = blockIdx.x * (2 * QT), head = blockIdx.y, img = blockIdx.z;
   const int T = (p.kv_len + KT - 1) / KT;
+  const int ntiles = (p.rows - q0 > QT) ? 2 : 1;
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
     for (int s = 0; s < NS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_free[s], 128); }
-    mbar_init(p_full, 128);
-    mbar_init(p_free, 1);
+    for (int t = 0; t < 2; ++t) { mbar_init(&s_full[t], 1); mbar_init(&p_full[t], QT); mbar_init(&o_done[t], 1); }
     mbar_fence_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
   }
@@ -97,12 +148,13 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_o = tmem_base + 256;
 
   if (warp == 0) {
     if (lane == 0) {
-      mbar_expect_tx(q_full, Cfg::kQBytes);
-      for (int a = 0; a < HD / 64; ++a) tma_load_2d(q_s + a * (QT * 128), &tmQ, head * HD + a * 64, img * p.rows + q0, q_full);
+      mbar_expect_tx(q_full, ntiles * Cfg::kQBytes);
+      for (int t = 0; t < ntiles; ++t)
+        for (int a = 0; a < HD / 64; ++a)
+          tma_load_2d(q_s + t * Cfg::kQBytes + a * (QT * 128), &tmQ, head * HD + a * 64, img * p.rows + q0 + t * QT, q_full);
       for (int j = 0; j < T; ++j) {
         const int s = j % NS;
         const uint32_t ph = (j / NS) & 1;
@@ -120,132 +172,114 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (lane == 0) {
       constexpr uint32_t idesc_qk = umma_idesc_bf16(QT, KT);
       constexpr uint32_t idesc_pv = umma_idesc_bf16(QT, HD);
-      bool ok = mbar_wait(q_full, 0);
-      if (!ok) report(p.status, DEV_TIMEOUT_MMA);
-      const uint32_t q_addr = smem_u32(q_s), p_addr = smem_u32(p_s);
-      for (int j = 0; ok && j <= T; ++j) {
-        if (j < T) {
-          const int s = j % NS;
-          if (!mbar_wait(&k_full[s], (j / NS) & 1) || !mbar_wait(&s_free[j & 1], ((j >> 1) & 1) ^ 1)) {
-            report(p.status, DEV_TIMEOUT_MMA); ok = false; break;
-          }
-          tc_fence_after();
-          const uint32_t k_addr = smem_u32(k_s + s * Cfg::kKBytes);
-          const uint32_t d = tmem_base + (j & 1) * KT;
+      const uint32_t q_addr = smem_u32(q_s);
+      // S_t = Q_t K^T for the key tile in stage s
+      auto issue_qk = [&](int t, int s) {
+        const uint32_t k_addr = smem_u32(k_s + s * Cfg::kKBytes);
+        const uint32_t qa = q_addr + t * Cfg::kQBytes;
 #pragma unroll
-          for (int kk = 0; kk < HD / 16; ++kk) {
-            const uint32_t off = (kk >> 2) * (QT * 128) + (kk & 3) * 32;
-            umma_bf16(d, umma_desc_k_sw128(q_addr + off), umma_desc_k_sw128(k_addr + off), idesc_qk, kk != 0);
-          }
-          umma_commit(&k_empty[s]);
-          umma_commit(&s_full[j & 1]);
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * (QT * 128) + (kk & 3) * 32;
+          umma_bf16(tmem_base + t * KT, umma_desc_k_sw128(qa + off), umma_desc_k_sw128(k_addr + off), idesc_qk, kk != 0);
         }
-        if (j > 0) {
-          const int jj = j - 1, s = jj % NS;
-          if (!mbar_wait(&v_full[s], (jj / NS) & 1) || !mbar_wait(p_full, jj & 1)) {
-            report(p.status, DEV_TIMEOUT_MMA); ok = false; break;
-          }
+        umma_commit(&s_full[t]);
+      };
+      bool ok = mbar_wait(q_full, 0) && mbar_wait(&k_full[0], 0);
+      if (!ok) report(p.status, DEV_TIMEOUT_MMA);
+      if (ok) {
+        tc_fence_after();
+        for (int t = 0; t < ntiles; ++t) issue_qk(t, 0);
+        umma_commit(&k_empty[0]);
+      }
+      for (int j = 0; ok && j < T; ++j) {
+        const int s = j % NS, sn = (j + 1) % NS;
+        const bool more = j + 1 < T;
+        if (!mbar_wait(&v_full[s], (j / NS) & 1) || (more && !mbar_wait(&k_full[sn], ((j + 1) / NS) & 1))) {
+          report(p.status, DEV_TIMEOUT_MMA); ok = false; break;
+        }
+        const uint32_t v_addr = smem_u32(v_s + s * Cfg::kVBytes);
+        for (int t = 0; t < ntiles; ++t) {
+          if (!mbar_wait(&p_full[t], j & 1)) { report(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
           tc_fence_after();
-          const uint32_t v_addr = smem_u32(v_s + s * Cfg::kVBytes);
+          const uint32_t p_tmem = tmem_base + t * KT;              // P_t over the first 64 columns of S_t
+          const uint32_t o_tmem = tmem_base + 256 + t * 128;
 #pragma unroll
           for (int kk = 0; kk < KT / 16; ++kk) {
-            const uint32_t a_off = (kk >> 2) * (QT * 128) + (kk & 3) * 32;
             const uint32_t b_off = (kk >> 2) * (HD * 128) + (kk & 3) * 32;
-            umma_bf16(tmem_o, umma_desc_k_sw128(p_addr + a_off), umma_desc_k_sw128(v_addr + b_off), idesc_pv, (jj | kk) != 0);
+            umma_bf16_ts(o_tmem, p_tmem + kk * 8, umma_desc_k_sw128(v_addr + b_off), idesc_pv, (j | kk) != 0);
           }
-          umma_commit(&v_empty[s]);
-          umma_commit(p_free);
+          umma_commit(&o_done[t]);
+          if (more) issue_qk(t, sn);
         }
+        if (!ok) break;
+        umma_commit(&v_empty[s]);
+        if (more) umma_commit(&k_empty[sn]);
       }
     }
   } else {
-    // ---- softmax + output: thread = one query row ----
-    const int quarter = warp & 3;
+    // ---- softmax + output: thread = one query row of tile t ----
+    const int t = (warp - 2) >> 2;
+    const int quarter = warp & 3;                 // the TMEM lanes this warp may touch
     const int r = quarter * 32 + lane;
     const uint32_t lane_off = uint32_t(quarter * 32) << 16;
-    float m_run = -INFINITY, l_run = 0.f;
-    bool ok = true;
-    for (int j = 0; j < T; ++j) {
-      if (!mbar_wait(&s_full[j & 1], (j >> 1) & 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); ok = false; break; }
+    const uint32_t s_addr = tmem_base + lane_off + t * KT;
+    const uint32_t o_addr = tmem_base + lane_off + 256 + t * 128;
+    if (t < ntiles) {
+      float m_run = -INFINITY, l_run = 0.f;
+      bool ok = true;
+      for (int j = 0; j < T; ++j) {
+        if (!mbar_wait(&s_full[t], j & 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); ok = false; break; }
+        tc_fence_after();
+        const int valid = p.kv_len - j * KT;  // >= 1
+        const bool tail = valid < KT;
+        const float mx = (tail ? tile_row_max<true>(s_addr, valid) : tile_row_max<false>(s_addr, valid)) * p.scale_log2;
+        // Raise the running maximum only when it would grow by more than the threshold: probabilities
+        // may then exceed 1 (by at most 2^threshold), which fp32 sums and bf16 P hold without loss.
+        float alpha = 1.f;
+        if (mx > m_run + kRescaleThreshold) {
+          alpha = fast_exp2(m_run - mx);  // 0 on the first tile (m_run = -inf)
+          m_run = mx;
+        }
+        // S_t of tile j was issued after P V of tile j-1, so O_t is at rest here.
+        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+          for (int c = 0; c < HD / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(o_addr + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+            tmem_st32(o_addr + c * 32, o);
+          }
+        }
+        const float rs = tail ? tile_exp_store<true>(s_addr, s_addr, p.scale_log2, m_run, valid)
+                              : tile_exp_store<false>(s_addr, s_addr, p.scale_log2, m_run, valid);
+        l_run = fmaf(l_run, alpha, rs);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&p_full[t]);
+      }
+      if (ok && !mbar_wait(&o_done[t], (T - 1) & 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); ok = false; }
       tc_fence_after();
-      float sc[KT];
-#pragma unroll
-      for (int c = 0; c < KT / 32; ++c) {
-        uint32_t t[32];
-        tmem_ld32(tmem_base + lane_off + (j & 1) * KT + c * 32, t);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) sc[c * 32 + i] = __uint_as_float(t[i]);
-      }
-      tmem_wait_ld();
-      tc_fence_before();
-      mbar_arrive(&s_free[j & 1]);
-      const int valid = p.kv_len - j * KT;  // >= 1
-      float mx = -INFINITY;
-#pragma unroll
-      for (int i = 0; i < KT; ++i) {
-        if (i >= valid) sc[i] = -INFINITY;
-        mx = fmaxf(mx, sc[i]);
-      }
-      const float m_new = fmaxf(m_run, mx * p.scale_log2);
-      const float alpha = fast_exp2(m_run - m_new);  // 0 on the first tile (m_run = -inf)
-      float rs = 0.f;
-#pragma unroll
-      for (int i = 0; i < KT; ++i) {
-        sc[i] = fast_exp2(fmaf(sc[i], p.scale_log2, -m_new));
-        rs += sc[i];
-      }
-      l_run = fmaf(l_run, alpha, rs);
-      m_run = m_new;
-      // P buffer free and O stable once P V of the previous tile has completed
-      if (!mbar_wait(p_free, (j & 1) ^ 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); ok = false; break; }
-      tc_fence_after();
-      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+      if (ok) {
+        const float inv_l = 1.f / l_run;
+        const int row = q0 + t * QT + r;
+        __nv_bfloat16* dst = p.out + ((size_t)img * p.rows + row) * p.C + head * HD;
 #pragma unroll
         for (int c = 0; c < HD / 32; ++c) {
-          uint32_t t[32];
-          tmem_ld32(tmem_o + lane_off + c * 32, t);
+          uint32_t o[32];
+          tmem_ld32(o_addr + c * 32, o);
           tmem_wait_ld();
+          if (row < p.rows) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) t[i] = __float_as_uint(__uint_as_float(t[i]) * alpha);
-          tmem_st32(tmem_o + lane_off + c * 32, t);
-        }
-        tmem_wait_st();
-      }
-      // bf16 probabilities -> shared memory, K-major rows of 128 bytes with the 128-byte swizzle
-#pragma unroll
-      for (int c8 = 0; c8 < KT / 8; ++c8) {
-        uint4 o;
-        o.x = pack_bf16x2(sc[8 * c8 + 0], sc[8 * c8 + 1]); o.y = pack_bf16x2(sc[8 * c8 + 2], sc[8 * c8 + 3]);
-        o.z = pack_bf16x2(sc[8 * c8 + 4], sc[8 * c8 + 5]); o.w = pack_bf16x2(sc[8 * c8 + 6], sc[8 * c8 + 7]);
-        const int atom = c8 >> 3, chunk = c8 & 7;
-        *reinterpret_cast<uint4*>(p_s + atom * (QT * 128) + r * 128 + ((chunk ^ (r & 7)) << 4)) = o;
-      }
-      fence_async_smem();
-      tc_fence_before();
-      mbar_arrive(p_full);
-    }
-    if (ok) {
-      if (!mbar_wait(p_free, (T - 1) & 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); ok = false; }
-    }
-    tc_fence_after();
-    if (ok) {
-      const float inv_l = 1.f / l_run;
-      const int row = q0 + r;
-      __nv_bfloat16* dst = p.out + ((size_t)img * p.rows + row) * p.C + head * HD;
-#pragma unroll
-      for (int c = 0; c < HD / 32; ++c) {
-        uint32_t t[32];
-        tmem_ld32(tmem_o + lane_off + c * 32, t);
-        tmem_wait_ld();
-        if (row < p.rows) {
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint4 o;
-            o.x = pack_bf16x2(__uint_as_float(t[8 * g + 0]) * inv_l, __uint_as_float(t[8 * g + 1]) * inv_l);
-            o.y = pack_bf16x2(__uint_as_float(t[8 * g + 2]) * inv_l, __uint_as_float(t[8 * g + 3]) * inv_l);
-            o.z = pack_bf16x2(__uint_as_float(t[8 * g + 4]) * inv_l, __uint_as_float(t[8 * g + 5]) * inv_l);
-            o.w = pack_bf16x2(__uint_as_float(t[8 * g + 6]) * inv_l, __uint_as_float(t[8 * g + 7]) * inv_l);
-            reinterpret_cast<uint4*>(dst + c * 32)[g] = o;
+            for (int g = 0; g < 4; ++g) {
+              uint4 v;
+              v.x = pack_bf16x2(__uint_as_float(o[8 * g + 0]) * inv_l, __uint_as_float(o[8 * g + 1]) * inv_l);
+              v.y = pack_bf16x2(__uint_as_float(o[8 * g + 2]) * inv_l, __uint_as_float(o[8 * g + 3]) * inv_l);
+              v.z = pack_bf16x2(__uint_as_float(o[8 * g + 4]) * inv_l, __uint_as_float(o[8 * g + 5]) * inv_l);
+              v.w = pack_bf16x2(__uint_as_float(o[8 * g + 6]) * inv_l, __uint_as_float(o[8 * g + 7]) * inv_l);
+              reinterpret_cast<uint4*>(dst + c * 32)[g] = v;
+            }
           }
         }
       }
@@ -273,7 +307,7 @@ template <int HD> fv_status launch_hd(const AttnArgs& a, cudaStream_t st) {
   p.rows = a.rows; p.C = a.C; p.kv_len = a.kv_len; p.kv_capacity = a.kv_capacity;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   p.status = a.status;
-  dim3 grid((a.rows + QT - 1) / QT, a.H, a.B);
+  dim3 grid((a.rows + 2 * QT - 1) / (2 * QT), a.H, a.B);
   LaunchScope scope(KC_ATTENTION, 1, 4.0 * a.B * (double)a.rows * a.kv_len * a.C, st);
   attention_kernel<HD><<<grid, kAttnThreads, AttnCfg<HD>::kSmemBytes, st>>>(tmQ, tmK, tmV, p);
   return cudaGetLastError() == cudaSuccess ? FV_OK : FV_ERR_CUDA;
