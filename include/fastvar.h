@@ -215,11 +215,16 @@ fv_status fv_restore_residual(float *x_dev, const void *y_dev, const void *cache
  *   epilogue 2: fp32 residual: out[m,n] += gamma[m / rows_per_image, n] * (acc + bias)  (out fp32;
  *               gamma NULL = 1; if aux_dev != NULL the bf16 value of acc+bias is also stored there).
  *   K % 8 == 0, N % 8 == 0, all pointers 16-byte aligned.  bias_dev may be NULL.
- *   status_dev: int32 device word that receives a non-zero code if a bounded wait expires (or NULL). */
+ *   status_dev: int32 device word that receives a non-zero code if a bounded wait expires (or NULL).
+ *   splitk_ws_dev: NULL, or scratch of fv_gemm_splitk_workspace_bytes() bytes whose first 4096 bytes are
+ *               zero (the kernel leaves them zero): shapes with too few output tiles to occupy the GPU
+ *               (few rows against a large weight matrix) are then split along K, the slices' fp32
+ *               partial sums added in slice order.  CAPACITY if splitk_ws_bytes is too small. */
+size_t fv_gemm_splitk_workspace_bytes(void);
 fv_status fv_gemm_bf16(const void *a_dev, const void *w_dev, const void *bias_dev, int32_t M,
                        int32_t N, int32_t K, int32_t epilogue, void *out_dev, void *aux_dev,
                        const float *gamma_dev, int32_t mod_stride, int32_t rows_per_image,
-                       int32_t *status_dev, void *stream);
+                       int32_t *status_dev, void *splitk_ws_dev, size_t splitk_ws_bytes, void *stream);
 
 /* Flash-style attention over a KV cache (Sec. 3.1 KV cache; Sec. 3.3: pivotal queries attend to the
  * cached keys of all earlier scales plus the current pivotal keys; no mask inside a step).

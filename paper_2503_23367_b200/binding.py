@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "FV_OK", 1: "FV_ERR_INVALID_ARG", 2: "FV_ERR_BAD_STATE", 3: "
 EXPORTS = ["fv_status_string", "fv_k_for", "fv_prune_select_workspace_bytes", "fv_prune_select", "fv_restore",
            "fv_workspace_bytes", "fv_kv_bytes", "fv_cache_bytes", "fv_create", "fv_destroy", "fv_reset",
            "fv_get_state", "fv_set_state", "fv_kv_pointers", "fv_cache_pointer", "fv_prepare_text",
-           "fv_device_status", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_gemm_bf16", "fv_attention",
+           "fv_device_status", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_gemm_bf16", "fv_gemm_splitk_workspace_bytes", "fv_attention",
            "fv_kernel_launches", "fv_profile_enable", "fv_profile_read",
            "fv_prune_select_static", "fv_prune_select_static_capacity"]
 
@@ -81,7 +81,8 @@ def lib() -> C.CDLL:
         L.fv_restore_residual.restype = C.c_int
         L.fv_restore_residual.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp]
         L.fv_gemm_bf16.restype = C.c_int
-        L.fv_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp]
+        L.fv_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, sz, vp]
+        L.fv_gemm_splitk_workspace_bytes.restype = sz; L.fv_gemm_splitk_workspace_bytes.argtypes = []
         L.fv_attention.restype = C.c_int
         L.fv_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp]
         L.fv_prune_select_static_capacity.restype = sz; L.fv_prune_select_static_capacity.argtypes = []
@@ -200,7 +201,8 @@ def fv_restore_residual(x: torch.Tensor, y: torch.Tensor, cache: torch.Tensor, i
 def fv_gemm_bf16(a: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor], epilogue: int = 0,
                  out: Optional[torch.Tensor] = None, aux: Optional[torch.Tensor] = None,
                  gamma: Optional[torch.Tensor] = None, mod_stride: int = 0, rows_per_image: int = 0,
-                 status: Optional[torch.Tensor] = None) -> torch.Tensor:
+                 status: Optional[torch.Tensor] = None, splitk_ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """splitk_ws: uint8 scratch of fv_gemm_splitk_workspace_bytes() bytes, first 4096 zero, or None (no K split)."""
     M, K = a.shape
     N = w.shape[0]
     assert w.shape[1] == K and a.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
@@ -208,7 +210,8 @@ def fv_gemm_bf16(a: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor],
         assert epilogue in (0, 1)
         out = torch.empty((M, N), dtype=torch.bfloat16, device=a.device)
     _check(lib().fv_gemm_bf16(_ptr(a), _ptr(w), _ptr(bias), M, N, K, epilogue, _ptr(out), _ptr(aux), _ptr(gamma),
-                              mod_stride, rows_per_image, _ptr(status), _stream()), "fv_gemm_bf16")
+                              mod_stride, rows_per_image, _ptr(status), _ptr(splitk_ws),
+                              0 if splitk_ws is None else splitk_ws.numel(), _stream()), "fv_gemm_bf16")
     return out
 
 

@@ -30,6 +30,7 @@ struct fv_ctx {
   char *a_buf = nullptr, *q_buf = nullptr, *o_buf = nullptr, *y_buf = nullptr, *h_buf = nullptr;
   int32_t *idx = nullptr, *inv = nullptr;
   void* sel_ws = nullptr;
+  void* splitk_ws = nullptr;
   size_t kv_block_bytes = 0, k_bytes = 0, text_k_bytes = 0, text_block_bytes = 0, cache_sub_bytes = 0;
 };
 
@@ -50,7 +51,7 @@ cudaError_t ensure_init() {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 struct Layout {
-  size_t status, a, q, o, y, hbuf, idx, inv, sel, total;
+  size_t status, a, q, o, y, hbuf, idx, inv, sel, splitk, total;
 };
 
 int max_tokens(const fv_config* c) {
@@ -83,6 +84,7 @@ Layout workspace_layout(const fv_config* c) {
   l.idx = take(M * 4);
   l.inv = take(M * 4);
   l.sel = take(select_workspace_bytes(c->B_max, max_tokens(c), c->C));
+  l.splitk = take(gemm_splitk_ws_bytes());
   l.total = off;
   return l;
 }
@@ -170,14 +172,16 @@ fv_status fv_restore_residual(float* x_dev, const void* y_dev, const void* cache
 
 fv_status fv_gemm_bf16(const void* a_dev, const void* w_dev, const void* bias_dev, int32_t M, int32_t N, int32_t K,
                        int32_t epilogue, void* out_dev, void* aux_dev, const float* gamma_dev, int32_t mod_stride,
-                       int32_t rows_per_image, int32_t* status_dev, void* stream) {
+                       int32_t rows_per_image, int32_t* status_dev, void* splitk_ws_dev, size_t splitk_ws_bytes, void* stream) {
   if (!a_dev || !w_dev || !out_dev || epilogue < 0 || epilogue > 2) return FV_ERR_INVALID_ARG;
+  if (splitk_ws_dev && (splitk_ws_bytes < gemm_splitk_ws_bytes() || !aligned16(splitk_ws_dev))) return FV_ERR_CAPACITY;
   if (!aligned16(a_dev) || !aligned16(w_dev) || !aligned16(out_dev) || (bias_dev && !aligned16(bias_dev))) return FV_ERR_INVALID_ARG;
   if (ensure_init() != cudaSuccess) return FV_ERR_CUDA;
   GemmArgs g{};
   g.a = a_dev; g.w = w_dev; g.bias = bias_dev; g.M = M; g.N = N; g.K = K; g.epilogue = epilogue; g.out = out_dev;
   g.aux = aux_dev; g.gamma = gamma_dev; g.mod_stride = mod_stride; g.rows_per_image = rows_per_image > 0 ? rows_per_image : M;
   g.status = status_dev;
+  g.splitk_ws = splitk_ws_dev;
   return launch_gemm(g, static_cast<cudaStream_t>(stream));
 }
 
@@ -192,6 +196,8 @@ fv_status fv_attention(const void* q_dev, const void* k_dev, const void* vt_dev,
 }
 
 // ------------------------------------------------------------------------------------------------ context
+
+size_t fv_gemm_splitk_workspace_bytes(void) { return gemm_splitk_ws_bytes(); }
 
 size_t fv_workspace_bytes(const fv_config* cfg) { return config_ok(cfg) ? workspace_layout(cfg).total : 0; }
 
@@ -263,9 +269,11 @@ fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, v
   c->idx = reinterpret_cast<int32_t*>(c->ws + lay.idx);
   c->inv = reinterpret_cast<int32_t*>(c->ws + lay.inv);
   c->sel_ws = c->ws + lay.sel;
+  c->splitk_ws = c->ws + lay.splitk;
   // Never-written KV rows must read as zeros (they meet zero probabilities in P*V).
   if (cudaMemset(kv_dev, 0, fv_kv_bytes(cfg)) != cudaSuccess || cudaMemset(c->status, 0, 256) != cudaSuccess ||
       cudaMemset(c->sel_ws, 0, select_ticket_bytes(cfg->B_max)) != cudaSuccess ||
+      cudaMemset(c->splitk_ws, 0, gemm_splitk_ticket_bytes()) != cudaSuccess ||
       cudaDeviceSynchronize() != cudaSuccess) {
     delete c;
     return FV_ERR_CUDA;
@@ -322,7 +330,7 @@ fv_status fv_prepare_text(fv_ctx* ctx, int32_t B, void* stream) {
     g.a = ctx->text; g.w = ctx->w_kv_x[l]; g.bias = nullptr; g.M = B * c.cross_len; g.N = 2 * c.C; g.K = c.C;
     g.epilogue = EPI_QKV_SPLIT; g.out = nullptr; g.q_cols = 0; g.C = c.C; g.rows_per_image = c.cross_len;
     g.k_cache = text_k(ctx, l); g.vt_cache = text_k(ctx, l) + ctx->text_k_bytes; g.kv_capacity = c.cross_len; g.kv_offset = 0;
-    g.status = ctx->status;
+    g.status = ctx->status; g.splitk_ws = ctx->splitk_ws;
     fv_status s = launch_gemm(g, static_cast<cudaStream_t>(stream));
     if (s != FV_OK) return s;
   }
@@ -410,7 +418,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
       if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
       // ---- branch on the compact rows
       GemmArgs g{};
-      g.status = ctx->status; g.rows_per_image = k; g.mod_stride = mod_stride;
+      g.status = ctx->status; g.rows_per_image = k; g.mod_stride = mod_stride; g.splitk_ws = ctx->splitk_ws;
       const void* last_in = nullptr; const void* last_w = nullptr; const void* last_b = nullptr; int last_K = C;
       if (kind == 0) {
         g.a = ctx->a_buf; g.w = ctx->w_qkv[l]; g.bias = ctx->b_qkv[l]; g.M = M; g.N = 3 * C; g.K = C;
@@ -443,7 +451,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
       }
       // ---- last projection, then Cached Token Restoration + gate + residual
       GemmArgs o{};
-      o.status = ctx->status; o.rows_per_image = k; o.mod_stride = mod_stride;
+      o.status = ctx->status; o.rows_per_image = k; o.mod_stride = mod_stride; o.splitk_ws = ctx->splitk_ws;
       o.a = last_in; o.w = last_w; o.bias = last_b; o.M = M; o.N = C; o.K = last_K;
       if (pruned) {
         o.epilogue = EPI_BF16; o.out = ctx->y_buf;

@@ -13,6 +13,10 @@
 //              handed back as soon as it is in registers, so the epilogue of tile i runs under the
 //              MMAs of tile i+1.
 // BN (128 / 192 / 256) is picked per shape on the host to minimise rounds x tile width on the SM count.
+// Shapes with too few tiles to occupy the GPU (the small scale steps, where the GEMM is a stream of
+// weights) are split along K: work item = (tile, K slice), every slice leaves its fp32 partial rows in
+// a scratch buffer, and the last slice of a tile to arrive adds them in slice order and runs the
+// epilogue, so the result does not depend on arrival order.
 // Every wait is bounded; on expiry a code is written to the status word and the CTA unwinds normally.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -53,6 +57,9 @@ struct GemmDev {
   __nv_bfloat16* vt_cache;
   int kv_capacity, kv_offset;
   int32_t* status;
+  int splits, kb_per_split;   // K slices per tile (1 = no split) and 64-wide k-blocks per slice
+  float* sk_partial;          // [tile][slice][128][BN] fp32 partial accumulators
+  unsigned int* sk_tickets;   // [tile] arrival counters, zero between launches
 };
 
 __device__ __forceinline__ float gelu_tanh_fast(float v) {
@@ -157,7 +164,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmDev& p, const uint32_t 
   }
 }
 
-template <int BN>
+template <int BN, bool SPLIT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
   using Cfg = GemmCfg<BN>;
@@ -169,11 +176,13 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   uint64_t* acc_full = empty_bar + STAGES;   // [2]
   uint64_t* acc_empty = acc_full + 2;        // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* sk_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_m = (p.M + BM - 1) / BM;
   const int tiles_n = (p.N + BN - 1) / BN;
-  const int total_tiles = tiles_m * tiles_n;
+  const int splits = SPLIT ? p.splits : 1;
+  const int total_tiles = tiles_m * tiles_n * splits;   // work items: (tile, K slice), slice fastest
   const int num_kb = (p.K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
@@ -193,9 +202,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      for (int item = blockIdx.x; ok && item < total_tiles; item += gridDim.x) {
+        const int tile = item / splits, slice = item - tile * splits;
         const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        const int kb0 = slice * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           if (!mbar_wait(&empty_bar[s], ph ^ 1)) { report(p.status, DEV_TIMEOUT_TMA); ok = false; break; }
@@ -211,12 +222,14 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
       uint32_t it = 0, lt = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++lt) {
+      for (int item = blockIdx.x; ok && item < total_tiles; item += gridDim.x, ++lt) {
         const uint32_t buf = lt & 1;
         if (!mbar_wait(&acc_empty[buf], ((lt >> 1) & 1) ^ 1)) { report(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
         tc_fence_after();
         const uint32_t d = tmem_base + buf * Cfg::kAccStride;
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        const int slice = item % splits;
+        const int kb0 = slice * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           if (!mbar_wait(&full_bar[s], ph)) { report(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
@@ -226,7 +239,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           const uint64_t bdesc = umma_desc_k_sw128(a_addr + kATileBytes);
 #pragma unroll
           for (int kk = 0; kk < BK / 16; ++kk)
-            umma_bf16(d, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0);
+            umma_bf16(d, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb > kb0) || kk != 0);
           umma_commit(&empty_bar[s]);
         }
         if (ok) umma_commit(&acc_full[buf]);
@@ -237,8 +250,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int quarter = warp & 3;
     const uint32_t lane_off = uint32_t(quarter * 32) << 16;
     uint32_t lt = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
+    for (int item = blockIdx.x; item < total_tiles; item += gridDim.x, ++lt) {
       const uint32_t buf = lt & 1;
+      const int tile = item / splits, slice = item - tile * splits;
       const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
       const int row = m0 + quarter * 32 + lane;
       const bool row_ok = row < p.M;
@@ -247,20 +261,73 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int img = row_ok ? row / p.rows_per_image : 0;
       const int jrow = row_ok ? row - img * p.rows_per_image : 0;
       const uint32_t t0 = tmem_base + lane_off + buf * Cfg::kAccStride;
+      if (!SPLIT) {
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 64) {
-        // two chunks in flight: the second load overlaps the first chunk's stores
-        uint32_t r0[32], r1[32];
-        tmem_ld32(t0 + c0, r0);
-        tmem_ld32(t0 + c0 + 32, r1);
-        tmem_wait_ld();
-        if (c0 + 64 >= BN) {  // accumulator fully in registers: hand the buffer back to the MMA warp
-          tc_fence_before();
-          mbar_arrive(&acc_empty[buf]);
+        for (int c0 = 0; c0 < BN; c0 += 64) {
+          // two chunks in flight: the second load overlaps the first chunk's stores
+          uint32_t r0[32], r1[32];
+          tmem_ld32(t0 + c0, r0);
+          tmem_ld32(t0 + c0 + 32, r1);
+          tmem_wait_ld();
+          if (c0 + 64 >= BN) {  // accumulator fully in registers: hand the buffer back to the MMA warp
+            tc_fence_before();
+            mbar_arrive(&acc_empty[buf]);
+          }
+          const int col = n0 + c0;
+          if (row_ok && col < p.N) epilogue_chunk(p, r0, row, img, jrow, col);
+          if (row_ok && col + 32 < p.N) epilogue_chunk(p, r1, row, img, jrow, col + 32);
         }
-        const int col = n0 + c0;
-        if (row_ok && col < p.N) epilogue_chunk(p, r0, row, img, jrow, col);
-        if (row_ok && col + 32 < p.N) epilogue_chunk(p, r1, row, img, jrow, col + 32);
+      } else {
+        // ---- K-split: park this slice's partial rows, then the last slice to arrive finishes the tile
+        float* mine = p.sk_partial + ((size_t)item * BM + (quarter * 32 + lane)) * BN;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t r0[32];
+          tmem_ld32(t0 + c0, r0);
+          tmem_wait_ld();
+          if (row_ok && n0 + c0 < p.N) {
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+              __stcg(reinterpret_cast<uint4*>(mine + c0) + g, make_uint4(r0[4 * g], r0[4 * g + 1], r0[4 * g + 2], r0[4 * g + 3]));
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(&acc_empty[buf]);
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (threadIdx.x == 64) {
+          const unsigned int prev = atomicAdd(p.sk_tickets + tile, 1u);
+          const int last = (prev == (unsigned int)(p.splits - 1));
+          if (last) p.sk_tickets[tile] = 0u;
+          *sk_flag = last;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const int last = *sk_flag;
+        asm volatile("bar.sync 1, 128;" ::: "memory");  // flag consumed before the next item may rewrite it
+        if (last) {
+          __threadfence();
+          const float* base = p.sk_partial + ((size_t)tile * p.splits * BM + (quarter * 32 + lane)) * BN;
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            const int col = n0 + c0;
+            if (!(row_ok && col < p.N)) continue;
+            float acc[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+            for (int sl = 0; sl < p.splits; ++sl) {
+              const float4* src = reinterpret_cast<const float4*>(base + (size_t)sl * BM * BN + c0);
+#pragma unroll
+              for (int g = 0; g < 8; ++g) {
+                const float4 v = __ldcg(src + g);
+                acc[4 * g] += v.x; acc[4 * g + 1] += v.y; acc[4 * g + 2] += v.z; acc[4 * g + 3] += v.w;
+              }
+            }
+            uint32_t r0[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r0[i] = __float_as_uint(acc[i]);
+            epilogue_chunk(p, r0, row, img, jrow, col);
+          }
+        }
       }
     }
   }
@@ -287,8 +354,8 @@ void load_encode() {
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
 }
 
-template <int BN> cudaError_t set_attr() {
-  return cudaFuncSetAttribute(gemm_bf16_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<BN>::kSmemBytes);
+template <int BN, bool SPLIT> cudaError_t set_attr() {
+  return cudaFuncSetAttribute(gemm_bf16_kernel<BN, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<BN>::kSmemBytes);
 }
 
 }  // namespace
@@ -307,9 +374,10 @@ bool make_tmap_bf16_2d(void* tmap_out, const void* base, uint64_t rows, uint64_t
 }
 
 cudaError_t gemm_init() {
-  cudaError_t e = set_attr<128>();
-  if (e == cudaSuccess) e = set_attr<192>();
-  if (e == cudaSuccess) e = set_attr<256>();
+  cudaError_t e = set_attr<128, false>();
+  if (e == cudaSuccess) e = set_attr<128, true>();
+  if (e == cudaSuccess) e = set_attr<192, false>();
+  if (e == cudaSuccess) e = set_attr<256, false>();
   if (e != cudaSuccess) return e;
   int dev = 0;
   e = cudaGetDevice(&dev);
@@ -332,14 +400,37 @@ static int pick_bn(int tiles_m, int N, int sms) {
   return best;
 }
 
+// K-split scratch: room for two work items per SM of the widest tile, after 4 KB of arrival counters.
+constexpr size_t kSplitTicketBytes = 4096;
+constexpr int kSplitMaxItems = 2 * 148;
+size_t gemm_splitk_ticket_bytes() { return kSplitTicketBytes; }
+size_t gemm_splitk_ws_bytes() { return kSplitTicketBytes + (size_t)kSplitMaxItems * BM * 128 * sizeof(float); }
+
+// How many K slices for a shape that leaves SMs idle.  A CTA pulls its operands at roughly 100 GB/s and
+// pays a few microseconds of fixed cost, so slicing only pays for long K (>= 64 k-blocks), and a slice
+// keeps at least 16 k-blocks.  The last arriver re-reads slices x rows x 512 bytes, which grows with M.
+static int pick_splits(long tiles, int num_kb, int sms) {
+  if (tiles * 2 > sms || num_kb < 64) return 1;
+  int s = (int)(sms / tiles);
+  if (s > num_kb / 16) s = num_kb / 16;
+  if (s < 2) return 1;
+  const int per = (num_kb + s - 1) / s;
+  return (num_kb + per - 1) / per;  // no empty slice
+}
+
 template <int BN>
 static cudaError_t launch_bn(const GemmArgs& g, const GemmDev& p, int tiles_m, cudaStream_t st) {
   alignas(64) CUtensorMap tmA, tmB;
   if (!make_tmap_bf16_2d(&tmA, g.a, g.M, g.K, BM)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16_2d(&tmB, g.w, g.N, g.K, BN)) return cudaErrorInvalidValue;
-  const long tiles = (long)tiles_m * ((g.N + BN - 1) / BN);
+  const long tiles = (long)tiles_m * ((g.N + BN - 1) / BN) * p.splits;
   const int grid = (int)(tiles < g_num_sms ? tiles : g_num_sms);
-  gemm_bf16_kernel<BN><<<grid, kGemmThreads, GemmCfg<BN>::kSmemBytes, st>>>(tmA, tmB, p);
+  if (p.splits > 1) {
+    if constexpr (BN == 128) gemm_bf16_kernel<128, true><<<grid, kGemmThreads, GemmCfg<128>::kSmemBytes, st>>>(tmA, tmB, p);
+    else return cudaErrorInvalidValue;
+  } else {
+    gemm_bf16_kernel<BN, false><<<grid, kGemmThreads, GemmCfg<BN>::kSmemBytes, st>>>(tmA, tmB, p);
+  }
   return cudaGetLastError();
 }
 
@@ -348,8 +439,21 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   if (g.rows_per_image <= 0) return FV_ERR_INVALID_ARG;
   if (g.epilogue == EPI_QKV_SPLIT && (g.C % 128 || g.q_cols % 128)) return FV_ERR_UNSUPPORTED;
   const int tiles_m = (g.M + BM - 1) / BM;
-  const int bn = pick_bn(tiles_m, g.N, g_num_sms);
+  int bn = pick_bn(tiles_m, g.N, g_num_sms);
   GemmDev p;
+  p.splits = 1; p.kb_per_split = (g.K + BK - 1) / BK; p.sk_partial = nullptr; p.sk_tickets = nullptr;
+  if (g.splitk_ws) {
+    const int num_kb = (g.K + BK - 1) / BK;
+    const long tiles128 = (long)tiles_m * ((g.N + 127) / 128);
+    const int sp = pick_splits(tiles128, num_kb, g_num_sms);
+    if (sp > 1 && tiles128 * sp <= kSplitMaxItems && tiles128 * sizeof(unsigned int) <= kSplitTicketBytes) {
+      bn = 128;
+      p.splits = sp;
+      p.kb_per_split = (num_kb + sp - 1) / sp;
+      p.sk_tickets = static_cast<unsigned int*>(g.splitk_ws);
+      p.sk_partial = reinterpret_cast<float*>(static_cast<char*>(g.splitk_ws) + kSplitTicketBytes);
+    }
+  }
   p.bias = static_cast<const __nv_bfloat16*>(g.bias);
   p.M = g.M; p.N = g.N; p.K = g.K; p.epilogue = g.epilogue; p.out = g.out; p.aux = g.aux; p.gamma = g.gamma;
   p.mod_stride = g.mod_stride; p.rows_per_image = g.rows_per_image; p.q_cols = g.q_cols; p.C = g.C;

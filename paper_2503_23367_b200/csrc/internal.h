@@ -76,8 +76,11 @@ struct GemmArgs {
   void* vt_cache;      // [B, C, kv_capacity] bf16
   int kv_capacity, kv_offset;
   int32_t* status;     // device status word or null
+  void* splitk_ws;     // scratch for K-split partials (gemm_splitk_ws_bytes(), tickets at its head zero) or null
 };
 cudaError_t gemm_init();
+size_t gemm_splitk_ws_bytes();      // size of the K-split scratch
+size_t gemm_splitk_ticket_bytes();  // its leading bytes that must be zero before first use
 fv_status launch_gemm(const GemmArgs& g, cudaStream_t st);
 
 // ---- attention.cu : flash-style attention over the KV cache ------------------------------------

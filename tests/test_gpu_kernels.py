@@ -177,6 +177,40 @@ def test_gemm_bf16(M, N, K, epilogue):
     assert err <= MAX_ABS and cos >= MIN_COS, (err, cos)
 
 
+SPLITK_CASES = [(2, 2048, 8192), (2, 6144, 2048), (85, 768, 256), (128, 8192, 2048), (288, 2048, 2048), (300, 1024, 4096), (7, 136, 1024),
+                (1640, 6144, 2048)]   # the last shape has enough tiles: the scratch is passed but no split is taken
+
+
+@pytest.mark.parametrize("M,N,K", SPLITK_CASES)
+@pytest.mark.parametrize("epilogue", [0, 1])
+def test_gemm_bf16_split_along_k(M, N, K, epilogue):
+    """Few rows against a large weight matrix: K slices on different CTAs, partial sums added in slice order."""
+    a = I.normal_bf16(73, (M, K), 1.0 if K <= 2048 else 0.5)
+    w = I.normal_bf16(74, (N, K), 0.02)
+    b = I.normal_bf16(75, (N,), 0.02)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = torch.zeros(fv.lib().fv_gemm_splitk_workspace_bytes(), dtype=torch.uint8, device=DEV)
+    ad, wd, bd = bf16_dev(a), bf16_dev(w), bf16_dev(b)
+    out = fv.fv_gemm_bf16(ad, wd, bd, epilogue=epilogue, status=status, splitk_ws=ws)
+    out2 = fv.fv_gemm_bf16(ad, wd, bd, epilogue=epilogue, status=status, splitk_ws=ws)   # counters were left at zero
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(out, out2)                       # arrival order does not change the sum
+    assert int(ws[:4096].to(torch.int32).sum().item()) == 0
+    ref = O.linear(I.bf16_bits_to_f32(a), I.bf16_bits_to_f32(w), I.bf16_bits_to_f32(b))
+    if epilogue == 1:
+        ref = O.gelu_tanh(ref)
+    err, cos = per_token_errors(bf16_host(out), ref)
+    assert err <= MAX_ABS and cos >= MIN_COS, (err, cos)
+
+
+def test_gemm_split_along_k_refuses_small_scratch():
+    a = torch.zeros((2, 256), dtype=torch.bfloat16, device=DEV); w = torch.zeros((256, 256), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(fv.FvError) as e:
+        fv.fv_gemm_bf16(a, w, None, splitk_ws=torch.zeros(4096, dtype=torch.uint8, device=DEV))
+    assert e.value.code == 3
+
+
 def test_gemm_residual_epilogue_with_cache_copy():
     B, rows, N, K = 2, 100, 256, 512
     M = B * rows
