@@ -221,6 +221,11 @@ fv_status fv_restore_residual(float *x_dev, const void *y_dev, const void *cache
  *               (few rows against a large weight matrix) are then split along K, the slices' fp32
  *               partial sums added in slice order.  CAPACITY if splitk_ws_bytes is too small. */
 size_t fv_gemm_splitk_workspace_bytes(void);
+/* Test / profiling hook (process-wide): which GEMM kernel fv_gemm_bf16 and the step use when no K split is
+ * taken.  0 = chosen per shape (default); 1 = one CTA per 128-row tile, width chosen per shape; 2 = CTA
+ * pairs sharing 256 x 256 tiles (tcgen05 cta_group::2); 3 = CTA pairs, 256 x 128 tiles; 4 / 5 / 6 = one CTA
+ * per tile of width 128 / 192 / 256.  INVALID_ARG outside 0..6. */
+fv_status fv_gemm_force_path(int32_t path);
 fv_status fv_gemm_bf16(const void *a_dev, const void *w_dev, const void *bias_dev, int32_t M,
                        int32_t N, int32_t K, int32_t epilogue, void *out_dev, void *aux_dev,
                        const float *gamma_dev, int32_t mod_stride, int32_t rows_per_image,

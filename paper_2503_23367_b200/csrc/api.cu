@@ -199,6 +199,12 @@ fv_status fv_attention(const void* q_dev, const void* k_dev, const void* vt_dev,
 
 size_t fv_gemm_splitk_workspace_bytes(void) { return gemm_splitk_ws_bytes(); }
 
+fv_status fv_gemm_force_path(int32_t path) {
+  if (path < 0 || path > 6) return FV_ERR_INVALID_ARG;
+  gemm_force_path(path);
+  return FV_OK;
+}
+
 size_t fv_workspace_bytes(const fv_config* cfg) { return config_ok(cfg) ? workspace_layout(cfg).total : 0; }
 
 size_t fv_kv_bytes(const fv_config* cfg) {

@@ -23,10 +23,13 @@
 
 #include <mutex>
 
+#include "gemm_epilogue.cuh"
 #include "internal.h"
 #include "sm100.cuh"
 
 namespace fv {
+
+using namespace gemm_detail;
 
 namespace {
 
@@ -43,126 +46,6 @@ template <int BN> struct GemmCfg {
   static constexpr int kAccStride = (BN == 128) ? 128 : 256;  // column offset of the second accumulator
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
-
-struct GemmDev {
-  const __nv_bfloat16* bias;
-  int M, N, K;
-  int epilogue;
-  void* out;
-  void* aux;
-  const float* gamma;
-  int mod_stride, rows_per_image;
-  int q_cols, C;
-  __nv_bfloat16* k_cache;
-  __nv_bfloat16* vt_cache;
-  int kv_capacity, kv_offset;
-  int32_t* status;
-  int splits, kb_per_split;   // K slices per tile (1 = no split) and 64-wide k-blocks per slice
-  float* sk_partial;          // [tile][slice][128][BN] fp32 partial accumulators
-  unsigned int* sk_tickets;   // [tile] arrival counters, zero between launches
-};
-
-__device__ __forceinline__ float gelu_tanh_fast(float v) {
-  const float u = 0.7978845608028654f * fmaf(0.044715f * v * v, v, v);
-  float t;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
-  return 0.5f * v * (1.f + t);
-}
-
-__device__ __forceinline__ void report(int32_t* status, int code) {
-  if (status) atomicCAS(status, 0, code);
-}
-
-// One 32-column chunk of one accumulator row: bias, optional GELU, then the epilogue's store.
-__device__ __forceinline__ void epilogue_chunk(const GemmDev& p, const uint32_t (&r)[32], int row, int img, int jrow, int col) {
-  float v[32];
-  if (p.bias) {
-    const uint4* bp = reinterpret_cast<const uint4*>(p.bias + col);
-#pragma unroll
-    for (int g = 0; g < 4; ++g) {
-      if (col + 8 * g < p.N) {
-        uint4 bb = __ldg(bp + g);
-        const uint32_t u[4] = {bb.x, bb.y, bb.z, bb.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          v[8 * g + 2 * i] = __uint_as_float(r[8 * g + 2 * i]) + __uint_as_float(u[i] << 16);
-          v[8 * g + 2 * i + 1] = __uint_as_float(r[8 * g + 2 * i + 1]) + __uint_as_float(u[i] & 0xFFFF0000u);
-        }
-      } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v[8 * g + i] = 0.f;
-      }
-    }
-  } else {
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-  }
-  if (p.epilogue == EPI_GELU_BF16) {
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = gelu_tanh_fast(v[i]);
-  }
-  if (p.epilogue == EPI_BF16 || p.epilogue == EPI_GELU_BF16 || (p.epilogue == EPI_QKV_SPLIT && col < p.q_cols)) {
-    const int ld = (p.epilogue == EPI_QKV_SPLIT) ? p.q_cols : p.N;
-    uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + (size_t)row * ld + col);
-#pragma unroll
-    for (int g = 0; g < 4; ++g) {
-      if (col + 8 * g < p.N) {
-        uint4 o;
-        o.x = pack_bf16x2(v[8 * g + 0], v[8 * g + 1]); o.y = pack_bf16x2(v[8 * g + 2], v[8 * g + 3]);
-        o.z = pack_bf16x2(v[8 * g + 4], v[8 * g + 5]); o.w = pack_bf16x2(v[8 * g + 6], v[8 * g + 7]);
-        dst[g] = o;
-      }
-    }
-  } else if (p.epilogue == EPI_RESIDUAL) {
-    float4* xr = reinterpret_cast<float4*>(static_cast<float*>(p.out) + (size_t)row * p.N + col);
-    const float4* gp = p.gamma ? reinterpret_cast<const float4*>(p.gamma + (size_t)img * p.mod_stride + col) : nullptr;
-    uint4* ap = p.aux ? reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.aux) + (size_t)row * p.N + col) : nullptr;
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      if (col + 4 * g < p.N) {
-        float4 xv = xr[g];
-        if (gp) {
-          float4 gg = __ldg(gp + g);
-          xv.x = fmaf(gg.x, v[4 * g + 0], xv.x); xv.y = fmaf(gg.y, v[4 * g + 1], xv.y);
-          xv.z = fmaf(gg.z, v[4 * g + 2], xv.z); xv.w = fmaf(gg.w, v[4 * g + 3], xv.w);
-        } else {
-          xv.x += v[4 * g + 0]; xv.y += v[4 * g + 1]; xv.z += v[4 * g + 2]; xv.w += v[4 * g + 3];
-        }
-        xr[g] = xv;
-      }
-    }
-    if (ap) {
-#pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        if (col + 8 * g < p.N) {
-          uint4 o;
-          o.x = pack_bf16x2(v[8 * g + 0], v[8 * g + 1]); o.y = pack_bf16x2(v[8 * g + 2], v[8 * g + 3]);
-          o.z = pack_bf16x2(v[8 * g + 4], v[8 * g + 5]); o.w = pack_bf16x2(v[8 * g + 6], v[8 * g + 7]);
-          ap[g] = o;
-        }
-      }
-    }
-  } else {  // EPI_QKV_SPLIT, K or V part
-    const int kc = col - p.q_cols;
-    const size_t krow = (size_t)img * p.kv_capacity + p.kv_offset + jrow;
-    if (kc < p.C) {
-      uint4* dst = reinterpret_cast<uint4*>(p.k_cache + krow * p.C + kc);
-#pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        uint4 o;
-        o.x = pack_bf16x2(v[8 * g + 0], v[8 * g + 1]); o.y = pack_bf16x2(v[8 * g + 2], v[8 * g + 3]);
-        o.z = pack_bf16x2(v[8 * g + 4], v[8 * g + 5]); o.w = pack_bf16x2(v[8 * g + 6], v[8 * g + 7]);
-        dst[g] = o;
-      }
-    } else {
-      // V is kept transposed ([image, channel, key]) so that P*V reads it K-major; for a fixed
-      // channel the 32 lanes write 32 consecutive keys.
-      __nv_bfloat16* dst = p.vt_cache + ((size_t)img * p.C + (kc - p.C)) * p.kv_capacity + p.kv_offset + jrow;
-#pragma unroll
-      for (int i = 0; i < 32; ++i) dst[(size_t)i * p.kv_capacity] = __float2bfloat16_rn(v[i]);
-    }
-  }
-}
 
 template <int BN, bool SPLIT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
@@ -378,6 +261,7 @@ cudaError_t gemm_init() {
   if (e == cudaSuccess) e = set_attr<128, true>();
   if (e == cudaSuccess) e = set_attr<192, false>();
   if (e == cudaSuccess) e = set_attr<256, false>();
+  if (e == cudaSuccess) e = gemm_pair_init();
   if (e != cudaSuccess) return e;
   int dev = 0;
   e = cudaGetDevice(&dev);
@@ -385,17 +269,26 @@ cudaError_t gemm_init() {
   return cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
 }
 
-// Tile width for a shape: the persistent grid runs ceil(tiles / SMs) rounds of BN-wide tiles, so pick
-// the BN with the smallest rounds x BN (128-wide tiles pay ~10 % for their shared-memory read rate).
-static int pick_bn(int tiles_m, int N, int sms) {
-  const int cand[3] = {256, 192, 128};
-  int best = 128;
+// Kernel and tile width for a shape.  Measured on B200, one launch costs about
+//     fixed + rounds x k-blocks x per_kblock
+// where rounds = ceil(tiles / resident CTAs or pairs): the operand pipeline is bound by the latency of
+// its loads (all of shared memory is in flight), so a k-block costs about the same whatever the tile
+// width, and wider tiles / CTA pairs win by needing fewer rounds and less L2 traffic per flop.
+struct TileChoice { int bn; bool pair; };
+static TileChoice pick_tile(int M, int N, int K, int sms) {
+  const int num_kb = (K + BK - 1) / BK;
+  struct Cand { int bn; bool pair; double fixed_us, kb_us; };
+  const Cand cand[4] = {{128, false, 8.5, 0.271}, {192, false, 10.4, 0.278}, {256, false, 10.1, 0.361}, {256, true, 14.0, 0.297}};
+  TileChoice best{128, false};
   double best_cost = 1e30;
-  for (int bn : cand) {
-    const long tiles = (long)tiles_m * ((N + bn - 1) / bn);
-    const long rounds = (tiles + sms - 1) / sms;
-    const double cost = (double)rounds * bn * (bn == 128 ? 1.1 : 1.0);
-    if (cost < best_cost - 1e-9) { best_cost = cost; best = bn; }
+  for (const Cand& c : cand) {
+    if (c.pair && M <= 256) continue;
+    const int rows = c.pair ? 256 : 128;
+    const int slots = c.pair ? sms / 2 : sms;
+    const long tiles = (long)((M + rows - 1) / rows) * ((N + c.bn - 1) / c.bn);
+    const long rounds = (tiles + slots - 1) / slots;
+    const double cost = c.fixed_us + (double)rounds * num_kb * c.kb_us;
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = TileChoice{c.bn, c.pair}; }
   }
   return best;
 }
@@ -434,12 +327,20 @@ static cudaError_t launch_bn(const GemmArgs& g, const GemmDev& p, int tiles_m, c
   return cudaGetLastError();
 }
 
+static int g_force_path = 0;
+void gemm_force_path(int path) { g_force_path = path; }
+
 fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   if (g.M <= 0 || g.N <= 0 || g.K <= 0 || (g.K % 8) || (g.N % 8) || !g.a || !g.w) return FV_ERR_INVALID_ARG;
   if (g.rows_per_image <= 0) return FV_ERR_INVALID_ARG;
   if (g.epilogue == EPI_QKV_SPLIT && (g.C % 128 || g.q_cols % 128)) return FV_ERR_UNSUPPORTED;
   const int tiles_m = (g.M + BM - 1) / BM;
-  int bn = pick_bn(tiles_m, g.N, g_num_sms);
+  TileChoice tc = pick_tile(g.M, g.N, g.K, g_num_sms);
+  if (g_force_path == 1 && tc.pair) tc = TileChoice{256, false};
+  if (g_force_path == 2) tc = TileChoice{256, true};
+  if (g_force_path == 3) tc = TileChoice{128, true};
+  if (g_force_path >= 4 && g_force_path <= 6) tc = TileChoice{128 + 64 * (g_force_path - 4), false};
+  int bn = tc.bn;
   GemmDev p;
   p.splits = 1; p.kb_per_split = (g.K + BK - 1) / BK; p.sk_partial = nullptr; p.sk_tickets = nullptr;
   if (g.splitk_ws) {
@@ -460,6 +361,10 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   p.k_cache = static_cast<__nv_bfloat16*>(g.k_cache); p.vt_cache = static_cast<__nv_bfloat16*>(g.vt_cache);
   p.kv_capacity = g.kv_capacity; p.kv_offset = g.kv_offset; p.status = g.status;
   LaunchScope scope(KC_GEMM, 1, 2.0 * g.M * (double)g.N * g.K, st);
+  if (p.splits == 1 && tc.pair) {
+    cudaError_t e2 = launch_gemm_pair(g, p, bn, st);
+    return e2 == cudaSuccess ? FV_OK : FV_ERR_CUDA;
+  }
   cudaError_t e = bn == 256 ? launch_bn<256>(g, p, tiles_m, st) : (bn == 192 ? launch_bn<192>(g, p, tiles_m, st) : launch_bn<128>(g, p, tiles_m, st));
   return e == cudaSuccess ? FV_OK : FV_ERR_CUDA;
 }

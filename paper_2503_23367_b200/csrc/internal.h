@@ -79,6 +79,8 @@ struct GemmArgs {
   void* splitk_ws;     // scratch for K-split partials (gemm_splitk_ws_bytes(), tickets at its head zero) or null
 };
 cudaError_t gemm_init();
+// Test / profiling hook: 0 = choose per shape, 1 = one-CTA kernel, 2 = CTA-pair kernel 256x256, 3 = CTA-pair 256x128.
+void gemm_force_path(int path);
 size_t gemm_splitk_ws_bytes();      // size of the K-split scratch
 size_t gemm_splitk_ticket_bytes();  // its leading bytes that must be zero before first use
 fv_status launch_gemm(const GemmArgs& g, cudaStream_t st);

@@ -211,6 +211,28 @@ def test_gemm_split_along_k_refuses_small_scratch():
     assert e.value.code == 3
 
 
+@pytest.mark.parametrize("path", [2, 3])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (300, 512, 256), (7, 136, 72), (1000, 1024, 1024), (130, 1920, 1920),
+                                   (1640, 6144, 2048), (1844, 2048, 8192)])
+def test_gemm_bf16_on_cta_pairs(M, N, K, path):
+    """The CTA-pair kernel (two CTAs share a 256-row tile, tcgen05 cta_group::2), forced for every shape,
+    ragged M / N tails included; both tile widths."""
+    a = I.normal_bf16(76, (M, K), 1.0 if K <= 2048 else 0.5)
+    w = I.normal_bf16(77, (N, K), 0.02)
+    b = I.normal_bf16(78, (N,), 0.02)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    assert fv.lib().fv_gemm_force_path(path) == 0
+    try:
+        out = fv.fv_gemm_bf16(bf16_dev(a), bf16_dev(w), bf16_dev(b), epilogue=1, status=status)
+        torch.cuda.synchronize()
+    finally:
+        fv.lib().fv_gemm_force_path(0)
+    assert int(status.item()) == 0
+    ref = O.gelu_tanh(O.linear(I.bf16_bits_to_f32(a), I.bf16_bits_to_f32(w), I.bf16_bits_to_f32(b)))
+    err, cos = per_token_errors(bf16_host(out), ref)
+    assert err <= MAX_ABS and cos >= MIN_COS, (err, cos)
+
+
 def test_gemm_residual_epilogue_with_cache_copy():
     B, rows, N, K = 2, 100, 256, 512
     M = B * rows
