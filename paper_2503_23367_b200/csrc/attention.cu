@@ -131,6 +131,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   uint64_t* o_done = p_full + 2;     // [2] the latest P V of query tile t has completed
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_done + 2);
 
+  pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = blockIdx.x * (2 * QT), head = blockIdx.y, img = blockIdx.z;
   const int T = (p.kv_len + KT - 1) / KT;
@@ -148,6 +149,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();  // set-up above overlaps the previous kernel; Q / K / V and the output are touched only from here
 
   if (warp == 0) {
     if (lane == 0) {
@@ -309,8 +311,8 @@ template <int HD> fv_status launch_hd(const AttnArgs& a, cudaStream_t st) {
   p.status = a.status;
   dim3 grid((a.rows + 2 * QT - 1) / (2 * QT), a.H, a.B);
   LaunchScope scope(KC_ATTENTION, 1, 4.0 * a.B * (double)a.rows * a.kv_len * a.C, st);
-  attention_kernel<HD><<<grid, kAttnThreads, AttnCfg<HD>::kSmemBytes, st>>>(tmQ, tmK, tmV, p);
-  return cudaGetLastError() == cudaSuccess ? FV_OK : FV_ERR_CUDA;
+  return launch_pdl(attention_kernel<HD>, grid, dim3(kAttnThreads), AttnCfg<HD>::kSmemBytes, st, tmQ, tmK, tmV, p) == cudaSuccess
+             ? FV_OK : FV_ERR_CUDA;
 }
 
 }  // namespace

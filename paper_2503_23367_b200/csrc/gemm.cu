@@ -61,6 +61,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* sk_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
+  pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_m = (p.M + BM - 1) / BM;
   const int tiles_n = (p.N + BN - 1) / BN;
@@ -80,6 +81,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();  // set-up above overlaps the previous kernel; operands and outputs are touched only from here
 
   if (warp == 0) {
     if (lane == 0) {
@@ -319,12 +321,11 @@ static cudaError_t launch_bn(const GemmArgs& g, const GemmDev& p, int tiles_m, c
   const long tiles = (long)tiles_m * ((g.N + BN - 1) / BN) * p.splits;
   const int grid = (int)(tiles < g_num_sms ? tiles : g_num_sms);
   if (p.splits > 1) {
-    if constexpr (BN == 128) gemm_bf16_kernel<128, true><<<grid, kGemmThreads, GemmCfg<128>::kSmemBytes, st>>>(tmA, tmB, p);
+    if constexpr (BN == 128) return launch_pdl(gemm_bf16_kernel<128, true>, dim3(grid), dim3(kGemmThreads), GemmCfg<128>::kSmemBytes, st, tmA, tmB, p);
     else return cudaErrorInvalidValue;
   } else {
-    gemm_bf16_kernel<BN, false><<<grid, kGemmThreads, GemmCfg<BN>::kSmemBytes, st>>>(tmA, tmB, p);
+    return launch_pdl(gemm_bf16_kernel<BN, false>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::kSmemBytes, st, tmA, tmB, p);
   }
-  return cudaGetLastError();
 }
 
 static int g_force_path = 0;

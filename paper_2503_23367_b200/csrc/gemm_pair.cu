@@ -53,6 +53,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   uint64_t* acc_empty = acc_full + 2;        // [2] used in the leader: 256 arrivals
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
 
+  pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
@@ -74,6 +75,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();  // set-up above overlaps the previous kernel; operands and outputs are touched only from here
 
   if (warp == 0) {
     if (lane == 0) {
@@ -181,13 +183,9 @@ cudaError_t launch_gemm_pair(const GemmArgs& g, const GemmDev& p, int bn, cudaSt
   const long tiles = (long)((g.M + 2 * BM - 1) / (2 * BM)) * ((g.N + bn - 1) / bn);
   const int max_pairs = g_pair_sms / 2;
   const int pairs = (int)(tiles < max_pairs ? tiles : max_pairs);
-  if (bn == 256)
-    gemm_pair_kernel<256><<<2 * pairs, kThreads, PairCfg<256>::kSmemBytes, st>>>(tmA, tmB, p);
-  else if (bn == 128)
-    gemm_pair_kernel<128><<<2 * pairs, kThreads, PairCfg<128>::kSmemBytes, st>>>(tmA, tmB, p);
-  else
-    return cudaErrorInvalidValue;
-  return cudaGetLastError();
+  if (bn == 256) return launch_pdl(gemm_pair_kernel<256>, dim3(2 * pairs), dim3(kThreads), PairCfg<256>::kSmemBytes, st, tmA, tmB, p);
+  if (bn == 128) return launch_pdl(gemm_pair_kernel<128>, dim3(2 * pairs), dim3(kThreads), PairCfg<128>::kSmemBytes, st, tmA, tmB, p);
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace fv

@@ -10,6 +10,26 @@ namespace fv {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Launch with programmatic stream serialization: the grid may start (and run up to its
+// griddepcontrol.wait) while the kernel before it in the stream is still finishing, which hides launch
+// latency and per-CTA set-up between the many short dependent kernels of a scale step.  Every kernel
+// launched this way executes pdl_wait() before its first access to global memory that an earlier
+// kernel may write or read.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---- prof.cu : launch counting and optional per-kernel-class timing (CUDA events on the stream) ---
 enum KernelClass : int { KC_SELECT = 0, KC_GATHER_LN = 1, KC_GEMM = 2, KC_ATTENTION = 3, KC_RESTORE = 4, KC_COUNT = 5 };
 // Brackets the launches of one kernel class: counts `kernels` launches, adds `work` (algorithmic bytes

@@ -29,6 +29,8 @@ __global__ void __launch_bounds__(256) gather_ln_kernel(const float4* __restrict
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.y, j = blockIdx.x * 8 + warp;
   const bool live = j < k;
+  pdl_trigger();
+  pdl_wait();
   const int t = live ? (idx ? __ldg(idx + (size_t)b * k + j) : j) : 0;
   if (sigma) {
     const float4* sg = reinterpret_cast<const float4*>(sigma + (size_t)b * mod_stride);
@@ -115,6 +117,8 @@ __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restric
                                                                int ngroups, float4* __restrict__ chunk_partial,
                                                                float4* __restrict__ group_partial, unsigned int* tickets) {
   __shared__ const uint4* s_src[kColsumRows];
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.y, chunk = blockIdx.x;
   const int t0 = chunk * kColsumRows;
   const int rows = min(kColsumRows, n - t0);
@@ -176,6 +180,8 @@ __global__ void __launch_bounds__(256) restore_bf16_kernel(const uint4* __restri
                                                            const uint4* __restrict__ pivots, const int32_t* __restrict__ inv,
                                                            int n, int k, int h, int w, int C8, uint4* __restrict__ out,
                                                            int total_rows) {
+  pdl_trigger();
+  pdl_wait();
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= total_rows) return;
   const int b = warp / n, t = warp - b * n;
@@ -192,10 +198,8 @@ cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, i
                              const float* beta, int mod_stride, void* a_out, cudaStream_t st) {
   const int rows = B * k;
   LaunchScope scope(KC_GATHER_LN, 1, (double)rows * C * 6.0, st);
-  gather_ln_kernel<<<dim3((k + 7) / 8, B), 256, sigma ? (size_t)C * 8 : 0, st>>>(reinterpret_cast<const float4*>(x), idx, n, k, C / 4,
-                                                                                sigma, beta, mod_stride,
-                                                                                reinterpret_cast<uint2*>(a_out));
-  return cudaGetLastError();
+  return launch_pdl(gather_ln_kernel, dim3((k + 7) / 8, B), dim3(256), sigma ? (size_t)C * 8 : 0, st, reinterpret_cast<const float4*>(x),
+                    idx, n, k, C / 4, sigma, beta, mod_stride, reinterpret_cast<uint2*>(a_out));
 }
 
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv, const float* gamma,
@@ -206,22 +210,18 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
   if (colsum_ws) ws = select_ws_carve(colsum_ws, B, n, C);
   const int nchunks = (n + kColsumRows - 1) / kColsumRows;
   LaunchScope scope(KC_RESTORE, 1, (double)B * C * (8.0 * n + 2.0 * k + 2.0 * hc * wc), st);
-  restore_residual_kernel<<<dim3(nchunks, B), 256, 0, st>>>(reinterpret_cast<float4*>(x), reinterpret_cast<const uint4*>(y),
-                                                            reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k,
-                                                            h, w, hc, wc, C / 8, nchunks, ws.group, ws.ngroups,
-                                                            reinterpret_cast<float4*>(ws.chunk_partial),
-                                                            reinterpret_cast<float4*>(ws.group_partial), ws.tickets);
-  return cudaGetLastError();
+  return launch_pdl(restore_residual_kernel, dim3(nchunks, B), dim3(256), 0, st, reinterpret_cast<float4*>(x),
+                    reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h, w, hc, wc,
+                    C / 8, nchunks, ws.group, ws.ngroups, reinterpret_cast<float4*>(ws.chunk_partial),
+                    reinterpret_cast<float4*>(ws.group_partial), ws.tickets);
 }
 
 cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* pivots, const int32_t* inv, int B, int k,
                                 int h, int w, int C, void* out, cudaStream_t st) {
   const int rows = B * h * w;
   LaunchScope scope(KC_RESTORE, 1, (double)B * C * (2.0 * h * w + 2.0 * k + 2.0 * hc * wc), st);
-  restore_bf16_kernel<<<(rows + 7) / 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(cache), hc, wc,
-                                                      reinterpret_cast<const uint4*>(pivots), inv, h * w, k, h, w, C / 8,
-                                                      reinterpret_cast<uint4*>(out), rows);
-  return cudaGetLastError();
+  return launch_pdl(restore_bf16_kernel, dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const uint4*>(cache), hc, wc,
+                    reinterpret_cast<const uint4*>(pivots), inv, h * w, k, h, w, C / 8, reinterpret_cast<uint4*>(out), rows);
 }
 
 }  // namespace fv

@@ -28,6 +28,8 @@ constexpr size_t kTopkMaxSmem = ((size_t)kTopkMaxTokens + kTopkMaxTokens / 32) *
 __global__ void __launch_bounds__(256) colsum_chunk_kernel(const float4* __restrict__ x, int n, int C4, int nchunks, int group,
                                                            int ngroups, float4* __restrict__ chunk_partial,
                                                            float4* __restrict__ group_partial, unsigned int* tickets) {
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.y, chunk = blockIdx.x;
   const int r0 = chunk * kColsumRows;
   const int r1 = min(n, r0 + kColsumRows);
@@ -91,6 +93,8 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float
   __shared__ uint32_t s_prefix, s_remaining, s_near;
   __shared__ int s_last;
   const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_trigger();
+  pdl_wait();
 
   // ---- Eq. 4: the mean token of image b from the group partials (fixed order)
   {
@@ -252,10 +256,14 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float
   }
 }
 __global__ void inv_fill_kernel(int32_t* inv, size_t total) {
+  pdl_trigger();
+  pdl_wait();
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < total) inv[i] = -1;
 }
 __global__ void inv_scatter_kernel(const int32_t* __restrict__ idx, int B, int k, int n, int32_t* __restrict__ inv) {
+  pdl_trigger();
+  pdl_wait();
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= B * k) return;
   int b = i / k, j = i - b * k;
@@ -314,9 +322,8 @@ cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* i
   float* sc = score ? score : w.score;
   LaunchScope scope(KC_SELECT, have_partials ? 1 : 2, (double)B * n * C * 4.0 + 4.0 * B * n + 4.0 * B * ((double)k + n), st);
   if (!have_partials)
-    colsum_chunk_kernel<<<dim3(w.nchunks, B), 256, 0, st>>>(reinterpret_cast<const float4*>(x), n, C4, w.nchunks, w.group, w.ngroups,
-                                                            reinterpret_cast<float4*>(w.chunk_partial),
-                                                            reinterpret_cast<float4*>(w.group_partial), w.tickets);
+    launch_pdl(colsum_chunk_kernel, dim3(w.nchunks, B), dim3(256), 0, st, reinterpret_cast<const float4*>(x), n, C4, w.nchunks, w.group,
+               w.ngroups, reinterpret_cast<float4*>(w.chunk_partial), reinterpret_cast<float4*>(w.group_partial), w.tickets);
   const size_t keys_smem = ((size_t)n + n / 32 + 1) * 4;
   const size_t smem = keys_smem > (size_t)C * 4 ? keys_smem : (size_t)C * 4;
   // all CTAs resident at once: two per SM over the B images, never more than one warp per token row
@@ -324,17 +331,17 @@ cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* i
   const int need = (n + kTopkWarps - 1) / kTopkWarps;
   if (per_image > need) per_image = need;
   if (per_image < 1) per_image = 1;
-  score_topk_kernel<<<dim3(per_image, B), kTopkThreads, smem, st>>>(
-      reinterpret_cast<const float4*>(x), reinterpret_cast<const float4*>(w.group_partial), w.ngroups, n, C4, k, sc,
-      w.tickets + (size_t)B * kMaxGroups, idx, inv, near_tie);
+  launch_pdl(score_topk_kernel, dim3(per_image, B), dim3(kTopkThreads), smem, st, reinterpret_cast<const float4*>(x),
+             reinterpret_cast<const float4*>(w.group_partial), w.ngroups, n, C4, k, sc, w.tickets + (size_t)B * kMaxGroups, idx, inv,
+             near_tie);
   return cudaGetLastError();
 }
 
 cudaError_t launch_inv_from_idx(const int32_t* idx, int B, int k, int n, int32_t* inv, cudaStream_t st) {
   const size_t total = (size_t)B * n;
   LaunchScope scope(KC_SELECT, 2, 4.0 * B * ((double)k + n), st);
-  inv_fill_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(inv, total);
-  inv_scatter_kernel<<<(B * k + 255) / 256, 256, 0, st>>>(idx, B, k, n, inv);
+  launch_pdl(inv_fill_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, inv, total);
+  launch_pdl(inv_scatter_kernel, dim3((B * k + 255) / 256), dim3(256), 0, st, idx, B, k, n, inv);
   return cudaGetLastError();
 }
 
