@@ -16,7 +16,7 @@
 // Shapes with too few tiles to occupy the GPU (the small scale steps, where the GEMM is a stream of
 // weights) are split along K: work item = (tile, K slice), every slice leaves its fp32 partial rows in
 // a scratch buffer, and the last slice of a tile to arrive adds them in slice order and runs the
-// epilogue, so the result does not depend on arrival order.
+// epilogue, so the result does not depend on arrival order.  A K-split launch has one work item per CTA.
 // Every wait is bounded; on expiry a code is written to the status word and the CTA unwinds normally.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -60,6 +60,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   uint64_t* acc_empty = acc_full + 2;        // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* sk_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  uint64_t* fix_bar = reinterpret_cast<uint64_t*>(tmem_slot + 2);  // K-split: arrival of the slices' partials
 
   pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -72,6 +73,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 128); }
+    if (SPLIT) mbar_init(fix_bar, 1);
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
@@ -190,27 +192,58 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int last = *sk_flag;
         asm volatile("bar.sync 1, 128;" ::: "memory");  // flag consumed before the next item may rewrite it
         if (last) {
+          // The slices' partial rows are pulled into the (now idle) operand stages with bulk copies --
+          // one CTA cannot keep enough ordinary loads in flight to fetch them quickly -- and added
+          // there in slice order, the running sum living in slot 0; then every thread takes its row.
           __threadfence();
-          const float* base = p.sk_partial + ((size_t)tile * p.splits * BM + (quarter * 32 + lane)) * BN;
+          const int et = threadIdx.x - 64;                       // 0..127 among the epilogue threads
+          const int rows_valid = min(BM, p.M - m0);
+          const uint32_t slice_bytes = (uint32_t)rows_valid * BN * 4;
+          const int max_slots = (STAGES * Cfg::kStageBytes) / (int)slice_bytes;   // >= 3
+          const float* src0 = p.sk_partial + (size_t)tile * p.splits * BM * BN;
+          float4* slot0 = reinterpret_cast<float4*>(smem);
+          const int nf4 = rows_valid * (BN / 4);
+          int done = 0;
+          uint32_t phase = 0;
+          bool ok = true;
+          while (done < p.splits) {
+            const int first_slot = done == 0 ? 0 : 1;
+            const int cnt = min(max_slots - first_slot, p.splits - done);
+            if (et == 0) {
+              fence_proxy_async_all();   // earlier generic accesses to these slots / partials before the copies
+              mbar_expect_tx(fix_bar, (uint32_t)cnt * slice_bytes);
+              for (int i = 0; i < cnt; ++i)
+                bulk_load_1d(smem + (size_t)(first_slot + i) * slice_bytes, src0 + (size_t)(done + i) * BM * BN, slice_bytes, fix_bar);
+            }
+            if (!mbar_wait(fix_bar, phase)) { report(p.status, DEV_TIMEOUT_EPI); ok = false; break; }
+            phase ^= 1;
+            const int last_slot = first_slot + cnt - 1;
+            for (int f = et; f < nf4; f += 128) {
+              float4 acc = slot0[f];
+              for (int i = 1; i <= last_slot; ++i) {
+                const float4 v = reinterpret_cast<const float4*>(smem + (size_t)i * slice_bytes)[f];
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+              }
+              slot0[f] = acc;
+            }
+            done += cnt;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+          }
+          if (ok && row_ok) {
+            const float4* mysum = slot0 + (size_t)(quarter * 32 + lane) * (BN / 4);
 #pragma unroll 1
-          for (int c0 = 0; c0 < BN; c0 += 32) {
-            const int col = n0 + c0;
-            if (!(row_ok && col < p.N)) continue;
-            float acc[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) acc[i] = 0.f;
-            for (int sl = 0; sl < p.splits; ++sl) {
-              const float4* src = reinterpret_cast<const float4*>(base + (size_t)sl * BM * BN + c0);
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+              const int col = n0 + c0;
+              if (col >= p.N) break;
+              uint32_t r0[32];
 #pragma unroll
               for (int g = 0; g < 8; ++g) {
-                const float4 v = __ldcg(src + g);
-                acc[4 * g] += v.x; acc[4 * g + 1] += v.y; acc[4 * g + 2] += v.z; acc[4 * g + 3] += v.w;
+                const float4 v = mysum[c0 / 4 + g];
+                r0[4 * g] = __float_as_uint(v.x); r0[4 * g + 1] = __float_as_uint(v.y);
+                r0[4 * g + 2] = __float_as_uint(v.z); r0[4 * g + 3] = __float_as_uint(v.w);
               }
+              epilogue_chunk(p, r0, row, img, jrow, col);
             }
-            uint32_t r0[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) r0[i] = __float_as_uint(acc[i]);
-            epilogue_chunk(p, r0, row, img, jrow, col);
           }
         }
       }
@@ -301,14 +334,25 @@ constexpr int kSplitMaxItems = 2 * 148;
 size_t gemm_splitk_ticket_bytes() { return kSplitTicketBytes; }
 size_t gemm_splitk_ws_bytes() { return kSplitTicketBytes + (size_t)kSplitMaxItems * BM * 128 * sizeof(float); }
 
-// How many K slices for a shape that leaves SMs idle.  A CTA pulls its operands at roughly 100 GB/s and
-// pays a few microseconds of fixed cost, so slicing only pays for long K (>= 64 k-blocks), and a slice
-// keeps at least 16 k-blocks.  The last arriver re-reads slices x rows x 512 bytes, which grows with M.
-static int pick_splits(long tiles, int num_kb, int sms) {
-  if (tiles * 2 > sms || num_kb < 64) return 1;
+// How many K slices for a shape that leaves SMs idle.  A CTA's operand pipeline is bound by load latency
+// (a k-block every ~0.3 us whatever the tile), so spreading a tile's k-blocks over idle CTAs pays --
+// until the last arriver's work, pulling slices x rows x 512 bytes back in, outweighs it.  Measured:
+// long K (>= 64 k-blocks) gains at any row count with >= 16 k-blocks per slice; short K only gains
+// while rows x slices stays small (<= 256) and there are at least 4 slices of >= 4 k-blocks.
+static int pick_splits(long tiles, int M, int num_kb, int sms) {
+  if (tiles * 2 > sms || num_kb < 16) return 1;
   int s = (int)(sms / tiles);
-  if (s > num_kb / 16) s = num_kb / 16;
-  if (s < 2) return 1;
+  if (num_kb >= 64) {
+    const int rows = M < 128 ? M : 128;
+    if (s > num_kb / 16) s = num_kb / 16;
+    if (s > 512 / rows) s = 512 / rows;
+    if (s < 2) return 1;
+  } else {
+    const int rows = M < 128 ? M : 128;
+    if (s > num_kb / 4) s = num_kb / 4;
+    if (s > 256 / rows) s = 256 / rows;
+    if (s < 4) return 1;
+  }
   const int per = (num_kb + s - 1) / s;
   return (num_kb + per - 1) / per;  // no empty slice
 }
@@ -347,8 +391,8 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   if (g.splitk_ws) {
     const int num_kb = (g.K + BK - 1) / BK;
     const long tiles128 = (long)tiles_m * ((g.N + 127) / 128);
-    const int sp = pick_splits(tiles128, num_kb, g_num_sms);
-    if (sp > 1 && tiles128 * sp <= kSplitMaxItems && tiles128 * sizeof(unsigned int) <= kSplitTicketBytes) {
+    const int sp = pick_splits(tiles128, g.M, num_kb, g_num_sms);
+    if (sp > 1 && tiles128 * sp <= g_num_sms && tiles128 * sp <= kSplitMaxItems && tiles128 * sizeof(unsigned int) <= kSplitTicketBytes) {
       bn = 128;
       p.splits = sp;
       p.kb_per_split = (num_kb + sp - 1) / sp;
