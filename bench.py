@@ -401,9 +401,13 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer end-to-end leg")
     ap.add_argument("--skip-profile", action="store_true", help="omit the per-kernel-class timing passes")
     ap.add_argument("--skip-unpruned", action="store_true", help="omit the unpruned GPU comparison")
+    ap.add_argument("--blocks", type=int, default=0,
+                    help="profiling only: run this many transformer blocks instead of the workload's depth (the line says so; not a bench number)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = I.WORKLOADS[args.workload]
+    if args.blocks > 0:
+        wl = wl.with_depth(args.blocks)
     if args.impl == "reference":
         reference_arm(args, wl)
     else:

@@ -215,6 +215,9 @@ fv_status fv_restore_residual(float *x_dev, const void *y_dev, const void *cache
  *   epilogue 2: fp32 residual: out[m,n] += gamma[m / rows_per_image, n] * (acc + bias)  (out fp32;
  *               gamma NULL = 1; if aux_dev != NULL the bf16 value of acc+bias is also stored there).
  *   K % 8 == 0, N % 8 == 0, all pointers 16-byte aligned.  bias_dev may be NULL.
+ *   W is treated as a constant of the stream: its first tiles are requested as soon as the kernel starts,
+ *   which (programmatic dependent launch) can be while the kernel enqueued just before it is still
+ *   finishing -- do not produce W with that kernel.  A, bias and the outputs are touched only after it.
  *   status_dev: int32 device word that receives a non-zero code if a bounded wait expires (or NULL).
  *   splitk_ws_dev: NULL, or scratch of fv_gemm_splitk_workspace_bytes() bytes whose first 4096 bytes are
  *               zero (the kernel leaves them zero): shapes with too few output tiles to occupy the GPU

@@ -6,14 +6,15 @@
 // One CTA = 256 queries (two tiles of 128) of one head of one image; keys are consumed in tiles of 128.
 // The two query tiles take turns on the tensor core: while the softmax warps of one tile work on its
 // scores, the MMAs of the other tile run.
-//   warp 0   : TMA producer (both Q tiles once; K tiles [128 keys x hd]; V^T tiles [hd x 128 keys]).
-//   warp 1   : one lane issues tcgen05.mma.  Per key tile j and query tile t:  O_t += P_t V_j  with P_t
+//   warp 8   : TMA producer (both Q tiles once; K tiles [128 keys x hd]; V^T tiles [hd x 128 keys]).
+//   warp 9   : one lane issues tcgen05.mma.  Per key tile j and query tile t:  O_t += P_t V_j  with P_t
 //              read from TENSOR MEMORY (it overwrites the first 64 columns of S_t), then
 //              S_t = Q_t K_{j+1}^T.  MMAs of one thread execute in issue order, which is what makes
 //              the P_t / S_t aliasing safe.
-//   warps 2-5, 6-9: online softmax of tile 0 / tile 1, thread = query row.  Pass 1 reads the 128 scores
-//              from TMEM for the row maximum, pass 2 reads them again, exponentiates (base 2), sums,
-//              and writes bf16 probabilities back to TMEM.  The running maximum is only raised when
+//   warps 0-3, 4-7: online softmax of tile 0 / tile 1, thread = query row: the 128 scores of the row come
+//              out of TMEM in one go (four loads, one wait; the register file is re-divided between the
+//              warpgroups with setmaxnreg so that a thread can hold them), row maximum, base-2
+//              exponentials, row sum, and the bf16 probabilities go back to TMEM.  The running maximum is only raised when
 //              it would grow by more than 2^8, so the O accumulator (TMEM) is rescaled in place only
 //              on the rare tiles where that happens; the final O / l is written as bf16.
 // V is read transposed ([channel, key], keys contiguous), which makes it a K-major B operand.
@@ -30,7 +31,7 @@ namespace {
 
 constexpr int QT = 128;   // queries per tile (two tiles per CTA)
 constexpr int KT = 128;   // keys per tile
-constexpr int kAttnThreads = 320;
+constexpr int kAttnThreads = 384;   // warps 0-3 / 4-7: softmax of query tile 0 / 1; warp 8: TMA; warp 9: MMA; 10-11: idle
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 
 template <int HD> struct AttnCfg {
@@ -59,54 +60,44 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-// Row maximum over one 128-key score tile held in TMEM (lanes = rows).  MASK: keys >= valid are ignored.
+// The 128 scores of one row: TMEM -> registers (one wait for all four loads).  MASK: keys >= valid read -inf.
 template <bool MASK>
-__device__ __forceinline__ float tile_row_max(uint32_t s_addr, int valid) {
-  float mx = -INFINITY;
+__device__ __forceinline__ void tile_load_scores(uint32_t s_addr, int valid, float (&sc)[KT]) {
+  uint32_t a[32], b[32], c[32], d[32];
+  tmem_ld32(s_addr, a);
+  tmem_ld32(s_addr + 32, b);
+  tmem_ld32(s_addr + 64, c);
+  tmem_ld32(s_addr + 96, d);
+  tmem_wait_ld();
 #pragma unroll
-  for (int c = 0; c < KT / 64; ++c) {
-    uint32_t a[32], b[32];
-    tmem_ld32(s_addr + c * 64, a);
-    tmem_ld32(s_addr + c * 64 + 32, b);
-    tmem_wait_ld();
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      float va = __uint_as_float(a[i]), vb = __uint_as_float(b[i]);
-      if (MASK) {
-        if (c * 64 + i >= valid) va = -INFINITY;
-        if (c * 64 + 32 + i >= valid) vb = -INFINITY;
-      }
-      mx = fmaxf(mx, fmaxf(va, vb));
-    }
+  for (int i = 0; i < 32; ++i) {
+    sc[i] = __uint_as_float(a[i]); sc[32 + i] = __uint_as_float(b[i]);
+    sc[64 + i] = __uint_as_float(c[i]); sc[96 + i] = __uint_as_float(d[i]);
   }
-  return mx;
+  if (MASK) {
+#pragma unroll
+    for (int i = 0; i < KT; ++i)
+      if (i >= valid) sc[i] = -INFINITY;
+  }
 }
 
 // p = 2^(s * scale - m) for the 128 scores of a row; bf16 pairs written to TMEM columns [p_addr, +64);
-// returns the row sum of the UNROUNDED probabilities.
-template <bool MASK>
-__device__ __forceinline__ float tile_exp_store(uint32_t s_addr, uint32_t p_addr, float scale, float m, int valid) {
-  float rs = 0.f;
+// returns the row sum of the UNROUNDED probabilities.  Masked scores are -inf and give p = 0.
+__device__ __forceinline__ float tile_exp_store(const float (&sc)[KT], uint32_t p_addr, float scale, float m) {
+  float rs0 = 0.f, rs1 = 0.f;
 #pragma unroll
   for (int c = 0; c < KT / 32; ++c) {
-    uint32_t a[32];
-    tmem_ld32(s_addr + c * 32, a);
-    tmem_wait_ld();
     uint32_t pk[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-      float p0 = fast_exp2(fmaf(__uint_as_float(a[2 * i]), scale, -m));
-      float p1 = fast_exp2(fmaf(__uint_as_float(a[2 * i + 1]), scale, -m));
-      if (MASK) {
-        if (c * 32 + 2 * i >= valid) p0 = 0.f;
-        if (c * 32 + 2 * i + 1 >= valid) p1 = 0.f;
-      }
-      rs += p0 + p1;
+      const float p0 = fast_exp2(fmaf(sc[c * 32 + 2 * i], scale, -m));
+      const float p1 = fast_exp2(fmaf(sc[c * 32 + 2 * i + 1], scale, -m));
+      rs0 += p0; rs1 += p1;
       pk[i] = pack_bf16x2(p0, p1);
     }
     tmem_st16(p_addr + c * 16, pk);
   }
-  return rs;
+  return rs0 + rs1;
 }
 
 template <int HD>
@@ -144,14 +135,18 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     mbar_fence_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
   }
-  if (warp == 1) { tmem_alloc(tmem_slot, Cfg::kTmemCols); tmem_relinquish(); }
+  if (warp == 9) { tmem_alloc(tmem_slot, Cfg::kTmemCols); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();  // set-up above overlaps the previous kernel; Q / K / V and the output are touched only from here
 
-  if (warp == 0) {
+  // A softmax thread holds a whole score row (128 fp32) in registers, so the register file is re-divided
+  // between the warpgroups: 2 x 128 x 216 + 128 x 40 <= 64 K registers.
+  if (warp >= 8) {
+   asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+   if (warp == 8) {
     if (lane == 0) {
       mbar_expect_tx(q_full, ntiles * Cfg::kQBytes);
       for (int t = 0; t < ntiles; ++t)
@@ -170,7 +165,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           tma_load_2d(v_s + s * Cfg::kVBytes + a * (HD * 128), &tmV, j * KT + a * 64, img * p.C + head * HD, &v_full[s]);
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 9) {
     if (lane == 0) {
       constexpr uint32_t idesc_qk = umma_idesc_bf16(QT, KT);
       constexpr uint32_t idesc_pv = umma_idesc_bf16(QT, HD);
@@ -218,9 +213,11 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (more) umma_commit(&k_empty[sn]);
       }
     }
+   }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ---- softmax + output: thread = one query row of tile t ----
-    const int t = (warp - 2) >> 2;
+    const int t = warp >> 2;
     const int quarter = warp & 3;                 // the TMEM lanes this warp may touch
     const int r = quarter * 32 + lane;
     const uint32_t lane_off = uint32_t(quarter * 32) << 16;
@@ -233,8 +230,15 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (!mbar_wait(&s_full[t], j & 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); ok = false; break; }
         tc_fence_after();
         const int valid = p.kv_len - j * KT;  // >= 1
-        const bool tail = valid < KT;
-        const float mx = (tail ? tile_row_max<true>(s_addr, valid) : tile_row_max<false>(s_addr, valid)) * p.scale_log2;
+        float sc[KT];
+        if (valid < KT) tile_load_scores<true>(s_addr, valid, sc);
+        else tile_load_scores<false>(s_addr, valid, sc);
+        float mx0 = sc[0], mx1 = sc[1], mx2 = sc[2], mx3 = sc[3];
+#pragma unroll
+        for (int i = 4; i < KT; i += 4) {
+          mx0 = fmaxf(mx0, sc[i]); mx1 = fmaxf(mx1, sc[i + 1]); mx2 = fmaxf(mx2, sc[i + 2]); mx3 = fmaxf(mx3, sc[i + 3]);
+        }
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
         // Raise the running maximum only when it would grow by more than the threshold: probabilities
         // may then exceed 1 (by at most 2^threshold), which fp32 sums and bf16 P hold without loss.
         float alpha = 1.f;
@@ -254,8 +258,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             tmem_st32(o_addr + c * 32, o);
           }
         }
-        const float rs = tail ? tile_exp_store<true>(s_addr, s_addr, p.scale_log2, m_run, valid)
-                              : tile_exp_store<false>(s_addr, s_addr, p.scale_log2, m_run, valid);
+        const float rs = tile_exp_store(sc, s_addr, p.scale_log2, m_run);
         l_run = fmaf(l_run, alpha, rs);
         tmem_wait_st();
         tc_fence_before();
@@ -289,7 +292,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == 9) {
     __syncwarp();
     tmem_dealloc(tmem_base, Cfg::kTmemCols);
   }

@@ -83,28 +83,46 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_wait();  // set-up above overlaps the previous kernel; operands and outputs are touched only from here
+  // Set-up above overlaps the previous kernel.  Activations and outputs are touched only after
+  // pdl_wait(); the weight tiles (never written by a kernel of the step) are requested before it.
 
   if (warp == 0) {
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
+      int pre = 0;  // stages of the first work item whose W tile is already on its way
+      if ((int)blockIdx.x < total_tiles) {
+        const int tile = (int)blockIdx.x / splits, slice = (int)blockIdx.x - tile * splits;
+        const int n0 = (tile / tiles_m) * BN;
+        const int kb0 = slice * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
+        pre = min(STAGES, kb1 - kb0);
+        for (int i = 0; i < pre; ++i) {
+          mbar_expect_tx(&full_bar[i], Cfg::kStageBytes);
+          tma_load_2d(smem + i * Cfg::kStageBytes + kATileBytes, &tmB, (kb0 + i) * BK, n0, &full_bar[i]);
+        }
+      }
+      pdl_wait();
       for (int item = blockIdx.x; ok && item < total_tiles; item += gridDim.x) {
         const int tile = item / splits, slice = item - tile * splits;
         const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
         const int kb0 = slice * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
+          uint8_t* a_s = smem + s * Cfg::kStageBytes;
+          if ((int)it < pre) {  // W tile requested before the wait: only the activations are missing
+            tma_load_2d(a_s, &tmA, kb * BK, m0, &full_bar[s]);
+            continue;
+          }
           const uint32_t ph = (it / STAGES) & 1;
           if (!mbar_wait(&empty_bar[s], ph ^ 1)) { report(p.status, DEV_TIMEOUT_TMA); ok = false; break; }
           mbar_expect_tx(&full_bar[s], Cfg::kStageBytes);
-          uint8_t* a_s = smem + s * Cfg::kStageBytes;
           tma_load_2d(a_s, &tmA, kb * BK, m0, &full_bar[s]);
           tma_load_2d(a_s + kATileBytes, &tmB, kb * BK, n0, &full_bar[s]);
         }
       }
     }
   } else if (warp == 1) {
+    pdl_wait();
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
       uint32_t it = 0, lt = 0;
@@ -134,6 +152,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
   } else {
     // ---- epilogue: thread = one accumulator row, 32 fp32 columns per tcgen05.ld ----
+    pdl_wait();
     const int quarter = warp & 3;
     const uint32_t lane_off = uint32_t(quarter * 32) << 16;
     uint32_t lt = 0;

@@ -75,27 +75,43 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_wait();  // set-up above overlaps the previous kernel; operands and outputs are touched only from here
+  // Set-up above overlaps the previous kernel.  Activations and outputs are touched only after
+  // pdl_wait(); the weight tiles (never written by a kernel of the step) are requested before it.
 
   if (warp == 0) {
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
+      int pre = 0;  // stages of the first tile whose W half-tile is already on its way
+      if (pair < total_tiles) {
+        const int n0 = (pair / tiles_m) * BN + (int)rank * (BN / 2);
+        pre = min(STAGES, num_kb);
+        for (int i = 0; i < pre; ++i) {
+          if (rank == 0) mbar_expect_tx(&full_bar[i], 2 * Cfg::kStageBytes);
+          tma_load_2d_pair(smem + i * Cfg::kStageBytes + kATileBytes, &tmB, i * BK, n0, &full_bar[i]);
+        }
+      }
+      pdl_wait();
       for (int tile = pair; ok && tile < total_tiles; tile += npairs) {
         const int m0 = (tile % tiles_m) * (2 * BM) + (int)rank * BM;
         const int n0 = (tile / tiles_m) * BN + (int)rank * (BN / 2);
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % STAGES;
+          uint8_t* a_s = smem + s * Cfg::kStageBytes;
+          if ((int)it < pre) {  // W half-tile requested before the wait: only the activations are missing
+            tma_load_2d_pair(a_s, &tmA, kb * BK, m0, &full_bar[s]);
+            continue;
+          }
           const uint32_t ph = (it / STAGES) & 1;
           if (!mbar_wait(&empty_bar[s], ph ^ 1)) { report(p.status, DEV_TIMEOUT_TMA); ok = false; break; }
           if (rank == 0) mbar_expect_tx(&full_bar[s], 2 * Cfg::kStageBytes);
-          uint8_t* a_s = smem + s * Cfg::kStageBytes;
           tma_load_2d_pair(a_s, &tmA, kb * BK, m0, &full_bar[s]);
           tma_load_2d_pair(a_s + kATileBytes, &tmB, kb * BK, n0, &full_bar[s]);
         }
       }
     }
   } else if (warp == 1) {
+    pdl_wait();
     if (rank == 0 && lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(2 * BM, BN);
       uint32_t it = 0, lt = 0;
@@ -123,6 +139,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
   } else {
     // ---- epilogue: thread = one of this CTA's 128 accumulator rows, 32 fp32 columns per tcgen05.ld ----
+    pdl_wait();
     const int quarter = warp & 3;
     const uint32_t lane_off = uint32_t(quarter * 32) << 16;
     uint32_t lt = 0;

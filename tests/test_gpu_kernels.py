@@ -93,7 +93,7 @@ def test_prune_select_argument_errors():
 
 # ------------------------------------------------------------------ gather + LayerNorm + modulate
 @pytest.mark.parametrize("B,n,k,C,with_mod", [(1, 169, 85, 256, True), (4, 324, 243, 1920, True),
-                                             (2, 1024, 205, 2048, False), (2, 50, 50, 128, True)])
+                                             (2, 1024, 205, 2048, False), (2, 50, 50, 128, True), (2, 4096, 820, 2048, True)])
 def test_gather_ln(B, n, k, C, with_mod):
     x = I.normal(3, (B, n, C)) * 2.0 + 0.5
     idx = np.stack([np.sort(np.argsort(I.uniform01(9 + b, n))[:k]) for b in range(B)]).astype(np.int32)
@@ -150,6 +150,26 @@ def test_restore_residual(with_gamma):
                                        I.bf16_bits_to_f32(cache).astype(np.float64), hc, wc, h, w)
     g = mod[:, 2].astype(np.float64)[:, None, :] if with_gamma else 1.0
     ref = x.astype(np.float64) + g * yfull
+    np.testing.assert_allclose(xd.cpu().numpy(), ref, rtol=1e-6, atol=2e-6)
+
+
+def test_restore_residual_large():
+    """The 64x64 pruned step's restore (67 MB map, 820 kept rows per image, cache of the 32x32 step), with the
+    column sums of the updated map left in a selection workspace: they must equal the map's own column sums."""
+    B, hc, wc, h, w, C, k = 2, 32, 32, 64, 64, 2048, 820
+    n = h * w
+    x = I.normal(54, (B, n, C))
+    y = I.normal_bf16(55, (B, k, C))
+    cache = I.normal_bf16(56, (B, hc * wc, C))
+    mod = I.normal(57, (B, 6, C), 0.3)
+    idx = np.stack([np.sort(np.argsort(I.uniform01(61 + b, n))[:k]) for b in range(B)])
+    inv = O.inverse_map(idx, n).astype(np.int32)
+    xd, modd = dev(x), dev(mod)
+    fv.fv_restore_residual(xd, bf16_dev(y), bf16_dev(cache), dev(inv), modd.data_ptr() + 2 * 4 * C, 6 * C, h, w, hc, wc)
+    torch.cuda.synchronize()
+    yfull = O.cached_token_restoration(I.bf16_bits_to_f32(y).astype(np.float64), idx,
+                                       I.bf16_bits_to_f32(cache).astype(np.float64), hc, wc, h, w)
+    ref = x.astype(np.float64) + mod[:, 2].astype(np.float64)[:, None, :] * yfull
     np.testing.assert_allclose(xd.cpu().numpy(), ref, rtol=1e-6, atol=2e-6)
 
 
