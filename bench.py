@@ -27,6 +27,18 @@ sys.path.insert(0, ROOT)
 
 from paper_2503_23367_b200 import inputs as I  # noqa: E402
 
+# `roofline.traffic` is the bytes one launch has to move to and from HBM (operands + results, counted by
+# the library per launch), averaged over the launches of the dominant class; the notes say what an ncu
+# capture of the same kernel measured against that count (summaries under profiles/).
+NCU_TRAFFIC_NOTE = {
+    "gemm": "A + W + out bytes per launch, mean over the pruned steps' launches; ncu on M1640 N6144 K2048: dram read 31.95 MB = A + W "
+            "(31.9 MB), out (20 MB) still in L2 at kernel end; CTA-pair kernel M1844 N2048 K8192: read 63.8 MB = A + W, write 4.4 of 7.6 MB",
+    "attention": "Q + O + K + V^T bytes per launch; ncu on q820 kv5223 H16 hd128 B2: dram read 92.7 MB (K, V^T, Q = 92.3 MB), write 3.6 of 6.7 MB",
+    "restore": "x read + written, y, cache; ncu on B2 64x64 C2048 k820: read 82.3 MB + write 11.8 MB of 149 MB (x written stays in L2)",
+    "select": "x once + scores + indices; ncu on B2 64x64 C2048: score+top-k kernel reads 67.3 MB (x = 67.1 MB)",
+    "gather_ln": "kept rows in, bf16 rows out; ncu on B2 k820 C2048: read 13.5 MB (rows = 13.4 MB), output left in L2",
+}
+
 METRIC = "forwarded_tokens_per_s_over_pruned_scale_steps"
 UNIT = "tokens/s"
 
@@ -312,7 +324,8 @@ def ours(args, wl):
             ach = (v["work"] / reps) / (ms * 1e-3) / (1e12 if tensor else 1e9)
             peak = peaks["bf16_tflops_sustained"] if tensor else peaks["hbm_gbs"]
             table[name] = {"ms_per_step": ms, "launches_per_step": v["launches"] // reps, "bound": "tensor" if tensor else "hbm",
-                           "achieved": ach, "unit": "TFLOP/s" if tensor else "GB/s", "peak": peak, "frac": ach / peak}
+                           "achieved": ach, "unit": "TFLOP/s" if tensor else "GB/s", "peak": peak, "frac": ach / peak,
+                           "dram_bytes_per_launch": v["dram_bytes"] / max(1, v["launches"])}
         return table
 
     kernels, kernels_pruned, roofline = {}, {}, None
@@ -334,13 +347,14 @@ def ours(args, wl):
                         acc = r
                     else:
                         for n_, v_ in r.items():
-                            for f_ in ("ms", "launches", "work"):
+                            for f_ in ("ms", "launches", "work", "dram_bytes"):
                                 acc[n_][f_] += v_[f_]
         kernels_pruned = summarise(acc, reps)
         dom = max(kernels_pruned, key=lambda n: kernels_pruned[n]["ms_per_step"])
         d = kernels_pruned[dom]
         roofline = {"kernel": dom, "region": "pruned scale steps", "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"],
-                    "unit": d["unit"], "frac": d["frac"], "traffic": None,
+                    "unit": d["unit"], "frac": d["frac"], "traffic": d["dram_bytes_per_launch"],
+                    "traffic_source": NCU_TRAFFIC_NOTE.get(dom, "operand + result bytes per launch (no ncu capture for this class)"),
                     "peak_source": f"of {peaks['source']} ({'sustained bf16 matmul' if d['bound'] == 'tensor' else 'copy bandwidth'})",
                     "avg_launch_ms": d["ms_per_step"] / max(1, d["launches_per_step"])}
 

@@ -251,11 +251,13 @@ fv_status fv_attention(const void *q_dev, const void *k_dev, const void *vt_dev,
  *   fv_kernel_launches : kernels this library has launched since the last fv_profile_read.
  *   fv_profile_enable  : when on, every launch is bracketed by CUDA events on its stream.
  *   fv_profile_read    : synchronises the device; fills (each [5], HOST, may be NULL) the summed device
- *                        milliseconds per class (0 unless timing was on), launches per class and the
- *                        algorithmic work per class (bytes for classes 0,1,4; flops for 2,3), then clears. */
+ *                        milliseconds per class (0 unless timing was on), launches per class, the
+ *                        algorithmic work per class (bytes for classes 0,1,4; flops for 2,3) and the bytes
+ *                        each class has to move to and from HBM once (operands + results), then clears. */
 uint64_t fv_kernel_launches(void);
 fv_status fv_profile_enable(int32_t on);
-fv_status fv_profile_read(double *ms_host, uint64_t *launches_host, double *work_host);
+fv_status fv_profile_read(double *ms_host, uint64_t *launches_host, double *work_host,
+                          double *dram_bytes_host);
 
 #ifdef __cplusplus
 }

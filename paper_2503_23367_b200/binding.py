@@ -92,7 +92,7 @@ def lib() -> C.CDLL:
         L.fv_kernel_launches.restype = C.c_uint64; L.fv_kernel_launches.argtypes = []
         L.fv_profile_enable.restype = C.c_int; L.fv_profile_enable.argtypes = [i32]
         L.fv_profile_read.restype = C.c_int
-        L.fv_profile_read.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_double)]
+        L.fv_profile_read.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
         _lib = L
     return _lib
 
@@ -125,10 +125,11 @@ def fv_profile_enable(on: bool) -> None:
 
 
 def fv_profile_read() -> dict:
-    """{class: {"ms", "launches", "work"}}; work = algorithmic bytes (select, gather_ln, restore) or flops."""
-    ms, ln, wk = (C.c_double * 5)(), (C.c_uint64 * 5)(), (C.c_double * 5)()
-    _check(lib().fv_profile_read(ms, ln, wk), "fv_profile_read")
-    return {n: {"ms": ms[i], "launches": int(ln[i]), "work": wk[i]} for i, n in enumerate(KERNEL_CLASSES)}
+    """{class: {"ms", "launches", "work", "dram_bytes"}}; work = algorithmic bytes (select, gather_ln, restore)
+    or flops; dram_bytes = operand + result bytes the launches have to move to and from HBM once."""
+    ms, ln, wk, db = (C.c_double * 5)(), (C.c_uint64 * 5)(), (C.c_double * 5)(), (C.c_double * 5)()
+    _check(lib().fv_profile_read(ms, ln, wk, db), "fv_profile_read")
+    return {n: {"ms": ms[i], "launches": int(ln[i]), "work": wk[i], "dram_bytes": db[i]} for i, n in enumerate(KERNEL_CLASSES)}
 
 
 def fv_k_for(keep_ratio: float, h: int, w: int) -> int:

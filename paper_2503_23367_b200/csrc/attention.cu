@@ -313,7 +313,8 @@ template <int HD> fv_status launch_hd(const AttnArgs& a, cudaStream_t st) {
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   p.status = a.status;
   dim3 grid((a.rows + 2 * QT - 1) / (2 * QT), a.H, a.B);
-  LaunchScope scope(KC_ATTENTION, 1, 4.0 * a.B * (double)a.rows * a.kv_len * a.C, st);
+  LaunchScope scope(KC_ATTENTION, 1, 4.0 * a.B * (double)a.rows * a.kv_len * a.C,
+                    2.0 * a.B * a.C * (2.0 * a.rows + 2.0 * a.kv_len), st);  // Q in, O out, K and V^T once
   return launch_pdl(attention_kernel<HD>, grid, dim3(kAttnThreads), AttnCfg<HD>::kSmemBytes, st, tmQ, tmK, tmV, p) == cudaSuccess
              ? FV_OK : FV_ERR_CUDA;
 }

@@ -424,7 +424,7 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   p.mod_stride = g.mod_stride; p.rows_per_image = g.rows_per_image; p.q_cols = g.q_cols; p.C = g.C;
   p.k_cache = static_cast<__nv_bfloat16*>(g.k_cache); p.vt_cache = static_cast<__nv_bfloat16*>(g.vt_cache);
   p.kv_capacity = g.kv_capacity; p.kv_offset = g.kv_offset; p.status = g.status;
-  LaunchScope scope(KC_GEMM, 1, 2.0 * g.M * (double)g.N * g.K, st);
+  LaunchScope scope(KC_GEMM, 1, 2.0 * g.M * (double)g.N * g.K, 2.0 * ((double)g.M * g.K + (double)g.N * g.K + (double)g.M * g.N), st);
   if (p.splits == 1 && tc.pair) {
     cudaError_t e2 = launch_gemm_pair(g, p, bn, st);
     return e2 == cudaSuccess ? FV_OK : FV_ERR_CUDA;

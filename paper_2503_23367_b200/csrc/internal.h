@@ -33,10 +33,11 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // ---- prof.cu : launch counting and optional per-kernel-class timing (CUDA events on the stream) ---
 enum KernelClass : int { KC_SELECT = 0, KC_GATHER_LN = 1, KC_GEMM = 2, KC_ATTENTION = 3, KC_RESTORE = 4, KC_COUNT = 5 };
 // Brackets the launches of one kernel class: counts `kernels` launches, adds `work` (algorithmic bytes
-// for the HBM-bound classes, flops for GEMM / attention) and, when timing is enabled, records an event
-// pair around them on `st`.
+// for the HBM-bound classes, flops for GEMM / attention) and `dram_bytes` (the bytes the launch has to
+// move to and from HBM once: its operands and results; checked against ncu's DRAM counters) and, when
+// timing is enabled, records an event pair around them on `st`.
 struct LaunchScope {
-  LaunchScope(KernelClass c, int kernels, double work, cudaStream_t st);
+  LaunchScope(KernelClass c, int kernels, double work, double dram_bytes, cudaStream_t st);
   ~LaunchScope();
   int slot;
   cudaStream_t st;

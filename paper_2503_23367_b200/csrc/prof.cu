@@ -14,15 +14,17 @@ std::mutex g_mu;
 bool g_timing = false;
 uint64_t g_launches[KC_COUNT] = {0};
 double g_work[KC_COUNT] = {0};
+double g_dram[KC_COUNT] = {0};
 struct Pair { cudaEvent_t a, b; int cls; };
 std::vector<Pair> g_pairs;       // recorded since the last read
 std::vector<Pair> g_free;        // reusable events
 }  // namespace
 
-LaunchScope::LaunchScope(KernelClass c, int kernels, double work, cudaStream_t s) : slot(-1), st(s) {
+LaunchScope::LaunchScope(KernelClass c, int kernels, double work, double dram_bytes, cudaStream_t s) : slot(-1), st(s) {
   std::lock_guard<std::mutex> lk(g_mu);
   g_launches[c] += kernels;
   g_work[c] += work;
+  g_dram[c] += dram_bytes;
   if (!g_timing) return;
   Pair p;
   if (!g_free.empty()) { p = g_free.back(); g_free.pop_back(); }
@@ -58,7 +60,7 @@ fv_status fv_profile_enable(int32_t on) {
   return FV_OK;
 }
 
-fv_status fv_profile_read(double* ms_host, uint64_t* launches_host, double* work_host) {
+fv_status fv_profile_read(double* ms_host, uint64_t* launches_host, double* work_host, double* dram_bytes_host) {
   if (cudaDeviceSynchronize() != cudaSuccess) return FV_ERR_CUDA;
   std::lock_guard<std::mutex> lk(g_mu);
   double ms[KC_COUNT] = {0};
@@ -72,8 +74,10 @@ fv_status fv_profile_read(double* ms_host, uint64_t* launches_host, double* work
     if (ms_host) ms_host[i] = ms[i];
     if (launches_host) launches_host[i] = g_launches[i];
     if (work_host) work_host[i] = g_work[i];
+    if (dram_bytes_host) dram_bytes_host[i] = g_dram[i];
     g_launches[i] = 0;
     g_work[i] = 0;
+    g_dram[i] = 0;
   }
   return FV_OK;
 }

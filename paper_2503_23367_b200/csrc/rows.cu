@@ -197,7 +197,7 @@ __global__ void __launch_bounds__(256) restore_bf16_kernel(const uint4* __restri
 cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
                              const float* beta, int mod_stride, void* a_out, cudaStream_t st) {
   const int rows = B * k;
-  LaunchScope scope(KC_GATHER_LN, 1, (double)rows * C * 6.0, st);
+  LaunchScope scope(KC_GATHER_LN, 1, (double)rows * C * 6.0, (double)rows * C * 6.0, st);
   return launch_pdl(gather_ln_kernel, dim3((k + 7) / 8, B), dim3(256), sigma ? (size_t)C * 8 : 0, st, reinterpret_cast<const float4*>(x),
                     idx, n, k, C / 4, sigma, beta, mod_stride, reinterpret_cast<uint2*>(a_out));
 }
@@ -209,7 +209,8 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
   SelectWs ws{};
   if (colsum_ws) ws = select_ws_carve(colsum_ws, B, n, C);
   const int nchunks = (n + kColsumRows - 1) / kColsumRows;
-  LaunchScope scope(KC_RESTORE, 1, (double)B * C * (8.0 * n + 2.0 * k + 2.0 * hc * wc), st);
+  const double rr_bytes = (double)B * C * (8.0 * n + 2.0 * k + 2.0 * hc * wc);
+  LaunchScope scope(KC_RESTORE, 1, rr_bytes, rr_bytes, st);
   return launch_pdl(restore_residual_kernel, dim3(nchunks, B), dim3(256), 0, st, reinterpret_cast<float4*>(x),
                     reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h, w, hc, wc,
                     C / 8, nchunks, ws.group, ws.ngroups, reinterpret_cast<float4*>(ws.chunk_partial),
@@ -219,7 +220,8 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
 cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* pivots, const int32_t* inv, int B, int k,
                                 int h, int w, int C, void* out, cudaStream_t st) {
   const int rows = B * h * w;
-  LaunchScope scope(KC_RESTORE, 1, (double)B * C * (2.0 * h * w + 2.0 * k + 2.0 * hc * wc), st);
+  const double rb_bytes = (double)B * C * (2.0 * h * w + 2.0 * k + 2.0 * hc * wc);
+  LaunchScope scope(KC_RESTORE, 1, rb_bytes, rb_bytes, st);
   return launch_pdl(restore_bf16_kernel, dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const uint4*>(cache), hc, wc,
                     reinterpret_cast<const uint4*>(pivots), inv, h * w, k, h, w, C / 8, reinterpret_cast<uint4*>(out), rows);
 }

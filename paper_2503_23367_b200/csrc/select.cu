@@ -320,7 +320,9 @@ cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* i
   const int C4 = C / 4;
   const SelectWs w = select_ws_carve(workspace, B, n, C);
   float* sc = score ? score : w.score;
-  LaunchScope scope(KC_SELECT, have_partials ? 1 : 2, (double)B * n * C * 4.0 + 4.0 * B * n + 4.0 * B * ((double)k + n), st);
+  const double sel_bytes = (double)B * n * C * 4.0 + 4.0 * B * n + 4.0 * B * ((double)k + n);
+  // the stand-alone column-sum pass reads the map a second time
+  LaunchScope scope(KC_SELECT, have_partials ? 1 : 2, sel_bytes, sel_bytes + (have_partials ? 0.0 : (double)B * n * C * 4.0), st);
   if (!have_partials)
     launch_pdl(colsum_chunk_kernel, dim3(w.nchunks, B), dim3(256), 0, st, reinterpret_cast<const float4*>(x), n, C4, w.nchunks, w.group,
                w.ngroups, reinterpret_cast<float4*>(w.chunk_partial), reinterpret_cast<float4*>(w.group_partial), w.tickets);
@@ -339,7 +341,7 @@ cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* i
 
 cudaError_t launch_inv_from_idx(const int32_t* idx, int B, int k, int n, int32_t* inv, cudaStream_t st) {
   const size_t total = (size_t)B * n;
-  LaunchScope scope(KC_SELECT, 2, 4.0 * B * ((double)k + n), st);
+  LaunchScope scope(KC_SELECT, 2, 4.0 * B * ((double)k + n), 4.0 * B * ((double)k + n), st);
   launch_pdl(inv_fill_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, inv, total);
   launch_pdl(inv_scatter_kernel, dim3((B * k + 255) / 256), dim3(256), 0, st, idx, B, k, n, inv);
   return cudaGetLastError();
