@@ -91,6 +91,74 @@ def test_infinity_shape_cross_attention_forced_indices():
     check_forced(wl)
 
 
+def _bf16_t(bits):
+    return torch.from_numpy(bits.view(np.int16)).to(DEV).view(torch.bfloat16)
+
+
+def test_full_size_last_pruned_step_of_the_bench_workload():
+    """The 64x64 step of infinity_2b_1k at FULL width and batch (B 2, C 2048, 16 heads of 128, 512 text
+    tokens, keep 0.2 -> 820 kept rows per image, 4403 cached keys per image) -- the shapes and launch
+    configuration bench.py times -- on one transformer block (depth only repeats the same launches).
+    The KV prefix of the earlier scales and the sublayer caches are seeded bf16 values placed on both
+    sides.  Every output row is compared, not a sample: forced-index mode for the floating point, and
+    the first selection (identical input on both sides) for the indices."""
+    wl = I.WORKLOADS["infinity_2b_1k"].with_depth(1)
+    step = len(wl.sides) - 1
+    side = wl.sides[step]
+    kv_before = sum(O.kept_count(wl.keep[i], wl.sides[i], wl.sides[i]) if wl.keep[i] < 1 else wl.tokens(i) for i in range(step))
+    n_c = wl.tokens(wl.cache_step)
+    mt = I.model_tensors(wl)
+    x = I.step_input(wl, step, "structured")
+    kpre = I.normal_bf16(wl.seed + 900, (wl.B, kv_before, wl.C))
+    vpre = I.normal_bf16(wl.seed + 950, (wl.B, kv_before, wl.C))
+    caches = {name: I.normal_bf16(wl.seed + 990 + j, (wl.B, n_c, wl.C), 0.5) for j, name in enumerate(SUB_NAMES[wl.n_sub])}
+    widen = lambda bits: I.bf16_bits_to_f32(bits).astype(np.float64)
+    # ---- oracle
+    orc = make_oracle(wl, mt)
+    orc.step, orc.kv_len = step, kv_before
+    orc.Kc[0] = [widen(kpre[b]) for b in range(wl.B)]
+    orc.Vc[0] = [widen(vpre[b]) for b in range(wl.B)]
+    orc.cache[0] = {name: widen(c) for name, c in caches.items()}
+    tr = {}
+    ref = orc.var_step(x, step, wl.keep[step], trace=tr)
+    k = O.kept_count(wl.keep[step], side, side)
+    assert k == 820 and kv_before == 4403 and orc.kv_len == kv_before + k
+    # ---- CUDA path, oracle's indices forced
+    ctx = make_ctx(wl, mt)
+
+    def place_state():
+        kview, vview = ctx.kv_views(0)
+        kview[:, :kv_before].copy_(_bf16_t(kpre))
+        vview[:, :, :kv_before].copy_(_bf16_t(np.ascontiguousarray(vpre.transpose(0, 2, 1))))
+        for si, name in enumerate(SUB_NAMES[wl.n_sub]):
+            ctx.cache_view(0, si).copy_(_bf16_t(caches[name]))
+        ctx.set_state(step, kv_before)
+        ctx.prepare_text(wl.B)
+
+    place_state()
+    forced = torch.from_numpy(trace_to_index_tensor(wl, tr)).to(DEV)
+    xd = torch.from_numpy(x).to(DEV)
+    got = ctx.var_step(xd, step, wl.keep[step], forced_idx=forced).cpu().numpy()
+    assert ctx.device_status() == 0 and ctx.state() == (step + 1, kv_before + k)
+    err, cos = per_token_errors(got, ref)
+    assert err <= MAX_ABS and cos >= MIN_COS, (err, cos)
+    # rows that were not forwarded anywhere in the block only ever received restored cache rows
+    # ---- free running: the first selection sees the same x on both sides
+    place_state()
+    trace = torch.zeros((wl.L, wl.n_sub, wl.B, k), dtype=torch.int32, device=DEV)
+    ctx.var_step(xd, step, wl.keep[step], idx_trace=trace)
+    assert ctx.device_status() == 0
+    idx_g = trace[0, 0].cpu().numpy().astype(np.int64)
+    idx_o, s_o = tr[(0, "attn")]["idx"], tr[(0, "attn")]["score"]
+    for b in range(wl.B):
+        assert np.all(np.diff(idx_g[b]) > 0)
+        diff = np.setxor1d(idx_g[b], idx_o[b])
+        if len(diff):
+            tau = np.sort(s_o[b])[::-1][k - 1]
+            assert np.all(np.abs(s_o[b, diff] - tau) <= 1e-5 * tau), "index mismatch away from a near-tie"
+    ctx.close()
+
+
 def test_free_running_selection_matches_oracle_on_identical_input():
     wl = I.WORKLOADS["tiny"]
     mt = I.model_tensors(wl)
