@@ -26,6 +26,14 @@ Readings taken where the paper is silent or inconsistent (each is also listed in
     1/sqrt(head_dim), biases on qkv / out / fc1 / fc2, optional cross-attention to text with plain
     LN, no biases and no gate.
 
+Granularity.  The paper wraps EVERY attention / FFN layer with the selection / restoration pair
+(Sec. 3.3 "Implementation"); that is `granularity="sublayer"`, the default.  `granularity="step"` is the
+coarser variant in which the pair wraps the whole stack of blocks of a scale step: one selection on the
+step's input token map, all blocks run on the kept rows only (their residual stream stays compact), and
+one restoration from the cached OUTPUT token map of step K-N.  It is a different approximation (its
+unkept tokens take the previous scale's output, interpolated, instead of accumulating cached layer
+outputs); it is not the paper's configuration and is pinned only by its own invariants.
+
 Parity pins: every function here is pinned by tests/test_oracle_pins.py (closed forms, brute force,
 invariants, library special cases).  The end-to-end activation values of a whole step have no
 printed example in the paper: "parity unpinned" for `VarOracle.var_step` as a whole beyond the
@@ -201,7 +209,9 @@ class VarOracle:
     """
 
     def __init__(self, L: int, C: int, H: int, sides_hw: Sequence[Sequence[int]], cache_step: int,
-                 weights: Dict, B: int, cross_len: int = 0):
+                 weights: Dict, B: int, cross_len: int = 0, granularity: str = "sublayer"):
+        assert granularity in ("sublayer", "step")
+        self.granularity = granularity
         self.L, self.C, self.H, self.B = L, C, H, B
         self.hw = [tuple(s) for s in sides_hw]
         self.cache_step = cache_step
@@ -216,6 +226,7 @@ class VarOracle:
         self.Kc = [[np.zeros((0, self.C)) for _ in range(self.B)] for _ in range(self.L)]
         self.Vc = [[np.zeros((0, self.C)) for _ in range(self.B)] for _ in range(self.L)]
         self.cache: List[Dict[str, np.ndarray]] = [dict() for _ in range(self.L)]
+        self.step_cache: Optional[np.ndarray] = None   # granularity "step": output token map of step K-N
 
     # -- one wrapped sublayer on compact rows ---------------------------------------------------
     def _branch(self, l: int, sub: str, xp: np.ndarray) -> np.ndarray:
@@ -263,6 +274,8 @@ class VarOracle:
         assert n == h * w_ and B == self.B and C == self.C
         pruned = keep_ratio < 1.0
         k = kept_count(keep_ratio, h, w_) if pruned else n
+        if self.granularity == "step":
+            return self._var_step_whole(x, scale_idx, pruned, k, forced_idx, trace)
         for l in range(self.L):
             mod = np.asarray(self.w["mod"][l], dtype=F64)
             for sub in self.subs:
@@ -297,6 +310,42 @@ class VarOracle:
         self.kv_len += k
         self.step += 1
         return x
+
+    def _var_step_whole(self, x: np.ndarray, scale_idx: int, pruned: bool, k: int,
+                        forced_idx: Optional[Dict], trace: Optional[Dict]) -> np.ndarray:
+        """granularity "step": PTS once on the step input, all blocks on the kept rows (compact residual
+        stream), CTR once from the cached output map of the caching step.  `forced_idx[("step",)]`
+        overrides the selection; `trace[("step",)]` receives idx / score."""
+        h, w_ = self.hw[scale_idx]
+        idx, score = None, None
+        xc = x
+        if pruned:
+            score = pts_score(x)
+            idx = np.asarray(forced_idx[("step",)], dtype=np.int64) if forced_idx is not None else pts_topk(score, k)
+            xc = pts_gather(x, idx)
+        if trace is not None:
+            trace[("step",)] = {"idx": idx, "score": score}
+        for l in range(self.L):
+            mod = np.asarray(self.w["mod"][l], dtype=F64)
+            for sub in self.subs:
+                y = self._branch(l, sub, xc)
+                if sub == "attn":
+                    xc = xc + mod[:, 2][:, None, :] * y
+                elif sub == "ffn":
+                    xc = xc + mod[:, 5][:, None, :] * y
+                else:
+                    xc = xc + y
+        if scale_idx == self.cache_step:
+            assert not pruned, "the caching step is the last unpruned step"
+            self.step_cache = xc.copy()
+        if pruned:
+            hc, wc = self.hw[self.cache_step]
+            out = cached_token_restoration(xc, idx, self.step_cache, hc, wc, h, w_)
+        else:
+            out = xc
+        self.kv_len += k
+        self.step += 1
+        return out
 
     def run_schedule(self, inputs: Sequence[np.ndarray], keep: Sequence[float]) -> List[np.ndarray]:
         """All steps 0..K-1 in order; inputs[k] is the token map entering step k."""

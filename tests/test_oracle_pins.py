@@ -322,9 +322,9 @@ def test_unpruned_schedule_equals_block_causal_sequence_forward(cross_len):
     assert orc.kv_len == sum(s * s for s in wl.sides)
 
 
-def _run(wl, w, xs, keep, cache_step, **kw):
+def _run(wl, w, xs, keep, cache_step, granularity="sublayer", **kw):
     orc = O.VarOracle(wl.L, wl.C, wl.H, [(s, s) for s in wl.sides], cache_step=cache_step, weights=w,
-                      B=wl.B, cross_len=wl.cross_len)
+                      B=wl.B, cross_len=wl.cross_len, granularity=granularity)
     outs, traces = [], []
     for i, x in enumerate(xs):
         tr = {}
@@ -396,6 +396,63 @@ def test_images_are_independent():
     wl1 = I.Workload("t1", L=1, C=wl.C, H=wl.H, B=1, sides=wl.sides, keep=wl.keep, seed=wl.seed)
     w1 = dict(w); w1["mod"] = w["mod"][:, 1:2]
     _, one, _ = _run(wl1, w1, [x[1:2] for x in xs], keep, cache_step=2)
+    np.testing.assert_allclose(both[4][1:2], one[4], rtol=1e-12, atol=1e-13)
+
+
+# ------------------------------------------------------------------ per-step granularity (the coarser variant)
+@pytest.mark.parametrize("cross_len", [0, 4])
+def test_step_granularity_unpruned_and_keep_all_equal_the_unpruned_forward(cross_len):
+    wl, mt, w = _tiny_model(cross_len=cross_len)
+    xs = [I.step_input(wl, s) for s in range(len(wl.sides))]
+    _, ref, _ = _run(wl, w, xs, [1.0] * 5, cache_step=2)                      # paper granularity, unpruned
+    _, got, _ = _run(wl, w, xs, [1.0] * 5, cache_step=2, granularity="step")
+    for a, b in zip(got, ref):
+        np.testing.assert_array_equal(a, b)                                   # no pruning: the same arithmetic
+    almost = 1.0 - 1e-7                                                       # PTS / CTR run, k = n
+    _, got, tr = _run(wl, w, xs, [1.0, 1.0, 1.0, almost, almost], cache_step=2, granularity="step")
+    for a, b in zip(got, ref):
+        np.testing.assert_allclose(a, b, rtol=1e-11, atol=1e-12)
+    assert (tr[4][("step",)]["idx"] == np.arange(36)).all()
+
+
+def test_step_granularity_pivot_rows_and_restored_rows():
+    """Kept rows: the blocks only ever see the compact rows, so with the SAME index set forced on every
+    sublayer the paper-granularity oracle must give the same values on those rows.  Other rows: exactly
+    the cached output map of step K-N, nearest-upsampled.  KV cache: k rows per pruned step."""
+    wl, mt, w = _tiny_model(L=2, cross_len=3)
+    xs = [I.step_input(wl, s) for s in range(len(wl.sides))]
+    keep = [1.0, 1.0, 1.0, 0.5, 0.25]
+    orc, outs, tr = _run(wl, w, xs, keep, cache_step=2, granularity="step")
+    assert orc.kv_len == 1 + 4 + 9 + 8 + 9
+    np.testing.assert_array_equal(orc.step_cache, outs[2])                    # the cache is step 2's output map
+    h, hc = wl.sides[4], wl.sides[2]
+    src = O.nearest_source(h, h, hc, hc)
+    idx = tr[4][("step",)]["idx"]
+    assert idx.shape == (wl.B, 9) and (np.diff(idx, axis=1) > 0).all()
+    np.testing.assert_array_equal(idx, O.pts_topk(O.pts_score(xs[4]), 9))     # selected on the step input
+    for b in range(wl.B):
+        rest = np.setdiff1d(np.arange(h * h), idx[b])
+        np.testing.assert_array_equal(outs[4][b, rest], outs[2][b, src[rest]])
+    # same sets forced on every sublayer of the paper-granularity oracle, steps 3 and 4
+    forced3 = {(l, s): tr[3][("step",)]["idx"] for l in range(wl.L) for s in ("attn", "xattn", "ffn")}
+    forced4 = {(l, s): idx for l in range(wl.L) for s in ("attn", "xattn", "ffn")}
+    ref = O.VarOracle(wl.L, wl.C, wl.H, [(s, s) for s in wl.sides], cache_step=2, weights=w, B=wl.B, cross_len=wl.cross_len)
+    for i in range(3):
+        ref.var_step(xs[i], i, 1.0)
+    ref.var_step(xs[3], 3, keep[3], forced_idx=forced3)
+    out4 = ref.var_step(xs[4], 4, keep[4], forced_idx=forced4)
+    for b in range(wl.B):
+        np.testing.assert_allclose(outs[4][b, idx[b]], out4[b, idx[b]], rtol=1e-11, atol=1e-12)
+
+
+def test_step_granularity_images_are_independent():
+    wl, mt, w = _tiny_model(L=1, B=2)
+    xs = [I.step_input(wl, s) for s in range(len(wl.sides))]
+    keep = [1.0, 1.0, 1.0, 0.5, 0.5]
+    _, both, _ = _run(wl, w, xs, keep, cache_step=2, granularity="step")
+    wl1 = I.Workload("t1", L=1, C=wl.C, H=wl.H, B=1, sides=wl.sides, keep=wl.keep, seed=wl.seed)
+    w1 = dict(w); w1["mod"] = w["mod"][:, 1:2]
+    _, one, _ = _run(wl1, w1, [x[1:2] for x in xs], keep, cache_step=2, granularity="step")
     np.testing.assert_allclose(both[4][1:2], one[4], rtol=1e-12, atol=1e-13)
 
 
