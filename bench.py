@@ -358,12 +358,37 @@ def ours(args, wl):
                     "peak_source": f"of {peaks['source']} ({'sustained bf16 matmul' if d['bound'] == 'tensor' else 'copy bandwidth'})",
                     "avg_launch_ms": d["ms_per_step"] / max(1, d["launches_per_step"])}
 
+    # ---- the coarser granularity beside it: one selection and one restoration around the whole stack of
+    # blocks of a pruned step (not the paper's configuration, which is what `value` measures)
+    variant = None
+    ctx.close()
+    del ctx
+    torch.cuda.empty_cache()
+    if not args.skip_variant:
+        ctx_step = fv.FvContext(wl.L, wl.C, wl.H, hw, wl.cache_step, wl.B, cap, gt, cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio,
+                                device=dev, granularity=1)
+        for _ in range(3):
+            schedule(ctx_step, wl.keep)
+        barrier()
+        nv = max(2, min(args.steps, 5))
+        evv = [[torch.cuda.Event(enable_timing=True) for _ in range(S + 1)] for _ in range(nv)]
+        for k in range(nv):
+            schedule(ctx_step, wl.keep, evv[k])
+        barrier()
+        if ctx_step.device_status() != 0:
+            raise SystemExit("a kernel reported an expired wait")
+        v_total = max_over_ranks(statistics.mean(evv[k][0].elapsed_time(evv[k][S]) for k in range(nv)))
+        v_pruned = max_over_ranks(sum(statistics.mean(evv[k][i].elapsed_time(evv[k][i + 1]) for k in range(nv)) for i in pruned_steps))
+        variant = {"what": "selection and restoration once per scale step around all blocks (granularity 1), not the paper's per-layer wrapping",
+                   "value": world * fwd_tokens / (v_pruned * 1e-3), "unit": UNIT, "ms_per_step": v_total, "ms_per_image": v_total / wl.B,
+                   "ms_pruned_steps": v_pruned}
+        ctx_step.close()
+        del ctx_step
+        torch.cuda.empty_cache()
+
     # ---- the unpruned GPU step beside it (same kernels, keep_ratio = 1 everywhere)
     unpruned = None
     if not args.skip_unpruned:
-        ctx.close()
-        del ctx
-        torch.cuda.empty_cache()
         cap_full = sum(wl.tokens(i) for i in range(S))
         ctx_full = fv.FvContext(wl.L, wl.C, wl.H, hw, wl.cache_step, wl.B, cap_full, gt, cross_len=wl.cross_len,
                                 mlp_ratio=wl.mlp_ratio, device=dev)
@@ -400,7 +425,7 @@ def ours(args, wl):
             "ms_per_image": ms_per_step / wl.B, "ms_per_image_pruned_steps": pruned_ms / wl.B,
             "scale_step_ms": [round(t, 4) for t in step_ms], "wall_ms_per_step": t_wall * 1e3 / args.steps,
             "roofline": roofline, "kernels": kernels, "kernels_pruned_steps": kernels_pruned, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": gpu_launches,
-            "clocks": clocks, "unpruned_gpu": unpruned, "peaks": peaks}
+            "clocks": clocks, "unpruned_gpu": unpruned, "per_step_granularity": variant, "peaks": peaks}
     print(json.dumps(line))
 
 
@@ -415,6 +440,7 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer end-to-end leg")
     ap.add_argument("--skip-profile", action="store_true", help="omit the per-kernel-class timing passes")
     ap.add_argument("--skip-unpruned", action="store_true", help="omit the unpruned GPU comparison")
+    ap.add_argument("--skip-variant", action="store_true", help="omit the per-step-granularity comparison")
     ap.add_argument("--blocks", type=int, default=0,
                     help="profiling only: run this many transformer blocks instead of the workload's depth (the line says so; not a bench number)")
     args = ap.parse_args()

@@ -131,6 +131,8 @@ typedef struct {
   const int32_t *w;
   int32_t cache_step; /* 0-based index of step K-N, the last unpruned step; -1 = never cache       */
   int32_t kv_capacity;/* KV rows per image per block the caller provides room for; % 8 == 0        */
+  int32_t granularity;/* 0: selection / restoration around every attention and FFN layer (the paper).
+                         1: around the whole stack of blocks of a scale step (see fv_var_step)          */
 } fv_config;
 
 typedef struct { /* HOST arrays of length L holding DEVICE pointers; bf16 unless noted; borrowed   */
@@ -185,6 +187,12 @@ fv_status fv_device_status(fv_ctx *ctx, int32_t *code_host, void *stream);
  *               instead of selecting -- separates index parity from floating-point parity in tests.
  *   idx_trace_dev  NULL, or int32 [L, n_sub, B, k]: receives the kept indices of every sublayer.
  * n_sub = 3 with cross-attention else 2; sublayer order: self-attention, [cross-attention], FFN.
+ *
+ * granularity 1 (not the paper's configuration; the coarser reading "select once per scale step"): at a
+ * pruned step PTS runs once on tokens_dev, the kept rows are gathered into a compact fp32 residual stream,
+ * all L blocks run on those rows only (each block appends their K/V), and one CTR builds out_dev from the
+ * compact result and the cached OUTPUT map of step cache_step (fp32 [B_max, n_cache, C]; that is what the
+ * cache buffer then holds, fv_cache_pointer(ctx, 0, 0)).  forced_idx_dev / idx_trace_dev are int32 [B, k].
  * Errors: INVALID_ARG, BAD_STATE (wrong scale_idx; pruned step before the cache step),
  *         CAPACITY (kv_len + k > kv_capacity), CUDA. */
 fv_status fv_var_step(fv_ctx *ctx, const float *tokens_dev, int32_t B, int32_t scale_idx,

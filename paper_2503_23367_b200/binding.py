@@ -37,7 +37,7 @@ class fv_config(C.Structure):
     _fields_ = [("L", C.c_int32), ("C", C.c_int32), ("H", C.c_int32), ("mlp_ratio", C.c_int32),
                 ("cross_len", C.c_int32), ("B_max", C.c_int32), ("n_steps", C.c_int32),
                 ("h", C.POINTER(C.c_int32)), ("w", C.POINTER(C.c_int32)),
-                ("cache_step", C.c_int32), ("kv_capacity", C.c_int32)]
+                ("cache_step", C.c_int32), ("kv_capacity", C.c_int32), ("granularity", C.c_int32)]
 
 
 class fv_weights(C.Structure):
@@ -234,7 +234,7 @@ class FvContext:
     (`inputs.ModelTensors`) or as torch bf16 CUDA tensors with the same field names."""
 
     def __init__(self, L: int, Cw: int, H: int, sides_hw: Sequence[Sequence[int]], cache_step: int, B_max: int,
-                 kv_capacity: int, tensors, cross_len: int = 0, mlp_ratio: int = 4, device="cuda:0"):
+                 kv_capacity: int, tensors, cross_len: int = 0, mlp_ratio: int = 4, device="cuda:0", granularity: int = 0):
         self.dev = torch.device(device)
         self.L, self.C, self.H, self.B_max, self.cross_len = L, Cw, H, B_max, cross_len
         self.n_sub = 3 if cross_len else 2
@@ -242,8 +242,9 @@ class FvContext:
         self.kv_capacity = (kv_capacity + 7) // 8 * 8
         self._h = (C.c_int32 * len(self.hw))(*[s[0] for s in self.hw])
         self._w = (C.c_int32 * len(self.hw))(*[s[1] for s in self.hw])
+        self.granularity = granularity
         self.cfg = fv_config(L, Cw, H, mlp_ratio, cross_len, B_max, len(self.hw), self._h, self._w, cache_step,
-                             self.kv_capacity)
+                             self.kv_capacity, granularity)
         self._keep: List[torch.Tensor] = []
 
         def dev_bf16(a):
@@ -331,6 +332,8 @@ class FvContext:
         B = B or self.B_max
         nel = B * hc * wc * self.C
         off = p.value - self.cache.data_ptr()
+        if self.granularity == 1:      # the step-level cache: fp32 output map of the caching step
+            return self.cache[off: off + 4 * nel].view(torch.float32).view(B, hc * wc, self.C)
         return self.cache[off: off + 2 * nel].view(torch.bfloat16).view(B, hc * wc, self.C)
 
     def var_step(self, tokens: torch.Tensor, scale_idx: int, keep_ratio: float, out: Optional[torch.Tensor] = None,

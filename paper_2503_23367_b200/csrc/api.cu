@@ -31,6 +31,7 @@ struct fv_ctx {
   int32_t *idx = nullptr, *inv = nullptr;
   void* sel_ws = nullptr;
   void* splitk_ws = nullptr;
+  float* xc = nullptr;  // granularity 1: compact fp32 residual stream of a pruned step [B*k, C]
   size_t kv_block_bytes = 0, k_bytes = 0, text_k_bytes = 0, text_block_bytes = 0, cache_sub_bytes = 0;
 };
 
@@ -51,7 +52,7 @@ cudaError_t ensure_init() {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 struct Layout {
-  size_t status, a, q, o, y, hbuf, idx, inv, sel, splitk, total;
+  size_t status, a, q, o, y, hbuf, idx, inv, sel, splitk, xc, total;
 };
 
 int max_tokens(const fv_config* c) {
@@ -66,6 +67,7 @@ bool config_ok(const fv_config* c) {
   for (int i = 0; i < c->n_steps; ++i)
     if (c->h[i] <= 0 || c->w[i] <= 0) return false;
   if (c->cache_step >= c->n_steps) return false;
+  if (c->granularity != 0 && c->granularity != 1) return false;
   return true;
 }
 
@@ -85,6 +87,7 @@ Layout workspace_layout(const fv_config* c) {
   l.inv = take(M * 4);
   l.sel = take(select_workspace_bytes(c->B_max, max_tokens(c), c->C));
   l.splitk = take(gemm_splitk_ws_bytes());
+  l.xc = take(c->granularity == 1 ? M * C * 4 : 0);
   l.total = off;
   return l;
 }
@@ -217,6 +220,7 @@ size_t fv_kv_bytes(const fv_config* cfg) {
 size_t fv_cache_bytes(const fv_config* cfg) {
   if (!config_ok(cfg) || cfg->cache_step < 0) return 0;
   const size_t n_cache = (size_t)cfg->h[cfg->cache_step] * cfg->w[cfg->cache_step];
+  if (cfg->granularity == 1) return align_up((size_t)cfg->B_max * n_cache * cfg->C * 4, 1024);  // fp32 output map of the caching step
   const int n_sub = cfg->cross_len ? 3 : 2;
   return (size_t)cfg->L * n_sub * align_up((size_t)cfg->B_max * n_cache * cfg->C * 2, 1024);
 }
@@ -276,6 +280,7 @@ fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, v
   c->inv = reinterpret_cast<int32_t*>(c->ws + lay.inv);
   c->sel_ws = c->ws + lay.sel;
   c->splitk_ws = c->ws + lay.splitk;
+  c->xc = reinterpret_cast<float*>(c->ws + lay.xc);
   // Never-written KV rows must read as zeros (they meet zero probabilities in P*V).
   if (cudaMemset(kv_dev, 0, fv_kv_bytes(cfg)) != cudaSuccess || cudaMemset(c->status, 0, 256) != cudaSuccess ||
       cudaMemset(c->sel_ws, 0, select_ticket_bytes(cfg->B_max)) != cudaSuccess ||
@@ -321,6 +326,11 @@ fv_status fv_kv_pointers(const fv_ctx* ctx, int32_t block, void** k_dev, void** 
 
 fv_status fv_cache_pointer(const fv_ctx* ctx, int32_t block, int32_t sublayer, void** cache_dev) {
   if (!ctx || !cache_dev || block < 0 || block >= ctx->cfg.L || sublayer < 0 || sublayer >= ctx->n_sub || !ctx->cache) return FV_ERR_INVALID_ARG;
+  if (ctx->cfg.granularity == 1) {  // one step-level cache
+    if (block != 0 || sublayer != 0) return FV_ERR_INVALID_ARG;
+    *cache_dev = ctx->cache;
+    return FV_OK;
+  }
   *cache_dev = ctx->cache + ((size_t)block * ctx->n_sub + sublayer) * ctx->cache_sub_bytes;
   return FV_OK;
 }
@@ -376,7 +386,8 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   if (c.cross_len && scale_idx > 0 && !ctx->text_ready) return FV_ERR_BAD_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   float* x = out_dev;
-  if (out_dev != tokens_dev &&
+  // (per-step granularity, pruned step: the output map is written whole by the final restoration)
+  if (out_dev != tokens_dev && !(pruned && c.granularity == 1) &&
       cudaMemcpyAsync(out_dev, tokens_dev, (size_t)B * n * C * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
     return FV_ERR_CUDA;
   if (c.cross_len && scale_idx == 0) {
@@ -388,10 +399,31 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   const int mod_stride = 6 * C;
   fv_status s = FV_OK;
   cudaError_t e = cudaSuccess;
+  const bool whole_step = c.granularity == 1;
+  // Per sublayer (the paper): every sublayer selects from the full map x and restores into it.
+  // Per step: one selection here, the blocks then run on the compact rows xr = ctx->xc as if unpruned.
+  const bool sub_pruned = pruned && !whole_step;
+  float* xr = x;        // residual stream the blocks update
+  int nr = n;           // its rows per image
+  if (pruned && whole_step) {
+    const int32_t* idx = forced_idx_dev;
+    if (forced_idx_dev) {
+      e = launch_inv_from_idx(forced_idx_dev, B, k, n, ctx->inv, st);
+    } else {
+      idx = ctx->idx;
+      if (cudaMemsetAsync(ctx->sel_ws, 0, select_ticket_bytes(B), st) != cudaSuccess) return FV_ERR_CUDA;
+      e = launch_select(tokens_dev, B, n, C, k, ctx->idx, ctx->inv, nullptr, nullptr, ctx->sel_ws, false, st);
+    }
+    if (e != cudaSuccess) return FV_ERR_CUDA;
+    if (idx_trace_dev && cudaMemcpyAsync(idx_trace_dev, idx, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return FV_ERR_CUDA;
+    if (launch_gather_rows(tokens_dev, idx, B, n, k, C, ctx->xc, st) != cudaSuccess) return FV_ERR_CUDA;
+    xr = ctx->xc;
+    nr = k;
+  }
   // Column sums of x (Eq. 4) for the next selection are left in the selection scratch by the restore
   // kernel of the sublayer before it; only the first sublayer of a step has to sum the map itself.
   bool have_partials = false;
-  const bool selecting = pruned && !forced_idx_dev;
+  const bool selecting = sub_pruned && !forced_idx_dev;
   if (selecting && cudaMemsetAsync(ctx->sel_ws, 0, select_ticket_bytes(B), st) != cudaSuccess) return FV_ERR_CUDA;
 
   for (int l = 0; l < c.L && s == FV_OK; ++l) {
@@ -399,11 +431,11 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
     char* kbase = ctx->kv + (size_t)l * ctx->kv_block_bytes;
     for (int sub = 0; sub < ctx->n_sub && s == FV_OK; ++sub) {
       const int kind = (ctx->n_sub == 3) ? sub : (sub == 0 ? 0 : 2);  // 0 self-attention, 1 cross-attention, 2 FFN
-      char* cache_sub = ctx->cache ? ctx->cache + ((size_t)l * ctx->n_sub + sub) * ctx->cache_sub_bytes : nullptr;
+      char* cache_sub = (ctx->cache && !whole_step) ? ctx->cache + ((size_t)l * ctx->n_sub + sub) * ctx->cache_sub_bytes : nullptr;
       const size_t trace_off = ((size_t)l * ctx->n_sub + sub) * (size_t)B * k;
       // ---- Pivotal Token Selection
       const int32_t* idx = nullptr;
-      if (pruned) {
+      if (sub_pruned) {
         if (forced_idx_dev) {
           idx = forced_idx_dev + trace_off;
           e = launch_inv_from_idx(idx, B, k, n, ctx->inv, st);
@@ -420,7 +452,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
       const float* sigma = kind == 0 ? mod : (kind == 2 ? mod + 3 * C : nullptr);
       const float* beta = kind == 0 ? mod + C : (kind == 2 ? mod + 4 * C : nullptr);
       const float* gamma = kind == 0 ? mod + 2 * C : (kind == 2 ? mod + 5 * C : nullptr);
-      e = launch_gather_ln(x, idx, B, n, k, C, sigma, beta, mod_stride, ctx->a_buf, st);
+      e = launch_gather_ln(xr, idx, B, nr, k, C, sigma, beta, mod_stride, ctx->a_buf, st);
       if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
       // ---- branch on the compact rows
       GemmArgs g{};
@@ -459,7 +491,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
       GemmArgs o{};
       o.status = ctx->status; o.rows_per_image = k; o.mod_stride = mod_stride; o.splitk_ws = ctx->splitk_ws;
       o.a = last_in; o.w = last_w; o.bias = last_b; o.M = M; o.N = C; o.K = last_K;
-      if (pruned) {
+      if (sub_pruned) {
         o.epilogue = EPI_BF16; o.out = ctx->y_buf;
         s = launch_gemm(o, st);
         if (s != FV_OK) break;
@@ -469,11 +501,20 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
         have_partials = more;
       } else {
-        o.epilogue = EPI_RESIDUAL; o.out = x; o.gamma = gamma; o.aux = write_cache ? cache_sub : nullptr;
+        o.epilogue = EPI_RESIDUAL; o.out = xr; o.gamma = gamma; o.aux = (write_cache && !whole_step) ? cache_sub : nullptr;
         s = launch_gemm(o, st);
         if (s != FV_OK) break;
       }
     }
+  }
+  if (s != FV_OK) return s;
+  if (whole_step) {
+    if (write_cache &&
+        cudaMemcpyAsync(ctx->cache, x, (size_t)B * n * C * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return FV_ERR_CUDA;  // the step-level cache: this step's output map (image stride n*C == n_cache*C here)
+    if (pruned && launch_restore_rows_f32(reinterpret_cast<const float*>(ctx->cache), hc, wc, ctx->xc, ctx->inv, B, k, h, w, C,
+                                          out_dev, st) != cudaSuccess)
+      return FV_ERR_CUDA;
   }
   if (s != FV_OK) return s;
   ctx->kv_len += k;

@@ -75,6 +75,10 @@ cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, i
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv,
                                     const float* gamma, int mod_stride, int B, int k, int h, int w, int hc, int wc,
                                     int C, void* colsum_ws, cudaStream_t st);
+// Per-step granularity: fp32 gather of the kept rows, and fp32 restoration of the step's output map.
+cudaError_t launch_gather_rows(const float* x, const int32_t* idx, int B, int n, int k, int C, float* out, cudaStream_t st);
+cudaError_t launch_restore_rows_f32(const float* cache, int hc, int wc, const float* pivots, const int32_t* inv, int B, int k,
+                                    int h, int w, int C, float* out, cudaStream_t st);
 cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* pivots, const int32_t* inv, int B,
                                 int k, int h, int w, int C, void* out, cudaStream_t st);
 

@@ -192,6 +192,39 @@ __global__ void __launch_bounds__(256) restore_bf16_kernel(const uint4* __restri
   for (int c8 = lane; c8 < C8; c8 += 32) dst[c8] = __ldg(src + c8);
 }
 
+// Per-step granularity: compact copy of the kept rows of the fp32 token map (Algorithm 1's gather).
+// grid (ceil(k / 8), B): one warp per kept row.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const float4* __restrict__ x, const int32_t* __restrict__ idx, int n,
+                                                          int k, int C4, float4* __restrict__ out) {
+  pdl_trigger();
+  pdl_wait();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.y, j = blockIdx.x * 8 + warp;
+  if (j >= k) return;
+  const int t = __ldg(idx + (size_t)b * k + j);
+  const float4* src = x + ((size_t)b * n + t) * C4;
+  float4* dst = out + ((size_t)b * k + j) * C4;
+  for (int c4 = lane; c4 < C4; c4 += 32) dst[c4] = __ldg(src + c4);
+}
+
+// Per-step granularity: Cached Token Restoration of the step's output map (Eq. 6), fp32, a copy:
+// out[b,t,:] = inv[b,t] >= 0 ? pivots[b, inv[b,t], :] : cache[b, src(t), :].
+__global__ void __launch_bounds__(256) restore_rows_f32_kernel(const float4* __restrict__ cache, int hc, int wc,
+                                                               const float4* __restrict__ pivots, const int32_t* __restrict__ inv,
+                                                               int n, int k, int h, int w, int C4, float4* __restrict__ out,
+                                                               int total_rows) {
+  pdl_trigger();
+  pdl_wait();
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= total_rows) return;
+  const int b = warp / n, t = warp - b * n;
+  const int j = __ldg(inv + warp);
+  const float4* src = (j >= 0) ? pivots + ((size_t)b * k + j) * C4
+                               : cache + ((size_t)b * hc * wc + nearest_src(t, h, w, hc, wc)) * C4;
+  float4* dst = out + (size_t)warp * C4;
+  for (int c4 = lane; c4 < C4; c4 += 32) dst[c4] = __ldg(src + c4);
+}
+
 }  // namespace
 
 cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
@@ -224,6 +257,21 @@ cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* p
   LaunchScope scope(KC_RESTORE, 1, rb_bytes, rb_bytes, st);
   return launch_pdl(restore_bf16_kernel, dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const uint4*>(cache), hc, wc,
                     reinterpret_cast<const uint4*>(pivots), inv, h * w, k, h, w, C / 8, reinterpret_cast<uint4*>(out), rows);
+}
+
+cudaError_t launch_gather_rows(const float* x, const int32_t* idx, int B, int n, int k, int C, float* out, cudaStream_t st) {
+  LaunchScope scope(KC_GATHER_LN, 1, (double)B * k * C * 8.0, (double)B * k * C * 8.0, st);
+  return launch_pdl(gather_rows_kernel, dim3((k + 7) / 8, B), dim3(256), 0, st, reinterpret_cast<const float4*>(x), idx, n, k, C / 4,
+                    reinterpret_cast<float4*>(out));
+}
+
+cudaError_t launch_restore_rows_f32(const float* cache, int hc, int wc, const float* pivots, const int32_t* inv, int B, int k,
+                                    int h, int w, int C, float* out, cudaStream_t st) {
+  const int rows = B * h * w;
+  const double bytes = (double)B * C * 4.0 * ((double)h * w + k + (double)hc * wc);
+  LaunchScope scope(KC_RESTORE, 1, bytes, bytes, st);
+  return launch_pdl(restore_rows_f32_kernel, dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const float4*>(cache), hc, wc,
+                    reinterpret_cast<const float4*>(pivots), inv, h * w, k, h, w, C / 4, reinterpret_cast<float4*>(out), rows);
 }
 
 }  // namespace fv

@@ -12,17 +12,18 @@ from oracle import fastvar_oracle as O
 from paper_2503_23367_b200 import binding as fv
 from paper_2503_23367_b200 import inputs as I
 from tests.helpers import SUB_NAMES, make_oracle, per_token_errors, run_oracle, trace_to_index_tensor
+from tests.helpers import oracle_weights as helpers_oracle_weights
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 MAX_ABS, MIN_COS = 3e-2, 0.999
 
 
-def make_ctx(wl: I.Workload, mt: I.ModelTensors, unpruned=False) -> fv.FvContext:
+def make_ctx(wl: I.Workload, mt: I.ModelTensors, unpruned=False, granularity=0) -> fv.FvContext:
     cap = sum(wl.tokens(i) if (unpruned or wl.keep[i] >= 1.0) else O.kept_count(wl.keep[i], wl.sides[i], wl.sides[i])
               for i in range(len(wl.sides)))
     return fv.FvContext(wl.L, wl.C, wl.H, [(s, s) for s in wl.sides], wl.cache_step, wl.B, cap, mt,
-                        cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio, device=DEV)
+                        cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio, device=DEV, granularity=granularity)
 
 
 def gpu_schedule(ctx, wl, xs, forced=None, trace=False):
@@ -191,6 +192,73 @@ def test_free_running_selection_matches_oracle_on_identical_input():
                     agree.append(len(np.intersect1d(g[b], o[b])) / o.shape[1])
     assert min(agree) >= 0.9
     ctx.close()
+
+
+# ------------------------------------------------------------------ per-step granularity (the coarser variant)
+def check_step_granularity(wl, kind="iid"):
+    """One selection and one restoration around the whole stack of blocks, against the oracle's variant of
+    the same name: forced indices for the floating point, free running for the indices (the selection
+    sees the step input itself, identical on both sides)."""
+    mt = I.model_tensors(wl)
+    xs = [I.step_input(wl, i, kind) for i in range(len(wl.sides))]
+    orc = O.VarOracle(wl.L, wl.C, wl.H, [(s, s) for s in wl.sides], cache_step=wl.cache_step,
+                      weights=helpers_oracle_weights(mt), B=wl.B, cross_len=wl.cross_len, granularity="step")
+    ref, tr = [], []
+    for i, x in enumerate(xs):
+        t = {}
+        ref.append(orc.var_step(x, i, wl.keep[i], trace=t))
+        tr.append(t)
+    ctx = make_ctx(wl, mt, granularity=1)
+    for mode in ("forced", "free"):
+        ctx.reset()
+        for i, x in enumerate(xs):
+            xd = torch.from_numpy(x).to(DEV)
+            f = t = None
+            if wl.keep[i] < 1.0:
+                idx_o = tr[i][("step",)]["idx"]
+                if mode == "forced":
+                    f = torch.from_numpy(idx_o.astype(np.int32)).to(DEV)
+                else:
+                    t = torch.zeros(idx_o.shape, dtype=torch.int32, device=DEV)
+            got = ctx.var_step(xd, i, wl.keep[i], forced_idx=f, idx_trace=t).cpu().numpy()
+            if t is not None:
+                idx_g = t.cpu().numpy().astype(np.int64)
+                s_o = tr[i][("step",)]["score"]
+                same = True
+                for b in range(wl.B):
+                    assert np.all(np.diff(idx_g[b]) > 0)
+                    diff = np.setxor1d(idx_g[b], idx_o[b])
+                    if len(diff):
+                        same = False
+                        tau = np.sort(s_o[b])[::-1][idx_o.shape[1] - 1]
+                        assert np.all(np.abs(s_o[b, diff] - tau) <= 1e-5 * tau), "index mismatch away from a near-tie"
+                if not same:
+                    continue        # a near-tie went the other way: the floating-point check ran in forced mode
+            err, cos = per_token_errors(got, ref[i])
+            assert err <= MAX_ABS and cos >= MIN_COS, f"{mode} step {i} side {wl.sides[i]}: max-abs {err:.4g}, cos {cos:.6f}"
+            if wl.keep[i] < 1.0:     # rows that were not kept are exact copies of the cached output map
+                hc = wl.sides[wl.cache_step]
+                src = O.nearest_source(wl.sides[i], wl.sides[i], hc, hc)
+                cache = ctx.cache_view(0, 0, wl.B).cpu().numpy()
+                idx_used = tr[i][("step",)]["idx"] if mode == "forced" else idx_g
+                for b in range(wl.B):
+                    rest = np.setdiff1d(np.arange(wl.tokens(i)), idx_used[b])
+                    assert np.array_equal(got[b, rest], cache[b, src[rest]])
+        assert ctx.device_status() == 0 and ctx.state() == (len(xs), orc.kv_len)
+    ctx.close()
+
+
+def test_step_granularity_tiny_schedule():
+    check_step_granularity(I.WORKLOADS["tiny"])
+    check_step_granularity(I.WORKLOADS["tiny"], kind="structured")
+
+
+def test_step_granularity_infinity_shape_with_cross_attention():
+    base = I.WORKLOADS["infinity_2b_1k"]
+    sides = (1, 2, 4, 8, 12, 16, 24)
+    wl = I.Workload("inf-short", L=2, C=base.C, H=base.H, B=2, sides=sides,
+                    keep=(1.0, 1.0, 1.0, 1.0, 1.0, 0.6, 0.4), cross_len=64, seed=base.seed)
+    check_step_granularity(wl)
 
 
 def test_keep_ratio_one_is_the_unpruned_path_and_is_deterministic():
