@@ -197,6 +197,7 @@ class ClockSampler:
 def ours(args, wl):
     from paper_2503_23367_b200 import binding as fv
     from paper_2503_23367_b200 import build as fv_build
+    from paper_2503_23367_b200 import replicas as R
     rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
@@ -214,11 +215,11 @@ def ours(args, wl):
 
     S = len(wl.sides)
     pruned_steps = [i for i in range(S) if wl.keep[i] < 1.0]
-    gt = GpuTensors(wl, dev, seed=wl.seed + rank)
+    gt = GpuTensors(wl, dev, seed=wl.seed)          # replicas: the same weights on every rank
     cap = sum(kept(wl, i) for i in range(S))
     hw = [(s, s) for s in wl.sides]
     ctx = fv.FvContext(wl.L, wl.C, wl.H, hw, wl.cache_step, wl.B, cap, gt, cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio, device=dev)
-    g = torch.Generator(device=dev); g.manual_seed(wl.seed + 77 + rank)
+    g = torch.Generator(device=dev); g.manual_seed(R.rank_seed(wl.seed + 77, rank))   # its own images
     xs = [torch.randn(wl.B, wl.tokens(i), wl.C, generator=g, device=dev, dtype=torch.float32) for i in range(S)]
     outs = [torch.empty_like(x) for x in xs]
 
@@ -234,15 +235,11 @@ def ours(args, wl):
     def barrier():
         torch.cuda.synchronize()
         if world > 1:
-            dist.barrier()
+            R.barrier()
             torch.cuda.synchronize()
 
     def max_over_ranks(v: float) -> float:
-        if world == 1:
-            return v
-        t = torch.tensor([v], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return R.max_over_ranks(v, device=dev)
 
     for _ in range(args.warmup):
         schedule(ctx, wl.keep)
