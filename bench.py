@@ -56,6 +56,8 @@ def kept(wl: I.Workload, i: int, pruned: bool = True) -> int:
     n = wl.tokens(i)
     if not pruned or wl.keep[i] >= 1.0:
         return n
+    if wl.keep[i] == 0.0:
+        return 0                      # skipped step: nothing forwarded, nothing cached
     import math
     return min(n, max(1, int(math.ceil(wl.keep[i] * n - 1e-9))))
 
@@ -73,7 +75,7 @@ def oracle_sample(wl: I.Workload):
                                               "w_q_x", "w_kv_x", "w_o_x")}
     w["mod"] = mt.mod.astype(np.float64)
     w["text"] = None if mt.text is None else I.bf16_bits_to_f32(mt.text).astype(np.float64)
-    steps = [i for i in range(len(wl.sides)) if wl.keep[i] < 1.0]
+    steps = [i for i in range(len(wl.sides)) if 0.0 < wl.keep[i] < 1.0]   # skipped steps cost the oracle nothing worth timing
     n_c = wl.tokens(wl.cache_step)
     subs = ("attn", "xattn", "ffn") if wl.cross_len else ("attn", "ffn")
     xs = {i: I.step_input(wl, i) for i in steps}

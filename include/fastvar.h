@@ -153,7 +153,7 @@ typedef struct { /* HOST arrays of length L holding DEVICE pointers; bf16 unless
 
 size_t fv_workspace_bytes(const fv_config *cfg); /* scratch for fv_var_step                         */
 size_t fv_kv_bytes(const fv_config *cfg);        /* KV cache of all blocks (+ text K/V)             */
-size_t fv_cache_bytes(const fv_config *cfg);     /* sublayer caches y_{K-N} of all blocks           */
+size_t fv_cache_bytes(const fv_config *cfg);     /* output map of step K-N (fp32) + sublayer caches  */
 
 /* Builds a context over caller-owned buffers (sizes from the three queries above, 1024-byte aligned).
  * Clears the KV buffer once (synchronously) so that never-written rows hold zeros.
@@ -182,7 +182,9 @@ fv_status fv_device_status(fv_ctx *ctx, int32_t *code_host, void *stream);
  *   tokens_dev  [B, h*w, C] fp32: residual stream entering block 0 at this scale.
  *   out_dev     [B, h*w, C] fp32: residual stream after block L-1 (may alias tokens_dev).
  *   scale_idx   must equal the context's next step (steps are taken in order).
- *   keep_ratio  1.0 = unpruned path (no select / gather / restore work at all); < 1 = FastVAR.
+ *   keep_ratio  1.0 = unpruned path (no select / gather / restore work at all); in (0, 1) = FastVAR;
+ *               0.0 = the step is skipped (the paper's 100 % pruning ratio, Sec. 4.1): out_dev is the output
+ *               map of step cache_step interpolated (nearest) to this scale, nothing enters the KV cache.
  *   forced_idx_dev NULL, or int32 [L, n_sub, B, k]: use these kept indices (ascending per image)
  *               instead of selecting -- separates index parity from floating-point parity in tests.
  *   idx_trace_dev  NULL, or int32 [L, n_sub, B, k]: receives the kept indices of every sublayer.

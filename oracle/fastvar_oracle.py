@@ -226,7 +226,7 @@ class VarOracle:
         self.Kc = [[np.zeros((0, self.C)) for _ in range(self.B)] for _ in range(self.L)]
         self.Vc = [[np.zeros((0, self.C)) for _ in range(self.B)] for _ in range(self.L)]
         self.cache: List[Dict[str, np.ndarray]] = [dict() for _ in range(self.L)]
-        self.step_cache: Optional[np.ndarray] = None   # granularity "step": output token map of step K-N
+        self.step_cache: Optional[np.ndarray] = None   # output token map of step K-N (granularity "step"; skipped steps)
 
     # -- one wrapped sublayer on compact rows ---------------------------------------------------
     def _branch(self, l: int, sub: str, xp: np.ndarray) -> np.ndarray:
@@ -272,6 +272,15 @@ class VarOracle:
         B, n, C = x.shape
         h, w_ = self.hw[scale_idx]
         assert n == h * w_ and B == self.B and C == self.C
+        if keep_ratio == 0.0:
+            # Sec. 4.1 "Implementation Details": a 100 % pruning ratio drops every token -- the step is
+            # skipped and the intermediate output is interpolated to the target resolution.  Reading: the
+            # intermediate output is the output token map of the caching step (the last step that ran in
+            # full); nothing enters the KV cache.
+            assert self.step_cache is not None and scale_idx > self.cache_step
+            hc, wc = self.hw[self.cache_step]
+            self.step += 1
+            return ctr_upsample(self.step_cache, hc, wc, h, w_)
         pruned = keep_ratio < 1.0
         k = kept_count(keep_ratio, h, w_) if pruned else n
         if self.granularity == "step":
@@ -307,6 +316,8 @@ class VarOracle:
                     x = x + mod[:, 5][:, None, :] * yfull
                 else:
                     x = x + yfull
+        if scale_idx == self.cache_step:
+            self.step_cache = x.copy()          # output map of the caching step (used by skipped steps)
         self.kv_len += k
         self.step += 1
         return x

@@ -31,6 +31,7 @@ struct fv_ctx {
   int32_t *idx = nullptr, *inv = nullptr;
   void* sel_ws = nullptr;
   void* splitk_ws = nullptr;
+  float* step_cache = nullptr;  // fp32 output map of the caching step [B_max, n_cache, C] (skipped steps; granularity 1)
   float* xc = nullptr;  // granularity 1: compact fp32 residual stream of a pruned step [B*k, C]
   size_t kv_block_bytes = 0, k_bytes = 0, text_k_bytes = 0, text_block_bytes = 0, cache_sub_bytes = 0;
 };
@@ -220,9 +221,12 @@ size_t fv_kv_bytes(const fv_config* cfg) {
 size_t fv_cache_bytes(const fv_config* cfg) {
   if (!config_ok(cfg) || cfg->cache_step < 0) return 0;
   const size_t n_cache = (size_t)cfg->h[cfg->cache_step] * cfg->w[cfg->cache_step];
-  if (cfg->granularity == 1) return align_up((size_t)cfg->B_max * n_cache * cfg->C * 4, 1024);  // fp32 output map of the caching step
+  // the fp32 output map of the caching step comes first (restored by skipped steps and by granularity 1) ...
+  const size_t step_bytes = align_up((size_t)cfg->B_max * n_cache * cfg->C * 4, 1024);
+  if (cfg->granularity == 1) return step_bytes;
+  // ... then, for the paper's granularity, one bf16 cache per wrapped sublayer
   const int n_sub = cfg->cross_len ? 3 : 2;
-  return (size_t)cfg->L * n_sub * align_up((size_t)cfg->B_max * n_cache * cfg->C * 2, 1024);
+  return step_bytes + (size_t)cfg->L * n_sub * align_up((size_t)cfg->B_max * n_cache * cfg->C * 2, 1024);
 }
 
 fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, void* cache_dev, void* workspace_dev,
@@ -262,7 +266,10 @@ fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, v
   c->mod = wts->mod_dev;
   c->text = wts->text_dev;
   c->kv = static_cast<char*>(kv_dev);
-  c->cache = static_cast<char*>(cache_dev);
+  c->step_cache = static_cast<float*>(cache_dev);
+  c->cache = (cache_dev && cfg->cache_step >= 0) ? static_cast<char*>(cache_dev) +
+                             align_up((size_t)cfg->B_max * cfg->h[cfg->cache_step] * cfg->w[cfg->cache_step] * cfg->C * 4, 1024)
+                       : nullptr;
   c->ws = static_cast<char*>(workspace_dev);
   c->n_sub = cfg->cross_len ? 3 : 2;
   c->n_max = max_tokens(cfg);
@@ -328,7 +335,7 @@ fv_status fv_cache_pointer(const fv_ctx* ctx, int32_t block, int32_t sublayer, v
   if (!ctx || !cache_dev || block < 0 || block >= ctx->cfg.L || sublayer < 0 || sublayer >= ctx->n_sub || !ctx->cache) return FV_ERR_INVALID_ARG;
   if (ctx->cfg.granularity == 1) {  // one step-level cache
     if (block != 0 || sublayer != 0) return FV_ERR_INVALID_ARG;
-    *cache_dev = ctx->cache;
+    *cache_dev = ctx->step_cache;
     return FV_OK;
   }
   *cache_dev = ctx->cache + ((size_t)block * ctx->n_sub + sublayer) * ctx->cache_sub_bytes;
@@ -372,10 +379,24 @@ fv_status fv_device_status(fv_ctx* ctx, int32_t* code_host, void* stream) {
 fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t scale_idx, double keep_ratio, float* out_dev,
                       const int32_t* forced_idx_dev, int32_t* idx_trace_dev, void* stream) {
   if (!ctx || !tokens_dev || !out_dev || B <= 0 || B > ctx->cfg.B_max) return FV_ERR_INVALID_ARG;
-  if (!(keep_ratio > 0.0) || keep_ratio > 1.0 || !aligned16(tokens_dev) || !aligned16(out_dev)) return FV_ERR_INVALID_ARG;
+  if (!(keep_ratio >= 0.0) || keep_ratio > 1.0 || !aligned16(tokens_dev) || !aligned16(out_dev)) return FV_ERR_INVALID_ARG;
   const fv_config& c = ctx->cfg;
   if (scale_idx < 0 || scale_idx >= c.n_steps) return FV_ERR_INVALID_ARG;
   if (scale_idx != ctx->next_step) return FV_ERR_BAD_STATE;
+  if (keep_ratio == 0.0) {
+    // Skipped step (the paper's 100 % pruning ratio, Sec. 4.1): no token is forwarded, nothing enters the
+    // KV cache; the output is the caching step's output map interpolated to this scale.
+    if (c.cache_step < 0 || scale_idx <= c.cache_step) return FV_ERR_BAD_STATE;
+    if (forced_idx_dev || idx_trace_dev) return FV_ERR_INVALID_ARG;
+    cudaStream_t st0 = static_cast<cudaStream_t>(stream);
+    const int h0 = c.h[scale_idx], w0 = c.w[scale_idx];
+    if (launch_inv_fill(B, h0 * w0, ctx->inv, st0) != cudaSuccess) return FV_ERR_CUDA;
+    if (launch_restore_rows_f32(ctx->step_cache, c.h[c.cache_step], c.w[c.cache_step], ctx->step_cache, ctx->inv, B, 0, h0, w0, c.C,
+                                out_dev, st0) != cudaSuccess)
+      return FV_ERR_CUDA;
+    ctx->next_step += 1;
+    return FV_OK;
+  }
   const bool pruned = keep_ratio < 1.0;
   if (pruned && (c.cache_step < 0 || scale_idx <= c.cache_step)) return FV_ERR_BAD_STATE;
   if (!pruned && (forced_idx_dev || idx_trace_dev)) return FV_ERR_INVALID_ARG;
@@ -508,14 +529,12 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
     }
   }
   if (s != FV_OK) return s;
-  if (whole_step) {
-    if (write_cache &&
-        cudaMemcpyAsync(ctx->cache, x, (size_t)B * n * C * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-      return FV_ERR_CUDA;  // the step-level cache: this step's output map (image stride n*C == n_cache*C here)
-    if (pruned && launch_restore_rows_f32(reinterpret_cast<const float*>(ctx->cache), hc, wc, ctx->xc, ctx->inv, B, k, h, w, C,
-                                          out_dev, st) != cudaSuccess)
-      return FV_ERR_CUDA;
-  }
+  if (write_cache &&
+      cudaMemcpyAsync(ctx->step_cache, x, (size_t)B * n * C * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return FV_ERR_CUDA;  // the step-level cache: this step's output map (image stride n*C == n_cache*C here)
+  if (whole_step && pruned &&
+      launch_restore_rows_f32(ctx->step_cache, hc, wc, ctx->xc, ctx->inv, B, k, h, w, C, out_dev, st) != cudaSuccess)
+    return FV_ERR_CUDA;
   if (s != FV_OK) return s;
   ctx->kv_len += k;
   ctx->next_step += 1;

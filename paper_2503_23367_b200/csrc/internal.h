@@ -66,6 +66,7 @@ SelectWs select_ws_carve(void* workspace, int B, int n, int C);
 cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* idx, int32_t* inv, float* score,
                           int32_t* near_tie, void* workspace, bool have_partials, cudaStream_t st);
 cudaError_t launch_inv_from_idx(const int32_t* idx, int B, int k, int n, int32_t* inv, cudaStream_t st);
+cudaError_t launch_inv_fill(int B, int n, int32_t* inv, cudaStream_t st);  // every token unkept (-1)
 cudaError_t select_init();  // one-time function attributes
 
 // ---- rows.cu : gather + LayerNorm + modulate, restore (+ gate and residual) ----------------------

@@ -339,6 +339,12 @@ cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* i
   return cudaGetLastError();
 }
 
+cudaError_t launch_inv_fill(int B, int n, int32_t* inv, cudaStream_t st) {
+  const size_t total = (size_t)B * n;
+  LaunchScope scope(KC_SELECT, 1, 4.0 * total, 4.0 * total, st);
+  return launch_pdl(inv_fill_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, inv, total);
+}
+
 cudaError_t launch_inv_from_idx(const int32_t* idx, int B, int k, int n, int32_t* inv, cudaStream_t st) {
   const size_t total = (size_t)B * n;
   LaunchScope scope(KC_SELECT, 2, 4.0 * B * ((double)k + n), 4.0 * B * ((double)k + n), st);

@@ -132,6 +132,11 @@ WORKLOADS: Dict[str, Workload] = {
     "infinity_2b_1k": Workload("infinity_2b_1k", L=32, C=2048, H=16, B=2, sides=_INF1K,
                                keep=_keeps(_INF1K, {40: 0.6, 48: 0.4, 64: 0.2}),
                                cross_len=512, seed=4000),
+    # the paper's own Infinity schedule (Sec. 4.1): pruning ratios {40, 50, 100, 100} % on the last four
+    # scale steps, i.e. keep 0.6 / 0.5 and two skipped steps
+    "infinity_2b_1k_paper": Workload("infinity_2b_1k_paper", L=32, C=2048, H=16, B=2, sides=_INF1K,
+                                     keep=_keeps(_INF1K, {32: 0.6, 40: 0.5, 48: 0.0, 64: 0.0}),
+                                     cross_len=512, seed=4000),
     "infinity_2b_2k": Workload("infinity_2b_2k", L=32, C=2048, H=16, B=1, sides=_INF2K,
                                keep=_keeps(_INF2K, {64: 0.2, 80: 0.2, 96: 0.2, 128: 0.2}),
                                cross_len=512, seed=5000),

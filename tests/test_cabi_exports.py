@@ -56,4 +56,4 @@ def test_argument_validation_happens_before_any_launch(lib):
     cfg = fv.fv_config(2, 256, 4, 4, 0, 1, 2, h, w, 0, 80)
     assert lib.fv_workspace_bytes(ctypes.byref(cfg)) > 64 * 256 * 2 * 4
     assert lib.fv_kv_bytes(ctypes.byref(cfg)) == 2 * 2 * 80 * 256 * 2
-    assert lib.fv_cache_bytes(ctypes.byref(cfg)) == 2 * 2 * 16 * 256 * 2
+    assert lib.fv_cache_bytes(ctypes.byref(cfg)) == 16 * 256 * 4 + 2 * 2 * 16 * 256 * 2   # fp32 output map + sublayer caches

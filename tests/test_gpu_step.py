@@ -261,6 +261,37 @@ def test_step_granularity_infinity_shape_with_cross_attention():
     check_step_granularity(wl)
 
 
+@pytest.mark.parametrize("granularity", [0, 1])
+def test_skipped_step_keep_ratio_zero(granularity):
+    """keep_ratio = 0 (the paper's 100 % pruning ratio): the output is an exact copy of rows of the caching
+    step's output map (nearest interpolation), the KV cache does not grow, the next pruned step still runs."""
+    base = I.WORKLOADS["tiny"]
+    keep = tuple(base.keep[:8]) + (0.0, 0.5)                  # sides ..., 10 (cache step 7), 13 skipped, 16 pruned
+    wl = I.Workload("tiny-skip", L=base.L, C=base.C, H=base.H, B=base.B, sides=base.sides, keep=keep, seed=base.seed)
+    assert wl.cache_step == 7
+    mt = I.model_tensors(wl)
+    xs = [I.step_input(wl, i) for i in range(len(wl.sides))]
+    orc = O.VarOracle(wl.L, wl.C, wl.H, [(s, s) for s in wl.sides], cache_step=wl.cache_step, weights=helpers_oracle_weights(mt),
+                      B=wl.B, cross_len=wl.cross_len, granularity="step" if granularity else "sublayer")
+    ctx = make_ctx(wl, mt, granularity=granularity)
+    outs = []
+    for i, x in enumerate(xs):
+        tr = {}
+        ref = orc.var_step(x, i, wl.keep[i], trace=tr)
+        forced = None
+        if 0.0 < wl.keep[i] < 1.0:
+            forced = torch.from_numpy(tr[("step",)]["idx"].astype(np.int32) if granularity else trace_to_index_tensor(wl, tr)).to(DEV)
+        got = ctx.var_step(torch.from_numpy(x).to(DEV), i, wl.keep[i], forced_idx=forced).cpu().numpy()
+        outs.append(got)
+        err, cos = per_token_errors(got, ref)
+        assert err <= MAX_ABS and cos >= MIN_COS, (i, err, cos)
+        assert ctx.state() == (i + 1, orc.kv_len)
+    src = O.nearest_source(13, 13, 10, 10)
+    assert np.array_equal(outs[8], outs[7][:, src])          # a copy of the cached map's rows, bit for bit
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
 def test_keep_ratio_one_is_the_unpruned_path_and_is_deterministic():
     wl = I.WORKLOADS["tiny"]
     mt = I.model_tensors(wl)
@@ -290,7 +321,10 @@ def test_state_and_argument_errors():
         ctx.var_step(x0, 0, 0.5)                                         # pruned before the cache step
     assert e.value.code == 2
     with pytest.raises(fv.FvError) as e:
-        ctx.var_step(x0, 0, 0.0)
+        ctx.var_step(x0, 0, 0.0)                                         # nothing cached yet to interpolate
+    assert e.value.code == 2
+    with pytest.raises(fv.FvError) as e:
+        ctx.var_step(x0, 0, -0.1)
     assert e.value.code == 1
     ctx.var_step(x0, 0, 1.0)
     assert ctx.state() == (1, 1)

@@ -445,6 +445,22 @@ def test_step_granularity_pivot_rows_and_restored_rows():
         np.testing.assert_allclose(outs[4][b, idx[b]], out4[b, idx[b]], rtol=1e-11, atol=1e-12)
 
 
+@pytest.mark.parametrize("granularity", ["sublayer", "step"])
+def test_skipped_step_is_the_interpolated_output_of_the_caching_step(granularity):
+    """keep_ratio = 0 (the paper's 100 % pruning ratio): no token is forwarded, the step's output is the
+    nearest-neighbour interpolation of the caching step's output map (checked against the library's
+    interpolate), the KV cache does not grow, and a later step still runs."""
+    wl, mt, w = _tiny_model(L=1)
+    xs = [I.step_input(wl, s) for s in range(len(wl.sides))]
+    orc, outs, _ = _run(wl, w, xs, [1.0, 1.0, 1.0, 0.0, 0.5], cache_step=2, granularity=granularity)
+    hc, h = wl.sides[2], wl.sides[3]
+    t = torch.from_numpy(outs[2]).reshape(wl.B, hc, hc, wl.C).permute(0, 3, 1, 2)
+    up = F.interpolate(t, size=(h, h), mode="nearest").permute(0, 2, 3, 1).reshape(wl.B, h * h, wl.C).numpy()
+    np.testing.assert_array_equal(outs[3], up)
+    assert orc.kv_len == 1 + 4 + 9 + 0 + 18 and orc.step == 5
+    assert outs[4].shape == xs[4].shape
+
+
 def test_step_granularity_images_are_independent():
     wl, mt, w = _tiny_model(L=1, B=2)
     xs = [I.step_input(wl, s) for s in range(len(wl.sides))]
