@@ -68,13 +68,13 @@ fv_status fv_prune_select(const float *x_dev, int32_t B, int32_t h, int32_t w, i
  * exists for the deployment reason below.)  Some hosts of this library may not call cudaMalloc: a
  * serving process that split all device memory into fixed pools at start-up, or a plug-in that must
  * not touch the allocator because allocation synchronises the device under its pipeline.  They
- * cannot provide `workspace_dev`, so this variant keeps the scratch (partial column sums, mean token,
- * scores) in a fixed array inside the library's device image: fv_prune_select_static_capacity()
+ * cannot provide `workspace_dev`, so this variant keeps the scratch (arrival counters, partial column
+ * sums, scores) in a fixed array inside the library's device image: fv_prune_select_static_capacity()
  * bytes (8 MiB), held by every GPU that loads the library until the process exits.
  *   - Inputs and outputs are still the caller's; arguments as in fv_prune_select, minus the workspace.
  *   - It allocates nothing: no cudaMalloc / cudaFree, no allocating library routine.  Shapes whose
  *     scratch need, fv_prune_select_workspace_bytes(B, h*w, C), exceeds the capacity are refused with
- *     FV_ERR_CAPACITY (e.g. B = 2, 64x64 tokens, C = 2048 needs 2.1 MiB; B = 1, 128x128, C = 2048 needs
+ *     FV_ERR_CAPACITY (e.g. B = 2, 64x64 tokens, C = 2048 needs 2.2 MiB; B = 1, 128x128, C = 2048 needs
  *     4.1 MiB; B = 4 at 128x128, C = 2048 does not fit).
  *   - The first call on each device looks up the array's device address (with that device current);
  *     make that first call outside any stream capture.

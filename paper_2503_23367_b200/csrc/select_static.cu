@@ -2,8 +2,8 @@
 // buffer because they cannot allocate one -- e.g. a serving loop whose device memory was carved up
 // once at start-up (every byte belongs to a pool with a fixed budget), or a host plug-in that is not
 // allowed to call the CUDA allocator, whose implicit device synchronisation would stall its pipeline.
-// The selection kernels need scratch beyond their inputs and outputs (partial column sums, the mean
-// token, the scores); here that scratch is a fixed array that lives in the library's own device image.
+// The selection kernels need scratch beyond their inputs and outputs (arrival counters, partial column
+// sums, the scores); here that scratch is a fixed array that lives in the library's own device image.
 //
 // The array below exists once per GPU that loads this library and stays resident until the process
 // exits.  In HOST code its name is only a handle (not a device address): the device address is
