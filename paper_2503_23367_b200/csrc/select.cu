@@ -23,7 +23,7 @@ constexpr int kTopkWarps = kTopkThreads / 32;
 // Keys sit in shared memory with one pad word per 32, so that both access patterns of the top-k are
 // free of bank conflicts: consecutive lanes on consecutive tokens, and each lane on its own contiguous run.
 __device__ __forceinline__ int KI(int i) { return i + (i >> 5); }
-constexpr size_t kTopkMaxSmem = ((size_t)kTopkMaxTokens + kTopkMaxTokens / 32) * 4;
+constexpr size_t kTopkMaxSmem = ((size_t)kTopkMaxTokens + kTopkMaxTokens / 32 + 1) * 4;
 
 __global__ void __launch_bounds__(256) colsum_chunk_kernel(const float4* __restrict__ x, int n, int C4, int nchunks, int group,
                                                            int ngroups, float4* __restrict__ chunk_partial,

@@ -34,6 +34,7 @@ SELECT_CASES = [  # B, h, w, C, keep, kind
     (2, 64, 64, 2048, 0.2, "structured"), (1, 1, 1, 256, 0.5, "iid"), (3, 5, 7, 260, 0.3, "iid"),
     (2, 40, 40, 2048, 0.6, "structured"), (1, 3, 2, 8, 1.0, "iid"), (2, 33, 31, 128, 0.01, "iid"),
     (1, 128, 128, 2048, 0.2, "iid"),        # 2K zero-shot step: 16384 tokens, map larger than L2
+    (1, 192, 256, 64, 0.1, "iid"),          # 49152 tokens: the largest map the top-k CTA holds in shared memory
 ]
 
 
@@ -82,6 +83,10 @@ def test_prune_select_ties_go_to_lowest_index():
 
 
 def test_prune_select_argument_errors():
+    big = torch.zeros((1, 193 * 256, 8), device=DEV)                      # one row of tokens beyond the largest map
+    with pytest.raises(fv.FvError) as e:
+        fv.fv_prune_select(big, 193, 256, 0.5)
+    assert e.value.code == 4
     x = torch.zeros((1, 4, 8), device=DEV)
     with pytest.raises(fv.FvError) as e:
         fv.fv_prune_select(x, 2, 2, 0.0)
