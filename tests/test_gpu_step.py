@@ -292,6 +292,32 @@ def test_skipped_step_keep_ratio_zero(granularity):
     ctx.close()
 
 
+def test_non_square_maps_and_partial_batch():
+    """Token maps need not be square, and a call may use fewer images than the context was built for."""
+    hw = [(1, 1), (2, 3), (3, 5), (5, 8), (7, 12), (10, 17)]
+    keep = [1.0, 1.0, 1.0, 1.0, 0.5, 0.3]
+    L, C, H, B_max, B = 2, 128, 2, 3, 2
+    wl = I.Workload("rect", L=L, C=C, H=H, B=B_max, sides=tuple(h for h, _ in hw), keep=tuple(keep), cross_len=8, seed=77)
+    mt = I.model_tensors(wl)
+    w = helpers_oracle_weights(mt)
+    w = dict(w); w["mod"] = w["mod"][:, :B]; w["text"] = w["text"][:B]
+    orc = O.VarOracle(L, C, H, hw, cache_step=3, weights=w, B=B, cross_len=8)
+    cap = sum(O.kept_count(r, h, ww) if r < 1 else h * ww for r, (h, ww) in zip(keep, hw))
+    ctx = fv.FvContext(L, C, H, hw, 3, B_max, cap, mt, cross_len=8, device=DEV)
+    for i, (h, ww) in enumerate(hw):
+        x = I.token_map(500 + i, B, h, ww, C)
+        tr = {}
+        ref = orc.var_step(x, i, keep[i], trace=tr)
+        forced = None
+        if keep[i] < 1.0:
+            forced = torch.from_numpy(np.stack([np.stack([tr[(l, s)]["idx"] for s in SUB_NAMES[3]]) for l in range(L)]).astype(np.int32)).to(DEV)
+        got = ctx.var_step(torch.from_numpy(x).to(DEV), i, keep[i], forced_idx=forced).cpu().numpy()
+        err, cos = per_token_errors(got, ref)
+        assert err <= MAX_ABS and cos >= MIN_COS, (i, err, cos)
+    assert ctx.device_status() == 0 and ctx.state() == (len(hw), orc.kv_len)
+    ctx.close()
+
+
 def test_keep_ratio_one_is_the_unpruned_path_and_is_deterministic():
     wl = I.WORKLOADS["tiny"]
     mt = I.model_tensors(wl)
