@@ -31,6 +31,8 @@ struct fv_ctx {
   int32_t *idx = nullptr, *inv = nullptr;
   void* sel_ws = nullptr;
   void* splitk_ws = nullptr;
+  cudaStream_t side = nullptr;           // the unkept rows of a restoration run here, beside the sublayer's branch
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   float* step_cache = nullptr;  // fp32 output map of the caching step [B_max, n_cache, C] (skipped steps; granularity 1)
   float* xc = nullptr;  // granularity 1: compact fp32 residual stream of a pruned step [B*k, C]
   size_t kv_block_bytes = 0, k_bytes = 0, text_k_bytes = 0, text_block_bytes = 0, cache_sub_bytes = 0;
@@ -171,7 +173,7 @@ fv_status fv_restore_residual(float* x_dev, const void* y_dev, const void* cache
   if (!x_dev || !y_dev || !cache_dev || !inv_dev || B <= 0 || k <= 0 || h <= 0 || w <= 0 || hc <= 0 || wc <= 0) return FV_ERR_INVALID_ARG;
   if (C <= 0 || (C % 8)) return FV_ERR_INVALID_ARG;
   return cuda_status(launch_restore_residual(x_dev, y_dev, cache_dev, inv_dev, gamma_dev, mod_stride, B, k, h, w, hc, wc, C,
-                                             nullptr, static_cast<cudaStream_t>(stream)));
+                                             nullptr, 0, static_cast<cudaStream_t>(stream)));
 }
 
 fv_status fv_gemm_bf16(const void* a_dev, const void* w_dev, const void* bias_dev, int32_t M, int32_t N, int32_t K,
@@ -292,15 +294,24 @@ fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, v
   if (cudaMemset(kv_dev, 0, fv_kv_bytes(cfg)) != cudaSuccess || cudaMemset(c->status, 0, 256) != cudaSuccess ||
       cudaMemset(c->sel_ws, 0, select_ticket_bytes(cfg->B_max)) != cudaSuccess ||
       cudaMemset(c->splitk_ws, 0, gemm_splitk_ticket_bytes()) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
       cudaDeviceSynchronize() != cudaSuccess) {
-    delete c;
+    fv_destroy(c);
     return FV_ERR_CUDA;
   }
   *out = c;
   return FV_OK;
 }
 
-void fv_destroy(fv_ctx* ctx) { delete ctx; }
+void fv_destroy(fv_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->side) { cudaStreamSynchronize(ctx->side); cudaStreamDestroy(ctx->side); }
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+  delete ctx;
+}
 
 fv_status fv_reset(fv_ctx* ctx) {
   if (!ctx) return FV_ERR_INVALID_ARG;
@@ -473,6 +484,16 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
       const float* sigma = kind == 0 ? mod : (kind == 2 ? mod + 3 * C : nullptr);
       const float* beta = kind == 0 ? mod + C : (kind == 2 ? mod + 4 * C : nullptr);
       const float* gamma = kind == 0 ? mod + 2 * C : (kind == 2 ? mod + 5 * C : nullptr);
+      const bool more = selecting && !(l == c.L - 1 && sub == ctx->n_sub - 1);
+      if (sub_pruned) {
+        // Cached Token Restoration of the rows that were NOT kept needs only the selection and the cache:
+        // it runs on the side stream while the gather and the branch below work on the kept rows (the two
+        // touch disjoint rows of x).
+        if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
+        e = launch_restore_residual(x, ctx->y_buf, cache_sub, ctx->inv, gamma, mod_stride, B, k, h, w, hc, wc, C,
+                                    more ? ctx->sel_ws : nullptr, 1, ctx->side);
+        if (e != cudaSuccess || cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) { s = FV_ERR_CUDA; break; }
+      }
       e = launch_gather_ln(xr, idx, B, nr, k, C, sigma, beta, mod_stride, ctx->a_buf, st);
       if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
       // ---- branch on the compact rows
@@ -516,9 +537,9 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         o.epilogue = EPI_BF16; o.out = ctx->y_buf;
         s = launch_gemm(o, st);
         if (s != FV_OK) break;
-        const bool more = selecting && !(l == c.L - 1 && sub == ctx->n_sub - 1);
+        if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
         e = launch_restore_residual(x, ctx->y_buf, cache_sub, ctx->inv, gamma, mod_stride, B, k, h, w, hc, wc, C,
-                                    more ? ctx->sel_ws : nullptr, st);
+                                    more ? ctx->sel_ws : nullptr, 2, st);
         if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
         have_partials = more;
       } else {

@@ -73,9 +73,10 @@ cudaError_t select_init();  // one-time function attributes
 cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
                              const float* beta, int mod_stride, void* a_out, cudaStream_t st);
 // colsum_ws: null, or the selection workspace that receives the column sums of the updated x.
+// part: 0 = every row; 1 = the rows that were not kept; 2 = the kept rows (and the fold of the column sums).
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv,
                                     const float* gamma, int mod_stride, int B, int k, int h, int w, int hc, int wc,
-                                    int C, void* colsum_ws, cudaStream_t st);
+                                    int C, void* colsum_ws, int part, cudaStream_t st);
 // Per-step granularity: fp32 gather of the kept rows, and fp32 restoration of the step's output map.
 cudaError_t launch_gather_rows(const float* x, const int32_t* idx, int B, int n, int k, int C, float* out, cudaStream_t st);
 cudaError_t launch_restore_rows_f32(const float* cache, int hc, int wc, const float* pivots, const int32_t* inv, int B, int k,

@@ -110,13 +110,19 @@ __device__ __forceinline__ void bf16x8_to_float(const uint4& p, float (&f)[8]) {
 // source, two float4 of x) for all rows of the chunk, so the column sums of the updated rows -- the
 // next sublayer's Eq. 4 -- fall out of the same registers with no cross-thread reduction.  The source
 // row of every token is resolved once into shared memory; the x rows do not wait for it.
+// `part` splits the work so that the bulk of it can run beside the sublayer's GEMMs and attention:
+//   0 : every row;  1 : only the rows that were NOT kept (they depend on the selection and the cache alone:
+//   column sums start at zero and are left as the chunk partial);  2 : only the kept rows (after the
+//   branch has produced y: column sums continue from the chunk partial of part 1, then the group fold).
 __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restrict__ x, const uint4* __restrict__ y,
                                                                const uint4* __restrict__ cache, const int32_t* __restrict__ inv,
                                                                const float* __restrict__ gamma, int mod_stride, int n, int k,
                                                                int h, int w, int hc, int wc, int C8, int nchunks, int group,
                                                                int ngroups, float4* __restrict__ chunk_partial,
-                                                               float4* __restrict__ group_partial, unsigned int* tickets) {
+                                                               float4* __restrict__ group_partial, unsigned int* tickets,
+                                                               int part) {
   __shared__ const uint4* s_src[kColsumRows];
+  __shared__ int s_on[kColsumRows];
   pdl_trigger();
   pdl_wait();
   const int b = blockIdx.y, chunk = blockIdx.x;
@@ -127,6 +133,7 @@ __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restric
     const int j = __ldg(inv + (size_t)b * n + t);
     s_src[threadIdx.x] = (j >= 0) ? y + ((size_t)b * k + j) * C8
                                   : cache + ((size_t)b * hc * wc + nearest_src(t, h, w, hc, wc)) * C8;
+    s_on[threadIdx.x] = part == 0 || (part == 1) == (j < 0);
   }
   __syncthreads();
   float4* xbase = x + ((size_t)b * n + t0) * C8 * 2;
@@ -137,12 +144,16 @@ __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restric
       g0 = __ldg(g + 2 * c8); g1 = __ldg(g + 2 * c8 + 1);
     }
     float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+    if (part == 2 && chunk_partial) {  // continue the sums of the rows updated by part 1
+      const float4* cp = chunk_partial + ((size_t)b * nchunks + chunk) * C8 * 2 + 2 * c8;
+      a0 = __ldcg(cp); a1 = __ldcg(cp + 1);
+    }
     for (int r = 0; r < rows; r += 4) {
       uint4 p[4];
       float4 x0[4], x1[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        if (r + i < rows) {
+        if (r + i < rows && s_on[r + i]) {
           float4* xr = xbase + (size_t)(r + i) * C8 * 2 + 2 * c8;
           x0[i] = xr[0]; x1[i] = xr[1];
           p[i] = __ldg(s_src[r + i] + c8);
@@ -150,7 +161,7 @@ __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restric
       }
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        if (r + i < rows) {
+        if (r + i < rows && s_on[r + i]) {
           float f[8];
           bf16x8_to_float(p[i], f);
           float4 u0 = x0[i], u1 = x1[i];
@@ -173,7 +184,8 @@ __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restric
       cp[0] = a0; cp[1] = a1;
     }
   }
-  if (chunk_partial) fold_group_partials(b, chunk, nchunks, group, ngroups, C8 * 2, chunk_partial, group_partial, tickets);
+  if (chunk_partial && part != 1)
+    fold_group_partials(b, chunk, nchunks, group, ngroups, C8 * 2, chunk_partial, group_partial, tickets);
 }
 
 __global__ void __launch_bounds__(256) restore_bf16_kernel(const uint4* __restrict__ cache, int hc, int wc,
@@ -237,17 +249,28 @@ cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, i
 
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv, const float* gamma,
                                     int mod_stride, int B, int k, int h, int w, int hc, int wc, int C, void* colsum_ws,
-                                    cudaStream_t st) {
+                                    int part, cudaStream_t st) {
   const int n = h * w;
   SelectWs ws{};
   if (colsum_ws) ws = select_ws_carve(colsum_ws, B, n, C);
   const int nchunks = (n + kColsumRows - 1) / kColsumRows;
-  const double rr_bytes = (double)B * C * (8.0 * n + 2.0 * k + 2.0 * hc * wc);
+  // algorithmic bytes of the part: x read + written for its rows, its source rows
+  const double rows_x = part == 0 ? (double)n : (part == 1 ? (double)(n - k) : (double)k);
+  const double rr_bytes = (double)B * C * (8.0 * rows_x + (part != 1 ? 2.0 * k : 0.0) + (part != 2 ? 2.0 * hc * wc : 0.0));
   LaunchScope scope(KC_RESTORE, 1, rr_bytes, rr_bytes, st);
-  return launch_pdl(restore_residual_kernel, dim3(nchunks, B), dim3(256), 0, st, reinterpret_cast<float4*>(x),
-                    reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h, w, hc, wc,
-                    C / 8, nchunks, ws.group, ws.ngroups, reinterpret_cast<float4*>(ws.chunk_partial),
-                    reinterpret_cast<float4*>(ws.group_partial), ws.tickets);
+  if (part == 0)
+    return launch_pdl(restore_residual_kernel, dim3(nchunks, B), dim3(256), 0, st, reinterpret_cast<float4*>(x),
+                      reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h, w, hc, wc,
+                      C / 8, nchunks, ws.group, ws.ngroups, reinterpret_cast<float4*>(ws.chunk_partial),
+                      reinterpret_cast<float4*>(ws.group_partial), ws.tickets, part);
+  // The two halves of a split restoration are ordered against another stream by events: they are
+  // launched as ordinary stream work, not as programmatic dependents.
+  restore_residual_kernel<<<dim3(nchunks, B), 256, 0, st>>>(reinterpret_cast<float4*>(x), reinterpret_cast<const uint4*>(y),
+                                                            reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h,
+                                                            w, hc, wc, C / 8, nchunks, ws.group, ws.ngroups,
+                                                            reinterpret_cast<float4*>(ws.chunk_partial),
+                                                            reinterpret_cast<float4*>(ws.group_partial), ws.tickets, part);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* pivots, const int32_t* inv, int B, int k,
