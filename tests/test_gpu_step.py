@@ -191,6 +191,13 @@ def test_free_running_selection_matches_oracle_on_identical_input():
                     assert np.all(np.diff(g[b]) > 0) and g[b].min() >= 0 and g[b].max() < wl.tokens(i)
                     agree.append(len(np.intersect1d(g[b], o[b])) / o.shape[1])
     assert min(agree) >= 0.9
+    # the pruned path is deterministic: same inputs, bit-identical outputs and kept sets, run to run
+    # (column sums, K-split partial sums and the two-stream restoration all add in a fixed order)
+    again, traces2 = gpu_schedule(ctx, wl, xs, trace=True)
+    for i in range(len(xs)):
+        assert np.array_equal(got[i], again[i])
+        if traces[i] is not None:
+            assert np.array_equal(traces[i], traces2[i])
     ctx.close()
 
 
