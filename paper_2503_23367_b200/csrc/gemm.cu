@@ -44,17 +44,25 @@ template <int BN> struct GemmCfg {
   static constexpr int kStages = (BN == 256) ? 4 : (BN == 192 ? 5 : 6);
   static constexpr int kTmemCols = (BN == 128) ? 256 : 512;  // two accumulators, power of two
   static constexpr int kAccStride = (BN == 128) ? 128 : 256;  // column offset of the second accumulator
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  // operand stages | per-warp bias slices | barriers | (residual-epilogue kernels only) one turning tile per warp
+  static constexpr int smem_bytes(bool resid) {
+    return kStages * kStageBytes + kBiasSmemBytes + 256 /*barriers*/ + (resid ? kResidSmemBytes : 0) + 1024 /*alignment slack*/;
+  }
 };
 
-template <int BN, bool SPLIT>
+// RESID: the instantiation launched for the residual epilogue.  It is a kernel of its own because that epilogue
+// needs ~90 more registers per thread; the others stay small enough for a bandwidth-bound kernel of another
+// stream (the restoration of the rows that were not kept) to share the SMs with them.
+template <int BN, bool SPLIT, bool RESID>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
   using Cfg = GemmCfg<BN>;
   constexpr int STAGES = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::kStageBytes);
+  uint4* bias_s = reinterpret_cast<uint4*>(smem + STAGES * Cfg::kStageBytes);   // per-warp bias slice of the tile
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::kStageBytes + kBiasSmemBytes);
+  float* resid_s = reinterpret_cast<float*>(smem + STAGES * Cfg::kStageBytes + kBiasSmemBytes + 256);   // RESID: one tile per warp
   uint64_t* empty_bar = full_bar + STAGES;
   uint64_t* acc_full = empty_bar + STAGES;   // [2]
   uint64_t* acc_empty = acc_full + 2;        // [2]
@@ -162,12 +170,39 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
       const int row = m0 + quarter * 32 + lane;
       const bool row_ok = row < p.M;
+      uint4* bias_w = bias_s + quarter * 32;
+      stage_bias(p, bias_w, lane, n0, BN);
+      // residual epilogue (images of fewer than 32 rows take the row-per-thread path below): the first chunk
+      // of `out` is on its way while the accumulator is computed
+      const bool resid = RESID && p.rows_per_image >= 32;
+      ResidRows rr;
+      float4 xa[8], xb[8];
+      if (resid) {
+        rr = resid_rows(p, lane, m0 + quarter * 32);
+        residual_load_x(p, rr, xa, lane, n0);
+      }
       if (!mbar_wait(&acc_full[buf], (lt >> 1) & 1)) { report(p.status, DEV_TIMEOUT_EPI); break; }
       tc_fence_after();
       const int img = row_ok ? row / p.rows_per_image : 0;
       const int jrow = row_ok ? row - img * p.rows_per_image : 0;
       const uint32_t t0 = tmem_base + lane_off + buf * Cfg::kAccStride;
-      if (!SPLIT) {
+      if (resid) {   // whole warp: rows are re-distributed over the lanes
+        float* tile_s = resid_s + quarter * (32 * kResidTilePitch);
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ++ch) {   // rolled: the code of one chunk is fetched once and then reused
+          uint32_t r0[32];
+          tmem_ld32(t0 + 32 * ch, r0);
+          if (ch + 1 < BN / 32) residual_load_x(p, rr, xb, lane, n0 + 32 * (ch + 1));
+          tmem_wait_ld();
+          if (ch == BN / 32 - 1) {  // accumulator fully in registers: hand the buffer back to the MMA warp
+            tc_fence_before();
+            mbar_arrive(&acc_empty[buf]);
+          }
+          if (n0 + 32 * ch < p.N) residual_chunk(p, rr, r0, xa, tile_s, lane, n0 + 32 * ch, bias_w + 4 * ch);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) xa[i] = xb[i];
+        }
+      } else if (!SPLIT) {
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 64) {
           // two chunks in flight: the second load overlaps the first chunk's stores
@@ -180,8 +215,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             mbar_arrive(&acc_empty[buf]);
           }
           const int col = n0 + c0;
-          if (row_ok && col < p.N) epilogue_chunk(p, r0, row, img, jrow, col);
-          if (row_ok && col + 32 < p.N) epilogue_chunk(p, r1, row, img, jrow, col + 32);
+          if (row_ok && col < p.N) epilogue_chunk(p, r0, row, img, jrow, col, bias_w + c0 / 8);
+          if (row_ok && col + 32 < p.N) epilogue_chunk(p, r1, row, img, jrow, col + 32, bias_w + c0 / 8 + 4);
         }
       } else {
         // ---- K-split: park this slice's partial rows, then the last slice to arrive finishes the tile
@@ -261,7 +296,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 r0[4 * g] = __float_as_uint(v.x); r0[4 * g + 1] = __float_as_uint(v.y);
                 r0[4 * g + 2] = __float_as_uint(v.z); r0[4 * g + 3] = __float_as_uint(v.w);
               }
-              epilogue_chunk(p, r0, row, img, jrow, col);
+              epilogue_chunk(p, r0, row, img, jrow, col, bias_w + c0 / 8);
             }
           }
         }
@@ -291,8 +326,8 @@ void load_encode() {
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
 }
 
-template <int BN, bool SPLIT> cudaError_t set_attr() {
-  return cudaFuncSetAttribute(gemm_bf16_kernel<BN, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<BN>::kSmemBytes);
+template <int BN, bool SPLIT, bool RESID> cudaError_t set_attr() {
+  return cudaFuncSetAttribute(gemm_bf16_kernel<BN, SPLIT, RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<BN>::smem_bytes(RESID));
 }
 
 }  // namespace
@@ -311,10 +346,13 @@ bool make_tmap_bf16_2d(void* tmap_out, const void* base, uint64_t rows, uint64_t
 }
 
 cudaError_t gemm_init() {
-  cudaError_t e = set_attr<128, false>();
-  if (e == cudaSuccess) e = set_attr<128, true>();
-  if (e == cudaSuccess) e = set_attr<192, false>();
-  if (e == cudaSuccess) e = set_attr<256, false>();
+  cudaError_t e = set_attr<128, false, false>();
+  if (e == cudaSuccess) e = set_attr<128, true, false>();
+  if (e == cudaSuccess) e = set_attr<192, false, false>();
+  if (e == cudaSuccess) e = set_attr<256, false, false>();
+  if (e == cudaSuccess) e = set_attr<128, false, true>();
+  if (e == cudaSuccess) e = set_attr<192, false, true>();
+  if (e == cudaSuccess) e = set_attr<256, false, true>();
   if (e == cudaSuccess) e = gemm_pair_init();
   if (e != cudaSuccess) return e;
   int dev = 0;
@@ -384,10 +422,12 @@ static cudaError_t launch_bn(const GemmArgs& g, const GemmDev& p, int tiles_m, c
   const long tiles = (long)tiles_m * ((g.N + BN - 1) / BN) * p.splits;
   const int grid = (int)(tiles < g_num_sms ? tiles : g_num_sms);
   if (p.splits > 1) {
-    if constexpr (BN == 128) return launch_pdl(gemm_bf16_kernel<128, true>, dim3(grid), dim3(kGemmThreads), GemmCfg<128>::kSmemBytes, st, tmA, tmB, p);
+    if constexpr (BN == 128) return launch_pdl(gemm_bf16_kernel<128, true, false>, dim3(grid), dim3(kGemmThreads), GemmCfg<128>::smem_bytes(false), st, tmA, tmB, p);
     else return cudaErrorInvalidValue;
   } else {
-    return launch_pdl(gemm_bf16_kernel<BN, false>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::kSmemBytes, st, tmA, tmB, p);
+    if (p.epilogue == EPI_RESIDUAL)
+      return launch_pdl(gemm_bf16_kernel<BN, false, true>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::smem_bytes(true), st, tmA, tmB, p);
+    return launch_pdl(gemm_bf16_kernel<BN, false, false>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::smem_bytes(false), st, tmA, tmB, p);
   }
 }
 

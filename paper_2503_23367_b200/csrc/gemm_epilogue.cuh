@@ -38,15 +38,22 @@ __device__ __forceinline__ void report(int32_t* status, int code) {
   if (status) atomicCAS(status, 0, code);
 }
 
-// One 32-column chunk of one accumulator row: bias, optional GELU, then the epilogue's store.
-__device__ __forceinline__ void epilogue_chunk(const GemmDev& p, const uint32_t (&r)[32], int row, int img, int jrow, int col) {
-  float v[32];
+// The epilogue warps copy the bias slice of a tile (BN bf16 <= 512 bytes) into shared memory while they wait
+// for its accumulator, so that no chunk stalls on a global load of 64 bytes of bias.
+constexpr int kBiasSmemBytes = 4 * 512;   // one slice per epilogue warp
+__device__ __forceinline__ void stage_bias(const GemmDev& p, uint4* bias_w, int lane, int n0, int bn) {
+  if (p.bias && lane * 8 < bn && n0 + lane * 8 < p.N) bias_w[lane] = __ldg(reinterpret_cast<const uint4*>(p.bias + n0) + lane);
+  __syncwarp();
+}
+
+// acc + bias (+ GELU) of one 32-column chunk of one accumulator row; bias4 = the chunk's 32 bias values
+// in shared memory (ignored when the GEMM has no bias).
+__device__ __forceinline__ void chunk_values(const GemmDev& p, const uint32_t (&r)[32], int col, float (&v)[32], const uint4* bias4) {
   if (p.bias) {
-    const uint4* bp = reinterpret_cast<const uint4*>(p.bias + col);
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
       if (col + 8 * g < p.N) {
-        uint4 bb = __ldg(bp + g);
+        uint4 bb = bias4[g];
         const uint32_t u[4] = {bb.x, bb.y, bb.z, bb.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -66,6 +73,92 @@ __device__ __forceinline__ void epilogue_chunk(const GemmDev& p, const uint32_t 
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = gelu_tanh_fast(v[i]);
   }
+}
+
+// ---- residual epilogue: out[row, :] += gamma[image of row] * (acc + bias), fp32 in place (+ bf16 copy) ----
+// The accumulator comes out of TMEM one row per thread; read-modify-writing the fp32 stream that way would
+// touch 32 different rows per instruction.  Each 32 x 32 chunk is therefore turned through the warp's
+// shared-memory tile (row pitch 36 floats: conflict-free both ways) so that lane l works on columns
+// 4 * (l & 7) .. +3 of rows (l >> 3) + 4 * i, i = 0..7: 8 lanes cover the 128 contiguous bytes of one row, and
+// a lane's column group is the same for all its rows, so the gate is one float4 per chunk.  One warp issues
+// the whole epilogue of its 32 rows with nothing to hide its instruction latencies behind, so the number
+// of instructions per chunk is what bounds it (measured: taking the loads and stores out changed nothing):
+// everything that does not depend on the chunk (row validity, the image boundary, the row pointers) is
+// set up once per tile.
+constexpr int kResidTilePitch = 36;
+constexpr int kResidSmemBytes = 4 * 32 * kResidTilePitch * 4;   // one tile per epilogue warp
+
+struct ResidRows {
+  float* out0;             // &out[first row of the lane, 4 * (lane & 7)] (column offset of the chunk not included)
+  __nv_bfloat16* aux0;     // same position in the bf16 copy, or nullptr
+  const float* gam0;       // gate vector of the image of the warp's first row (+ the lane's column offset), or nullptr
+  const float* gam1;       // gate vector of the next image
+  int n_rows;              // the lane's rows i < n_rows exist
+  int n_first;             // the lane's rows i < n_first belong to the first image, the others to the next one
+};
+
+// Valid when an image has at least 32 rows (a warp's 32 rows then span at most two images).
+__device__ __forceinline__ ResidRows resid_rows(const GemmDev& p, int lane, int row0) {
+  ResidRows rr;
+  const int r = row0 + (lane >> 3);
+  const int cl = 4 * (lane & 7);
+  rr.out0 = static_cast<float*>(p.out) + (size_t)r * p.N + cl;
+  rr.aux0 = p.aux ? static_cast<__nv_bfloat16*>(p.aux) + (size_t)r * p.N + cl : nullptr;
+  rr.n_rows = max(0, min(8, (p.M - r + 3) >> 2));
+  const int img0 = min(row0, p.M - 1) / p.rows_per_image;
+  rr.n_first = max(0, min(8, ((img0 + 1) * p.rows_per_image - r + 3) >> 2));
+  rr.gam0 = p.gamma ? p.gamma + (size_t)img0 * p.mod_stride + cl : nullptr;
+  rr.gam1 = p.gamma ? rr.gam0 + p.mod_stride : nullptr;
+  return rr;
+}
+
+// The lane's 8 float4 of `out` for the chunk at column `col`; fetched one chunk ahead of its use.
+__device__ __forceinline__ void residual_load_x(const GemmDev& p, const ResidRows& rr, float4 (&x)[8], int lane, int col) {
+  const bool col_ok = col + 4 * (lane & 7) < p.N;
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+    if (col_ok && i < rr.n_rows) x[i] = *reinterpret_cast<const float4*>(rr.out0 + (size_t)(4 * i) * p.N + col);
+}
+
+__device__ __forceinline__ void residual_chunk(const GemmDev& p, const ResidRows& rr, const uint32_t (&r)[32], const float4 (&x)[8],
+                                               float* tile, int lane, int col, const uint4* bias4) {
+  float v[32];
+  chunk_values(p, r, col, v, bias4);
+#pragma unroll
+  for (int g = 0; g < 8; ++g)
+    *reinterpret_cast<float4*>(tile + lane * kResidTilePitch + 4 * g) = make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+  __syncwarp();
+  if (col + 4 * (lane & 7) < p.N) {
+    float4 g0 = make_float4(1.f, 1.f, 1.f, 1.f), g1 = g0;
+    if (rr.gam0) {
+      g0 = __ldg(reinterpret_cast<const float4*>(rr.gam0 + col));
+      if (rr.n_first < rr.n_rows) g1 = __ldg(reinterpret_cast<const float4*>(rr.gam1 + col));
+    }
+    const float* trow = tile + (lane >> 3) * kResidTilePitch + 4 * (lane & 7);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (i < rr.n_rows) {
+        const float4 a = *reinterpret_cast<const float4*>(trow + 4 * i * kResidTilePitch);
+        const float4 gg = i < rr.n_first ? g0 : g1;
+        float4 xv = x[i];
+        xv.x = fmaf(gg.x, a.x, xv.x); xv.y = fmaf(gg.y, a.y, xv.y); xv.z = fmaf(gg.z, a.z, xv.z); xv.w = fmaf(gg.w, a.w, xv.w);
+        *reinterpret_cast<float4*>(rr.out0 + (size_t)(4 * i) * p.N + col) = xv;
+        if (rr.aux0) {
+          uint2 o;
+          o.x = pack_bf16x2(a.x, a.y); o.y = pack_bf16x2(a.z, a.w);
+          *reinterpret_cast<uint2*>(rr.aux0 + (size_t)(4 * i) * p.N + col) = o;
+        }
+      }
+    }
+  }
+  __syncwarp();
+}
+
+// One 32-column chunk of one accumulator row: bias, optional GELU, then the epilogue's store.
+__device__ __forceinline__ void epilogue_chunk(const GemmDev& p, const uint32_t (&r)[32], int row, int img, int jrow, int col,
+                                               const uint4* bias4) {
+  float v[32];
+  chunk_values(p, r, col, v, bias4);
   if (p.epilogue == EPI_BF16 || p.epilogue == EPI_GELU_BF16 || (p.epilogue == EPI_QKV_SPLIT && col < p.q_cols)) {
     const int ld = (p.epilogue == EPI_QKV_SPLIT) ? p.q_cols : p.N;
     uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + (size_t)row * ld + col);

@@ -37,17 +37,23 @@ template <int BN> struct PairCfg {
   static constexpr int kStages = (BN == 256) ? 6 : 7;
   static constexpr int kTmemCols = 512;    // two accumulators, 256 columns apart
   static constexpr int kAccStride = 256;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  // operand stages | per-warp bias slices | barriers | (residual-epilogue kernels only) one turning tile per warp
+  static constexpr int smem_bytes(bool resid) {
+    return kStages * kStageBytes + kBiasSmemBytes + 256 /*barriers*/ + (resid ? kResidSmemBytes : 0) + 1024 /*alignment slack*/;
+  }
 };
 
-template <int BN>
+// RESID: the instantiation launched for the residual epilogue (a kernel of its own: it needs far more registers).
+template <int BN, bool RESID>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
   using Cfg = PairCfg<BN>;
   constexpr int STAGES = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::kStageBytes);  // used in the leader
+  uint4* bias_s = reinterpret_cast<uint4*>(smem + STAGES * Cfg::kStageBytes);   // per-warp bias slice of the tile
+  float* resid_s = reinterpret_cast<float*>(smem + STAGES * Cfg::kStageBytes + kBiasSmemBytes + 256);   // RESID: one tile per warp
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::kStageBytes + kBiasSmemBytes);  // used in the leader
   uint64_t* empty_bar = full_bar + STAGES;   // one per CTA, completed by the leader's commits
   uint64_t* acc_full = empty_bar + STAGES;   // [2] one per CTA
   uint64_t* acc_empty = acc_full + 2;        // [2] used in the leader: 256 arrivals
@@ -148,24 +154,53 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int m0 = (tile % tiles_m) * (2 * BM) + (int)rank * BM, n0 = (tile / tiles_m) * BN;
       const int row = m0 + quarter * 32 + lane;
       const bool row_ok = row < p.M;
+      uint4* bias_w = bias_s + quarter * 32;
+      stage_bias(p, bias_w, lane, n0, BN);
+      // residual epilogue (images of fewer than 32 rows take the row-per-thread path below): the first chunk
+      // of `out` is on its way while the accumulator is computed
+      const bool resid = RESID && p.rows_per_image >= 32;
+      ResidRows rr;
+      float4 xa[8], xb[8];
+      if (resid) {
+        rr = resid_rows(p, lane, m0 + quarter * 32);
+        residual_load_x(p, rr, xa, lane, n0);
+      }
       if (!mbar_wait(&acc_full[buf], (lt >> 1) & 1)) { report(p.status, DEV_TIMEOUT_EPI); break; }
       tc_fence_after();
       const int img = row_ok ? row / p.rows_per_image : 0;
       const int jrow = row_ok ? row - img * p.rows_per_image : 0;
       const uint32_t t0 = tmem_base + lane_off + buf * Cfg::kAccStride;
+      if (resid) {   // whole warp: rows are re-distributed over the lanes
+        float* tile_s = resid_s + quarter * (32 * kResidTilePitch);
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 64) {
-        uint32_t r0[32], r1[32];
-        tmem_ld32(t0 + c0, r0);
-        tmem_ld32(t0 + c0 + 32, r1);
-        tmem_wait_ld();
-        if (c0 + 64 >= BN) {  // accumulator fully in registers: hand the buffer back to the leader's MMA warp
-          tc_fence_before();
-          mbar_arrive_cluster(&acc_empty[buf], 0);
+        for (int ch = 0; ch < BN / 32; ++ch) {   // rolled: the code of one chunk is fetched once and then reused
+          uint32_t r0[32];
+          tmem_ld32(t0 + 32 * ch, r0);
+          if (ch + 1 < BN / 32) residual_load_x(p, rr, xb, lane, n0 + 32 * (ch + 1));
+          tmem_wait_ld();
+          if (ch == BN / 32 - 1) {  // accumulator fully in registers: hand the buffer back to the MMA warp
+            tc_fence_before();
+            mbar_arrive_cluster(&acc_empty[buf], 0);
+          }
+          if (n0 + 32 * ch < p.N) residual_chunk(p, rr, r0, xa, tile_s, lane, n0 + 32 * ch, bias_w + 4 * ch);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) xa[i] = xb[i];
         }
-        const int col = n0 + c0;
-        if (row_ok && col < p.N) epilogue_chunk(p, r0, row, img, jrow, col);
-        if (row_ok && col + 32 < p.N) epilogue_chunk(p, r1, row, img, jrow, col + 32);
+      } else {
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 64) {
+          uint32_t r0[32], r1[32];
+          tmem_ld32(t0 + c0, r0);
+          tmem_ld32(t0 + c0 + 32, r1);
+          tmem_wait_ld();
+          if (c0 + 64 >= BN) {  // accumulator fully in registers: hand the buffer back to the leader's MMA warp
+            tc_fence_before();
+            mbar_arrive_cluster(&acc_empty[buf], 0);
+          }
+          const int col = n0 + c0;
+          if (row_ok && col < p.N) epilogue_chunk(p, r0, row, img, jrow, col, bias_w + c0 / 8);
+          if (row_ok && col + 32 < p.N) epilogue_chunk(p, r1, row, img, jrow, col + 32, bias_w + c0 / 8 + 4);
+        }
       }
     }
   }
@@ -182,10 +217,15 @@ int g_pair_sms = 148;
 
 }  // namespace
 
+template <int BN, bool RESID> static cudaError_t set_pair_attr() {
+  return cudaFuncSetAttribute(gemm_pair_kernel<BN, RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<BN>::smem_bytes(RESID));
+}
+
 cudaError_t gemm_pair_init() {
-  cudaError_t e = cudaFuncSetAttribute(gemm_pair_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<256>::kSmemBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(gemm_pair_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<128>::kSmemBytes);
+  cudaError_t e = set_pair_attr<256, false>();
+  if (e == cudaSuccess) e = set_pair_attr<128, false>();
+  if (e == cudaSuccess) e = set_pair_attr<256, true>();
+  if (e == cudaSuccess) e = set_pair_attr<128, true>();
   if (e != cudaSuccess) return e;
   int dev = 0;
   e = cudaGetDevice(&dev);
@@ -200,8 +240,11 @@ cudaError_t launch_gemm_pair(const GemmArgs& g, const GemmDev& p, int bn, cudaSt
   const long tiles = (long)((g.M + 2 * BM - 1) / (2 * BM)) * ((g.N + bn - 1) / bn);
   const int max_pairs = g_pair_sms / 2;
   const int pairs = (int)(tiles < max_pairs ? tiles : max_pairs);
-  if (bn == 256) return launch_pdl(gemm_pair_kernel<256>, dim3(2 * pairs), dim3(kThreads), PairCfg<256>::kSmemBytes, st, tmA, tmB, p);
-  if (bn == 128) return launch_pdl(gemm_pair_kernel<128>, dim3(2 * pairs), dim3(kThreads), PairCfg<128>::kSmemBytes, st, tmA, tmB, p);
+  const bool resid = p.epilogue == EPI_RESIDUAL;
+  if (bn == 256 && resid) return launch_pdl(gemm_pair_kernel<256, true>, dim3(2 * pairs), dim3(kThreads), PairCfg<256>::smem_bytes(true), st, tmA, tmB, p);
+  if (bn == 128 && resid) return launch_pdl(gemm_pair_kernel<128, true>, dim3(2 * pairs), dim3(kThreads), PairCfg<128>::smem_bytes(true), st, tmA, tmB, p);
+  if (bn == 256) return launch_pdl(gemm_pair_kernel<256, false>, dim3(2 * pairs), dim3(kThreads), PairCfg<256>::smem_bytes(false), st, tmA, tmB, p);
+  if (bn == 128) return launch_pdl(gemm_pair_kernel<128, false>, dim3(2 * pairs), dim3(kThreads), PairCfg<128>::smem_bytes(false), st, tmA, tmB, p);
   return cudaErrorInvalidValue;
 }
 
