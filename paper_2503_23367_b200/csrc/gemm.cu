@@ -263,6 +263,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           while (done < p.splits) {
             const int first_slot = done == 0 ? 0 : 1;
             const int cnt = min(max_slots - first_slot, p.splits - done);
+            if (cnt <= 0) { report(p.status, DEV_TIMEOUT_EPI); ok = false; break; }   // cannot happen while a slice fits the stages twice over
             if (et == 0) {
               fence_proxy_async_all();   // earlier generic accesses to these slots / partials before the copies
               mbar_expect_tx(fix_bar, (uint32_t)cnt * slice_bytes);
