@@ -231,3 +231,43 @@ def step_input(wl: Workload, step: int, kind: str = "iid") -> np.ndarray:
     """Token map entering scale step ``step`` of ``wl`` (fp32 ``[B, n, C]``)."""
     s = wl.sides[step]
     return token_map(wl.seed + 10_000 + 10 * step, wl.B, s, s, wl.C, kind)
+
+
+@dataclass
+class GenerationTensors:
+    """Step-invariant tensors of the synthetic generation loop around the scale step: the quantiser's
+    codebook ``[V, d]`` (fp32), the output head ``w_head [V, C]`` / ``b_head [V]`` (bf16 bits) with its
+    AdaLN vectors ``mod_head [B, 2, C]`` (sigma, beta; fp32), the map from accumulated code vectors to the
+    next scale's tokens ``w_in [C, d]`` / ``b_in [C]`` (fp32) and one position embedding per scale
+    ``pos[k] [n_k, C]`` (fp32)."""
+    codebook: Optional[np.ndarray] = None
+    w_head: Optional[np.ndarray] = None
+    b_head: Optional[np.ndarray] = None
+    mod_head: Optional[np.ndarray] = None
+    w_in: Optional[np.ndarray] = None
+    b_in: Optional[np.ndarray] = None
+    pos: List[np.ndarray] = field(default_factory=list)
+    start: Optional[np.ndarray] = None   # [B, n_0, C] fp32: the token map entering the first step
+
+
+def generation_tensors(wl: Workload, V: int = 4096, d: int = 32, w_std: float = 0.02) -> GenerationTensors:
+    """Draw the generation-loop tensors of ``wl`` (seeds ``wl.seed + 60 ..``).  The head's weights are larger
+    than the blocks' (std ``4 * w_std``) so that its logits spread over a few units, as a trained head's do."""
+    g = GenerationTensors()
+    g.codebook = normal(wl.seed + 60, (V, d), 1.0)
+    g.w_head = normal_bf16(wl.seed + 61, (V, wl.C), 4 * w_std)
+    g.b_head = normal_bf16(wl.seed + 62, (V,), w_std)
+    g.mod_head = normal(wl.seed + 63, (wl.B, 2, wl.C), 0.3)
+    g.w_in = normal(wl.seed + 64, (wl.C, d), 1.0 / math.sqrt(d))
+    g.b_in = normal(wl.seed + 65, (wl.C,), w_std)
+    g.pos = [normal(wl.seed + 70 + k, (wl.tokens(k), wl.C), 0.5) for k in range(len(wl.sides))]
+    g.start = normal(wl.seed + 66, (wl.B, wl.tokens(0), wl.C), 1.0)
+    return g
+
+
+def gumbel_noise(seed: int, shape: Sequence[int]) -> np.ndarray:
+    """Standard Gumbel draws -log(-log(u)) from the counter-based uniforms, fp32.  The sampler's random
+    numbers are an input of both implementations, so neither has to reproduce a generator."""
+    n = int(np.prod(shape))
+    u = uniform01(seed, n).astype(np.float64)
+    return (-np.log(-np.log(u))).astype(np.float32).reshape(shape)
