@@ -224,6 +224,7 @@ fv_status fv_restore_residual(float *x_dev, const void *y_dev, const void *cache
  *   epilogue 0: bf16 store to out [M, N].          1: tanh-GELU then bf16 store.
  *   epilogue 2: fp32 residual: out[m,n] += gamma[m / rows_per_image, n] * (acc + bias)  (out fp32;
  *               gamma NULL = 1; if aux_dev != NULL the bf16 value of acc+bias is also stored there).
+ *   epilogue 4: fp32 store of acc + bias to out [M, N] (aux_dev, gamma_dev ignored).  3 is not a public value.
  *   K % 8 == 0, N % 8 == 0, all pointers 16-byte aligned.  bias_dev may be NULL.
  *   W is treated as a constant of the stream: its first tiles are requested as soon as the kernel starts,
  *   which (programmatic dependent launch) can be while the kernel enqueued just before it is still
@@ -253,6 +254,79 @@ fv_status fv_gemm_bf16(const void *a_dev, const void *w_dev, const void *bias_de
 fv_status fv_attention(const void *q_dev, const void *k_dev, const void *vt_dev, int32_t B,
                        int32_t rows, int32_t H, int32_t C, int32_t kv_len, int32_t kv_capacity,
                        void *out_dev, int32_t *status_dev, void *stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * (4) The generation loop around the scale step -- Sec. 3.1: step k turns the token map of scale k into a
+ *     residual f_k and the running prediction follows Eq. 2,
+ *         r_k = interpolate(r_{k-1}, (h_k, w_k)) + f_k        (Eq. 3 is its unfolded form).
+ *     The paper does not say how f_k is read off the transformer output nor how the next token map is
+ *     built; this library and its CPU oracle take the plain construction of VAR-style models:
+ *         logits = (LayerNorm(y) * (1 + sigma_h) + beta_h) * W_head^T + b_head       (V codebook entries)
+ *         id     = argmax_v (logits_v + tau * noise_v), lowest id on ties   (noise NULL: greedy;
+ *                  standard Gumbel noise: a draw from softmax(logits / tau).  The noise is an INPUT.)
+ *         f_k    = codebook[id];   r_1 = f_1
+ *         x_{k+1} = interpolate(r_k, (h_{k+1}, w_{k+1})) * W_in^T + b_in + pos_{k+1}
+ *     interpolate = nearest neighbour, src = floor(dst * in / out) per axis, as for Eq. 6.            */
+
+/* Head + token choice for one scale step.
+ *   y_dev [B, n, C] fp32 (output of fv_var_step); mod_head_dev fp32 [B, 2, C] (sigma_h, beta_h);
+ *   w_head_dev bf16 [V, C]; b_head_dev bf16 [V] or NULL; noise_dev fp32 [B*n, V] or NULL;
+ *   ids_out_dev int32 [B, n]; logits_out_dev fp32 [B*n, V] or NULL (then the logits live in the workspace).
+ *   workspace_dev: fv_head_workspace_bytes(B*n, C, V) bytes, 256-byte aligned; status_dev as in fv_gemm_bf16.
+ *   The GEMM is the bf16 tensor-core GEMM (fp32 accumulation, fp32 logits); the comparison is exact on
+ *   those fp32 values.  V % 8 == 0, C % 8 == 0, C <= 2048.  Errors: INVALID_ARG, CAPACITY, CUDA. */
+size_t fv_head_workspace_bytes(int32_t rows, int32_t C, int32_t V);
+fv_status fv_head_tokens(const float *y_dev, int32_t B, int32_t n, int32_t C, const float *mod_head_dev,
+                         const void *w_head_dev, const void *b_head_dev, int32_t V,
+                         const float *noise_dev, float tau, int32_t *ids_out_dev, float *logits_out_dev,
+                         void *workspace_dev, size_t workspace_bytes, int32_t *status_dev, void *stream);
+
+/* Token choice alone: ids[r] = argmax_v (logits[r, v] + tau * noise[r, v]), lowest v on ties.
+ * logits_dev fp32 [rows, V]; noise_dev fp32 [rows, V] or NULL; V % 4 == 0. */
+fv_status fv_argmax_rows(const float *logits_dev, const float *noise_dev, float tau, int32_t rows,
+                         int32_t V, int32_t *ids_out_dev, void *stream);
+
+/* Eq. 2: r_out[b, t, :] = (r_prev ? r_prev[b, src(t), :] : 0) + codebook[ids[b, t], :].
+ *   ids_dev int32 [B, h*w] in [0, V) (an id outside is clamped and sets *status_dev, if given, to a
+ *   non-zero code); codebook_dev fp32 [V, d]; r_prev_dev fp32 [B, hp*wp, d] or NULL (first step);
+ *   r_out_dev fp32 [B, h*w, d] (must not alias r_prev_dev).  d % 4 == 0. */
+fv_status fv_residual_accumulate(const int32_t *ids_dev, int32_t B, int32_t h, int32_t w,
+                                 const float *codebook_dev, int32_t V, int32_t d,
+                                 const float *r_prev_dev, int32_t hp, int32_t wp, float *r_out_dev,
+                                 int32_t *status_dev, void *stream);
+
+/* Token map entering the next scale: x[b, t, :] = r[b, src(t), :] * W_in^T + b_in + pos[t, :].
+ *   r_dev fp32 [B, h*w, d]; w_in_dev fp32 [C, d]; b_in_dev fp32 [C] or NULL; pos_dev fp32 [h2*w2, C] or
+ *   NULL; x_out_dev fp32 [B, h2*w2, C].  d in {8, 16, 32, 64}; C % 4 == 0. */
+fv_status fv_next_scale_input(const float *r_dev, int32_t B, int32_t h, int32_t w, int32_t d, int32_t h2,
+                              int32_t w2, const float *w_in_dev, const float *b_in_dev,
+                              const float *pos_dev, int32_t C, float *x_out_dev, void *stream);
+
+typedef struct {
+  int32_t V, d;                 /* codebook entries and their width                                    */
+  const float *codebook_dev;    /* [V, d] fp32                                                         */
+  const void *w_head_dev;       /* [V, C] bf16                                                         */
+  const void *b_head_dev;       /* [V] bf16 or NULL                                                    */
+  const float *mod_head_dev;    /* [B_max, 2, C] fp32: sigma_h, beta_h                                 */
+  const float *w_in_dev;        /* [C, d] fp32                                                         */
+  const float *b_in_dev;        /* [C] fp32 or NULL                                                    */
+  const float *const *pos_dev;  /* HOST array [n_steps] of device pointers [h_k*w_k, C] (entry 0 unused; NULL entries = none) */
+  float tau;                    /* scale of the noise                                                  */
+} fv_generator;
+
+/* The whole K-step loop on `stream`: for every scale step of the context, fv_var_step, head + token
+ * choice, Eq. 2, and the next token map.  The context is reset first.
+ *   start_dev [B, h_0*w_0, C] fp32 : token map entering step 0 (not modified).
+ *   keep_host [n_steps]           : keep ratio per step, as for fv_var_step.
+ *   noise_host NULL, or HOST array [n_steps] of device pointers fp32 [B*h_k*w_k, V] (NULL entries = greedy).
+ *   ids_out_dev int32 [B * sum_k h_k*w_k]: step k's ids [B, h_k*w_k] start at B * sum_{j<k} h_j*w_j.
+ *   r_out_dev fp32 [B, h_K*w_K, d]: the final prediction r_K.
+ *   workspace_dev: fv_generate_workspace_bytes(ctx, gen) bytes, 1024-byte aligned.
+ * Errors: those of the calls it makes. */
+size_t fv_generate_workspace_bytes(const fv_ctx *ctx, const fv_generator *gen);
+fv_status fv_generate(fv_ctx *ctx, const fv_generator *gen, const float *start_dev, int32_t B,
+                      const double *keep_host, const float *const *noise_host, int32_t *ids_out_dev,
+                      float *r_out_dev, void *workspace_dev, size_t workspace_bytes, void *stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Measurement support (no counterpart in the paper; Appendix "efficiency profiling" motivates the

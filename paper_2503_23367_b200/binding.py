@@ -24,7 +24,9 @@ EXPORTS = ["fv_status_string", "fv_k_for", "fv_prune_select_workspace_bytes", "f
            "fv_get_state", "fv_set_state", "fv_kv_pointers", "fv_cache_pointer", "fv_prepare_text",
            "fv_device_status", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_gemm_bf16", "fv_gemm_splitk_workspace_bytes", "fv_gemm_force_path", "fv_attention",
            "fv_kernel_launches", "fv_profile_enable", "fv_profile_read",
-           "fv_prune_select_static", "fv_prune_select_static_capacity"]
+           "fv_prune_select_static", "fv_prune_select_static_capacity",
+           "fv_head_workspace_bytes", "fv_head_tokens", "fv_argmax_rows", "fv_residual_accumulate", "fv_next_scale_input",
+           "fv_generate_workspace_bytes", "fv_generate"]
 
 
 class FvError(RuntimeError):
@@ -44,6 +46,12 @@ class fv_weights(C.Structure):
     _fields_ = [(n, C.POINTER(C.c_void_p)) for n in
                 ("w_qkv", "b_qkv", "w_o", "b_o", "w_fc1", "b_fc1", "w_fc2", "b_fc2", "w_q_x", "w_kv_x", "w_o_x")] + \
                [("mod_dev", C.c_void_p), ("text_dev", C.c_void_p)]
+
+
+class fv_generator(C.Structure):
+    _fields_ = [("V", C.c_int32), ("d", C.c_int32), ("codebook_dev", C.c_void_p), ("w_head_dev", C.c_void_p),
+                ("b_head_dev", C.c_void_p), ("mod_head_dev", C.c_void_p), ("w_in_dev", C.c_void_p), ("b_in_dev", C.c_void_p),
+                ("pos_dev", C.POINTER(C.c_void_p)), ("tau", C.c_float)]
 
 
 _lib = None
@@ -89,6 +97,18 @@ def lib() -> C.CDLL:
         L.fv_prune_select_static_capacity.restype = sz; L.fv_prune_select_static_capacity.argtypes = []
         L.fv_prune_select_static.restype = C.c_int
         L.fv_prune_select_static.argtypes = [vp, i32, i32, i32, i32, dbl, vp, vp, vp, vp, C.POINTER(i32), vp]
+        f32 = C.c_float
+        L.fv_head_workspace_bytes.restype = sz; L.fv_head_workspace_bytes.argtypes = [i32, i32, i32]
+        L.fv_head_tokens.restype = C.c_int
+        L.fv_head_tokens.argtypes = [vp, i32, i32, i32, vp, vp, vp, i32, vp, f32, vp, vp, vp, sz, vp, vp]
+        L.fv_argmax_rows.restype = C.c_int; L.fv_argmax_rows.argtypes = [vp, vp, f32, i32, i32, vp, vp]
+        L.fv_residual_accumulate.restype = C.c_int
+        L.fv_residual_accumulate.argtypes = [vp, i32, i32, i32, vp, i32, i32, vp, i32, i32, vp, vp, vp]
+        L.fv_next_scale_input.restype = C.c_int
+        L.fv_next_scale_input.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, i32, vp, vp]
+        L.fv_generate_workspace_bytes.restype = sz; L.fv_generate_workspace_bytes.argtypes = [vp, C.POINTER(fv_generator)]
+        L.fv_generate.restype = C.c_int
+        L.fv_generate.argtypes = [vp, C.POINTER(fv_generator), vp, i32, C.POINTER(dbl), C.POINTER(vp), vp, vp, vp, sz, vp]
         L.fv_kernel_launches.restype = C.c_uint64; L.fv_kernel_launches.argtypes = []
         L.fv_profile_enable.restype = C.c_int; L.fv_profile_enable.argtypes = [i32]
         L.fv_profile_read.restype = C.c_int
@@ -226,6 +246,90 @@ def fv_attention(q: torch.Tensor, k_cache: torch.Tensor, vt_cache: torch.Tensor,
     _check(lib().fv_attention(_ptr(q), _ptr(k_cache), _ptr(vt_cache), B, rows, H, Cw, kv_len, cap, _ptr(out), _ptr(status),
                               _stream()), "fv_attention")
     return out
+
+
+def fv_argmax_rows(logits: torch.Tensor, noise: Optional[torch.Tensor] = None, tau: float = 1.0) -> torch.Tensor:
+    rows, V = logits.shape
+    ids = torch.empty(rows, dtype=torch.int32, device=logits.device)
+    _check(lib().fv_argmax_rows(_ptr(logits), _ptr(noise), float(tau), rows, V, _ptr(ids), _stream()), "fv_argmax_rows")
+    return ids
+
+
+def fv_head_tokens(y: torch.Tensor, mod_head: torch.Tensor, w_head: torch.Tensor, b_head: Optional[torch.Tensor],
+                   noise: Optional[torch.Tensor] = None, tau: float = 1.0, want_logits: bool = False,
+                   status: Optional[torch.Tensor] = None):
+    """y fp32 [B, n, C]; returns ids int32 [B, n] (and the fp32 logits [B*n, V] when asked)."""
+    B, n, Cw = y.shape
+    V = w_head.shape[0]
+    ws_bytes = lib().fv_head_workspace_bytes(B * n, Cw, V)
+    ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device=y.device)
+    wsp = (ws.data_ptr() + 255) // 256 * 256
+    ids = torch.empty((B, n), dtype=torch.int32, device=y.device)
+    logits = torch.empty((B * n, V), dtype=torch.float32, device=y.device) if want_logits else None
+    _check(lib().fv_head_tokens(_ptr(y), B, n, Cw, _ptr(mod_head), _ptr(w_head), _ptr(b_head), V, _ptr(noise), float(tau),
+                                _ptr(ids), _ptr(logits), wsp, ws_bytes, _ptr(status), _stream()), "fv_head_tokens")
+    return (ids, logits) if want_logits else ids
+
+
+def fv_residual_accumulate(ids: torch.Tensor, h: int, w: int, codebook: torch.Tensor, r_prev: Optional[torch.Tensor] = None,
+                           hp: int = 0, wp: int = 0, status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    B = ids.shape[0]
+    V, d = codebook.shape
+    out = torch.empty((B, h * w, d), dtype=torch.float32, device=ids.device)
+    _check(lib().fv_residual_accumulate(_ptr(ids), B, h, w, _ptr(codebook), V, d, _ptr(r_prev), hp, wp, _ptr(out), _ptr(status),
+                                        _stream()), "fv_residual_accumulate")
+    return out
+
+
+def fv_next_scale_input(r: torch.Tensor, h: int, w: int, h2: int, w2: int, w_in: torch.Tensor, b_in: Optional[torch.Tensor],
+                        pos: Optional[torch.Tensor]) -> torch.Tensor:
+    B, _, d = r.shape
+    Cw = w_in.shape[0]
+    out = torch.empty((B, h2 * w2, Cw), dtype=torch.float32, device=r.device)
+    _check(lib().fv_next_scale_input(_ptr(r), B, h, w, d, h2, w2, _ptr(w_in), _ptr(b_in), _ptr(pos), Cw, _ptr(out), _stream()),
+           "fv_next_scale_input")
+    return out
+
+
+class FvGenerator:
+    """Device copies of `inputs.GenerationTensors` and the fv_generate call for one context."""
+
+    def __init__(self, ctx: "FvContext", gt, tau: float = 1.0):
+        dev = ctx.dev
+        f32 = lambda a: torch.from_numpy(a).to(dev, torch.float32).contiguous()
+        bf = lambda a: torch.from_numpy(a.view("int16")).to(dev).view(torch.bfloat16).contiguous()
+        self.ctx = ctx
+        self.codebook, self.w_head, self.b_head = f32(gt.codebook), bf(gt.w_head), bf(gt.b_head)
+        self.mod_head, self.w_in, self.b_in = f32(gt.mod_head), f32(gt.w_in), f32(gt.b_in)
+        self.pos = [f32(p) for p in gt.pos]
+        self.V, self.d = self.codebook.shape
+        self._pos_arr = (C.c_void_p * len(self.pos))(*[p.data_ptr() for p in self.pos])
+        self.gen = fv_generator(self.V, self.d, self.codebook.data_ptr(), self.w_head.data_ptr(), self.b_head.data_ptr(),
+                                self.mod_head.data_ptr(), self.w_in.data_ptr(), self.b_in.data_ptr(),
+                                C.cast(self._pos_arr, C.POINTER(C.c_void_p)), float(tau))
+        nbytes = lib().fv_generate_workspace_bytes(ctx.ctx, C.byref(self.gen))
+        self.ws = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
+        self.ws_bytes = nbytes
+
+    def generate(self, start: torch.Tensor, keep: Sequence[float], noise: Optional[Sequence[Optional[torch.Tensor]]] = None):
+        """start fp32 [B, n_0, C].  Returns (ids per step: list of int32 [B, n_k], r_K fp32 [B, n_K, d])."""
+        B = start.shape[0]
+        hw = self.ctx.hw
+        ns = [h * w for h, w in hw]
+        ids = torch.empty(B * sum(ns), dtype=torch.int32, device=start.device)
+        r = torch.empty((B, ns[-1], self.d), dtype=torch.float32, device=start.device)
+        keep_arr = (C.c_double * len(hw))(*[float(k) for k in keep])
+        noise_arr = None
+        if noise is not None:
+            noise_arr = (C.c_void_p * len(hw))(*[None if t is None else t.data_ptr() for t in noise])
+        wsp = (self.ws.data_ptr() + 1023) // 1024 * 1024
+        _check(lib().fv_generate(self.ctx.ctx, C.byref(self.gen), _ptr(start), B, keep_arr, noise_arr, _ptr(ids), _ptr(r), wsp,
+                                 self.ws_bytes, _stream()), "fv_generate")
+        out, off = [], 0
+        for n in ns:
+            out.append(ids[off:off + B * n].view(B, n))
+            off += B * n
+        return out, r
 
 
 class FvContext:

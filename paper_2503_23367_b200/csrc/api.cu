@@ -38,6 +38,10 @@ struct fv_ctx {
   size_t kv_block_bytes = 0, k_bytes = 0, text_k_bytes = 0, text_block_bytes = 0, cache_sub_bytes = 0;
 };
 
+namespace fv {
+const fv_config* ctx_config(const fv_ctx* ctx) { return &ctx->cfg; }
+}  // namespace fv
+
 namespace {
 
 std::once_flag g_init_once;
@@ -179,7 +183,7 @@ fv_status fv_restore_residual(float* x_dev, const void* y_dev, const void* cache
 fv_status fv_gemm_bf16(const void* a_dev, const void* w_dev, const void* bias_dev, int32_t M, int32_t N, int32_t K,
                        int32_t epilogue, void* out_dev, void* aux_dev, const float* gamma_dev, int32_t mod_stride,
                        int32_t rows_per_image, int32_t* status_dev, void* splitk_ws_dev, size_t splitk_ws_bytes, void* stream) {
-  if (!a_dev || !w_dev || !out_dev || epilogue < 0 || epilogue > 2) return FV_ERR_INVALID_ARG;
+  if (!a_dev || !w_dev || !out_dev || epilogue < 0 || epilogue > 4 || epilogue == EPI_QKV_SPLIT) return FV_ERR_INVALID_ARG;
   if (splitk_ws_dev && (splitk_ws_bytes < gemm_splitk_ws_bytes() || !aligned16(splitk_ws_dev))) return FV_ERR_CAPACITY;
   if (!aligned16(a_dev) || !aligned16(w_dev) || !aligned16(out_dev) || (bias_dev && !aligned16(bias_dev))) return FV_ERR_INVALID_ARG;
   if (ensure_init() != cudaSuccess) return FV_ERR_CUDA;

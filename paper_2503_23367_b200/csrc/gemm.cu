@@ -174,7 +174,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       stage_bias(p, bias_w, lane, n0, BN);
       // residual epilogue (images of fewer than 32 rows take the row-per-thread path below): the first chunk
       // of `out` is on its way while the accumulator is computed
-      const bool resid = RESID && p.rows_per_image >= 32;
+      const bool resid = RESID && (p.rows_per_image >= 32 || p.epilogue == EPI_F32);
       ResidRows rr;
       float4 xa[8], xb[8];
       if (resid) {
@@ -426,7 +426,7 @@ static cudaError_t launch_bn(const GemmArgs& g, const GemmDev& p, int tiles_m, c
     if constexpr (BN == 128) return launch_pdl(gemm_bf16_kernel<128, true, false>, dim3(grid), dim3(kGemmThreads), GemmCfg<128>::smem_bytes(false), st, tmA, tmB, p);
     else return cudaErrorInvalidValue;
   } else {
-    if (p.epilogue == EPI_RESIDUAL)
+    if (p.epilogue == EPI_RESIDUAL || p.epilogue == EPI_F32)
       return launch_pdl(gemm_bf16_kernel<BN, false, true>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::smem_bytes(true), st, tmA, tmB, p);
     return launch_pdl(gemm_bf16_kernel<BN, false, false>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::smem_bytes(false), st, tmA, tmB, p);
   }
@@ -462,6 +462,7 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   }
   p.bias = static_cast<const __nv_bfloat16*>(g.bias);
   p.M = g.M; p.N = g.N; p.K = g.K; p.epilogue = g.epilogue; p.out = g.out; p.aux = g.aux; p.gamma = g.gamma;
+  if (g.epilogue == EPI_F32) { p.aux = nullptr; p.gamma = nullptr; }
   p.mod_stride = g.mod_stride; p.rows_per_image = g.rows_per_image; p.q_cols = g.q_cols; p.C = g.C;
   p.k_cache = static_cast<__nv_bfloat16*>(g.k_cache); p.vt_cache = static_cast<__nv_bfloat16*>(g.vt_cache);
   p.kv_capacity = g.kv_capacity; p.kv_offset = g.kv_offset; p.status = g.status;

@@ -75,7 +75,8 @@ __device__ __forceinline__ void chunk_values(const GemmDev& p, const uint32_t (&
   }
 }
 
-// ---- residual epilogue: out[row, :] += gamma[image of row] * (acc + bias), fp32 in place (+ bf16 copy) ----
+// ---- residual epilogue: out[row, :] += gamma[image of row] * (acc + bias), fp32 in place (+ bf16 copy);
+// also the plain fp32 result (EPI_F32: out = acc + bias, gamma and aux unused) ----
 // The accumulator comes out of TMEM one row per thread; read-modify-writing the fp32 stream that way would
 // touch 32 different rows per instruction.  Each 32 x 32 chunk is therefore turned through the warp's
 // shared-memory tile (row pitch 36 floats: conflict-free both ways) so that lane l works on columns
@@ -115,6 +116,11 @@ __device__ __forceinline__ ResidRows resid_rows(const GemmDev& p, int lane, int 
 // The lane's 8 float4 of `out` for the chunk at column `col`; fetched one chunk ahead of its use.
 __device__ __forceinline__ void residual_load_x(const GemmDev& p, const ResidRows& rr, float4 (&x)[8], int lane, int col) {
   const bool col_ok = col + 4 * (lane & 7) < p.N;
+  if (p.epilogue == EPI_F32) {   // plain fp32 result: nothing to add to
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    return;
+  }
 #pragma unroll
   for (int i = 0; i < 8; ++i)
     if (col_ok && i < rr.n_rows) x[i] = *reinterpret_cast<const float4*>(rr.out0 + (size_t)(4 * i) * p.N + col);
@@ -171,6 +177,11 @@ __device__ __forceinline__ void epilogue_chunk(const GemmDev& p, const uint32_t 
         dst[g] = o;
       }
     }
+  } else if (p.epilogue == EPI_F32) {
+    float4* xr = reinterpret_cast<float4*>(static_cast<float*>(p.out) + (size_t)row * p.N + col);
+#pragma unroll
+    for (int g = 0; g < 8; ++g)
+      if (col + 4 * g < p.N) xr[g] = make_float4(v[4 * g + 0], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
   } else if (p.epilogue == EPI_RESIDUAL) {
     float4* xr = reinterpret_cast<float4*>(static_cast<float*>(p.out) + (size_t)row * p.N + col);
     const float4* gp = p.gamma ? reinterpret_cast<const float4*>(p.gamma + (size_t)img * p.mod_stride + col) : nullptr;

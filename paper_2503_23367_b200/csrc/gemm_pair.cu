@@ -158,7 +158,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       stage_bias(p, bias_w, lane, n0, BN);
       // residual epilogue (images of fewer than 32 rows take the row-per-thread path below): the first chunk
       // of `out` is on its way while the accumulator is computed
-      const bool resid = RESID && p.rows_per_image >= 32;
+      const bool resid = RESID && (p.rows_per_image >= 32 || p.epilogue == EPI_F32);
       ResidRows rr;
       float4 xa[8], xb[8];
       if (resid) {
@@ -240,7 +240,7 @@ cudaError_t launch_gemm_pair(const GemmArgs& g, const GemmDev& p, int bn, cudaSt
   const long tiles = (long)((g.M + 2 * BM - 1) / (2 * BM)) * ((g.N + bn - 1) / bn);
   const int max_pairs = g_pair_sms / 2;
   const int pairs = (int)(tiles < max_pairs ? tiles : max_pairs);
-  const bool resid = p.epilogue == EPI_RESIDUAL;
+  const bool resid = p.epilogue == EPI_RESIDUAL || p.epilogue == EPI_F32;
   if (bn == 256 && resid) return launch_pdl(gemm_pair_kernel<256, true>, dim3(2 * pairs), dim3(kThreads), PairCfg<256>::smem_bytes(true), st, tmA, tmB, p);
   if (bn == 128 && resid) return launch_pdl(gemm_pair_kernel<128, true>, dim3(2 * pairs), dim3(kThreads), PairCfg<128>::smem_bytes(true), st, tmA, tmB, p);
   if (bn == 256) return launch_pdl(gemm_pair_kernel<256, false>, dim3(2 * pairs), dim3(kThreads), PairCfg<256>::smem_bytes(false), st, tmA, tmB, p);

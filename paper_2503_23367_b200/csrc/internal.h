@@ -85,14 +85,14 @@ cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* p
                                 int k, int h, int w, int C, void* out, cudaStream_t st);
 
 // ---- gemm.cu : tcgen05 GEMM with fused epilogues -----------------------------------------------
-enum GemmEpilogue : int { EPI_BF16 = 0, EPI_GELU_BF16 = 1, EPI_RESIDUAL = 2, EPI_QKV_SPLIT = 3 };
+enum GemmEpilogue : int { EPI_BF16 = 0, EPI_GELU_BF16 = 1, EPI_RESIDUAL = 2, EPI_QKV_SPLIT = 3, EPI_F32 = 4 };
 struct GemmArgs {
   const void* a;     // [M,K] bf16
   const void* w;     // [N,K] bf16
   const void* bias;  // [N] bf16 or null
   int M, N, K;
   int epilogue;
-  void* out;           // EPI_BF16/GELU: bf16 [M,N]; EPI_RESIDUAL: fp32 [M,N] in place; EPI_QKV_SPLIT: Q bf16 [M,q_cols]
+  void* out;           // EPI_BF16/GELU: bf16 [M,N]; EPI_RESIDUAL: fp32 [M,N] in place; EPI_F32: fp32 [M,N] written; EPI_QKV_SPLIT: Q bf16 [M,q_cols]
   void* aux;           // EPI_RESIDUAL: optional bf16 [M,N] copy of acc+bias
   const float* gamma;  // EPI_RESIDUAL: per-image gate or null
   int mod_stride;      // floats between images in gamma
@@ -128,4 +128,9 @@ fv_status launch_attention(const AttnArgs& a, cudaStream_t st);
 // 2-D bf16 row-major tensor [rows, cols] -> TMA descriptor with a (box_rows x 64) box and 128-byte swizzle.
 bool make_tmap_bf16_2d(void* tmap_out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 
+// generate.cu reads the step sizes of a context (api.cu owns the context's layout)
+}  // namespace fv
+struct fv_ctx;
+namespace fv {
+const fv_config* ctx_config(const fv_ctx* ctx);
 }  // namespace fv

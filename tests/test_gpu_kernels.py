@@ -277,6 +277,28 @@ def test_gemm_residual_epilogue_with_cache_copy():
     assert err <= MAX_ABS and cos >= MIN_COS
 
 
+@pytest.mark.parametrize("path", [0, 2, 3, 4, 5, 6])
+@pytest.mark.parametrize("M,N,K,rows_per_image,splitk", [(300, 512, 256, 300, False), (7, 136, 72, 7, False), (1000, 1032, 1024, 500, False),
+                                                          (2, 2048, 2048, 1, True), (130, 1920, 1920, 20, False)])
+def test_gemm_fp32_epilogue(M, N, K, rows_per_image, splitk, path):
+    """Epilogue 4: the fp32 value of acc + bias itself, on every kernel (one-CTA widths, CTA pairs, K split) and
+    with images shorter than a warp's 32 rows (the row-per-thread store path)."""
+    a = I.normal_bf16(85, (M, K)); w = I.normal_bf16(86, (N, K), 0.03); b = I.normal_bf16(87, (N,), 0.02)
+    out = torch.full((M, N), 7.0, dtype=torch.float32, device=DEV)          # must be overwritten, not added to
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = torch.zeros(fv.lib().fv_gemm_splitk_workspace_bytes(), dtype=torch.uint8, device=DEV) if splitk else None
+    assert fv.lib().fv_gemm_force_path(path) == 0
+    try:
+        fv.fv_gemm_bf16(bf16_dev(a), bf16_dev(w), bf16_dev(b), epilogue=4, out=out, rows_per_image=rows_per_image, status=status,
+                        splitk_ws=ws)
+        torch.cuda.synchronize()
+    finally:
+        fv.lib().fv_gemm_force_path(0)
+    assert int(status.item()) == 0
+    ref = O.linear(I.bf16_bits_to_f32(a), I.bf16_bits_to_f32(w), I.bf16_bits_to_f32(b))
+    assert np.abs(out.cpu().numpy() - ref).max() <= 2e-3      # fp32 accumulation of K bf16 x bf16 products
+
+
 # ------------------------------------------------------------------ attention over the KV cache
 ATTN_CASES = [  # B, rows, H, C, kv_len, cap
     (2, 85, 4, 256, 340, 344), (1, 300, 2, 256, 1000, 1024), (2, 128, 16, 1024, 485, 488), (1, 1, 4, 256, 1, 8),
