@@ -357,6 +357,33 @@ def ours(args, wl):
                     "peak_source": f"of {peaks['source']} ({'sustained bf16 matmul' if d['bound'] == 'tensor' else 'copy bandwidth'})",
                     "avg_launch_ms": d["ms_per_step"] / max(1, d["launches_per_step"])}
 
+    # ---- the generation loop around the step (Sec. 3.1, Eq. 2-3): head, greedy token choice, residual
+    # accumulation and the next token map after every step, all K steps in one fv_generate call
+    generation = None
+    if not args.skip_generation:
+        gen_t = I.generation_tensors(wl, V=4096, d=32)
+        fgen = fv.FvGenerator(ctx, gen_t)
+        start = torch.from_numpy(gen_t.start).to(dev)
+        for _ in range(2):
+            fgen.generate(start, wl.keep)
+        barrier()
+        ng = max(2, min(args.steps, 5))
+        before = fv.fv_profile_read()
+        evg = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ng)]
+        for a, b in evg:
+            a.record(); fgen.generate(start, wl.keep); b.record()
+        barrier()
+        if ctx.device_status() != 0:
+            raise SystemExit("a kernel reported an expired wait")
+        g_ms = max_over_ranks(statistics.mean(a.elapsed_time(b) for a, b in evg))
+        g_launches = sum(v["launches"] for v in fv.fv_profile_read().values()) // ng
+        generation = {"what": "fv_generate: every scale step followed by head (V = 4096), greedy token choice, Eq. 2 (d = 32) and "
+                              "the next token map; synthetic codebook and head",
+                      "ms_per_step": g_ms, "ms_per_image": g_ms / wl.B, "ms_outside_the_scale_steps": g_ms - ms_per_step,
+                      "gpu_launches": g_launches}
+        del fgen
+        torch.cuda.empty_cache()
+
     # ---- the coarser granularity beside it: one selection and one restoration around the whole stack of
     # blocks of a pruned step (not the paper's configuration, which is what `value` measures)
     variant = None
@@ -424,7 +451,8 @@ def ours(args, wl):
             "ms_per_image": ms_per_step / wl.B, "ms_per_image_pruned_steps": pruned_ms / wl.B,
             "scale_step_ms": [round(t, 4) for t in step_ms], "wall_ms_per_step": t_wall * 1e3 / args.steps,
             "roofline": roofline, "kernels": kernels, "kernels_pruned_steps": kernels_pruned, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": gpu_launches,
-            "clocks": clocks, "unpruned_gpu": unpruned, "per_step_granularity": variant, "peaks": peaks}
+            "clocks": clocks, "unpruned_gpu": unpruned, "per_step_granularity": variant, "generation_loop": generation,
+            "peaks": peaks}
     print(json.dumps(line))
 
 
@@ -439,6 +467,7 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer end-to-end leg")
     ap.add_argument("--skip-profile", action="store_true", help="omit the per-kernel-class timing passes")
     ap.add_argument("--skip-unpruned", action="store_true", help="omit the unpruned GPU comparison")
+    ap.add_argument("--skip-generation", action="store_true", help="omit the generation-loop (fv_generate) timing")
     ap.add_argument("--skip-variant", action="store_true", help="omit the per-step-granularity comparison")
     ap.add_argument("--blocks", type=int, default=0,
                     help="profiling only: run this many transformer blocks instead of the workload's depth (the line says so; not a bench number)")
