@@ -456,6 +456,75 @@ def ours(args, wl):
     print(json.dumps(line))
 
 
+def sweep(args, wl):
+    """Pruning-ratio and caching-step curves (the efficiency side of the paper's ablations on the pruning
+    ratio and on the number of pruned steps, with synthetic weights): one JSON line, `--sweep`."""
+    from dataclasses import replace
+    from paper_2503_23367_b200 import binding as fv
+    from paper_2503_23367_b200 import build as fv_build
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the pruned VAR step has no CPU path")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    fv_build.build()
+    fv.lib()
+    S = len(wl.sides)
+    gt = GpuTensors(wl, dev, seed=wl.seed)
+    g = torch.Generator(device=dev); g.manual_seed(wl.seed + 77)
+    xs = [torch.randn(wl.B, wl.tokens(i), wl.C, generator=g, device=dev, dtype=torch.float32) for i in range(S)]
+    outs = [torch.empty_like(x) for x in xs]
+    hw = [(s_, s_) for s_ in wl.sides]
+
+    def run(keep):
+        w2 = replace(wl, keep=tuple(keep))
+        pruned = [i for i in range(S) if keep[i] < 1.0]
+        cap = sum(kept(w2, i) for i in range(S))
+        ctx = fv.FvContext(wl.L, wl.C, wl.H, hw, w2.cache_step, wl.B, cap, gt, cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio, device=dev)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(S + 1)] for _ in range(3)]
+        for rep in range(5):
+            ctx.reset()
+            for i in range(S):
+                if rep >= 2:
+                    ev[rep - 2][i].record()
+                ctx.var_step(xs[i], i, keep[i], out=outs[i])
+            if rep >= 2:
+                ev[rep - 2][S].record()
+        torch.cuda.synchronize()
+        if ctx.device_status() != 0:
+            raise SystemExit("a kernel reported an expired wait")
+        total = statistics.mean(e[0].elapsed_time(e[S]) for e in ev)
+        step = [statistics.mean(e[i].elapsed_time(e[i + 1]) for e in ev) for i in range(S)]
+        ctx.close()
+        del ctx
+        torch.cuda.empty_cache()
+        return total, step, pruned, w2
+
+    base_total, base_step, _, _ = run((1.0,) * S)
+    default_pruned = [i for i in range(S) if wl.keep[i] < 1.0]
+    rows = []
+    for ratio in (0.25, 0.4, 0.5, 0.6, 0.75, 0.9):
+        keep = [1.0] * S
+        for i in default_pruned:
+            keep[i] = 1.0 - ratio
+        total, step, pruned, w2 = run(keep)
+        p_ms = sum(step[i] for i in pruned)
+        rows.append({"sweep": "pruning ratio on the workload's pruned steps", "pruning_ratio": ratio, "pruned_steps": len(pruned),
+                     "ms_per_image": total / wl.B, "speedup_whole_schedule": base_total / total,
+                     "speedup_pruned_steps": sum(base_step[i] for i in pruned) / p_ms,
+                     "forwarded_tokens_per_s": sum(wl.B * kept(w2, i) for i in pruned) / (p_ms * 1e-3)})
+    for n_pruned in (1, 2, 3, 4):
+        keep = [1.0] * S
+        for i in range(S - n_pruned, S):
+            keep[i] = 0.5
+        total, step, pruned, w2 = run(keep)
+        p_ms = sum(step[i] for i in pruned)
+        rows.append({"sweep": "number of pruned steps N at pruning ratio 0.5 (caching step K-N)", "pruned_steps": n_pruned,
+                     "cache_step": S - n_pruned - 1, "pruning_ratio": 0.5, "ms_per_image": total / wl.B,
+                     "speedup_whole_schedule": base_total / total, "speedup_pruned_steps": sum(base_step[i] for i in pruned) / p_ms,
+                     "forwarded_tokens_per_s": sum(wl.B * kept(w2, i) for i in pruned) / (p_ms * 1e-3)})
+    print(json.dumps({"sweep": rows, "workload": wl.name, "B": wl.B, "unpruned_ms_per_image": base_total / wl.B, "data": "synthetic"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -468,6 +537,7 @@ def main():
     ap.add_argument("--skip-profile", action="store_true", help="omit the per-kernel-class timing passes")
     ap.add_argument("--skip-unpruned", action="store_true", help="omit the unpruned GPU comparison")
     ap.add_argument("--skip-generation", action="store_true", help="omit the generation-loop (fv_generate) timing")
+    ap.add_argument("--sweep", action="store_true", help="print pruning-ratio and caching-step curves instead of the bench line")
     ap.add_argument("--skip-variant", action="store_true", help="omit the per-step-granularity comparison")
     ap.add_argument("--blocks", type=int, default=0,
                     help="profiling only: run this many transformer blocks instead of the workload's depth (the line says so; not a bench number)")
@@ -478,6 +548,8 @@ def main():
         wl = wl.with_depth(args.blocks)
     if args.impl == "reference":
         reference_arm(args, wl)
+    elif args.sweep:
+        sweep(args, wl)
     else:
         ours(args, wl)
 
