@@ -26,6 +26,21 @@ Readings taken where the paper is silent or inconsistent (each is also listed in
     1/sqrt(head_dim), biases on qkv / out / fc1 / fc2, optional cross-attention to text with plain
     LN, no biases and no gate.
 
+Backbone extras (all off by default; the paper names none of them, they belong to the backbones it prunes,
+so each is a reading stated here and pinned on its own):
+  * `interp_mode="bilinear"`: interpolate(.) of Eq. 6 as a bilinear blend with half-pixel centres
+    (source coordinate (dst + 0.5) * in / out - 0.5, clamped), the convention of library resizing routines.
+  * `qk_scale` [L, H]: cosine attention -- in the self-attention sublayer every head's query and key are
+    divided by their Euclidean norm (floored at 1e-12) and the query is multiplied by the head's scale.
+  * `rope_base`: two-dimensional rotary position embedding in the self-attention sublayer.  A token at
+    row y, column x of the (h, w) map of its scale sits at (y * h_K / h, x * w_K / w) in the frame of the
+    last scale, so that tokens of different scales covering the same image region get the same phase.  Of a
+    head's hd channels the first half is rotated by the row coordinate, the second by the column coordinate;
+    channel pairs (2j, 2j+1) of a half turn by coordinate * base^(-j / (hd/4)).  The position is that of the
+    token's ORIGINAL slot in the map: at a pruned step row j of the compact tensor is token idx[j], and it is
+    idx[j] that is rotated by -- the one place where pruning reaches into the attention arithmetic.
+    Order: normalise, then rotate (a rotation keeps the norm).  Values are not touched.
+
 Granularity.  The paper wraps EVERY attention / FFN layer with the selection / restoration pair
 (Sec. 3.3 "Implementation"); that is `granularity="sublayer"`, the default.  `granularity="step"` is the
 coarser variant in which the pair wraps the whole stack of blocks of a scale step: one selection on the
@@ -132,11 +147,36 @@ def ctr_upsample(cache: np.ndarray, hc: int, wc: int, h: int, w: int) -> np.ndar
     return cache[:, nearest_source(h, w, hc, wc), :]
 
 
+def bilinear_taps(n_out: int, n_in: int):
+    """Per destination index along one axis: the two source indices and the weight of the second one, for a
+    blend with half-pixel centres: s = (dst + 0.5) * n_in / n_out - 0.5 clamped to [0, n_in - 1]."""
+    i0 = np.empty(n_out, dtype=np.int64); i1 = np.empty(n_out, dtype=np.int64); t = np.empty(n_out, dtype=F64)
+    for o in range(n_out):
+        s = (o + 0.5) * n_in / n_out - 0.5
+        s = min(max(s, 0.0), n_in - 1.0)
+        i0[o] = int(math.floor(s))
+        i1[o] = min(i0[o] + 1, n_in - 1)
+        t[o] = s - i0[o]
+    return i0, i1, t
+
+
+def ctr_upsample_bilinear(cache: np.ndarray, hc: int, wc: int, h: int, w: int) -> np.ndarray:
+    """Eq. 6 with interpolate = bilinear.  cache [B,hc*wc,C] -> [B,h*w,C]."""
+    c = np.asarray(cache, dtype=F64).reshape(cache.shape[0], hc, wc, cache.shape[-1])
+    y0, y1, ty = bilinear_taps(h, hc)
+    x0, x1, tx = bilinear_taps(w, wc)
+    ty = ty[None, :, None, None]; tx = tx[None, None, :, None]
+    top = c[:, y0][:, :, x0] * (1 - tx) + c[:, y0][:, :, x1] * tx
+    bot = c[:, y1][:, :, x0] * (1 - tx) + c[:, y1][:, :, x1] * tx
+    return (top * (1 - ty) + bot * ty).reshape(cache.shape[0], h * w, cache.shape[-1])
+
+
 def cached_token_restoration(pivots: np.ndarray, idx: np.ndarray, cache: np.ndarray,
-                             hc: int, wc: int, h: int, w: int) -> np.ndarray:
+                             hc: int, wc: int, h: int, w: int, interp_mode: str = "nearest") -> np.ndarray:
     """Algorithm 1, second routine: upsample the cache to the current scale, then write the
     forwarded rows into their slots.  pivots [B,k,C], idx [B,k] -> [B,h*w,C]."""
-    out = np.array(ctr_upsample(np.asarray(cache, dtype=F64), hc, wc, h, w), dtype=F64, copy=True)
+    up = ctr_upsample if interp_mode == "nearest" else ctr_upsample_bilinear
+    out = np.array(up(np.asarray(cache, dtype=F64), hc, wc, h, w), dtype=F64, copy=True)
     for b in range(out.shape[0]):
         out[b, idx[b], :] = pivots[b]
     return out
@@ -178,6 +218,40 @@ def softmax_rows(s: np.ndarray) -> np.ndarray:
     return e / e.sum(axis=-1, keepdims=True)
 
 
+def qk_normalise(v: np.ndarray, H: int, scale: Optional[np.ndarray] = None, eps: float = 1e-12) -> np.ndarray:
+    """Every head's vector divided by its Euclidean norm (floored at eps), times scale[h] if given.  v [k,C]."""
+    k, C = v.shape
+    hd = C // H
+    vh = np.asarray(v, dtype=F64).reshape(k, H, hd)
+    out = vh / np.maximum(np.sqrt((vh ** 2).sum(-1, keepdims=True)), eps)
+    if scale is not None:
+        out = out * np.asarray(scale, dtype=F64)[None, :, None]
+    return out.reshape(k, C)
+
+
+def rope_angles(tokens: np.ndarray, h: int, w: int, h_last: int, w_last: int, hd: int, base: float) -> np.ndarray:
+    """Rotation angles [len(tokens), hd/2] of the tokens (row-major indices into the (h,w) map): columns
+    [0, hd/4) = row coordinate * base^(-j/(hd/4)), columns [hd/4, hd/2) = column coordinate * the same."""
+    quarter = hd // 4
+    tok = np.asarray(tokens, dtype=np.int64)
+    py = (tok // w).astype(F64) * h_last / h
+    px = (tok % w).astype(F64) * w_last / w
+    omega = np.asarray([base ** (-j / quarter) for j in range(quarter)], dtype=F64)
+    return np.concatenate([py[:, None] * omega[None, :], px[:, None] * omega[None, :]], axis=1)
+
+
+def apply_rope(v: np.ndarray, angles: np.ndarray, H: int) -> np.ndarray:
+    """Rotates channel pairs (2i, 2i+1) of every head by angles[:, i], i < hd/2.  v [k,C], angles [k,hd/2]."""
+    k, C = v.shape
+    hd = C // H
+    vh = np.asarray(v, dtype=F64).reshape(k, H, hd // 2, 2)
+    c, s_ = np.cos(angles)[:, None, :], np.sin(angles)[:, None, :]
+    out = np.empty_like(vh)
+    out[..., 0] = vh[..., 0] * c - vh[..., 1] * s_
+    out[..., 1] = vh[..., 0] * s_ + vh[..., 1] * c
+    return out.reshape(k, C)
+
+
 def attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, H: int) -> np.ndarray:
     """Multi-head softmax(q K^T / sqrt(hd)) V with a materialised attention matrix, no mask.
     q [k,C], K [Lkv,C], V [Lkv,C]; head h owns channels [h*hd, (h+1)*hd)."""
@@ -209,9 +283,12 @@ class VarOracle:
     """
 
     def __init__(self, L: int, C: int, H: int, sides_hw: Sequence[Sequence[int]], cache_step: int,
-                 weights: Dict, B: int, cross_len: int = 0, granularity: str = "sublayer"):
-        assert granularity in ("sublayer", "step")
+                 weights: Dict, B: int, cross_len: int = 0, granularity: str = "sublayer",
+                 interp_mode: str = "nearest", rope_base: Optional[float] = None, qk_scale: Optional[np.ndarray] = None):
+        assert granularity in ("sublayer", "step") and interp_mode in ("nearest", "bilinear")
         self.granularity = granularity
+        self.interp_mode, self.rope_base = interp_mode, rope_base
+        self.qk_scale = None if qk_scale is None else np.asarray(qk_scale, dtype=F64)      # [L, H]
         self.L, self.C, self.H, self.B = L, C, H, B
         self.hw = [tuple(s) for s in sides_hw]
         self.cache_step = cache_step
@@ -229,8 +306,9 @@ class VarOracle:
         self.step_cache: Optional[np.ndarray] = None   # output token map of step K-N (granularity "step"; skipped steps)
 
     # -- one wrapped sublayer on compact rows ---------------------------------------------------
-    def _branch(self, l: int, sub: str, xp: np.ndarray) -> np.ndarray:
-        """Sublayer branch output y for the compact rows xp [B,k,C] (before gate and residual)."""
+    def _branch(self, l: int, sub: str, xp: np.ndarray, tokens: Optional[np.ndarray] = None, scale_idx: int = 0) -> np.ndarray:
+        """Sublayer branch output y for the compact rows xp [B,k,C] (before gate and residual).
+        tokens [B,k]: the rows' original token indices in the map of scale `scale_idx` (rotary positions)."""
         w, mod = self.w, np.asarray(self.w["mod"][l], dtype=F64)      # mod [B,6,C]
         B = xp.shape[0]
         a = layernorm(xp)
@@ -239,6 +317,18 @@ class VarOracle:
             qkv = linear(a, w["w_qkv"][l], w["b_qkv"][l])
             q, kk, vv = qkv[..., :self.C], qkv[..., self.C:2 * self.C], qkv[..., 2 * self.C:]
             y = np.empty_like(xp)
+            if self.qk_scale is not None or self.rope_base is not None:
+                q, kk = np.array(q, copy=True), np.array(kk, copy=True)
+                h_, w_ = self.hw[scale_idx]
+                hl, wl = self.hw[-1]
+                for b in range(B):
+                    if self.qk_scale is not None:
+                        q[b] = qk_normalise(q[b], self.H, self.qk_scale[l])
+                        kk[b] = qk_normalise(kk[b], self.H)
+                    if self.rope_base is not None:
+                        ang = rope_angles(tokens[b], h_, w_, hl, wl, self.C // self.H, self.rope_base)
+                        q[b] = apply_rope(q[b], ang, self.H)
+                        kk[b] = apply_rope(kk[b], ang, self.H)
             for b in range(B):
                 # KV cache: all earlier (possibly pruned) scales plus the rows forwarded now
                 self.Kc[l][b] = np.concatenate([self.Kc[l][b][:self.kv_len], kk[b]], axis=0)
@@ -280,7 +370,8 @@ class VarOracle:
             assert self.step_cache is not None and scale_idx > self.cache_step
             hc, wc = self.hw[self.cache_step]
             self.step += 1
-            return ctr_upsample(self.step_cache, hc, wc, h, w_)
+            up = ctr_upsample if self.interp_mode == "nearest" else ctr_upsample_bilinear
+            return up(self.step_cache, hc, wc, h, w_)
         pruned = keep_ratio < 1.0
         k = kept_count(keep_ratio, h, w_) if pruned else n
         if self.granularity == "step":
@@ -299,13 +390,14 @@ class VarOracle:
                 else:
                     idx = None
                     xp = x
-                y = self._branch(l, sub, xp)
+                tokens = idx if pruned else np.broadcast_to(np.arange(n), (B, n))
+                y = self._branch(l, sub, xp, tokens, scale_idx)
                 if scale_idx == self.cache_step:
                     assert not pruned, "the caching step is the last unpruned step"
                     self.cache[l][sub] = y.copy()
                 if pruned:
                     hc, wc = self.hw[self.cache_step]
-                    yfull = cached_token_restoration(y, idx, self.cache[l][sub], hc, wc, h, w_)
+                    yfull = cached_token_restoration(y, idx, self.cache[l][sub], hc, wc, h, w_, self.interp_mode)
                 else:
                     yfull = y
                 if trace is not None:
@@ -336,10 +428,11 @@ class VarOracle:
             xc = pts_gather(x, idx)
         if trace is not None:
             trace[("step",)] = {"idx": idx, "score": score}
+        tokens = idx if pruned else np.broadcast_to(np.arange(x.shape[1]), x.shape[:2])
         for l in range(self.L):
             mod = np.asarray(self.w["mod"][l], dtype=F64)
             for sub in self.subs:
-                y = self._branch(l, sub, xc)
+                y = self._branch(l, sub, xc, tokens, scale_idx)
                 if sub == "attn":
                     xc = xc + mod[:, 2][:, None, :] * y
                 elif sub == "ffn":
@@ -351,7 +444,7 @@ class VarOracle:
             self.step_cache = xc.copy()
         if pruned:
             hc, wc = self.hw[self.cache_step]
-            out = cached_token_restoration(xc, idx, self.step_cache, hc, wc, h, w_)
+            out = cached_token_restoration(xc, idx, self.step_cache, hc, wc, h, w_, self.interp_mode)
         else:
             out = xc
         self.kv_len += k
