@@ -133,6 +133,15 @@ typedef struct {
   int32_t kv_capacity;/* KV rows per image per block the caller provides room for; % 8 == 0        */
   int32_t granularity;/* 0: selection / restoration around every attention and FFN layer (the paper).
                          1: around the whole stack of blocks of a scale step (see fv_var_step)          */
+  /* Optional pieces of the pruned backbones (the paper names none of them; 0 = off, the default):       */
+  float rope_base;    /* > 0: 2-D rotary positions on the self-attention's q and k.  Token (y, x) of the
+                         (h, w) map sits at (y*h_K/h, x*w_K/w) in the last scale's frame; of a head's hd
+                         channels the first half turns with the row, the second with the column coordinate,
+                         pair (2j, 2j+1) of a half by coordinate * rope_base^(-j/(hd/4)).  At a pruned step
+                         the angle is that of the token's ORIGINAL slot (its kept index), not of its row
+                         in the compact tensor.                                                          */
+  int32_t interp_mode;/* interpolate(.) of Eq. 6: 0 nearest (src = floor(dst*in/out)); 1 bilinear with
+                         half-pixel centres (src = (dst+0.5)*in/out - 0.5, clamped)                      */
 } fv_config;
 
 typedef struct { /* HOST arrays of length L holding DEVICE pointers; bf16 unless noted; borrowed   */
@@ -149,6 +158,9 @@ typedef struct { /* HOST arrays of length L holding DEVICE pointers; bf16 unless
   const void *const *w_o_x;  /* [C, C]                                                             */
   const float *mod_dev;      /* [L, B_max, 6, C] fp32: sigma1, beta1, gamma1, sigma2, beta2, gamma2 */
   const void *text_dev;      /* [B_max, cross_len, C] bf16 or NULL                                 */
+  const float *qk_scale_dev; /* NULL, or [L, H] fp32: cosine attention in the self-attention sublayer -- every
+                                head's q and k are divided by their Euclidean norm (floored at 1e-12) and q is
+                                multiplied by the head's scale; applied before the rotary rotation          */
 } fv_weights;
 
 size_t fv_workspace_bytes(const fv_config *cfg); /* scratch for fv_var_step                         */

@@ -39,13 +39,14 @@ class fv_config(C.Structure):
     _fields_ = [("L", C.c_int32), ("C", C.c_int32), ("H", C.c_int32), ("mlp_ratio", C.c_int32),
                 ("cross_len", C.c_int32), ("B_max", C.c_int32), ("n_steps", C.c_int32),
                 ("h", C.POINTER(C.c_int32)), ("w", C.POINTER(C.c_int32)),
-                ("cache_step", C.c_int32), ("kv_capacity", C.c_int32), ("granularity", C.c_int32)]
+                ("cache_step", C.c_int32), ("kv_capacity", C.c_int32), ("granularity", C.c_int32),
+                ("rope_base", C.c_float), ("interp_mode", C.c_int32)]
 
 
 class fv_weights(C.Structure):
     _fields_ = [(n, C.POINTER(C.c_void_p)) for n in
                 ("w_qkv", "b_qkv", "w_o", "b_o", "w_fc1", "b_fc1", "w_fc2", "b_fc2", "w_q_x", "w_kv_x", "w_o_x")] + \
-               [("mod_dev", C.c_void_p), ("text_dev", C.c_void_p)]
+               [("mod_dev", C.c_void_p), ("text_dev", C.c_void_p), ("qk_scale_dev", C.c_void_p)]
 
 
 class fv_generator(C.Structure):
@@ -338,7 +339,8 @@ class FvContext:
     (`inputs.ModelTensors`) or as torch bf16 CUDA tensors with the same field names."""
 
     def __init__(self, L: int, Cw: int, H: int, sides_hw: Sequence[Sequence[int]], cache_step: int, B_max: int,
-                 kv_capacity: int, tensors, cross_len: int = 0, mlp_ratio: int = 4, device="cuda:0", granularity: int = 0):
+                 kv_capacity: int, tensors, cross_len: int = 0, mlp_ratio: int = 4, device="cuda:0", granularity: int = 0,
+                 rope_base: float = 0.0, interp_mode: int = 0, qk_scale=None):
         self.dev = torch.device(device)
         self.L, self.C, self.H, self.B_max, self.cross_len = L, Cw, H, B_max, cross_len
         self.n_sub = 3 if cross_len else 2
@@ -348,7 +350,7 @@ class FvContext:
         self._w = (C.c_int32 * len(self.hw))(*[s[1] for s in self.hw])
         self.granularity = granularity
         self.cfg = fv_config(L, Cw, H, mlp_ratio, cross_len, B_max, len(self.hw), self._h, self._w, cache_step,
-                             self.kv_capacity, granularity)
+                             self.kv_capacity, granularity, float(rope_base), int(interp_mode))
         self._keep: List[torch.Tensor] = []
 
         def dev_bf16(a):
@@ -376,6 +378,11 @@ class FvContext:
         W.mod_dev = self.mod.data_ptr()
         self.text = dev_bf16(tensors.text) if cross_len else None
         W.text_dev = self.text.data_ptr() if cross_len else None
+        self.qk_scale = None
+        if qk_scale is not None:      # [L, H] fp32: cosine attention
+            self.qk_scale = (qk_scale if isinstance(qk_scale, torch.Tensor) else torch.from_numpy(qk_scale)).to(self.dev, torch.float32).contiguous()
+            assert tuple(self.qk_scale.shape) == (L, H)
+        W.qk_scale_dev = self.qk_scale.data_ptr() if self.qk_scale is not None else None
         self.weights = W
         Lb = lib()
         self.kv = torch.empty(Lb.fv_kv_bytes(C.byref(self.cfg)) + 1024, dtype=torch.uint8, device=self.dev)

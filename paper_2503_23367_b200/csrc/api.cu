@@ -35,6 +35,8 @@ struct fv_ctx {
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   float* step_cache = nullptr;  // fp32 output map of the caching step [B_max, n_cache, C] (skipped steps; granularity 1)
   float* xc = nullptr;  // granularity 1: compact fp32 residual stream of a pruned step [B*k, C]
+  const float* qk_scale = nullptr;      // [L, H] or null
+  std::vector<float*> rope_tab;         // per scale step: (cos, sin) table [h*w][hd/2][2], empty = no rotary positions
   size_t kv_block_bytes = 0, k_bytes = 0, text_k_bytes = 0, text_block_bytes = 0, cache_sub_bytes = 0;
 };
 
@@ -59,7 +61,7 @@ cudaError_t ensure_init() {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 struct Layout {
-  size_t status, a, q, o, y, hbuf, idx, inv, sel, splitk, xc, total;
+  size_t status, a, q, o, y, hbuf, idx, inv, sel, splitk, xc, rope, total;
 };
 
 int max_tokens(const fv_config* c) {
@@ -75,6 +77,8 @@ bool config_ok(const fv_config* c) {
     if (c->h[i] <= 0 || c->w[i] <= 0) return false;
   if (c->cache_step >= c->n_steps) return false;
   if (c->granularity != 0 && c->granularity != 1) return false;
+  if (c->interp_mode != 0 && c->interp_mode != 1) return false;
+  if (!(c->rope_base >= 0.f)) return false;
   return true;
 }
 
@@ -95,6 +99,10 @@ Layout workspace_layout(const fv_config* c) {
   l.sel = take(select_workspace_bytes(c->B_max, max_tokens(c), c->C));
   l.splitk = take(gemm_splitk_ws_bytes());
   l.xc = take(c->granularity == 1 ? M * C * 4 : 0);
+  size_t rope_bytes = 0;
+  if (c->rope_base > 0.f)
+    for (int i = 0; i < c->n_steps; ++i) rope_bytes += align_up((size_t)c->h[i] * c->w[i] * (c->C / c->H / 2) * 8, 1024);
+  l.rope = take(rope_bytes);
   l.total = off;
   return l;
 }
@@ -294,8 +302,19 @@ fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, v
   c->sel_ws = c->ws + lay.sel;
   c->splitk_ws = c->ws + lay.splitk;
   c->xc = reinterpret_cast<float*>(c->ws + lay.xc);
+  c->qk_scale = wts->qk_scale_dev;
+  bool rope_ok = true;
+  if (cfg->rope_base > 0.f) {
+    char* t = c->ws + lay.rope;
+    for (int i = 0; i < cfg->n_steps; ++i) {
+      c->rope_tab.push_back(reinterpret_cast<float*>(t));
+      rope_ok = rope_ok && launch_rope_table(c->rope_tab.back(), cfg->h[i], cfg->w[i], cfg->h[cfg->n_steps - 1], cfg->w[cfg->n_steps - 1], hd,
+                                             cfg->rope_base, nullptr) == cudaSuccess;
+      t += align_up((size_t)cfg->h[i] * cfg->w[i] * (hd / 2) * 8, 1024);
+    }
+  }
   // Never-written KV rows must read as zeros (they meet zero probabilities in P*V).
-  if (cudaMemset(kv_dev, 0, fv_kv_bytes(cfg)) != cudaSuccess || cudaMemset(c->status, 0, 256) != cudaSuccess ||
+  if (!rope_ok || cudaMemset(kv_dev, 0, fv_kv_bytes(cfg)) != cudaSuccess || cudaMemset(c->status, 0, 256) != cudaSuccess ||
       cudaMemset(c->sel_ws, 0, select_ticket_bytes(cfg->B_max)) != cudaSuccess ||
       cudaMemset(c->splitk_ws, 0, gemm_splitk_ticket_bytes()) != cudaSuccess ||
       cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
@@ -441,6 +460,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   const bool sub_pruned = pruned && !whole_step;
   float* xr = x;        // residual stream the blocks update
   int nr = n;           // its rows per image
+  const int32_t* step_idx = nullptr;   // per-step granularity: the kept indices of the whole step
   if (pruned && whole_step) {
     const int32_t* idx = forced_idx_dev;
     if (forced_idx_dev) {
@@ -455,6 +475,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
     if (launch_gather_rows(tokens_dev, idx, B, n, k, C, ctx->xc, st) != cudaSuccess) return FV_ERR_CUDA;
     xr = ctx->xc;
     nr = k;
+    step_idx = idx;
   }
   // Column sums of x (Eq. 4) for the next selection are left in the selection scratch by the restore
   // kernel of the sublayer before it; only the first sublayer of a step has to sum the map itself.
@@ -508,6 +529,11 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         g.a = ctx->a_buf; g.w = ctx->w_qkv[l]; g.bias = ctx->b_qkv[l]; g.M = M; g.N = 3 * C; g.K = C;
         g.epilogue = EPI_QKV_SPLIT; g.out = ctx->q_buf; g.q_cols = C; g.C = C;
         g.k_cache = kbase; g.vt_cache = kbase + ctx->k_bytes; g.kv_capacity = c.kv_capacity; g.kv_offset = ctx->kv_len;
+        // optional: cosine attention and rotary positions on q and k; a kept row's angle is that of its original slot
+        g.qk_scale = ctx->qk_scale ? ctx->qk_scale + (size_t)l * c.H : nullptr;
+        g.rope_table = ctx->rope_tab.empty() ? nullptr : ctx->rope_tab[scale_idx];
+        g.rope_idx = sub_pruned ? idx : step_idx;
+        g.head_dim = C / c.H;
         s = launch_gemm(g, st);
         if (s != FV_OK) break;
         AttnArgs a{};

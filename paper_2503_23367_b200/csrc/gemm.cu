@@ -50,14 +50,15 @@ template <int BN> struct GemmCfg {
   }
 };
 
-// RESID: the instantiation launched for the residual epilogue.  It is a kernel of its own because that epilogue
+// KIND 1 (RESID): the instantiation launched for the residual epilogue.  It is a kernel of its own because that epilogue
 // needs ~90 more registers per thread; the others stay small enough for a bandwidth-bound kernel of another
 // stream (the restoration of the rows that were not kept) to share the SMs with them.
-template <int BN, bool SPLIT, bool RESID>
+template <int BN, bool SPLIT, int KIND>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
   using Cfg = GemmCfg<BN>;
   constexpr int STAGES = Cfg::kStages;
+  constexpr bool RESID = KIND == 1;   // KIND 2: the QKV projection with cosine attention / rotary positions on Q and K
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint4* bias_s = reinterpret_cast<uint4*>(smem + STAGES * Cfg::kStageBytes);   // per-warp bias slice of the tile
@@ -202,6 +203,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
           for (int i = 0; i < 8; ++i) xa[i] = xb[i];
         }
+      } else if (KIND == 2) {
+        qkv_extras_tile<BN>(p, t0, row, row_ok, img, jrow, n0, bias_w);
+        tc_fence_before();
+        mbar_arrive(&acc_empty[buf]);
       } else if (!SPLIT) {
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 64) {
@@ -327,8 +332,8 @@ void load_encode() {
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
 }
 
-template <int BN, bool SPLIT, bool RESID> cudaError_t set_attr() {
-  return cudaFuncSetAttribute(gemm_bf16_kernel<BN, SPLIT, RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<BN>::smem_bytes(RESID));
+template <int BN, bool SPLIT, int KIND> cudaError_t set_attr() {
+  return cudaFuncSetAttribute(gemm_bf16_kernel<BN, SPLIT, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<BN>::smem_bytes(KIND == 1));
 }
 
 }  // namespace
@@ -347,13 +352,16 @@ bool make_tmap_bf16_2d(void* tmap_out, const void* base, uint64_t rows, uint64_t
 }
 
 cudaError_t gemm_init() {
-  cudaError_t e = set_attr<128, false, false>();
-  if (e == cudaSuccess) e = set_attr<128, true, false>();
-  if (e == cudaSuccess) e = set_attr<192, false, false>();
-  if (e == cudaSuccess) e = set_attr<256, false, false>();
-  if (e == cudaSuccess) e = set_attr<128, false, true>();
-  if (e == cudaSuccess) e = set_attr<192, false, true>();
-  if (e == cudaSuccess) e = set_attr<256, false, true>();
+  cudaError_t e = set_attr<128, false, 0>();
+  if (e == cudaSuccess) e = set_attr<128, true, 0>();
+  if (e == cudaSuccess) e = set_attr<192, false, 0>();
+  if (e == cudaSuccess) e = set_attr<256, false, 0>();
+  if (e == cudaSuccess) e = set_attr<128, false, 1>();
+  if (e == cudaSuccess) e = set_attr<192, false, 1>();
+  if (e == cudaSuccess) e = set_attr<256, false, 1>();
+  if (e == cudaSuccess) e = set_attr<128, false, 2>();
+  if (e == cudaSuccess) e = set_attr<192, false, 2>();
+  if (e == cudaSuccess) e = set_attr<256, false, 2>();
   if (e == cudaSuccess) e = gemm_pair_init();
   if (e != cudaSuccess) return e;
   int dev = 0;
@@ -423,12 +431,14 @@ static cudaError_t launch_bn(const GemmArgs& g, const GemmDev& p, int tiles_m, c
   const long tiles = (long)tiles_m * ((g.N + BN - 1) / BN) * p.splits;
   const int grid = (int)(tiles < g_num_sms ? tiles : g_num_sms);
   if (p.splits > 1) {
-    if constexpr (BN == 128) return launch_pdl(gemm_bf16_kernel<128, true, false>, dim3(grid), dim3(kGemmThreads), GemmCfg<128>::smem_bytes(false), st, tmA, tmB, p);
+    if constexpr (BN == 128) return launch_pdl(gemm_bf16_kernel<128, true, 0>, dim3(grid), dim3(kGemmThreads), GemmCfg<128>::smem_bytes(false), st, tmA, tmB, p);
     else return cudaErrorInvalidValue;
   } else {
     if (p.epilogue == EPI_RESIDUAL || p.epilogue == EPI_F32)
-      return launch_pdl(gemm_bf16_kernel<BN, false, true>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::smem_bytes(true), st, tmA, tmB, p);
-    return launch_pdl(gemm_bf16_kernel<BN, false, false>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::smem_bytes(false), st, tmA, tmB, p);
+      return launch_pdl(gemm_bf16_kernel<BN, false, 1>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::smem_bytes(true), st, tmA, tmB, p);
+    if (p.epilogue == EPI_QKV_SPLIT && (p.qk_scale || p.rope_table))
+      return launch_pdl(gemm_bf16_kernel<BN, false, 2>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::smem_bytes(false), st, tmA, tmB, p);
+    return launch_pdl(gemm_bf16_kernel<BN, false, 0>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::smem_bytes(false), st, tmA, tmB, p);
   }
 }
 
@@ -445,10 +455,17 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   if (g_force_path == 2) tc = TileChoice{256, true};
   if (g_force_path == 3) tc = TileChoice{128, true};
   if (g_force_path >= 4 && g_force_path <= 6) tc = TileChoice{128 + 64 * (g_force_path - 4), false};
+  // Q / K extras (cosine attention, rotary positions): one-CTA tiles that hold whole heads, no K split
+  const bool qk_extras = g.epilogue == EPI_QKV_SPLIT && (g.qk_scale || g.rope_table);
+  if (qk_extras) {
+    if (g.head_dim != 64 && g.head_dim != 128) return FV_ERR_UNSUPPORTED;
+    if (tc.pair) tc = TileChoice{256, false};
+    if (tc.bn % g.head_dim) tc.bn = 256;
+  }
   int bn = tc.bn;
   GemmDev p;
   p.splits = 1; p.kb_per_split = (g.K + BK - 1) / BK; p.sk_partial = nullptr; p.sk_tickets = nullptr;
-  if (g.splitk_ws) {
+  if (g.splitk_ws && !qk_extras) {
     const int num_kb = (g.K + BK - 1) / BK;
     const long tiles128 = (long)tiles_m * ((g.N + 127) / 128);
     const int sp = pick_splits(tiles128, g.M, num_kb, g_num_sms);
@@ -466,6 +483,10 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   p.mod_stride = g.mod_stride; p.rows_per_image = g.rows_per_image; p.q_cols = g.q_cols; p.C = g.C;
   p.k_cache = static_cast<__nv_bfloat16*>(g.k_cache); p.vt_cache = static_cast<__nv_bfloat16*>(g.vt_cache);
   p.kv_capacity = g.kv_capacity; p.kv_offset = g.kv_offset; p.status = g.status;
+  p.qk_scale = qk_extras ? g.qk_scale : nullptr;
+  p.rope_table = qk_extras ? reinterpret_cast<const float2*>(g.rope_table) : nullptr;
+  p.rope_idx = qk_extras ? g.rope_idx : nullptr;
+  p.head_dim = g.head_dim;
   LaunchScope scope(KC_GEMM, 1, 2.0 * g.M * (double)g.N * g.K, 2.0 * ((double)g.M * g.K + (double)g.N * g.K + (double)g.M * g.N), st);
   if (p.splits == 1 && tc.pair) {
     cudaError_t e2 = launch_gemm_pair(g, p, bn, st);

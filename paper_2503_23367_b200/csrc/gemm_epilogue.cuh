@@ -25,6 +25,11 @@ struct GemmDev {
   int splits, kb_per_split;   // K slices per tile (1 = no split) and 64-wide k-blocks per slice
   float* sk_partial;          // [tile][slice][128][BN] fp32 partial accumulators
   unsigned int* sk_tickets;   // [tile] arrival counters, zero between launches
+  // EPI_QKV_SPLIT extras on the Q and K columns (the instantiation of their own, KIND 2):
+  const float* qk_scale;      // [H] per-head query scale of cosine attention (q, k divided by their norm), or null
+  const float2* rope_table;   // [tokens of the scale][head_dim / 2] (cos, sin), or null
+  const int32_t* rope_idx;    // [B, rows_per_image] original token index of every row, or null (row j = token j)
+  int head_dim;
 };
 
 __device__ __forceinline__ float gelu_tanh_fast(float v) {
@@ -161,10 +166,16 @@ __device__ __forceinline__ void residual_chunk(const GemmDev& p, const ResidRows
 }
 
 // One 32-column chunk of one accumulator row: bias, optional GELU, then the epilogue's store.
+__device__ __forceinline__ void store_chunk(const GemmDev& p, const float (&v)[32], int row, int img, int jrow, int col);
 __device__ __forceinline__ void epilogue_chunk(const GemmDev& p, const uint32_t (&r)[32], int row, int img, int jrow, int col,
                                                const uint4* bias4) {
   float v[32];
   chunk_values(p, r, col, v, bias4);
+  store_chunk(p, v, row, img, jrow, col);
+}
+
+// The epilogue's store of 32 finished fp32 values of one row.
+__device__ __forceinline__ void store_chunk(const GemmDev& p, const float (&v)[32], int row, int img, int jrow, int col) {
   if (p.epilogue == EPI_BF16 || p.epilogue == EPI_GELU_BF16 || (p.epilogue == EPI_QKV_SPLIT && col < p.q_cols)) {
     const int ld = (p.epilogue == EPI_QKV_SPLIT) ? p.q_cols : p.N;
     uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + (size_t)row * ld + col);
@@ -229,6 +240,79 @@ __device__ __forceinline__ void epilogue_chunk(const GemmDev& p, const uint32_t 
       __nv_bfloat16* dst = p.vt_cache + ((size_t)img * p.C + (kc - p.C)) * p.kv_capacity + p.kv_offset + jrow;
 #pragma unroll
       for (int i = 0; i < 32; ++i) dst[(size_t)i * p.kv_capacity] = __float2bfloat16_rn(v[i]);
+    }
+  }
+}
+
+
+// ---- Q / K columns of the QKV projection with cosine attention and / or rotary positions (KIND 2) ----
+// One head's columns [col, col + head_dim) of one accumulator row (thread = row).  Cosine attention needs
+// the head's norm before any value can be stored, so the head's chunks are read from TMEM twice (the read is
+// cheap): once to sum the squares of acc + bias, once to scale, rotate and store.  The rotation angle belongs
+// to the token's ORIGINAL slot in the map (rope_idx), not to its row in the compact tensor.
+// Called by the whole warp (the TMEM loads are warp-wide); rows past M take part in the loads only.
+__device__ __forceinline__ void qk_head_epilogue(const GemmDev& p, uint32_t taddr, int row, bool row_ok, int img, int jrow, int col,
+                                                 const uint4* bias4, bool is_query) {
+  const int hd = p.head_dim;
+  float scale = 1.f;
+  if (p.qk_scale) {
+    float ss = 0.f;
+    for (int c = 0; c < hd; c += 32) {
+      uint32_t r[32];
+      float v[32];
+      tmem_ld32(taddr + c, r);
+      tmem_wait_ld();
+      chunk_values(p, r, col + c, v, bias4 + c / 8);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) ss = fmaf(v[i], v[i], ss);
+    }
+    scale = 1.f / fmaxf(sqrtf(ss), 1e-12f);
+    if (is_query) scale *= __ldg(p.qk_scale + (col % p.C) / hd);
+  }
+  const int token = (p.rope_idx && row_ok) ? __ldg(p.rope_idx + (size_t)img * p.rows_per_image + jrow) : jrow;
+  const float4* tab = (p.rope_table && row_ok) ? reinterpret_cast<const float4*>(p.rope_table + (size_t)token * (hd / 2)) : nullptr;
+  for (int c = 0; c < hd; c += 32) {
+    uint32_t r[32];
+    float v[32];
+    tmem_ld32(taddr + c, r);
+    tmem_wait_ld();
+    chunk_values(p, r, col + c, v, bias4 + c / 8);
+    if (p.qk_scale) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] *= scale;
+    }
+    if (tab) {
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {   // two channel pairs per float4 of (cos, sin, cos, sin)
+        const float4 cs = __ldg(tab + c / 4 + g);
+        const float a0 = v[4 * g], b0 = v[4 * g + 1], a1 = v[4 * g + 2], b1 = v[4 * g + 3];
+        v[4 * g] = a0 * cs.x - b0 * cs.y;
+        v[4 * g + 1] = a0 * cs.y + b0 * cs.x;
+        v[4 * g + 2] = a1 * cs.z - b1 * cs.w;
+        v[4 * g + 3] = a1 * cs.w + b1 * cs.z;
+      }
+    }
+    if (row_ok) store_chunk(p, v, row, img, jrow, col + c);
+  }
+}
+
+// All columns of one tile for KIND 2: Q and K heads through qk_head_epilogue, V columns as usual.
+template <int BN>
+__device__ __forceinline__ void qkv_extras_tile(const GemmDev& p, uint32_t t0, int row, bool row_ok, int img, int jrow, int n0,
+                                                const uint4* bias_w) {
+  const int hd = p.head_dim;
+  for (int c0 = 0; c0 < BN; c0 += hd) {
+    const int col = n0 + c0;
+    if (col >= p.N) break;
+    if (col < p.q_cols + p.C) {
+      qk_head_epilogue(p, t0 + c0, row, row_ok, img, jrow, col, bias_w + c0 / 8, col < p.q_cols);
+    } else {
+      for (int c = 0; c < hd; c += 32) {
+        uint32_t r[32];
+        tmem_ld32(t0 + c0 + c, r);
+        tmem_wait_ld();
+        if (row_ok) epilogue_chunk(p, r, row, img, jrow, col + c, bias_w + (c0 + c) / 8);
+      }
     }
   }
 }

@@ -104,7 +104,16 @@ struct GemmArgs {
   int kv_capacity, kv_offset;
   int32_t* status;     // device status word or null
   void* splitk_ws;     // scratch for K-split partials (gemm_splitk_ws_bytes(), tickets at its head zero) or null
+  // EPI_QKV_SPLIT extras on the Q and K columns (all null = none):
+  const float* qk_scale;      // [H] fp32: cosine attention (q, k divided by their per-head norm, q times this)
+  const float* rope_table;    // [tokens of the scale][head_dim/2][2] fp32 (cos, sin) of the rotary angles
+  const int32_t* rope_idx;    // [B, rows_per_image] original token of every row, or null (row j is token j)
+  int head_dim;               // 64 or 128 (needed with either extra)
 };
+// (cos, sin) of the 2-D rotary angles of every token of an (h, w) map placed in the (h_last, w_last) frame:
+// first head_dim/4 pairs turn with the row coordinate y * h_last / h, the rest with x * w_last / w, pair j of
+// either group at frequency base^(-j / (head_dim/4)).  table: [h*w][head_dim/2][2] fp32.
+cudaError_t launch_rope_table(float* table, int h, int w, int h_last, int w_last, int head_dim, float base, cudaStream_t st);
 cudaError_t gemm_init();
 // Test / profiling hook: 0 = choose per shape, 1 = one-CTA kernel, 2 = CTA-pair kernel 256x256, 3 = CTA-pair 256x128.
 void gemm_force_path(int path);

@@ -237,6 +237,23 @@ __global__ void __launch_bounds__(256) restore_rows_f32_kernel(const float4* __r
   for (int c4 = lane; c4 < C4; c4 += 32) dst[c4] = __ldg(src + c4);
 }
 
+
+// (cos, sin) of the rotary angles of every token of one scale; double precision (a few hundred thousand
+// evaluations per scale, once per context).
+__global__ void rope_table_kernel(float2* __restrict__ table, int h, int w, int h_last, int w_last, int half, double log2_base) {
+  const long total = (long)h * w * half;
+  const int quarter = half / 2;
+  for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
+    const int j = (int)(i % half);
+    const int t = (int)(i / half);
+    const int y = t / w, x = t - y * w;
+    const double pos = j < quarter ? (double)y * h_last / h : (double)x * w_last / w;
+    const double omega = exp2(-(double)(j % quarter) / quarter * log2_base);
+    double sn, cs;
+    sincos(pos * omega, &sn, &cs);
+    table[i] = make_float2((float)cs, (float)sn);
+  }
+}
 }  // namespace
 
 cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
@@ -295,6 +312,14 @@ cudaError_t launch_restore_rows_f32(const float* cache, int hc, int wc, const fl
   LaunchScope scope(KC_RESTORE, 1, bytes, bytes, st);
   return launch_pdl(restore_rows_f32_kernel, dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const float4*>(cache), hc, wc,
                     reinterpret_cast<const float4*>(pivots), inv, h * w, k, h, w, C / 4, reinterpret_cast<float4*>(out), rows);
+}
+
+cudaError_t launch_rope_table(float* table, int h, int w, int h_last, int w_last, int head_dim, float base, cudaStream_t st) {
+  const long total = (long)h * w * (head_dim / 2);
+  const long blocks = (total + 255) / 256;
+  rope_table_kernel<<<(unsigned)(blocks < 4096 ? blocks : 4096), 256, 0, st>>>(reinterpret_cast<float2*>(table), h, w, h_last, w_last,
+                                                                                head_dim / 2, log2((double)base));
+  return cudaGetLastError();
 }
 
 }  // namespace fv
