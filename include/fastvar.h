@@ -99,10 +99,13 @@ fv_status fv_prune_select_static(const float *x_dev, int32_t B, int32_t h, int32
  *   idx_dev        [B, k] int32       : their token indices (any order, no duplicates, in [0,h*w)).
  *   out_dev        [B, h*w, C] bf16.   C % 8 == 0.
  *   inv_scratch_dev[B, h*w] int32 scratch (overwritten).
+ *   interp_mode    0: nearest, as above (the default reading of the paper's mode-less interpolate).
+ *                  1: bilinear with half-pixel centres (source coordinate (dst+0.5)*in/out - 0.5 per axis,
+ *                     clamped): an unkept token is the fp32 blend of four cached rows, rounded to bf16 once.
  * Errors: INVALID_ARG, CUDA. */
 fv_status fv_restore(const void *cache_prev_dev, int32_t hc, int32_t wc, const void *pivots_dev,
                      const int32_t *idx_dev, int32_t B, int32_t k, int32_t h, int32_t w, int32_t C,
-                     void *out_dev, int32_t *inv_scratch_dev, void *stream);
+                     void *out_dev, int32_t *inv_scratch_dev, int32_t interp_mode, void *stream);
 
 /* ------------------------------------------------------------------------------------------------
  * (2) The pruned scale step -- Sec. 3.3 "Overview" and "Implementation", Fig. 3: at the pruned steps
@@ -226,11 +229,12 @@ fv_status fv_gather_ln(const float *x_dev, const int32_t *idx_dev, int32_t B, in
 
 /* Restore fused with gate and residual (Eq. 6 + the block's x += gamma * y):
  *   x[b,t,:] += gamma[b,:] * (inv[b,t] >= 0 ? y[b, inv[b,t], :] : cache[b, src(t), :]).
- * gamma_dev NULL = 1.  y, cache bf16; x fp32 in place.  C % 8 == 0. */
+ * gamma_dev NULL = 1.  y, cache bf16; x fp32 in place.  C % 8 == 0.  interp_mode as for fv_restore (with 1
+ * the cache term is the bilinear blend of four cached rows). */
 fv_status fv_restore_residual(float *x_dev, const void *y_dev, const void *cache_dev,
                               const int32_t *inv_dev, const float *gamma_dev, int32_t mod_stride,
                               int32_t B, int32_t k, int32_t h, int32_t w, int32_t hc, int32_t wc,
-                              int32_t C, void *stream);
+                              int32_t C, int32_t interp_mode, void *stream);
 
 /* tcgen05 GEMM  out = epilogue(A[M,K] * W[N,K]^T + bias), bf16 operands, fp32 accumulation in TMEM.
  *   epilogue 0: bf16 store to out [M, N].          1: tanh-GELU then bf16 store.

@@ -72,7 +72,7 @@ def lib() -> C.CDLL:
         L.fv_prune_select.restype = C.c_int
         L.fv_prune_select.argtypes = [vp, i32, i32, i32, i32, dbl, vp, vp, vp, vp, C.POINTER(i32), vp, sz, vp]
         L.fv_restore.restype = C.c_int
-        L.fv_restore.argtypes = [vp, i32, i32, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]
+        L.fv_restore.argtypes = [vp, i32, i32, vp, vp, i32, i32, i32, i32, i32, vp, vp, i32, vp]
         for f in ("fv_workspace_bytes", "fv_kv_bytes", "fv_cache_bytes"):
             getattr(L, f).restype = sz; getattr(L, f).argtypes = [C.POINTER(fv_config)]
         L.fv_create.restype = C.c_int
@@ -88,7 +88,7 @@ def lib() -> C.CDLL:
         L.fv_var_step.restype = C.c_int; L.fv_var_step.argtypes = [vp, vp, i32, i32, dbl, vp, vp, vp, vp]
         L.fv_gather_ln.restype = C.c_int; L.fv_gather_ln.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, i32, vp, vp]
         L.fv_restore_residual.restype = C.c_int
-        L.fv_restore_residual.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp]
+        L.fv_restore_residual.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp]
         L.fv_gemm_bf16.restype = C.c_int
         L.fv_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, sz, vp]
         L.fv_gemm_splitk_workspace_bytes.restype = sz; L.fv_gemm_splitk_workspace_bytes.argtypes = []
@@ -192,14 +192,14 @@ def fv_prune_select_static(x: torch.Tensor, h: int, w: int, keep_ratio: float, o
 
 
 def fv_restore(cache_prev: torch.Tensor, hc: int, wc: int, pivots: torch.Tensor, idx: torch.Tensor, h: int, w: int,
-               out: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """cache_prev bf16 [B,hc*wc,C], pivots bf16 [B,k,C], idx int32 [B,k] -> bf16 [B,h*w,C]."""
+               out: Optional[torch.Tensor] = None, interp_mode: int = 0) -> torch.Tensor:
+    """cache_prev bf16 [B,hc*wc,C], pivots bf16 [B,k,C], idx int32 [B,k] -> bf16 [B,h*w,C].  interp_mode 0 nearest, 1 bilinear."""
     B, k, Cw = pivots.shape
     if out is None:
         out = torch.empty((B, h * w, Cw), dtype=torch.bfloat16, device=pivots.device)
     inv = torch.empty((B, h * w), dtype=torch.int32, device=pivots.device)
     _check(lib().fv_restore(_ptr(cache_prev), hc, wc, _ptr(pivots), _ptr(idx), B, k, h, w, Cw, _ptr(out), _ptr(inv),
-                            _stream()), "fv_restore")
+                            int(interp_mode), _stream()), "fv_restore")
     return out
 
 
@@ -214,11 +214,11 @@ def fv_gather_ln(x: torch.Tensor, idx: Optional[torch.Tensor], sigma: Optional[t
 
 
 def fv_restore_residual(x: torch.Tensor, y: torch.Tensor, cache: torch.Tensor, inv: torch.Tensor,
-                        gamma: Optional[torch.Tensor], mod_stride: int, h: int, w: int, hc: int, wc: int) -> None:
+                        gamma: Optional[torch.Tensor], mod_stride: int, h: int, w: int, hc: int, wc: int, interp_mode: int = 0) -> None:
     B, n, Cw = x.shape
     k = y.shape[1]
     _check(lib().fv_restore_residual(_ptr(x), _ptr(y), _ptr(cache), _ptr(inv), _ptr(gamma), mod_stride, B, k, h, w, hc, wc,
-                                     Cw, _stream()), "fv_restore_residual")
+                                     Cw, int(interp_mode), _stream()), "fv_restore_residual")
 
 
 def fv_gemm_bf16(a: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor], epilogue: int = 0,

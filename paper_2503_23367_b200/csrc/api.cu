@@ -159,14 +159,15 @@ fv_status fv_prune_select(const float* x_dev, int32_t B, int32_t h, int32_t w, i
 
 fv_status fv_restore(const void* cache_prev_dev, int32_t hc, int32_t wc, const void* pivots_dev, const int32_t* idx_dev,
                      int32_t B, int32_t k, int32_t h, int32_t w, int32_t C, void* out_dev, int32_t* inv_scratch_dev,
-                     void* stream) {
+                     int32_t interp_mode, void* stream) {
   if (!cache_prev_dev || !pivots_dev || !idx_dev || !out_dev || !inv_scratch_dev) return FV_ERR_INVALID_ARG;
+  if (interp_mode != 0 && interp_mode != 1) return FV_ERR_INVALID_ARG;
   if (B <= 0 || k <= 0 || h <= 0 || w <= 0 || hc <= 0 || wc <= 0 || C <= 0 || (C % 8) || k > h * w) return FV_ERR_INVALID_ARG;
   if (!aligned16(cache_prev_dev) || !aligned16(pivots_dev) || !aligned16(out_dev)) return FV_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = launch_inv_from_idx(idx_dev, B, k, h * w, inv_scratch_dev, st);
   if (e != cudaSuccess) return FV_ERR_CUDA;
-  return cuda_status(launch_restore_bf16(cache_prev_dev, hc, wc, pivots_dev, inv_scratch_dev, B, k, h, w, C, out_dev, st));
+  return cuda_status(launch_restore_bf16(cache_prev_dev, hc, wc, pivots_dev, inv_scratch_dev, B, k, h, w, C, out_dev, interp_mode, st));
 }
 
 fv_status fv_gather_ln(const float* x_dev, const int32_t* idx_dev, int32_t B, int32_t n_tokens, int32_t k, int32_t C,
@@ -181,11 +182,12 @@ fv_status fv_gather_ln(const float* x_dev, const int32_t* idx_dev, int32_t B, in
 
 fv_status fv_restore_residual(float* x_dev, const void* y_dev, const void* cache_dev, const int32_t* inv_dev,
                               const float* gamma_dev, int32_t mod_stride, int32_t B, int32_t k, int32_t h, int32_t w,
-                              int32_t hc, int32_t wc, int32_t C, void* stream) {
+                              int32_t hc, int32_t wc, int32_t C, int32_t interp_mode, void* stream) {
+  if (interp_mode != 0 && interp_mode != 1) return FV_ERR_INVALID_ARG;
   if (!x_dev || !y_dev || !cache_dev || !inv_dev || B <= 0 || k <= 0 || h <= 0 || w <= 0 || hc <= 0 || wc <= 0) return FV_ERR_INVALID_ARG;
   if (C <= 0 || (C % 8)) return FV_ERR_INVALID_ARG;
   return cuda_status(launch_restore_residual(x_dev, y_dev, cache_dev, inv_dev, gamma_dev, mod_stride, B, k, h, w, hc, wc, C,
-                                             nullptr, 0, static_cast<cudaStream_t>(stream)));
+                                             nullptr, 0, interp_mode, static_cast<cudaStream_t>(stream)));
 }
 
 fv_status fv_gemm_bf16(const void* a_dev, const void* w_dev, const void* bias_dev, int32_t M, int32_t N, int32_t K,
@@ -426,7 +428,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
     const int h0 = c.h[scale_idx], w0 = c.w[scale_idx];
     if (launch_inv_fill(B, h0 * w0, ctx->inv, st0) != cudaSuccess) return FV_ERR_CUDA;
     if (launch_restore_rows_f32(ctx->step_cache, c.h[c.cache_step], c.w[c.cache_step], ctx->step_cache, ctx->inv, B, 0, h0, w0, c.C,
-                                out_dev, st0) != cudaSuccess)
+                                out_dev, c.interp_mode, st0) != cudaSuccess)
       return FV_ERR_CUDA;
     ctx->next_step += 1;
     return FV_OK;
@@ -516,7 +518,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         // touch disjoint rows of x).
         if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
         e = launch_restore_residual(x, ctx->y_buf, cache_sub, ctx->inv, gamma, mod_stride, B, k, h, w, hc, wc, C,
-                                    more ? ctx->sel_ws : nullptr, 1, ctx->side);
+                                    more ? ctx->sel_ws : nullptr, 1, c.interp_mode, ctx->side);
         if (e != cudaSuccess || cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) { s = FV_ERR_CUDA; break; }
       }
       e = launch_gather_ln(xr, idx, B, nr, k, C, sigma, beta, mod_stride, ctx->a_buf, st);
@@ -569,7 +571,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         if (s != FV_OK) break;
         if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
         e = launch_restore_residual(x, ctx->y_buf, cache_sub, ctx->inv, gamma, mod_stride, B, k, h, w, hc, wc, C,
-                                    more ? ctx->sel_ws : nullptr, 2, st);
+                                    more ? ctx->sel_ws : nullptr, 2, c.interp_mode, st);
         if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
         have_partials = more;
       } else {
@@ -584,7 +586,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
       cudaMemcpyAsync(ctx->step_cache, x, (size_t)B * n * C * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
     return FV_ERR_CUDA;  // the step-level cache: this step's output map (image stride n*C == n_cache*C here)
   if (whole_step && pruned &&
-      launch_restore_rows_f32(ctx->step_cache, hc, wc, ctx->xc, ctx->inv, B, k, h, w, C, out_dev, st) != cudaSuccess)
+      launch_restore_rows_f32(ctx->step_cache, hc, wc, ctx->xc, ctx->inv, B, k, h, w, C, out_dev, c.interp_mode, st) != cudaSuccess)
     return FV_ERR_CUDA;
   if (s != FV_OK) return s;
   ctx->kv_len += k;

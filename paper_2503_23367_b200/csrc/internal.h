@@ -74,15 +74,16 @@ cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, i
                              const float* beta, int mod_stride, void* a_out, cudaStream_t st);
 // colsum_ws: null, or the selection workspace that receives the column sums of the updated x.
 // part: 0 = every row; 1 = the rows that were not kept; 2 = the kept rows (and the fold of the column sums).
+// interp_mode (all restore launchers): 0 nearest, 1 bilinear with half-pixel centres.
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv,
                                     const float* gamma, int mod_stride, int B, int k, int h, int w, int hc, int wc,
-                                    int C, void* colsum_ws, int part, cudaStream_t st);
+                                    int C, void* colsum_ws, int part, int interp_mode, cudaStream_t st);
 // Per-step granularity: fp32 gather of the kept rows, and fp32 restoration of the step's output map.
 cudaError_t launch_gather_rows(const float* x, const int32_t* idx, int B, int n, int k, int C, float* out, cudaStream_t st);
 cudaError_t launch_restore_rows_f32(const float* cache, int hc, int wc, const float* pivots, const int32_t* inv, int B, int k,
-                                    int h, int w, int C, float* out, cudaStream_t st);
+                                    int h, int w, int C, float* out, int interp_mode, cudaStream_t st);
 cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* pivots, const int32_t* inv, int B,
-                                int k, int h, int w, int C, void* out, cudaStream_t st);
+                                int k, int h, int w, int C, void* out, int interp_mode, cudaStream_t st);
 
 // ---- gemm.cu : tcgen05 GEMM with fused epilogues -----------------------------------------------
 enum GemmEpilogue : int { EPI_BF16 = 0, EPI_GELU_BF16 = 1, EPI_RESIDUAL = 2, EPI_QKV_SPLIT = 3, EPI_F32 = 4 };

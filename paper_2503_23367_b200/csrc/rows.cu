@@ -96,6 +96,22 @@ __device__ __forceinline__ int nearest_src(int t, int h, int w, int hc, int wc) 
   return ((y * hc) / h) * wc + (xx * wc) / w;
 }
 
+// Bilinear interpolate(.) of Eq. 6 with half-pixel centres: the four source tokens of destination token t and
+// their weights (source coordinate (dst + 0.5) * in / out - 0.5 per axis, clamped to the map).
+struct BilinearTaps { int src[4]; float wt[4]; };
+__device__ __forceinline__ BilinearTaps bilinear_taps(int t, int h, int w, int hc, int wc) {
+  const int y = t / w, xx = t - y * w;
+  double sy = (y + 0.5) * (double)hc / h - 0.5, sx = (xx + 0.5) * (double)wc / w - 0.5;
+  sy = fmin(fmax(sy, 0.0), (double)(hc - 1)); sx = fmin(fmax(sx, 0.0), (double)(wc - 1));
+  const int y0 = (int)floor(sy), x0 = (int)floor(sx);
+  const int y1 = min(y0 + 1, hc - 1), x1 = min(x0 + 1, wc - 1);
+  const float ty = (float)(sy - y0), tx = (float)(sx - x0);
+  BilinearTaps b;
+  b.src[0] = y0 * wc + x0; b.src[1] = y0 * wc + x1; b.src[2] = y1 * wc + x0; b.src[3] = y1 * wc + x1;
+  b.wt[0] = (1.f - ty) * (1.f - tx); b.wt[1] = (1.f - ty) * tx; b.wt[2] = ty * (1.f - tx); b.wt[3] = ty * tx;
+  return b;
+}
+
 __device__ __forceinline__ void bf16x8_to_float(const uint4& p, float (&f)[8]) {
   const uint32_t u[4] = {p.x, p.y, p.z, p.w};
 #pragma unroll
@@ -238,6 +254,152 @@ __global__ void __launch_bounds__(256) restore_rows_f32_kernel(const float4* __r
 }
 
 
+// restore_residual_kernel with bilinear interpolation of the cache: an unkept token blends four cached rows
+// (fp32), a kept token takes its forwarded row.  Same CTA shape, row ownership and column-sum handling; two
+// rows in flight instead of four (four source rows each).  part 2 (kept rows only) never interpolates and
+// runs the kernel above.
+__global__ void __launch_bounds__(256) restore_residual_bilinear_kernel(float4* __restrict__ x, const uint4* __restrict__ y,
+                                                                        const uint4* __restrict__ cache, const int32_t* __restrict__ inv,
+                                                                        const float* __restrict__ gamma, int mod_stride, int n, int k,
+                                                                        int h, int w, int hc, int wc, int C8, int nchunks, int group,
+                                                                        int ngroups, float4* __restrict__ chunk_partial,
+                                                                        float4* __restrict__ group_partial, unsigned int* tickets,
+                                                                        int part) {
+  __shared__ const uint4* s_src[kColsumRows][4];
+  __shared__ float s_wt[kColsumRows][4];
+  __shared__ int s_on[kColsumRows];
+  pdl_trigger();
+  pdl_wait();
+  const int b = blockIdx.y, chunk = blockIdx.x;
+  const int t0 = chunk * kColsumRows;
+  const int rows = min(kColsumRows, n - t0);
+  if (threadIdx.x < rows) {
+    const int t = t0 + threadIdx.x;
+    const int j = __ldg(inv + (size_t)b * n + t);
+    if (j >= 0) {
+      for (int q = 0; q < 4; ++q) { s_src[threadIdx.x][q] = y + ((size_t)b * k + j) * C8; s_wt[threadIdx.x][q] = q == 0 ? 1.f : 0.f; }
+    } else {
+      const BilinearTaps bt = bilinear_taps(t, h, w, hc, wc);
+      for (int q = 0; q < 4; ++q) { s_src[threadIdx.x][q] = cache + ((size_t)b * hc * wc + bt.src[q]) * C8; s_wt[threadIdx.x][q] = bt.wt[q]; }
+    }
+    s_on[threadIdx.x] = part == 0 || (part == 1) == (j < 0);
+  }
+  __syncthreads();
+  float4* xbase = x + ((size_t)b * n + t0) * C8 * 2;
+  for (int c8 = threadIdx.x; c8 < C8; c8 += 256) {
+    float4 g0 = make_float4(1.f, 1.f, 1.f, 1.f), g1 = g0;
+    if (gamma) {
+      const float4* g = reinterpret_cast<const float4*>(gamma + (size_t)b * mod_stride);
+      g0 = __ldg(g + 2 * c8); g1 = __ldg(g + 2 * c8 + 1);
+    }
+    float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+    for (int r = 0; r < rows; r += 2) {
+      uint4 p[2][4];
+      float4 x0[2], x1[2];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        if (r + i < rows && s_on[r + i]) {
+          float4* xr = xbase + (size_t)(r + i) * C8 * 2 + 2 * c8;
+          x0[i] = xr[0]; x1[i] = xr[1];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) p[i][q] = __ldg(s_src[r + i][q] + c8);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        if (r + i < rows && s_on[r + i]) {
+          float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            float fq[8];
+            bf16x8_to_float(p[i][q], fq);
+            const float wq = s_wt[r + i][q];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = fmaf(wq, fq[e], f[e]);
+          }
+          float4 u0 = x0[i], u1 = x1[i];
+          u0.x = fmaf(g0.x, f[0], u0.x); u0.y = fmaf(g0.y, f[1], u0.y); u0.z = fmaf(g0.z, f[2], u0.z); u0.w = fmaf(g0.w, f[3], u0.w);
+          u1.x = fmaf(g1.x, f[4], u1.x); u1.y = fmaf(g1.y, f[5], u1.y); u1.z = fmaf(g1.z, f[6], u1.z); u1.w = fmaf(g1.w, f[7], u1.w);
+          float4* xr = xbase + (size_t)(r + i) * C8 * 2 + 2 * c8;
+          xr[0] = u0; xr[1] = u1;
+          a0.x += u0.x; a0.y += u0.y; a0.z += u0.z; a0.w += u0.w;
+          a1.x += u1.x; a1.y += u1.y; a1.z += u1.z; a1.w += u1.w;
+        }
+      }
+    }
+    if (chunk_partial) {
+      float4* cp = chunk_partial + ((size_t)b * nchunks + chunk) * C8 * 2 + 2 * c8;
+      cp[0] = a0; cp[1] = a1;
+    }
+  }
+  if (chunk_partial && part != 1)
+    fold_group_partials(b, chunk, nchunks, group, ngroups, C8 * 2, chunk_partial, group_partial, tickets);
+}
+
+// Plain restoration (no residual) with bilinear interpolation, one warp per output row; bf16 rows (8 per
+// uint4, blended in fp32 and rounded once) or fp32 rows.
+__global__ void __launch_bounds__(256) restore_bf16_bilinear_kernel(const uint4* __restrict__ cache, int hc, int wc,
+                                                                    const uint4* __restrict__ pivots, const int32_t* __restrict__ inv,
+                                                                    int n, int k, int h, int w, int C8, uint4* __restrict__ out,
+                                                                    int total_rows) {
+  pdl_trigger();
+  pdl_wait();
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= total_rows) return;
+  const int b = warp / n, t = warp - b * n;
+  const int j = inv[warp];
+  uint4* dst = out + (size_t)warp * C8;
+  if (j >= 0) {
+    const uint4* src = pivots + ((size_t)b * k + j) * C8;
+    for (int c8 = lane; c8 < C8; c8 += 32) dst[c8] = __ldg(src + c8);
+    return;
+  }
+  const BilinearTaps bt = bilinear_taps(t, h, w, hc, wc);
+  const uint4* base = cache + (size_t)b * hc * wc * C8;
+  for (int c8 = lane; c8 < C8; c8 += 32) {
+    float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      float fq[8];
+      bf16x8_to_float(__ldg(base + (size_t)bt.src[q] * C8 + c8), fq);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] = fmaf(bt.wt[q], fq[e], f[e]);
+    }
+    __nv_bfloat162 o[4] = {__floats2bfloat162_rn(f[0], f[1]), __floats2bfloat162_rn(f[2], f[3]), __floats2bfloat162_rn(f[4], f[5]),
+                           __floats2bfloat162_rn(f[6], f[7])};
+    dst[c8] = *reinterpret_cast<uint4*>(o);
+  }
+}
+
+__global__ void __launch_bounds__(256) restore_rows_f32_bilinear_kernel(const float4* __restrict__ cache, int hc, int wc,
+                                                                        const float4* __restrict__ pivots, const int32_t* __restrict__ inv,
+                                                                        int n, int k, int h, int w, int C4, float4* __restrict__ out,
+                                                                        int total_rows) {
+  pdl_trigger();
+  pdl_wait();
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= total_rows) return;
+  const int b = warp / n, t = warp - b * n;
+  const int j = __ldg(inv + warp);
+  float4* dst = out + (size_t)warp * C4;
+  if (j >= 0) {
+    const float4* src = pivots + ((size_t)b * k + j) * C4;
+    for (int c4 = lane; c4 < C4; c4 += 32) dst[c4] = __ldg(src + c4);
+    return;
+  }
+  const BilinearTaps bt = bilinear_taps(t, h, w, hc, wc);
+  const float4* base = cache + (size_t)b * hc * wc * C4;
+  for (int c4 = lane; c4 < C4; c4 += 32) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float4 v = __ldg(base + (size_t)bt.src[q] * C4 + c4);
+      acc.x = fmaf(bt.wt[q], v.x, acc.x); acc.y = fmaf(bt.wt[q], v.y, acc.y); acc.z = fmaf(bt.wt[q], v.z, acc.z); acc.w = fmaf(bt.wt[q], v.w, acc.w);
+    }
+    dst[c4] = acc;
+  }
+}
+
 // (cos, sin) of the rotary angles of every token of one scale; double precision (a few hundred thousand
 // evaluations per scale, once per context).
 __global__ void rope_table_kernel(float2* __restrict__ table, int h, int w, int h_last, int w_last, int half, double log2_base) {
@@ -266,7 +428,7 @@ cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, i
 
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv, const float* gamma,
                                     int mod_stride, int B, int k, int h, int w, int hc, int wc, int C, void* colsum_ws,
-                                    int part, cudaStream_t st) {
+                                    int part, int interp_mode, cudaStream_t st) {
   const int n = h * w;
   SelectWs ws{};
   if (colsum_ws) ws = select_ws_carve(colsum_ws, B, n, C);
@@ -275,27 +437,27 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
   const double rows_x = part == 0 ? (double)n : (part == 1 ? (double)(n - k) : (double)k);
   const double rr_bytes = (double)B * C * (8.0 * rows_x + (part != 1 ? 2.0 * k : 0.0) + (part != 2 ? 2.0 * hc * wc : 0.0));
   LaunchScope scope(KC_RESTORE, 1, rr_bytes, rr_bytes, st);
+  auto* kern = (interp_mode == 1 && part != 2) ? restore_residual_bilinear_kernel : restore_residual_kernel;
   if (part == 0)
-    return launch_pdl(restore_residual_kernel, dim3(nchunks, B), dim3(256), 0, st, reinterpret_cast<float4*>(x),
+    return launch_pdl(kern, dim3(nchunks, B), dim3(256), 0, st, reinterpret_cast<float4*>(x),
                       reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h, w, hc, wc,
                       C / 8, nchunks, ws.group, ws.ngroups, reinterpret_cast<float4*>(ws.chunk_partial),
                       reinterpret_cast<float4*>(ws.group_partial), ws.tickets, part);
   // The two halves of a split restoration are ordered against another stream by events: they are
   // launched as ordinary stream work, not as programmatic dependents.
-  restore_residual_kernel<<<dim3(nchunks, B), 256, 0, st>>>(reinterpret_cast<float4*>(x), reinterpret_cast<const uint4*>(y),
-                                                            reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h,
-                                                            w, hc, wc, C / 8, nchunks, ws.group, ws.ngroups,
-                                                            reinterpret_cast<float4*>(ws.chunk_partial),
-                                                            reinterpret_cast<float4*>(ws.group_partial), ws.tickets, part);
+  kern<<<dim3(nchunks, B), 256, 0, st>>>(reinterpret_cast<float4*>(x), reinterpret_cast<const uint4*>(y),
+                                         reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h, w, hc, wc, C / 8, nchunks,
+                                         ws.group, ws.ngroups, reinterpret_cast<float4*>(ws.chunk_partial),
+                                         reinterpret_cast<float4*>(ws.group_partial), ws.tickets, part);
   return cudaGetLastError();
 }
 
 cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* pivots, const int32_t* inv, int B, int k,
-                                int h, int w, int C, void* out, cudaStream_t st) {
+                                int h, int w, int C, void* out, int interp_mode, cudaStream_t st) {
   const int rows = B * h * w;
   const double rb_bytes = (double)B * C * (2.0 * h * w + 2.0 * k + 2.0 * hc * wc);
   LaunchScope scope(KC_RESTORE, 1, rb_bytes, rb_bytes, st);
-  return launch_pdl(restore_bf16_kernel, dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const uint4*>(cache), hc, wc,
+  return launch_pdl(interp_mode == 1 ? restore_bf16_bilinear_kernel : restore_bf16_kernel, dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const uint4*>(cache), hc, wc,
                     reinterpret_cast<const uint4*>(pivots), inv, h * w, k, h, w, C / 8, reinterpret_cast<uint4*>(out), rows);
 }
 
@@ -306,11 +468,11 @@ cudaError_t launch_gather_rows(const float* x, const int32_t* idx, int B, int n,
 }
 
 cudaError_t launch_restore_rows_f32(const float* cache, int hc, int wc, const float* pivots, const int32_t* inv, int B, int k,
-                                    int h, int w, int C, float* out, cudaStream_t st) {
+                                    int h, int w, int C, float* out, int interp_mode, cudaStream_t st) {
   const int rows = B * h * w;
   const double bytes = (double)B * C * 4.0 * ((double)h * w + k + (double)hc * wc);
   LaunchScope scope(KC_RESTORE, 1, bytes, bytes, st);
-  return launch_pdl(restore_rows_f32_kernel, dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const float4*>(cache), hc, wc,
+  return launch_pdl(interp_mode == 1 ? restore_rows_f32_bilinear_kernel : restore_rows_f32_kernel, dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const float4*>(cache), hc, wc,
                     reinterpret_cast<const float4*>(pivots), inv, h * w, k, h, w, C / 4, reinterpret_cast<float4*>(out), rows);
 }
 

@@ -95,3 +95,15 @@ def test_extras_at_model_width():
     """Infinity-like head count at full width (C = 2048, 16 heads of 128), one block, three scales."""
     wl = I.Workload("w", L=1, C=2048, H=16, B=2, sides=(4, 12, 20), keep=(1.0, 1.0, 0.4), cross_len=0, seed=77)
     run_both(wl, rope_base=10000.0, qk=True)
+
+
+@pytest.mark.parametrize("granularity", [0, 1])
+def test_bilinear_restoration_in_the_step(granularity):
+    """interp_mode 1 through the whole step, both granularities (the per-sublayer caches and the step-level
+    fp32 cache), structured maps so that neighbouring cached rows differ."""
+    run_both(wl_small(64), granularity=granularity, interp_mode=1, kind="structured")
+
+
+def test_bilinear_skipped_step_and_all_options_together():
+    run_both(wl_small(64, keep_last=(0.5, 0.0)), interp_mode=1, kind="structured")
+    run_both(wl_small(128, cross_len=8), rope_base=100.0, qk=True, interp_mode=1)
