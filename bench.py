@@ -412,6 +412,32 @@ def ours(args, wl):
         del ctx_step
         torch.cuda.empty_cache()
 
+    # ---- the optional backbone pieces switched on (cosine attention, rotary positions, bilinear restoration)
+    extras = None
+    if not args.skip_variant:
+        qk_scale = torch.full((wl.L, wl.H), 10.0, device=dev)
+        ctx_x = fv.FvContext(wl.L, wl.C, wl.H, hw, wl.cache_step, wl.B, cap, gt, cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio,
+                             device=dev, rope_base=10000.0, interp_mode=1, qk_scale=qk_scale)
+        for _ in range(3):
+            schedule(ctx_x, wl.keep)
+        barrier()
+        nx = max(2, min(args.steps, 5))
+        evx = [[torch.cuda.Event(enable_timing=True) for _ in range(S + 1)] for _ in range(nx)]
+        for k in range(nx):
+            schedule(ctx_x, wl.keep, evx[k])
+        barrier()
+        if ctx_x.device_status() != 0:
+            raise SystemExit("a kernel reported an expired wait")
+        x_total = max_over_ranks(statistics.mean(evx[k][0].elapsed_time(evx[k][S]) for k in range(nx)))
+        x_pruned = max_over_ranks(sum(statistics.mean(evx[k][i].elapsed_time(evx[k][i + 1]) for k in range(nx)) for i in pruned_steps))
+        extras = {"what": "same schedule with cosine attention + 2-D rotary positions (by original token index) in the QKV epilogue and "
+                          "bilinear interpolation of the cache in the restoration",
+                  "value": world * fwd_tokens / (x_pruned * 1e-3), "unit": UNIT, "ms_per_step": x_total, "ms_per_image": x_total / wl.B,
+                  "ms_pruned_steps": x_pruned}
+        ctx_x.close()
+        del ctx_x
+        torch.cuda.empty_cache()
+
     # ---- the unpruned GPU step beside it (same kernels, keep_ratio = 1 everywhere)
     unpruned = None
     if not args.skip_unpruned:
@@ -451,7 +477,7 @@ def ours(args, wl):
             "ms_per_image": ms_per_step / wl.B, "ms_per_image_pruned_steps": pruned_ms / wl.B,
             "scale_step_ms": [round(t, 4) for t in step_ms], "wall_ms_per_step": t_wall * 1e3 / args.steps,
             "roofline": roofline, "kernels": kernels, "kernels_pruned_steps": kernels_pruned, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": gpu_launches,
-            "clocks": clocks, "unpruned_gpu": unpruned, "per_step_granularity": variant, "generation_loop": generation,
+            "clocks": clocks, "unpruned_gpu": unpruned, "per_step_granularity": variant, "backbone_options": extras, "generation_loop": generation,
             "peaks": peaks}
     print(json.dumps(line))
 

@@ -100,6 +100,8 @@ struct ResidRows {
   const float* gam0;       // gate vector of the image of the warp's first row (+ the lane's column offset), or nullptr
   const float* gam1;       // gate vector of the next image
   int n_rows;              // the lane's rows i < n_rows exist
+  int n_load;              // ... and are read before they are written (n_rows, or 0 for the plain fp32 result: a
+                           // count, not a branch, so that the reads stay plain predicated loads issued together)
   int n_first;             // the lane's rows i < n_first belong to the first image, the others to the next one
 };
 
@@ -111,6 +113,7 @@ __device__ __forceinline__ ResidRows resid_rows(const GemmDev& p, int lane, int 
   rr.out0 = static_cast<float*>(p.out) + (size_t)r * p.N + cl;
   rr.aux0 = p.aux ? static_cast<__nv_bfloat16*>(p.aux) + (size_t)r * p.N + cl : nullptr;
   rr.n_rows = max(0, min(8, (p.M - r + 3) >> 2));
+  rr.n_load = p.epilogue == EPI_F32 ? 0 : rr.n_rows;
   const int img0 = min(row0, p.M - 1) / p.rows_per_image;
   rr.n_first = max(0, min(8, ((img0 + 1) * p.rows_per_image - r + 3) >> 2));
   rr.gam0 = p.gamma ? p.gamma + (size_t)img0 * p.mod_stride + cl : nullptr;
@@ -121,14 +124,9 @@ __device__ __forceinline__ ResidRows resid_rows(const GemmDev& p, int lane, int 
 // The lane's 8 float4 of `out` for the chunk at column `col`; fetched one chunk ahead of its use.
 __device__ __forceinline__ void residual_load_x(const GemmDev& p, const ResidRows& rr, float4 (&x)[8], int lane, int col) {
   const bool col_ok = col + 4 * (lane & 7) < p.N;
-  if (p.epilogue == EPI_F32) {   // plain fp32 result: nothing to add to
-#pragma unroll
-    for (int i = 0; i < 8; ++i) x[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    return;
-  }
 #pragma unroll
   for (int i = 0; i < 8; ++i)
-    if (col_ok && i < rr.n_rows) x[i] = *reinterpret_cast<const float4*>(rr.out0 + (size_t)(4 * i) * p.N + col);
+    if (col_ok && i < rr.n_load) x[i] = *reinterpret_cast<const float4*>(rr.out0 + (size_t)(4 * i) * p.N + col);
 }
 
 __device__ __forceinline__ void residual_chunk(const GemmDev& p, const ResidRows& rr, const uint32_t (&r)[32], const float4 (&x)[8],
@@ -151,7 +149,7 @@ __device__ __forceinline__ void residual_chunk(const GemmDev& p, const ResidRows
       if (i < rr.n_rows) {
         const float4 a = *reinterpret_cast<const float4*>(trow + 4 * i * kResidTilePitch);
         const float4 gg = i < rr.n_first ? g0 : g1;
-        float4 xv = x[i];
+        float4 xv = i < rr.n_load ? x[i] : make_float4(0.f, 0.f, 0.f, 0.f);
         xv.x = fmaf(gg.x, a.x, xv.x); xv.y = fmaf(gg.y, a.y, xv.y); xv.z = fmaf(gg.z, a.z, xv.z); xv.w = fmaf(gg.w, a.w, xv.w);
         *reinterpret_cast<float4*>(rr.out0 + (size_t)(4 * i) * p.N + col) = xv;
         if (rr.aux0) {
