@@ -334,6 +334,25 @@ def test_gemm_fp32_epilogue(M, N, K, rows_per_image, splitk, path):
     assert np.abs(out.cpu().numpy() - ref).max() <= 2e-3      # fp32 accumulation of K bf16 x bf16 products
 
 
+@pytest.mark.parametrize("rows,N,K", [(960, 2048, 2048), (820, 2048, 8192)])
+def test_gemm_residual_epilogue_at_step_shapes(rows, N, K):
+    """The out-projection and second MLP GEMM of the unpruned 32x32 / pruned 64x64 steps of the bench workload
+    (B = 2), gate + residual into the fp32 stream, rows of two images inside one warp's 32 rows."""
+    B = 2
+    M = B * rows
+    a = I.normal_bf16(88, (M, K), 1.0 if K <= 2048 else 0.5); w = I.normal_bf16(89, (N, K), 0.02); b = I.normal_bf16(90, (N,), 0.02)
+    x = I.normal(91, (M, N)); mod = I.normal(92, (B, 6, N), 0.3)
+    xd, modd = dev(x), dev(mod)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    fv.fv_gemm_bf16(bf16_dev(a), bf16_dev(w), bf16_dev(b), epilogue=2, out=xd, gamma=modd.data_ptr() + 2 * 4 * N, mod_stride=6 * N,
+                    rows_per_image=rows, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    y = O.linear(I.bf16_bits_to_f32(a), I.bf16_bits_to_f32(w), I.bf16_bits_to_f32(b))
+    ref = x.astype(np.float64) + np.repeat(mod[:, 2].astype(np.float64), rows, axis=0) * y
+    assert np.abs(xd.cpu().numpy() - ref).max() <= 2e-3
+
+
 # ------------------------------------------------------------------ attention over the KV cache
 ATTN_CASES = [  # B, rows, H, C, kv_len, cap
     (2, 85, 4, 256, 340, 344), (1, 300, 2, 256, 1000, 1024), (2, 128, 16, 1024, 485, 488), (1, 1, 4, 256, 1, 8),
