@@ -293,6 +293,29 @@ def test_gemm_bf16_on_cta_pairs(M, N, K, path):
     assert err <= MAX_ABS and cos >= MIN_COS, (err, cos)
 
 
+@pytest.mark.parametrize("epilogue", [0, 1])
+@pytest.mark.parametrize("M,N,K,splitk", [(128, 128, 64, False), (7, 136, 72, False), (300, 1024, 4096, True), (32, 2048, 2048, True),
+                                          (128, 2048, 8192, True), (1000, 1032, 1024, False), (2, 2048, 8192, True)])
+def test_gemm_bf16_width_64_tiles(M, N, K, splitk, epilogue):
+    """The 64-wide tile (chosen by itself for few rows against a narrow output), forced for every shape, with
+    and without the K split."""
+    a = I.normal_bf16(93, (M, K), 1.0 if K <= 2048 else 0.5); w = I.normal_bf16(94, (N, K), 0.02); b = I.normal_bf16(95, (N,), 0.02)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = torch.zeros(fv.lib().fv_gemm_splitk_workspace_bytes(), dtype=torch.uint8, device=DEV) if splitk else None
+    assert fv.lib().fv_gemm_force_path(7) == 0
+    try:
+        out = fv.fv_gemm_bf16(bf16_dev(a), bf16_dev(w), bf16_dev(b), epilogue=epilogue, status=status, splitk_ws=ws)
+        torch.cuda.synchronize()
+    finally:
+        fv.lib().fv_gemm_force_path(0)
+    assert int(status.item()) == 0
+    ref = O.linear(I.bf16_bits_to_f32(a), I.bf16_bits_to_f32(w), I.bf16_bits_to_f32(b))
+    if epilogue == 1:
+        ref = O.gelu_tanh(ref)
+    err, cos = per_token_errors(bf16_host(out), ref)
+    assert err <= MAX_ABS and cos >= MIN_COS, (err, cos)
+
+
 def test_gemm_residual_epilogue_with_cache_copy():
     B, rows, N, K = 2, 100, 256, 512
     M = B * rows
@@ -312,7 +335,7 @@ def test_gemm_residual_epilogue_with_cache_copy():
     assert err <= MAX_ABS and cos >= MIN_COS
 
 
-@pytest.mark.parametrize("path", [0, 2, 3, 4, 5, 6])
+@pytest.mark.parametrize("path", [0, 2, 3, 4, 5, 6, 7])
 @pytest.mark.parametrize("M,N,K,rows_per_image,splitk", [(300, 512, 256, 300, False), (7, 136, 72, 7, False), (1000, 1032, 1024, 500, False),
                                                           (2, 2048, 2048, 1, True), (130, 1920, 1920, 20, False)])
 def test_gemm_fp32_epilogue(M, N, K, rows_per_image, splitk, path):
