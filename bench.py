@@ -32,7 +32,7 @@ from paper_2503_23367_b200 import inputs as I  # noqa: E402
 # capture of the same kernel measured against that count (summaries under profiles/).
 NCU_TRAFFIC_NOTE = {
     "gemm": "A + W + out bytes per launch, mean over the pruned steps' launches; ncu on M1640 N6144 K2048: dram read 31.95 MB = A + W "
-            "(31.9 MB), out (20 MB) still in L2 at kernel end; CTA-pair kernel M1844 N2048 K8192: read 63.8 MB = A + W, write 4.4 of 7.6 MB",
+            "(31.9 MB), out (20 MB) still in L2 at kernel end; CTA-pair kernel M1844 N2048 K8192: read 63.8 MB = A + W, write 3.8 of 7.6 MB",
     "attention": "Q + O + K + V^T bytes per launch; ncu on q820 kv5223 H16 hd128 B2: dram read 92.7 MB (K, V^T, Q = 92.3 MB), write 3.6 of 6.7 MB",
     "restore": "x read + written, y, cache; ncu on B2 64x64 C2048 k820: read 82.3 MB + write 11.8 MB of 149 MB (x written stays in L2)",
     "select": "x once + scores + indices; ncu on B2 64x64 C2048: score+top-k kernel reads 67.3 MB (x = 67.1 MB)",
