@@ -28,17 +28,32 @@ __global__ void __launch_bounds__(256) argmax_rows_kernel(const float4* __restri
   const float4* np = noise ? noise + (size_t)row * V4 : nullptr;
   float best = -INFINITY;
   int bi = INT_MAX;
-  for (int j = lane; j < V4; j += 32) {
-    float4 z = __ldcs(lp + j);
+  for (int j0 = 0; j0 < V4; j0 += 128) {   // four loads per lane in flight
+    float4 z[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int j = j0 + lane + 32 * i;
+      z[i] = j < V4 ? __ldcs(lp + j) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    }
     if (np) {
-      const float4 g = __ldcs(np + j);
-      z.x = fmaf(tau, g.x, z.x); z.y = fmaf(tau, g.y, z.y); z.z = fmaf(tau, g.z, z.z); z.w = fmaf(tau, g.w, z.w);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int j = j0 + lane + 32 * i;
+        if (j < V4) {
+          const float4 g = __ldcs(np + j);
+          z[i].x = fmaf(tau, g.x, z[i].x); z[i].y = fmaf(tau, g.y, z[i].y); z[i].z = fmaf(tau, g.z, z[i].z); z[i].w = fmaf(tau, g.w, z[i].w);
+        }
+      }
     }
     // indices grow within a lane, so a strict comparison keeps the first occurrence
-    if (z.x > best) { best = z.x; bi = 4 * j; }
-    if (z.y > best) { best = z.y; bi = 4 * j + 1; }
-    if (z.z > best) { best = z.z; bi = 4 * j + 2; }
-    if (z.w > best) { best = z.w; bi = 4 * j + 3; }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int j = j0 + lane + 32 * i;
+      if (z[i].x > best) { best = z[i].x; bi = 4 * j; }
+      if (z[i].y > best) { best = z[i].y; bi = 4 * j + 1; }
+      if (z[i].z > best) { best = z[i].z; bi = 4 * j + 2; }
+      if (z[i].w > best) { best = z[i].w; bi = 4 * j + 3; }
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -83,7 +98,8 @@ template <int D>
 __global__ void __launch_bounds__(256) next_input_kernel(const float* __restrict__ r, int h, int w, int h2, int w2, const float* __restrict__ w_in,
                                                          const float* __restrict__ b_in, const float* __restrict__ pos, int C, int B,
                                                          float* __restrict__ x_out) {
-  __shared__ float r_s[kNextTokens][D];
+  __shared__ __align__(16) float r_s[kNextTokens][D];
+  __shared__ int s_t2[kNextTokens];      // token index inside the next map (row of pos), per staged token
   pdl_trigger();
   const int n = h * w, n2 = h2 * w2;
   const long rows = (long)B * n2;
@@ -98,6 +114,7 @@ __global__ void __launch_bounds__(256) next_input_kernel(const float* __restrict
       const int y = t2 / w2, x = t2 - y * w2;
       const int src = (int)(((long)y * h) / h2) * w + (int)(((long)x * w) / w2);
       v = r[((size_t)b * n + src) * D + j];
+      if (j == 0) s_t2[t] = t2;
     }
     r_s[t][j] = v;
   }
@@ -111,19 +128,28 @@ __global__ void __launch_bounds__(256) next_input_kernel(const float* __restrict
       wr[j] = q.x; wr[j + 1] = q.y; wr[j + 2] = q.z; wr[j + 3] = q.w;
     }
     const float bias = b_in ? __ldg(b_in + c) : 0.f;
-    for (int t = 0; t < t_valid; ++t) {
-      const long row = row0 + t;
-      const int t2 = (int)(row % n2);
-      float acc = 0.f;
+    float* out = x_out + (size_t)row0 * C + c;
+    for (int t0 = 0; t0 < t_valid; t0 += 8) {   // eight tokens at a time: their position-embedding loads go out together
+      float pe[8];
 #pragma unroll
-      for (int j = 0; j < D; ++j) acc = fmaf(r_s[t][j], wr[j], acc);
-      acc += bias;
-      if (pos) acc += __ldg(pos + (size_t)t2 * C + c);
-      x_out[(size_t)row * C + c] = acc;
+      for (int u = 0; u < 8; ++u) pe[u] = (pos && t0 + u < t_valid) ? __ldg(pos + (size_t)s_t2[t0 + u] * C + c) : 0.f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (t0 + u < t_valid) {
+          float acc = 0.f;
+#pragma unroll
+          for (int j = 0; j < D; j += 4) {      // the token's vector is read as float4 broadcasts
+            const float4 q = *reinterpret_cast<const float4*>(&r_s[t0 + u][j]);
+            acc = fmaf(q.x, wr[j], acc); acc = fmaf(q.y, wr[j + 1], acc); acc = fmaf(q.z, wr[j + 2], acc); acc = fmaf(q.w, wr[j + 3], acc);
+          }
+          acc += bias;
+          acc += pe[u];
+          out[(size_t)(t0 + u) * C] = acc;
+        }
+      }
     }
   }
 }
-
 
 struct HeadLayout { size_t a, logits, splitk, total; };
 HeadLayout head_layout(int rows, int C, int V, bool own_logits) {
