@@ -30,6 +30,8 @@ Backbone extras (all off by default; the paper names none of them, they belong t
 so each is a reading stated here and pinned on its own):
   * `interp_mode="bilinear"`: interpolate(.) of Eq. 6 as a bilinear blend with half-pixel centres
     (source coordinate (dst + 0.5) * in / out - 0.5, clamped), the convention of library resizing routines.
+    `interp_mode="bicubic"`: separable cubic convolution (Keys' kernel, a = -0.75) over 4 x 4 cached tokens at
+    the same half-pixel coordinates, tap indices clamped to the map.
   * `qk_scale` [L, H]: cosine attention -- in the self-attention sublayer every head's query and key are
     divided by their Euclidean norm (floored at 1e-12) and the query is multiplied by the head's scale.
   * `rope_base`: two-dimensional rotary position embedding in the self-attention sublayer.  A token at
@@ -171,11 +173,45 @@ def ctr_upsample_bilinear(cache: np.ndarray, hc: int, wc: int, h: int, w: int) -
     return (top * (1 - ty) + bot * ty).reshape(cache.shape[0], h * w, cache.shape[-1])
 
 
+def bicubic_taps(n_out: int, n_in: int, a: float = -0.75):
+    """Per destination index along one axis: four source indices (clamped to the map) and their weights under
+    cubic convolution (Keys' kernel with a = -0.75) at half-pixel centres, s = (dst + 0.5) * n_in / n_out - 0.5:
+    W(d) = (a+2)|d|^3 - (a+3)|d|^2 + 1 for |d| <= 1,  a|d|^3 - 5a|d|^2 + 8a|d| - 4a for 1 < |d| < 2."""
+    def kern(dist: float) -> float:
+        dist = abs(dist)
+        if dist <= 1.0:
+            return (a + 2.0) * dist ** 3 - (a + 3.0) * dist ** 2 + 1.0
+        if dist < 2.0:
+            return a * dist ** 3 - 5.0 * a * dist ** 2 + 8.0 * a * dist - 4.0 * a
+        return 0.0
+    idx = np.empty((n_out, 4), dtype=np.int64); wt = np.empty((n_out, 4), dtype=F64)
+    for o in range(n_out):
+        s = (o + 0.5) * n_in / n_out - 0.5
+        i0 = int(math.floor(s))
+        for q in range(4):
+            pos = i0 - 1 + q
+            idx[o, q] = min(max(pos, 0), n_in - 1)
+            wt[o, q] = kern(s - pos)
+    return idx, wt
+
+
+def ctr_upsample_bicubic(cache: np.ndarray, hc: int, wc: int, h: int, w: int) -> np.ndarray:
+    """Eq. 6 with interpolate = bicubic (separable cubic convolution).  cache [B,hc*wc,C] -> [B,h*w,C]."""
+    c = np.asarray(cache, dtype=F64).reshape(cache.shape[0], hc, wc, cache.shape[-1])
+    yi, yw = bicubic_taps(h, hc)
+    xi, xw = bicubic_taps(w, wc)
+    out = np.zeros((cache.shape[0], h, w, cache.shape[-1]), dtype=F64)
+    for qy in range(4):
+        for qx in range(4):
+            out += c[:, yi[:, qy]][:, :, xi[:, qx]] * (yw[:, qy][None, :, None, None] * xw[:, qx][None, None, :, None])
+    return out.reshape(cache.shape[0], h * w, cache.shape[-1])
+
+
 def cached_token_restoration(pivots: np.ndarray, idx: np.ndarray, cache: np.ndarray,
                              hc: int, wc: int, h: int, w: int, interp_mode: str = "nearest") -> np.ndarray:
     """Algorithm 1, second routine: upsample the cache to the current scale, then write the
     forwarded rows into their slots.  pivots [B,k,C], idx [B,k] -> [B,h*w,C]."""
-    up = ctr_upsample if interp_mode == "nearest" else ctr_upsample_bilinear
+    up = {"nearest": ctr_upsample, "bilinear": ctr_upsample_bilinear, "bicubic": ctr_upsample_bicubic}[interp_mode]
     out = np.array(up(np.asarray(cache, dtype=F64), hc, wc, h, w), dtype=F64, copy=True)
     for b in range(out.shape[0]):
         out[b, idx[b], :] = pivots[b]
@@ -285,7 +321,7 @@ class VarOracle:
     def __init__(self, L: int, C: int, H: int, sides_hw: Sequence[Sequence[int]], cache_step: int,
                  weights: Dict, B: int, cross_len: int = 0, granularity: str = "sublayer",
                  interp_mode: str = "nearest", rope_base: Optional[float] = None, qk_scale: Optional[np.ndarray] = None):
-        assert granularity in ("sublayer", "step") and interp_mode in ("nearest", "bilinear")
+        assert granularity in ("sublayer", "step") and interp_mode in ("nearest", "bilinear", "bicubic")
         self.granularity = granularity
         self.interp_mode, self.rope_base = interp_mode, rope_base
         self.qk_scale = None if qk_scale is None else np.asarray(qk_scale, dtype=F64)      # [L, H]
@@ -370,7 +406,7 @@ class VarOracle:
             assert self.step_cache is not None and scale_idx > self.cache_step
             hc, wc = self.hw[self.cache_step]
             self.step += 1
-            up = ctr_upsample if self.interp_mode == "nearest" else ctr_upsample_bilinear
+            up = {"nearest": ctr_upsample, "bilinear": ctr_upsample_bilinear, "bicubic": ctr_upsample_bicubic}[self.interp_mode]
             return up(self.step_cache, hc, wc, h, w_)
         pruned = keep_ratio < 1.0
         k = kept_count(keep_ratio, h, w_) if pruned else n

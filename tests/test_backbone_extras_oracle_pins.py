@@ -23,6 +23,20 @@ def test_bilinear_restoration_equals_library_resize(hc, wc, h, w):
     np.testing.assert_allclose(O.ctr_upsample_bilinear(np.full((1, hc * wc, 1), 3.5), hc, wc, h, w), 3.5, atol=1e-12)
 
 
+@pytest.mark.parametrize("hc,wc,h,w", [(2, 2, 4, 4), (3, 5, 7, 8), (4, 4, 4, 4), (5, 3, 6, 9), (1, 1, 3, 2), (6, 6, 4, 3), (8, 8, 16, 12)])
+def test_bicubic_restoration_equals_library_resize(hc, wc, h, w):
+    rng = np.random.default_rng(hc * 10 + w)
+    cache = rng.standard_normal((2, hc * wc, 3))
+    got = O.ctr_upsample_bicubic(cache, hc, wc, h, w)
+    t = torch.from_numpy(cache).reshape(2, hc, wc, 3).permute(0, 3, 1, 2)
+    lib = F.interpolate(t, size=(h, w), mode="bicubic", align_corners=False).permute(0, 2, 3, 1).reshape(2, h * w, 3).numpy()
+    np.testing.assert_allclose(got, lib, rtol=1e-11, atol=1e-11)
+    # the four weights of a tap set sum to one: a constant map stays constant
+    np.testing.assert_allclose(O.ctr_upsample_bicubic(np.full((1, hc * wc, 1), -2.25), hc, wc, h, w), -2.25, atol=1e-12)
+    idx, wt = O.bicubic_taps(h, hc)
+    np.testing.assert_allclose(wt.sum(1), 1.0, atol=1e-12)
+
+
 def test_bilinear_restoration_keeps_pivots_and_blends_elsewhere():
     rng = np.random.default_rng(3)
     cache = rng.standard_normal((1, 4, 3)); piv = rng.standard_normal((1, 2, 3)); idx = np.array([[1, 14]])
