@@ -102,6 +102,8 @@ fv_status fv_prune_select_static(const float *x_dev, int32_t B, int32_t h, int32
  *   interp_mode    0: nearest, as above (the default reading of the paper's mode-less interpolate).
  *                  1: bilinear with half-pixel centres (source coordinate (dst+0.5)*in/out - 0.5 per axis,
  *                     clamped): an unkept token is the fp32 blend of four cached rows, rounded to bf16 once.
+ *                  2: bicubic at the same coordinates (cubic convolution with a = -0.75 over 4 x 4 cached
+ *                     tokens, tap indices clamped to the map), blended in fp32, rounded once.
  * Errors: INVALID_ARG, CUDA. */
 fv_status fv_restore(const void *cache_prev_dev, int32_t hc, int32_t wc, const void *pivots_dev,
                      const int32_t *idx_dev, int32_t B, int32_t k, int32_t h, int32_t w, int32_t C,
@@ -144,7 +146,8 @@ typedef struct {
                          the angle is that of the token's ORIGINAL slot (its kept index), not of its row
                          in the compact tensor.                                                          */
   int32_t interp_mode;/* interpolate(.) of Eq. 6: 0 nearest (src = floor(dst*in/out)); 1 bilinear with
-                         half-pixel centres (src = (dst+0.5)*in/out - 0.5, clamped)                      */
+                         half-pixel centres (src = (dst+0.5)*in/out - 0.5, clamped); 2 bicubic (cubic
+                         convolution, a = -0.75, 4 x 4 cached tokens, tap indices clamped to the map)     */
 } fv_config;
 
 typedef struct { /* HOST arrays of length L holding DEVICE pointers; bf16 unless noted; borrowed   */

@@ -77,7 +77,7 @@ bool config_ok(const fv_config* c) {
     if (c->h[i] <= 0 || c->w[i] <= 0) return false;
   if (c->cache_step >= c->n_steps) return false;
   if (c->granularity != 0 && c->granularity != 1) return false;
-  if (c->interp_mode != 0 && c->interp_mode != 1) return false;
+  if (c->interp_mode < 0 || c->interp_mode > 2) return false;
   if (!(c->rope_base >= 0.f)) return false;
   return true;
 }
@@ -161,7 +161,7 @@ fv_status fv_restore(const void* cache_prev_dev, int32_t hc, int32_t wc, const v
                      int32_t B, int32_t k, int32_t h, int32_t w, int32_t C, void* out_dev, int32_t* inv_scratch_dev,
                      int32_t interp_mode, void* stream) {
   if (!cache_prev_dev || !pivots_dev || !idx_dev || !out_dev || !inv_scratch_dev) return FV_ERR_INVALID_ARG;
-  if (interp_mode != 0 && interp_mode != 1) return FV_ERR_INVALID_ARG;
+  if (interp_mode < 0 || interp_mode > 2) return FV_ERR_INVALID_ARG;
   if (B <= 0 || k <= 0 || h <= 0 || w <= 0 || hc <= 0 || wc <= 0 || C <= 0 || (C % 8) || k > h * w) return FV_ERR_INVALID_ARG;
   if (!aligned16(cache_prev_dev) || !aligned16(pivots_dev) || !aligned16(out_dev)) return FV_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -183,7 +183,7 @@ fv_status fv_gather_ln(const float* x_dev, const int32_t* idx_dev, int32_t B, in
 fv_status fv_restore_residual(float* x_dev, const void* y_dev, const void* cache_dev, const int32_t* inv_dev,
                               const float* gamma_dev, int32_t mod_stride, int32_t B, int32_t k, int32_t h, int32_t w,
                               int32_t hc, int32_t wc, int32_t C, int32_t interp_mode, void* stream) {
-  if (interp_mode != 0 && interp_mode != 1) return FV_ERR_INVALID_ARG;
+  if (interp_mode < 0 || interp_mode > 2) return FV_ERR_INVALID_ARG;
   if (!x_dev || !y_dev || !cache_dev || !inv_dev || B <= 0 || k <= 0 || h <= 0 || w <= 0 || hc <= 0 || wc <= 0) return FV_ERR_INVALID_ARG;
   if (C <= 0 || (C % 8)) return FV_ERR_INVALID_ARG;
   return cuda_status(launch_restore_residual(x_dev, y_dev, cache_dev, inv_dev, gamma_dev, mod_stride, B, k, h, w, hc, wc, C,

@@ -439,6 +439,8 @@ static cudaError_t launch_bn(const GemmArgs& g, const GemmDev& p, int tiles_m, c
   } else {
     if (p.epilogue == EPI_RESIDUAL || p.epilogue == EPI_F32)
       return launch_pdl(gemm_bf16_kernel<BN, false, 1>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::smem_bytes(true), st, tmA, tmB, p);
+    if constexpr (BN < 128)
+      if (p.epilogue == EPI_QKV_SPLIT && (p.qk_scale || p.rope_table)) return cudaErrorInvalidValue;   // never chosen for them
     if constexpr (BN >= 128)
       if (p.epilogue == EPI_QKV_SPLIT && (p.qk_scale || p.rope_table))
         return launch_pdl(gemm_bf16_kernel<BN, false, 2>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::smem_bytes(false), st, tmA, tmB, p);
@@ -469,6 +471,7 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   if (qk_extras) {
     if (g.head_dim != 64 && g.head_dim != 128) return FV_ERR_UNSUPPORTED;
     if (tc.pair) tc = TileChoice{256, false};
+    if (tc.bn < 128) tc.bn = 128;            // the extras exist for tiles of at least 128 columns
     if (tc.bn % g.head_dim) tc.bn = 256;
   }
   int bn = tc.bn;

@@ -96,19 +96,49 @@ __device__ __forceinline__ int nearest_src(int t, int h, int w, int hc, int wc) 
   return ((y * hc) / h) * wc + (xx * wc) / w;
 }
 
-// Bilinear interpolate(.) of Eq. 6 with half-pixel centres: the four source tokens of destination token t and
-// their weights (source coordinate (dst + 0.5) * in / out - 0.5 per axis, clamped to the map).
-struct BilinearTaps { int src[4]; float wt[4]; };
-__device__ __forceinline__ BilinearTaps bilinear_taps(int t, int h, int w, int hc, int wc) {
+// interpolate(.) of Eq. 6 beyond nearest neighbour, half-pixel centres (source coordinate
+// (dst + 0.5) * in / out - 0.5 per axis): the source tokens of destination token t and their weights.
+//   TAPS 4 : bilinear (coordinate clamped to the map, two taps per axis);
+//   TAPS 16: bicubic, separable cubic convolution (Keys' kernel, a = -0.75), four taps per axis with the
+//            tap indices clamped to the map.
+template <int TAPS> struct InterpTaps { int src[TAPS]; float wt[TAPS]; };
+
+__device__ __forceinline__ void cubic_axis(int o, int n_out, int n_in, int (&idx)[4], float (&wt)[4]) {
+  const double a = -0.75;
+  const double s = (o + 0.5) * (double)n_in / n_out - 0.5;
+  const int i0 = (int)floor(s);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int pos = i0 - 1 + q;
+    const double d = fabs(s - pos);
+    const double wv = d <= 1.0 ? ((a + 2.0) * d - (a + 3.0)) * d * d + 1.0 : (d < 2.0 ? ((a * d - 5.0 * a) * d + 8.0 * a) * d - 4.0 * a : 0.0);
+    idx[q] = min(max(pos, 0), n_in - 1);
+    wt[q] = (float)wv;
+  }
+}
+
+template <int TAPS>
+__device__ __forceinline__ InterpTaps<TAPS> interp_taps(int t, int h, int w, int hc, int wc) {
   const int y = t / w, xx = t - y * w;
-  double sy = (y + 0.5) * (double)hc / h - 0.5, sx = (xx + 0.5) * (double)wc / w - 0.5;
-  sy = fmin(fmax(sy, 0.0), (double)(hc - 1)); sx = fmin(fmax(sx, 0.0), (double)(wc - 1));
-  const int y0 = (int)floor(sy), x0 = (int)floor(sx);
-  const int y1 = min(y0 + 1, hc - 1), x1 = min(x0 + 1, wc - 1);
-  const float ty = (float)(sy - y0), tx = (float)(sx - x0);
-  BilinearTaps b;
-  b.src[0] = y0 * wc + x0; b.src[1] = y0 * wc + x1; b.src[2] = y1 * wc + x0; b.src[3] = y1 * wc + x1;
-  b.wt[0] = (1.f - ty) * (1.f - tx); b.wt[1] = (1.f - ty) * tx; b.wt[2] = ty * (1.f - tx); b.wt[3] = ty * tx;
+  InterpTaps<TAPS> b;
+  if constexpr (TAPS == 4) {
+    double sy = (y + 0.5) * (double)hc / h - 0.5, sx = (xx + 0.5) * (double)wc / w - 0.5;
+    sy = fmin(fmax(sy, 0.0), (double)(hc - 1)); sx = fmin(fmax(sx, 0.0), (double)(wc - 1));
+    const int y0 = (int)floor(sy), x0 = (int)floor(sx);
+    const int y1 = min(y0 + 1, hc - 1), x1 = min(x0 + 1, wc - 1);
+    const float ty = (float)(sy - y0), tx = (float)(sx - x0);
+    b.src[0] = y0 * wc + x0; b.src[1] = y0 * wc + x1; b.src[2] = y1 * wc + x0; b.src[3] = y1 * wc + x1;
+    b.wt[0] = (1.f - ty) * (1.f - tx); b.wt[1] = (1.f - ty) * tx; b.wt[2] = ty * (1.f - tx); b.wt[3] = ty * tx;
+  } else {
+    int yi[4], xi[4];
+    float yw[4], xw[4];
+    cubic_axis(y, h, hc, yi, yw);
+    cubic_axis(xx, w, wc, xi, xw);
+#pragma unroll
+    for (int qy = 0; qy < 4; ++qy)
+#pragma unroll
+      for (int qx = 0; qx < 4; ++qx) { b.src[4 * qy + qx] = yi[qy] * wc + xi[qx]; b.wt[4 * qy + qx] = yw[qy] * xw[qx]; }
+  }
   return b;
 }
 
@@ -254,19 +284,21 @@ __global__ void __launch_bounds__(256) restore_rows_f32_kernel(const float4* __r
 }
 
 
-// restore_residual_kernel with bilinear interpolation of the cache: an unkept token blends four cached rows
-// (fp32), a kept token takes its forwarded row.  Same CTA shape, row ownership and column-sum handling; two
-// rows in flight instead of four (four source rows each).  part 2 (kept rows only) never interpolates and
+// restore_residual_kernel with bilinear (TAPS 4) or bicubic (TAPS 16) interpolation of the cache: an unkept
+// token blends TAPS cached rows (fp32), a kept token takes its forwarded row.  Same CTA shape, row ownership
+// and column-sum handling; fewer rows in flight (two, or one with sixteen source rows).  part 2 (kept rows only) never interpolates and
 // runs the kernel above.
-__global__ void __launch_bounds__(256) restore_residual_bilinear_kernel(float4* __restrict__ x, const uint4* __restrict__ y,
+template <int TAPS>
+__global__ void __launch_bounds__(256) restore_residual_interp_kernel(float4* __restrict__ x, const uint4* __restrict__ y,
                                                                         const uint4* __restrict__ cache, const int32_t* __restrict__ inv,
                                                                         const float* __restrict__ gamma, int mod_stride, int n, int k,
                                                                         int h, int w, int hc, int wc, int C8, int nchunks, int group,
                                                                         int ngroups, float4* __restrict__ chunk_partial,
                                                                         float4* __restrict__ group_partial, unsigned int* tickets,
                                                                         int part) {
-  __shared__ const uint4* s_src[kColsumRows][4];
-  __shared__ float s_wt[kColsumRows][4];
+  constexpr int ROWS = TAPS == 4 ? 2 : 1;   // rows in flight per thread
+  __shared__ const uint4* s_src[kColsumRows][TAPS];
+  __shared__ float s_wt[kColsumRows][TAPS];
   __shared__ int s_on[kColsumRows];
   pdl_trigger();
   pdl_wait();
@@ -277,10 +309,10 @@ __global__ void __launch_bounds__(256) restore_residual_bilinear_kernel(float4* 
     const int t = t0 + threadIdx.x;
     const int j = __ldg(inv + (size_t)b * n + t);
     if (j >= 0) {
-      for (int q = 0; q < 4; ++q) { s_src[threadIdx.x][q] = y + ((size_t)b * k + j) * C8; s_wt[threadIdx.x][q] = q == 0 ? 1.f : 0.f; }
+      for (int q = 0; q < TAPS; ++q) { s_src[threadIdx.x][q] = y + ((size_t)b * k + j) * C8; s_wt[threadIdx.x][q] = q == 0 ? 1.f : 0.f; }
     } else {
-      const BilinearTaps bt = bilinear_taps(t, h, w, hc, wc);
-      for (int q = 0; q < 4; ++q) { s_src[threadIdx.x][q] = cache + ((size_t)b * hc * wc + bt.src[q]) * C8; s_wt[threadIdx.x][q] = bt.wt[q]; }
+      const InterpTaps<TAPS> bt = interp_taps<TAPS>(t, h, w, hc, wc);
+      for (int q = 0; q < TAPS; ++q) { s_src[threadIdx.x][q] = cache + ((size_t)b * hc * wc + bt.src[q]) * C8; s_wt[threadIdx.x][q] = bt.wt[q]; }
     }
     s_on[threadIdx.x] = part == 0 || (part == 1) == (j < 0);
   }
@@ -293,24 +325,24 @@ __global__ void __launch_bounds__(256) restore_residual_bilinear_kernel(float4* 
       g0 = __ldg(g + 2 * c8); g1 = __ldg(g + 2 * c8 + 1);
     }
     float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
-    for (int r = 0; r < rows; r += 2) {
-      uint4 p[2][4];
-      float4 x0[2], x1[2];
+    for (int r = 0; r < rows; r += ROWS) {
+      uint4 p[ROWS][TAPS];
+      float4 x0[ROWS], x1[ROWS];
 #pragma unroll
-      for (int i = 0; i < 2; ++i) {
+      for (int i = 0; i < ROWS; ++i) {
         if (r + i < rows && s_on[r + i]) {
           float4* xr = xbase + (size_t)(r + i) * C8 * 2 + 2 * c8;
           x0[i] = xr[0]; x1[i] = xr[1];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) p[i][q] = __ldg(s_src[r + i][q] + c8);
+          for (int q = 0; q < TAPS; ++q) p[i][q] = __ldg(s_src[r + i][q] + c8);
         }
       }
 #pragma unroll
-      for (int i = 0; i < 2; ++i) {
+      for (int i = 0; i < ROWS; ++i) {
         if (r + i < rows && s_on[r + i]) {
           float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
+          for (int q = 0; q < TAPS; ++q) {
             float fq[8];
             bf16x8_to_float(p[i][q], fq);
             const float wq = s_wt[r + i][q];
@@ -336,9 +368,10 @@ __global__ void __launch_bounds__(256) restore_residual_bilinear_kernel(float4* 
     fold_group_partials(b, chunk, nchunks, group, ngroups, C8 * 2, chunk_partial, group_partial, tickets);
 }
 
-// Plain restoration (no residual) with bilinear interpolation, one warp per output row; bf16 rows (8 per
-// uint4, blended in fp32 and rounded once) or fp32 rows.
-__global__ void __launch_bounds__(256) restore_bf16_bilinear_kernel(const uint4* __restrict__ cache, int hc, int wc,
+// Plain restoration (no residual) with bilinear / bicubic interpolation, one warp per output row; bf16 rows
+// (8 per uint4, blended in fp32 and rounded once) or fp32 rows.
+template <int TAPS>
+__global__ void __launch_bounds__(256) restore_bf16_interp_kernel(const uint4* __restrict__ cache, int hc, int wc,
                                                                     const uint4* __restrict__ pivots, const int32_t* __restrict__ inv,
                                                                     int n, int k, int h, int w, int C8, uint4* __restrict__ out,
                                                                     int total_rows) {
@@ -354,12 +387,12 @@ __global__ void __launch_bounds__(256) restore_bf16_bilinear_kernel(const uint4*
     for (int c8 = lane; c8 < C8; c8 += 32) dst[c8] = __ldg(src + c8);
     return;
   }
-  const BilinearTaps bt = bilinear_taps(t, h, w, hc, wc);
+  const InterpTaps<TAPS> bt = interp_taps<TAPS>(t, h, w, hc, wc);
   const uint4* base = cache + (size_t)b * hc * wc * C8;
   for (int c8 = lane; c8 < C8; c8 += 32) {
     float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < TAPS; ++q) {
       float fq[8];
       bf16x8_to_float(__ldg(base + (size_t)bt.src[q] * C8 + c8), fq);
 #pragma unroll
@@ -371,7 +404,8 @@ __global__ void __launch_bounds__(256) restore_bf16_bilinear_kernel(const uint4*
   }
 }
 
-__global__ void __launch_bounds__(256) restore_rows_f32_bilinear_kernel(const float4* __restrict__ cache, int hc, int wc,
+template <int TAPS>
+__global__ void __launch_bounds__(256) restore_rows_f32_interp_kernel(const float4* __restrict__ cache, int hc, int wc,
                                                                         const float4* __restrict__ pivots, const int32_t* __restrict__ inv,
                                                                         int n, int k, int h, int w, int C4, float4* __restrict__ out,
                                                                         int total_rows) {
@@ -387,12 +421,12 @@ __global__ void __launch_bounds__(256) restore_rows_f32_bilinear_kernel(const fl
     for (int c4 = lane; c4 < C4; c4 += 32) dst[c4] = __ldg(src + c4);
     return;
   }
-  const BilinearTaps bt = bilinear_taps(t, h, w, hc, wc);
+  const InterpTaps<TAPS> bt = interp_taps<TAPS>(t, h, w, hc, wc);
   const float4* base = cache + (size_t)b * hc * wc * C4;
   for (int c4 = lane; c4 < C4; c4 += 32) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < TAPS; ++q) {
       const float4 v = __ldg(base + (size_t)bt.src[q] * C4 + c4);
       acc.x = fmaf(bt.wt[q], v.x, acc.x); acc.y = fmaf(bt.wt[q], v.y, acc.y); acc.z = fmaf(bt.wt[q], v.z, acc.z); acc.w = fmaf(bt.wt[q], v.w, acc.w);
     }
@@ -437,7 +471,8 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
   const double rows_x = part == 0 ? (double)n : (part == 1 ? (double)(n - k) : (double)k);
   const double rr_bytes = (double)B * C * (8.0 * rows_x + (part != 1 ? 2.0 * k : 0.0) + (part != 2 ? 2.0 * hc * wc : 0.0));
   LaunchScope scope(KC_RESTORE, 1, rr_bytes, rr_bytes, st);
-  auto* kern = (interp_mode == 1 && part != 2) ? restore_residual_bilinear_kernel : restore_residual_kernel;
+  auto* kern = (interp_mode == 0 || part == 2) ? restore_residual_kernel
+               : (interp_mode == 1 ? restore_residual_interp_kernel<4> : restore_residual_interp_kernel<16>);
   if (part == 0)
     return launch_pdl(kern, dim3(nchunks, B), dim3(256), 0, st, reinterpret_cast<float4*>(x),
                       reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h, w, hc, wc,
@@ -457,7 +492,7 @@ cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* p
   const int rows = B * h * w;
   const double rb_bytes = (double)B * C * (2.0 * h * w + 2.0 * k + 2.0 * hc * wc);
   LaunchScope scope(KC_RESTORE, 1, rb_bytes, rb_bytes, st);
-  return launch_pdl(interp_mode == 1 ? restore_bf16_bilinear_kernel : restore_bf16_kernel, dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const uint4*>(cache), hc, wc,
+  return launch_pdl(interp_mode == 0 ? restore_bf16_kernel : (interp_mode == 1 ? restore_bf16_interp_kernel<4> : restore_bf16_interp_kernel<16>), dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const uint4*>(cache), hc, wc,
                     reinterpret_cast<const uint4*>(pivots), inv, h * w, k, h, w, C / 8, reinterpret_cast<uint4*>(out), rows);
 }
 
@@ -472,7 +507,8 @@ cudaError_t launch_restore_rows_f32(const float* cache, int hc, int wc, const fl
   const int rows = B * h * w;
   const double bytes = (double)B * C * 4.0 * ((double)h * w + k + (double)hc * wc);
   LaunchScope scope(KC_RESTORE, 1, bytes, bytes, st);
-  return launch_pdl(interp_mode == 1 ? restore_rows_f32_bilinear_kernel : restore_rows_f32_kernel, dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const float4*>(cache), hc, wc,
+  return launch_pdl(interp_mode == 0 ? restore_rows_f32_kernel
+                                     : (interp_mode == 1 ? restore_rows_f32_interp_kernel<4> : restore_rows_f32_interp_kernel<16>), dim3((rows + 7) / 8), dim3(256), 0, st, reinterpret_cast<const float4*>(cache), hc, wc,
                     reinterpret_cast<const float4*>(pivots), inv, h * w, k, h, w, C / 4, reinterpret_cast<float4*>(out), rows);
 }
 

@@ -32,7 +32,7 @@ def run_both(wl, granularity=0, rope_base=0.0, qk=False, interp_mode=0, kind="ii
     qk_scale = (6.0 + 8.0 * I.uniform01(wl.seed + 5, wl.L * wl.H).reshape(wl.L, wl.H)).astype(np.float32) if qk else None
     sizes = [(s, s) for s in wl.sides]
     orc = O.VarOracle(wl.L, wl.C, wl.H, sizes, cache_step=wl.cache_step, weights=oracle_weights(mt), B=wl.B, cross_len=wl.cross_len,
-                      granularity="step" if granularity else "sublayer", interp_mode="bilinear" if interp_mode else "nearest",
+                      granularity="step" if granularity else "sublayer", interp_mode=("nearest", "bilinear", "bicubic")[interp_mode],
                       rope_base=rope_base or None, qk_scale=qk_scale)
     ref, forced = [], []
     for i, x in enumerate(xs):
@@ -97,13 +97,15 @@ def test_extras_at_model_width():
     run_both(wl, rope_base=10000.0, qk=True)
 
 
+@pytest.mark.parametrize("mode", [1, 2])
 @pytest.mark.parametrize("granularity", [0, 1])
-def test_bilinear_restoration_in_the_step(granularity):
-    """interp_mode 1 through the whole step, both granularities (the per-sublayer caches and the step-level
-    fp32 cache), structured maps so that neighbouring cached rows differ."""
-    run_both(wl_small(64), granularity=granularity, interp_mode=1, kind="structured")
+def test_bilinear_restoration_in_the_step(granularity, mode):
+    """interp_mode 1 (bilinear) and 2 (bicubic) through the whole step, both granularities (the per-sublayer caches
+    and the step-level fp32 cache), structured maps so that neighbouring cached rows differ."""
+    run_both(wl_small(64), granularity=granularity, interp_mode=mode, kind="structured")
 
 
 def test_bilinear_skipped_step_and_all_options_together():
     run_both(wl_small(64, keep_last=(0.5, 0.0)), interp_mode=1, kind="structured")
     run_both(wl_small(128, cross_len=8), rope_base=100.0, qk=True, interp_mode=1)
+    run_both(wl_small(64, keep_last=(0.5, 0.0)), interp_mode=2, kind="structured")
