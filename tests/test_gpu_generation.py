@@ -20,7 +20,7 @@ T = lambda a, dt=torch.float32: torch.from_numpy(np.ascontiguousarray(a)).to(DEV
 BF = lambda bits: torch.from_numpy(bits.view("int16")).to(DEV).view(torch.bfloat16).contiguous()
 
 
-@pytest.mark.parametrize("rows,V", [(1, 4), (7, 64), (300, 4096), (5, 100), (2050, 1000)])
+@pytest.mark.parametrize("rows,V", [(1, 4), (7, 64), (300, 4096), (5, 100), (2050, 1000), (8192, 4096)])
 @pytest.mark.parametrize("with_noise", [False, True])
 def test_argmax_rows_bit_exact(rows, V, with_noise):
     """Same fp32 logits on both sides: ids are bit-exact without noise (pure comparisons, ties to the lowest
