@@ -257,7 +257,9 @@ size_t fv_gemm_splitk_workspace_bytes(void);
 /* Test / profiling hook (process-wide): which GEMM kernel fv_gemm_bf16 and the step use when no K split is
  * taken.  0 = chosen per shape (default); 1 = one CTA per 128-row tile, width chosen per shape; 2 = CTA
  * pairs sharing 256 x 256 tiles (tcgen05 cta_group::2); 3 = CTA pairs, 256 x 128 tiles; 4 / 5 / 6 = one CTA
- * per tile of width 128 / 192 / 256; 7 = one CTA per tile of width 64.  INVALID_ARG outside 0..7. */
+ * per tile of width 128 / 192 / 256; 7 = one CTA per tile of width 64; 8 / 9 = K split over a cluster of 4 / 2
+ * CTAs per 128-wide tile, 10 / 11 = the same with 64-wide tiles (partials reduced through distributed shared
+ * memory; no scratch).  INVALID_ARG outside 0..11. */
 fv_status fv_gemm_force_path(int32_t path);
 fv_status fv_gemm_bf16(const void *a_dev, const void *w_dev, const void *bias_dev, int32_t M,
                        int32_t N, int32_t K, int32_t epilogue, void *out_dev, void *aux_dev,

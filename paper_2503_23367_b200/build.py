@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libfastvar.so")
-SOURCES = ["select.cu", "rows.cu", "gemm.cu", "gemm_pair.cu", "attention.cu", "api.cu", "prof.cu", "select_static.cu", "generate.cu"]
+SOURCES = ["select.cu", "rows.cu", "gemm.cu", "gemm_pair.cu", "gemm_cluster.cu", "attention.cu", "api.cu", "prof.cu", "select_static.cu", "generate.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

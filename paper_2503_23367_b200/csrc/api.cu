@@ -220,7 +220,7 @@ fv_status fv_attention(const void* q_dev, const void* k_dev, const void* vt_dev,
 size_t fv_gemm_splitk_workspace_bytes(void) { return gemm_splitk_ws_bytes(); }
 
 fv_status fv_gemm_force_path(int32_t path) {
-  if (path < 0 || path > 7) return FV_ERR_INVALID_ARG;
+  if (path < 0 || path > 11) return FV_ERR_INVALID_ARG;
   gemm_force_path(path);
   return FV_OK;
 }

@@ -366,6 +366,7 @@ cudaError_t gemm_init() {
   if (e == cudaSuccess) e = set_attr<192, false, 2>();
   if (e == cudaSuccess) e = set_attr<256, false, 2>();
   if (e == cudaSuccess) e = gemm_pair_init();
+  if (e == cudaSuccess) e = gemm_cluster_init();
   if (e != cudaSuccess) return e;
   int dev = 0;
   e = cudaGetDevice(&dev);
@@ -500,7 +501,33 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   p.rope_table = qk_extras ? reinterpret_cast<const float2*>(g.rope_table) : nullptr;
   p.rope_idx = qk_extras ? g.rope_idx : nullptr;
   p.head_dim = g.head_dim;
+  // Few tiles against a long K (every GEMM of the small scale steps): split K over the CTAs of a cluster, the
+  // partials reduced through distributed shared memory.  Measured back to back on B200 (us, against the best
+  // of the other paths): N 2048 K 2048: 6.6 / 7.4 / 8.0 / 12.0 / 12.4 at M = 2 / 32 / 128 / 288 / 512 (9.7 /
+  // 9.7 / 12.7 / 13.7 / 14.0); N 2048 K 8192: 14.9 / 15.0 / 15.9 / 26.9 / 27.5 (14.9 / 15.9 / 20.8 / 29.5 /
+  // 35.6); N 6144 K 2048 at M <= 128: 13.2 / 11.4 / 13.8 (14.4 / 14.1 / 14.3); N 8192: 13.6 / 12.0 / 14.3
+  // (17.7 / 14.6 / 15.1).  Which of the three shapes wins follows the tile counts:
+  int cluster_slices = 0, cluster_bn = 0;
+  if (g_force_path == 0 && !qk_extras) {
+    const int num_kb = (g.K + BK - 1) / BK;
+    const long t128 = (long)tiles_m * ((g.N + 127) / 128), t64 = (long)tiles_m * ((g.N + 63) / 64);
+    if (num_kb >= 8) {
+      if (g.M > 16 && t64 * 4 <= g_num_sms) { cluster_bn = 64; cluster_slices = 4; }
+      else if (t128 * 4 <= g_num_sms) { cluster_bn = 128; cluster_slices = 4; }
+      else if (t128 * 2 <= g_num_sms) { cluster_bn = 128; cluster_slices = 2; }
+    }
+  }
+  if (g_force_path >= 8 && g_force_path <= 11 && !qk_extras) {   // 8: 128 wide x 4 slices, 9: 128 x 2, 10: 64 x 4, 11: 64 x 2
+    cluster_bn = g_force_path <= 9 ? 128 : 64;
+    cluster_slices = (g_force_path & 1) ? 2 : 4;
+  }
+  if (cluster_slices) {
+    const int num_kb = (g.K + BK - 1) / BK;
+    p.splits = 1; p.sk_partial = nullptr; p.sk_tickets = nullptr;
+    p.kb_per_split = (num_kb + cluster_slices - 1) / cluster_slices;
+  }
   LaunchScope scope(KC_GEMM, 1, 2.0 * g.M * (double)g.N * g.K, 2.0 * ((double)g.M * g.K + (double)g.N * g.K + (double)g.M * g.N), st);
+  if (cluster_slices) return launch_gemm_cluster(g, p, cluster_bn, cluster_slices, st) == cudaSuccess ? FV_OK : FV_ERR_CUDA;
   if (p.splits == 1 && tc.pair) {
     cudaError_t e2 = launch_gemm_pair(g, p, bn, st);
     return e2 == cudaSuccess ? FV_OK : FV_ERR_CUDA;

@@ -317,6 +317,11 @@ __device__ __forceinline__ void qkv_extras_tile(const GemmDev& p, uint32_t t0, i
 
 }  // namespace gemm_detail
 
+// gemm_cluster.cu: K split inside a cluster of `slices` CTAs per tile (partials reduced through distributed
+// shared memory); bn in {64, 128}, slices in {2, 4}, p.kb_per_split k-blocks per CTA.
+cudaError_t gemm_cluster_init();
+cudaError_t launch_gemm_cluster(const GemmArgs& g, const gemm_detail::GemmDev& p, int bn, int slices, cudaStream_t st);
+
 // gemm_pair.cu: the CTA-pair kernel (256 x bn tiles, bn in {128, 256}); same argument block and epilogues.
 cudaError_t gemm_pair_init();
 cudaError_t launch_gemm_pair(const GemmArgs& g, const gemm_detail::GemmDev& p, int bn, cudaStream_t st);

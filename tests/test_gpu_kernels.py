@@ -318,6 +318,33 @@ def test_gemm_bf16_width_64_tiles(M, N, K, splitk, epilogue):
     assert err <= MAX_ABS and cos >= MIN_COS, (err, cos)
 
 
+@pytest.mark.parametrize("path", [8, 9, 10, 11])
+@pytest.mark.parametrize("epilogue", [0, 1])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (7, 136, 72), (300, 1024, 4096), (32, 2048, 2048), (128, 2048, 8192), (2, 6144, 2048),
+                                   (200, 1032, 1024), (2, 2048, 8192), (130, 192, 128)])
+def test_gemm_bf16_split_inside_a_cluster(M, N, K, epilogue, path):
+    """K split over the 2 or 4 CTAs of a cluster (partials reduced through distributed shared memory), 128- and
+    64-wide tiles, forced for every shape: ragged rows and columns, fewer k-blocks than CTAs (K = 64, 72, 128: some
+    CTAs of the cluster then have nothing to add), and twice in a row with identical bits."""
+    a = I.normal_bf16(96, (M, K), 1.0 if K <= 2048 else 0.5); w = I.normal_bf16(97, (N, K), 0.02); b = I.normal_bf16(98, (N,), 0.02)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ad, wd, bd = bf16_dev(a), bf16_dev(w), bf16_dev(b)
+    assert fv.lib().fv_gemm_force_path(path) == 0
+    try:
+        out = fv.fv_gemm_bf16(ad, wd, bd, epilogue=epilogue, status=status)
+        out2 = fv.fv_gemm_bf16(ad, wd, bd, epilogue=epilogue, status=status)
+        torch.cuda.synchronize()
+    finally:
+        fv.lib().fv_gemm_force_path(0)
+    assert int(status.item()) == 0
+    assert torch.equal(out, out2)
+    ref = O.linear(I.bf16_bits_to_f32(a), I.bf16_bits_to_f32(w), I.bf16_bits_to_f32(b))
+    if epilogue == 1:
+        ref = O.gelu_tanh(ref)
+    err, cos = per_token_errors(bf16_host(out), ref)
+    assert err <= MAX_ABS and cos >= MIN_COS, (err, cos)
+
+
 def test_gemm_residual_epilogue_with_cache_copy():
     B, rows, N, K = 2, 100, 256, 512
     M = B * rows
