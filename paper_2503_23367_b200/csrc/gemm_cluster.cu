@@ -25,12 +25,18 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int kThreads = 192;
-constexpr int kATileBytes = BM * BK * 2;  // 16 KB
 
-template <int BN> struct ClusterCfg {
+// AROWS: rows of A that are actually loaded per k-block (32 when the GEMM has at most 32 rows, else 128).  The
+// MMA always reads a 128-row A tile from shared memory; with AROWS = 32 the rows beyond the 4 KB that were
+// loaded are whatever follows in shared memory (the stage's own W tile, the next stage, the buffers behind the
+// ring -- all inside the allocation).  They only feed accumulator rows >= 32, which belong to no row of the
+// output and are neither reduced nor stored.  The 12 KB saved per stage buy a deeper ring: more weight bytes
+// in flight per SM, which is what bounds these launches.
+template <int BN, int AROWS> struct ClusterCfg {
+  static constexpr int kATile = AROWS * BK * 2;
   static constexpr int kBTileBytes = BN * BK * 2;
-  static constexpr int kStageBytes = kATileBytes + kBTileBytes;
-  static constexpr int kStages = (BN == 128) ? 4 : 6;
+  static constexpr int kStageBytes = kATile + kBTileBytes;
+  static constexpr int kStages = AROWS == 32 ? ((BN == 128) ? 7 : 10) : ((BN == 128) ? 4 : 6);
   static constexpr int kTmemCols = BN;                      // one accumulator (64 or 128: powers of two)
   static constexpr int kRedPitch = BN + 4;                  // floats per row of the reduce buffer (bank spread)
   static constexpr int kRedBytes = BM * kRedPitch * 4;      // [S sources][128/S rows][pitch] = 128 rows in all
@@ -47,10 +53,11 @@ __device__ __forceinline__ void st_cluster_f4(uint32_t addr, uint32_t a, uint32_
   asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-template <int BN, int S>
+template <int BN, int S, int AROWS>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
-  using Cfg = ClusterCfg<BN>;
+  using Cfg = ClusterCfg<BN, AROWS>;
+  constexpr int kATileBytes = Cfg::kATile;
   constexpr int STAGES = Cfg::kStages;
   constexpr int ROWS_PER = BM / S;        // rows of the tile each CTA finishes
   constexpr int CHUNKS = BN / 32;         // 32-column chunks per row
@@ -203,44 +210,53 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   }
 }
 
-template <int BN, int S> cudaError_t set_attr() {
-  cudaError_t e = cudaFuncSetAttribute(gemm_cluster_kernel<BN, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, ClusterCfg<BN>::kSmemBytes);
-  return e;
+template <int BN, int S, int AROWS> cudaError_t set_attr() {
+  return cudaFuncSetAttribute(gemm_cluster_kernel<BN, S, AROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, ClusterCfg<BN, AROWS>::kSmemBytes);
 }
 
-template <int BN, int S>
+template <int BN, int S, int AROWS>
 cudaError_t launch(const GemmArgs& g, const GemmDev& p, long tiles, cudaStream_t st) {
   alignas(64) CUtensorMap tmA, tmB;
-  if (!make_tmap_bf16_2d(&tmA, g.a, g.M, g.K, BM)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16_2d(&tmA, g.a, g.M, g.K, AROWS)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16_2d(&tmB, g.w, g.N, g.K, BN)) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)(tiles * S)); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = ClusterCfg<BN>::kSmemBytes; cfg.stream = st;
+  cfg.gridDim = dim3((unsigned)(tiles * S)); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = ClusterCfg<BN, AROWS>::kSmemBytes; cfg.stream = st;
   cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   at[1].id = cudaLaunchAttributeClusterDimension;
   at[1].val.clusterDim.x = S; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<BN, S>, tmA, tmB, p);
+  return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<BN, S, AROWS>, tmA, tmB, p);
 }
 
 }  // namespace
 
 cudaError_t gemm_cluster_init() {
-  cudaError_t e = set_attr<128, 2>();
-  if (e == cudaSuccess) e = set_attr<128, 4>();
-  if (e == cudaSuccess) e = set_attr<64, 2>();
-  if (e == cudaSuccess) e = set_attr<64, 4>();
+  cudaError_t e = set_attr<128, 2, 128>();
+  if (e == cudaSuccess) e = set_attr<128, 4, 128>();
+  if (e == cudaSuccess) e = set_attr<64, 2, 128>();
+  if (e == cudaSuccess) e = set_attr<64, 4, 128>();
+  if (e == cudaSuccess) e = set_attr<128, 2, 32>();
+  if (e == cudaSuccess) e = set_attr<128, 4, 32>();
+  if (e == cudaSuccess) e = set_attr<64, 2, 32>();
+  if (e == cudaSuccess) e = set_attr<64, 4, 32>();
   return e;
 }
 
 // bn in {64, 128}, slices in {2, 4}; p.kb_per_split k-blocks per CTA.
 cudaError_t launch_gemm_cluster(const GemmArgs& g, const GemmDev& p, int bn, int slices, cudaStream_t st) {
   const long tiles = (long)((g.M + BM - 1) / BM) * ((g.N + bn - 1) / bn);
-  if (bn == 128 && slices == 2) return launch<128, 2>(g, p, tiles, st);
-  if (bn == 128 && slices == 4) return launch<128, 4>(g, p, tiles, st);
-  if (bn == 64 && slices == 2) return launch<64, 2>(g, p, tiles, st);
-  if (bn == 64 && slices == 4) return launch<64, 4>(g, p, tiles, st);
+  if (g.M <= 32) {   // at most 32 rows: short A tiles, deeper ring
+    if (bn == 128 && slices == 2) return launch<128, 2, 32>(g, p, tiles, st);
+    if (bn == 128 && slices == 4) return launch<128, 4, 32>(g, p, tiles, st);
+    if (bn == 64 && slices == 2) return launch<64, 2, 32>(g, p, tiles, st);
+    if (bn == 64 && slices == 4) return launch<64, 4, 32>(g, p, tiles, st);
+  }
+  if (bn == 128 && slices == 2) return launch<128, 2, 128>(g, p, tiles, st);
+  if (bn == 128 && slices == 4) return launch<128, 4, 128>(g, p, tiles, st);
+  if (bn == 64 && slices == 2) return launch<64, 2, 128>(g, p, tiles, st);
+  if (bn == 64 && slices == 4) return launch<64, 4, 128>(g, p, tiles, st);
   return cudaErrorInvalidValue;
 }
 
