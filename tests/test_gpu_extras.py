@@ -109,3 +109,32 @@ def test_bilinear_skipped_step_and_all_options_together():
     run_both(wl_small(64, keep_last=(0.5, 0.0)), interp_mode=1, kind="structured")
     run_both(wl_small(128, cross_len=8), rope_base=100.0, qk=True, interp_mode=1)
     run_both(wl_small(64, keep_last=(0.5, 0.0)), interp_mode=2, kind="structured")
+
+
+def test_all_options_on_non_square_maps_with_a_partial_batch():
+    """Rotary coordinates on rectangular maps (rows and columns scale by different factors towards the last map),
+    bicubic restoration, cosine attention, cross-attention, and fewer images than the context was built for."""
+    hw = [(1, 1), (2, 3), (3, 5), (5, 8), (7, 12), (10, 17)]
+    keep = [1.0, 1.0, 1.0, 1.0, 0.5, 0.3]
+    L, C, H, B_max, B = 2, 128, 2, 3, 2
+    wl = I.Workload("rect", L=L, C=C, H=H, B=B_max, sides=tuple(h for h, _ in hw), keep=tuple(keep), cross_len=8, seed=79)
+    mt = I.model_tensors(wl)
+    sharpen_attention(mt, C)
+    qk_scale = (6.0 + 8.0 * I.uniform01(5, L * H).reshape(L, H)).astype(np.float32)
+    w = dict(oracle_weights(mt)); w["mod"] = w["mod"][:, :B]; w["text"] = w["text"][:B]
+    orc = O.VarOracle(L, C, H, hw, cache_step=3, weights=w, B=B, cross_len=8, interp_mode="bicubic", rope_base=50.0, qk_scale=qk_scale)
+    cap = sum(O.kept_count(r, h, ww) if r < 1 else h * ww for r, (h, ww) in zip(keep, hw))
+    ctx = fv.FvContext(L, C, H, hw, 3, B_max, cap, mt, cross_len=8, device=DEV, rope_base=50.0, interp_mode=2, qk_scale=qk_scale)
+    names = ("attn", "xattn", "ffn")
+    for i, (h, ww) in enumerate(hw):
+        x = I.token_map(600 + i, B, h, ww, C, "structured")
+        tr = {}
+        ref = orc.var_step(x, i, keep[i], trace=tr)
+        forced = None
+        if keep[i] < 1.0:
+            forced = torch.from_numpy(np.stack([np.stack([tr[(l, s)]["idx"] for s in names]) for l in range(L)]).astype(np.int32)).to(DEV)
+        got = ctx.var_step(torch.from_numpy(x).to(DEV), i, keep[i], forced_idx=forced).cpu().numpy()
+        err, cos = per_token_errors(got, ref)
+        assert err <= MAX_ABS and cos >= MIN_COS, (i, err, cos)
+    assert ctx.device_status() == 0
+    ctx.close()
