@@ -277,9 +277,7 @@ def ours(args, wl):
         for i in range(S):
             if events is not None:
                 events[i].record()
-            xs[i].copy_(hx[i], non_blocking=True)
-            ctx.var_step(xs[i], i, wl.keep[i], out=outs[i])
-            ho[i].copy_(outs[i], non_blocking=True)
+            ctx.var_step_host(hx[i], i, wl.keep[i], ho[i])      # C ABI call with host buffers: H2D, step, D2H on the stream
         if events is not None:
             events[S].record()
 

@@ -594,4 +594,26 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   return FV_OK;
 }
 
+// fv_var_step for callers whose token maps live in host memory: copy in, step, copy out, all enqueued on `stream`.
+size_t fv_var_step_host_staging_bytes(const fv_config* cfg) {
+  if (!config_ok(cfg)) return 0;
+  return 2 * align_up((size_t)cfg->B_max * max_tokens(cfg) * cfg->C * sizeof(float), 1024);
+}
+
+fv_status fv_var_step_host(fv_ctx* ctx, const float* tokens_host, int32_t B, int32_t scale_idx, double keep_ratio, float* out_host,
+                           void* staging_dev, size_t staging_bytes, void* stream) {
+  if (!ctx || !tokens_host || !out_host || !staging_dev || B <= 0 || B > ctx->cfg.B_max) return FV_ERR_INVALID_ARG;
+  if (scale_idx < 0 || scale_idx >= ctx->cfg.n_steps || (reinterpret_cast<uintptr_t>(staging_dev) & 1023u)) return FV_ERR_INVALID_ARG;
+  if (staging_bytes < fv_var_step_host_staging_bytes(&ctx->cfg)) return FV_ERR_CAPACITY;
+  const fv_config& c = ctx->cfg;
+  const size_t bytes = (size_t)B * c.h[scale_idx] * c.w[scale_idx] * c.C * sizeof(float);
+  float* in_dev = static_cast<float*>(staging_dev);
+  float* out_dev = reinterpret_cast<float*>(static_cast<char*>(staging_dev) + fv_var_step_host_staging_bytes(&ctx->cfg) / 2);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(in_dev, tokens_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return FV_ERR_CUDA;
+  const fv_status s = fv_var_step(ctx, in_dev, B, scale_idx, keep_ratio, out_dev, nullptr, nullptr, stream);
+  if (s != FV_OK) return s;
+  return cuda_status(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, st));
+}
+
 }  // extern "C"

@@ -367,3 +367,24 @@ def test_state_and_argument_errors():
         ctx.var_step(x9, 9, 0.5)
     assert e.value.code == 3
     ctx.close()
+
+
+def test_step_with_host_buffers_equals_the_device_call():
+    """fv_var_step_host (pinned host token maps in, host result out) gives the bits of fv_var_step."""
+    wl = I.WORKLOADS["tiny"]
+    mt = I.model_tensors(wl)
+    xs = [I.step_input(wl, i) for i in range(len(wl.sides))]
+    ctx = make_ctx(wl, mt)
+    ref, _ = gpu_schedule(ctx, wl, xs)
+    ctx.reset()
+    for i, x in enumerate(xs):
+        hin = torch.from_numpy(x).pin_memory()
+        hout = torch.empty_like(hin).pin_memory()
+        ctx.var_step_host(hin, i, wl.keep[i], hout)
+        torch.cuda.synchronize()
+        assert np.array_equal(hout.numpy(), ref[i])
+    assert ctx.device_status() == 0
+    with pytest.raises(fv.FvError) as e:      # staging too small
+        fv._check(fv.lib().fv_var_step_host(ctx.ctx, hin.data_ptr(), 1, 0, 1.0, hout.data_ptr(), 1024, 16, None), "fv_var_step_host")
+    assert e.value.code == 3
+    ctx.close()
