@@ -369,6 +369,9 @@ fv_status fv_generate(fv_ctx *ctx, const fv_generator *gen, const float *start_d
  *                        milliseconds per class (0 unless timing was on), launches per class, the
  *                        algorithmic work per class (bytes for classes 0,1,4; flops for 2,3) and the bytes
  *                        each class has to move to and from HBM once (operands + results), then clears. */
+/* sizeof(fv_config), sizeof(fv_weights), sizeof(fv_generator) as this library was compiled: a binding checks
+ * its own struct definitions against them before passing any struct. */
+void fv_struct_sizes(size_t *sizes3_host);
 uint64_t fv_kernel_launches(void);
 fv_status fv_profile_enable(int32_t on);
 fv_status fv_profile_read(double *ms_host, uint64_t *launches_host, double *work_host,

@@ -26,7 +26,7 @@ EXPORTS = ["fv_status_string", "fv_k_for", "fv_prune_select_workspace_bytes", "f
            "fv_kernel_launches", "fv_profile_enable", "fv_profile_read",
            "fv_prune_select_static", "fv_prune_select_static_capacity",
            "fv_head_workspace_bytes", "fv_head_tokens", "fv_argmax_rows", "fv_residual_accumulate", "fv_next_scale_input",
-           "fv_generate_workspace_bytes", "fv_generate", "fv_var_step_host_staging_bytes", "fv_var_step_host"]
+           "fv_generate_workspace_bytes", "fv_generate", "fv_var_step_host_staging_bytes", "fv_var_step_host", "fv_struct_sizes"]
 
 
 class FvError(RuntimeError):
@@ -116,6 +116,12 @@ def lib() -> C.CDLL:
         L.fv_profile_enable.restype = C.c_int; L.fv_profile_enable.argtypes = [i32]
         L.fv_profile_read.restype = C.c_int
         L.fv_profile_read.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        L.fv_struct_sizes.restype = None; L.fv_struct_sizes.argtypes = [C.POINTER(sz)]
+        sizes = (sz * 3)()
+        L.fv_struct_sizes(sizes)
+        mine = (C.sizeof(fv_config), C.sizeof(fv_weights), C.sizeof(fv_generator))
+        if tuple(sizes) != mine:
+            raise RuntimeError(f"struct layouts of binding.py {mine} and libfastvar.so {tuple(sizes)} differ: rebuild the library")
         _lib = L
     return _lib
 

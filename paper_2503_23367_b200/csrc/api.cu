@@ -616,4 +616,9 @@ fv_status fv_var_step_host(fv_ctx* ctx, const float* tokens_host, int32_t B, int
   return cuda_status(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, st));
 }
 
+void fv_struct_sizes(size_t* sizes3_host) {
+  if (!sizes3_host) return;
+  sizes3_host[0] = sizeof(fv_config); sizes3_host[1] = sizeof(fv_weights); sizes3_host[2] = sizeof(fv_generator);
+}
+
 }  // extern "C"

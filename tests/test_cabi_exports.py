@@ -57,3 +57,10 @@ def test_argument_validation_happens_before_any_launch(lib):
     assert lib.fv_workspace_bytes(ctypes.byref(cfg)) > 64 * 256 * 2 * 4
     assert lib.fv_kv_bytes(ctypes.byref(cfg)) == 2 * 2 * 80 * 256 * 2
     assert lib.fv_cache_bytes(ctypes.byref(cfg)) == 16 * 256 * 4 + 2 * 2 * 16 * 256 * 2   # fp32 output map + sublayer caches
+
+
+def test_struct_layouts_match_the_library(lib):
+    import ctypes as C
+    sizes = (C.c_size_t * 3)()
+    lib.fv_struct_sizes(sizes)
+    assert tuple(sizes) == (C.sizeof(fv.fv_config), C.sizeof(fv.fv_weights), C.sizeof(fv.fv_generator))
