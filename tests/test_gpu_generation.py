@@ -200,3 +200,29 @@ def test_fv_generate_equals_its_stages_and_follows_the_oracle(keep):
     if compared == len(recs):
         np.testing.assert_allclose(r_a.cpu().numpy(), recs[-1]["r"], rtol=0, atol=1e-5)
     ctx.close()
+
+
+def test_head_tokens_at_the_last_scale_of_the_bench_workload_sampled_rows():
+    """The head at full size (B = 2, 64x64 tokens, C = 2048, V = 4096: the launch configuration the bench times);
+    the oracle computes a sample of rows (rows are independent), every sampled logit and id is checked."""
+    B, n, C, V = 2, 4096, 2048, 4096
+    y = I.normal(61, (B, n, C), 1.5) + 0.3
+    wl = I.Workload("h", L=1, C=C, H=16, B=B, sides=(1,), keep=(1.0,), cross_len=0, seed=19)
+    # head weights at the blocks' scale (std 0.02): |logits| stays below ~7, where one bf16 rounding of the
+    # normalised activations keeps a K = 2048 dot product inside the 3e-2 bar
+    gt = I.generation_tensors(wl, V=V, d=32, w_std=0.005)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ids, logits = fv.fv_head_tokens(T(y), T(gt.mod_head), BF(gt.w_head), BF(gt.b_head), want_logits=True, status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    ids = ids.cpu().numpy(); lg = logits.cpu().numpy().reshape(B, n, V)
+    rows = np.unique((I.uniform01(62, 96) * n).astype(np.int64))
+    rows = np.concatenate([rows, [0, 127, 128, n - 1]])             # tile edges of the GEMM too
+    wh, bh = I.bf16_bits_to_f32(gt.w_head), I.bf16_bits_to_f32(gt.b_head)
+    ref = G.head_logits(y[:, rows], gt.mod_head[:, 0], gt.mod_head[:, 1], wh, bh)
+    assert np.abs(lg[:, rows] - ref).max() <= LOGIT_TOL
+    ref_ids, margin = G.choose_tokens(ref)
+    clear = margin > 2 * LOGIT_TOL
+    np.testing.assert_array_equal(ids[:, rows][clear], ref_ids[clear])
+    # every id (all 8192 rows) is the exact argmax of the GPU's own fp32 logits
+    np.testing.assert_array_equal(ids, lg.argmax(-1))
