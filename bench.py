@@ -277,7 +277,8 @@ def ours(args, wl):
         for i in range(S):
             if events is not None:
                 events[i].record()
-            ctx.var_step_host(hx[i], i, wl.keep[i], ho[i])      # C ABI call with host buffers: H2D, step, D2H on the stream
+            ctx.var_step_host(hx[i], i, wl.keep[i], ho[i])      # C ABI call with host buffers: H2D, step, D2H
+        ctx.host_io_flush()                                     # the last results have landed before the region ends
         if events is not None:
             events[S].record()
 

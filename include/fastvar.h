@@ -219,15 +219,21 @@ fv_status fv_var_step(fv_ctx *ctx, const float *tokens_dev, int32_t B, int32_t s
                       double keep_ratio, float *out_dev, const int32_t *forced_idx_dev,
                       int32_t *idx_trace_dev, void *stream);
 
-/* fv_var_step with the token maps in HOST memory (pinned memory makes the copies asynchronous): enqueues on
- * `stream` the copy of tokens_host [B, h*w, C] fp32 to the device, the step, and the copy of its result to
- * out_host [B, h*w, C].  Nothing is synchronised: out_host is valid once the stream has run.
- *   staging_dev: device scratch of fv_var_step_host_staging_bytes(cfg) bytes, 1024-byte aligned (the step's
- *   input and output maps at their largest).  No forced indices / trace.  Errors: those of fv_var_step, CAPACITY. */
+/* fv_var_step with the token maps in HOST memory (pinned memory makes the copies asynchronous).  Enqueues the
+ * copy of tokens_host [B, h*w, C] fp32 to the device, the step (on `stream`), and the copy of its result to
+ * out_host [B, h*w, C].  The copies run on two streams owned by the context, ordered against `stream` by events
+ * over two staging buffers per direction, so the input of the next call and the result of the previous one
+ * travel while a step computes.  tokens_host must hold its data when the call is made (the copy does not wait
+ * for earlier work of `stream`).  out_host is valid after fv_host_io_flush(ctx, stream) and the completion of
+ * `stream`.
+ *   staging_dev: device scratch of fv_var_step_host_staging_bytes(cfg) bytes, 1024-byte aligned (two input and
+ *   two output maps at their largest).  No forced indices / trace.  Errors: those of fv_var_step, CAPACITY.
+ * fv_host_io_flush makes `stream` wait for every result copy enqueued so far. */
 size_t fv_var_step_host_staging_bytes(const fv_config *cfg);
 fv_status fv_var_step_host(fv_ctx *ctx, const float *tokens_host, int32_t B, int32_t scale_idx,
                            double keep_ratio, float *out_host, void *staging_dev, size_t staging_bytes,
                            void *stream);
+fv_status fv_host_io_flush(fv_ctx *ctx, void *stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Building blocks of the step, exported for kernel-level parity tests and profiling.            */

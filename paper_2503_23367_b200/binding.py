@@ -26,7 +26,7 @@ EXPORTS = ["fv_status_string", "fv_k_for", "fv_prune_select_workspace_bytes", "f
            "fv_kernel_launches", "fv_profile_enable", "fv_profile_read",
            "fv_prune_select_static", "fv_prune_select_static_capacity",
            "fv_head_workspace_bytes", "fv_head_tokens", "fv_argmax_rows", "fv_residual_accumulate", "fv_next_scale_input",
-           "fv_generate_workspace_bytes", "fv_generate", "fv_var_step_host_staging_bytes", "fv_var_step_host", "fv_struct_sizes"]
+           "fv_generate_workspace_bytes", "fv_generate", "fv_var_step_host_staging_bytes", "fv_var_step_host", "fv_host_io_flush", "fv_struct_sizes"]
 
 
 class FvError(RuntimeError):
@@ -112,6 +112,7 @@ def lib() -> C.CDLL:
         L.fv_generate.argtypes = [vp, C.POINTER(fv_generator), vp, i32, C.POINTER(dbl), C.POINTER(vp), vp, vp, vp, sz, vp]
         L.fv_var_step_host_staging_bytes.restype = sz; L.fv_var_step_host_staging_bytes.argtypes = [C.POINTER(fv_config)]
         L.fv_var_step_host.restype = C.c_int; L.fv_var_step_host.argtypes = [vp, vp, i32, i32, dbl, vp, vp, sz, vp]
+        L.fv_host_io_flush.restype = C.c_int; L.fv_host_io_flush.argtypes = [vp, vp]
         L.fv_kernel_launches.restype = C.c_uint64; L.fv_kernel_launches.argtypes = []
         L.fv_profile_enable.restype = C.c_int; L.fv_profile_enable.argtypes = [i32]
         L.fv_profile_read.restype = C.c_int
@@ -456,7 +457,8 @@ class FvContext:
         return self.cache[off: off + 2 * nel].view(torch.bfloat16).view(B, hc * wc, self.C)
 
     def var_step_host(self, tokens_host: torch.Tensor, scale_idx: int, keep_ratio: float, out_host: torch.Tensor) -> torch.Tensor:
-        """fv_var_step_host: token maps in (pinned) host memory; copies and step are enqueued on the current stream."""
+        """fv_var_step_host: token maps in (pinned) host memory; the step runs on the current stream, the copies on the
+        context's own streams.  Call host_io_flush() and synchronise before reading out_host."""
         assert not tokens_host.is_cuda and not out_host.is_cuda and tokens_host.dtype == torch.float32
         assert tokens_host.is_contiguous() and out_host.is_contiguous()
         if getattr(self, "_staging", None) is None:
@@ -467,6 +469,9 @@ class FvContext:
         _check(lib().fv_var_step_host(self.ctx, tokens_host.data_ptr(), tokens_host.shape[0], scale_idx, float(keep_ratio),
                                       out_host.data_ptr(), sp, self._staging_bytes, _stream()), "fv_var_step_host")
         return out_host
+
+    def host_io_flush(self) -> None:
+        _check(lib().fv_host_io_flush(self.ctx, _stream()), "fv_host_io_flush")
 
     def var_step(self, tokens: torch.Tensor, scale_idx: int, keep_ratio: float, out: Optional[torch.Tensor] = None,
                  forced_idx: Optional[torch.Tensor] = None, idx_trace: Optional[torch.Tensor] = None) -> torch.Tensor:

@@ -35,6 +35,11 @@ struct fv_ctx {
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   float* step_cache = nullptr;  // fp32 output map of the caching step [B_max, n_cache, C] (skipped steps; granularity 1)
   float* xc = nullptr;  // granularity 1: compact fp32 residual stream of a pruned step [B*k, C]
+  // fv_var_step_host: copy streams and the events that order two staging buffers per direction
+  cudaStream_t io_in = nullptr, io_out = nullptr;
+  cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_used[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr}, ev_copied[2] = {nullptr, nullptr};
+  bool used_rec[2] = {false, false}, copied_rec[2] = {false, false};
+  unsigned io_count = 0;
   const float* qk_scale = nullptr;      // [L, H] or null
   std::vector<float*> rope_tab;         // per scale step: (cos, sin) table [h*w][hd/2][2], empty = no rotary positions
   size_t kv_block_bytes = 0, k_bytes = 0, text_k_bytes = 0, text_block_bytes = 0, cache_sub_bytes = 0;
@@ -335,6 +340,11 @@ void fv_destroy(fv_ctx* ctx) {
   if (ctx->side) { cudaStreamSynchronize(ctx->side); cudaStreamDestroy(ctx->side); }
   if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
   if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+  if (ctx->io_in) { cudaStreamSynchronize(ctx->io_in); cudaStreamDestroy(ctx->io_in); }
+  if (ctx->io_out) { cudaStreamSynchronize(ctx->io_out); cudaStreamDestroy(ctx->io_out); }
+  for (int i = 0; i < 2; ++i)
+    for (cudaEvent_t e : {ctx->ev_in[i], ctx->ev_used[i], ctx->ev_out[i], ctx->ev_copied[i]})
+      if (e) cudaEventDestroy(e);
   delete ctx;
 }
 
@@ -594,10 +604,12 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   return FV_OK;
 }
 
-// fv_var_step for callers whose token maps live in host memory: copy in, step, copy out, all enqueued on `stream`.
+// fv_var_step for callers whose token maps live in host memory.  The copies run on two streams of the context
+// (one per direction) over two staging buffers per direction, ordered against the caller's stream by events:
+// the input of call i+1 travels while call i computes, and the result of call i travels while call i+1 computes.
 size_t fv_var_step_host_staging_bytes(const fv_config* cfg) {
   if (!config_ok(cfg)) return 0;
-  return 2 * align_up((size_t)cfg->B_max * max_tokens(cfg) * cfg->C * sizeof(float), 1024);
+  return 4 * align_up((size_t)cfg->B_max * max_tokens(cfg) * cfg->C * sizeof(float), 1024);
 }
 
 fv_status fv_var_step_host(fv_ctx* ctx, const float* tokens_host, int32_t B, int32_t scale_idx, double keep_ratio, float* out_host,
@@ -605,15 +617,47 @@ fv_status fv_var_step_host(fv_ctx* ctx, const float* tokens_host, int32_t B, int
   if (!ctx || !tokens_host || !out_host || !staging_dev || B <= 0 || B > ctx->cfg.B_max) return FV_ERR_INVALID_ARG;
   if (scale_idx < 0 || scale_idx >= ctx->cfg.n_steps || (reinterpret_cast<uintptr_t>(staging_dev) & 1023u)) return FV_ERR_INVALID_ARG;
   if (staging_bytes < fv_var_step_host_staging_bytes(&ctx->cfg)) return FV_ERR_CAPACITY;
+  if (!ctx->io_in) {
+    bool ok = cudaStreamCreateWithFlags(&ctx->io_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&ctx->io_out, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i)
+      for (cudaEvent_t* e : {&ctx->ev_in[i], &ctx->ev_used[i], &ctx->ev_out[i], &ctx->ev_copied[i]})
+        ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return FV_ERR_CUDA;
+  }
   const fv_config& c = ctx->cfg;
+  const size_t half = fv_var_step_host_staging_bytes(&c) / 4;
   const size_t bytes = (size_t)B * c.h[scale_idx] * c.w[scale_idx] * c.C * sizeof(float);
-  float* in_dev = static_cast<float*>(staging_dev);
-  float* out_dev = reinterpret_cast<float*>(static_cast<char*>(staging_dev) + fv_var_step_host_staging_bytes(&ctx->cfg) / 2);
+  const int p = (int)(ctx->io_count & 1u);
+  float* in_dev = reinterpret_cast<float*>(static_cast<char*>(staging_dev) + (size_t)p * half);
+  float* out_dev = reinterpret_cast<float*>(static_cast<char*>(staging_dev) + (size_t)(2 + p) * half);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (cudaMemcpyAsync(in_dev, tokens_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return FV_ERR_CUDA;
+  // in: this buffer's previous reader (the step two calls ago) must be done
+  if (ctx->used_rec[p] && cudaStreamWaitEvent(ctx->io_in, ctx->ev_used[p], 0) != cudaSuccess) return FV_ERR_CUDA;
+  if (cudaMemcpyAsync(in_dev, tokens_host, bytes, cudaMemcpyHostToDevice, ctx->io_in) != cudaSuccess ||
+      cudaEventRecord(ctx->ev_in[p], ctx->io_in) != cudaSuccess || cudaStreamWaitEvent(st, ctx->ev_in[p], 0) != cudaSuccess)
+    return FV_ERR_CUDA;
+  // out: this buffer's previous copy to the host must be done before the step overwrites it
+  if (ctx->copied_rec[p] && cudaStreamWaitEvent(st, ctx->ev_copied[p], 0) != cudaSuccess) return FV_ERR_CUDA;
   const fv_status s = fv_var_step(ctx, in_dev, B, scale_idx, keep_ratio, out_dev, nullptr, nullptr, stream);
   if (s != FV_OK) return s;
-  return cuda_status(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, st));
+  if (cudaEventRecord(ctx->ev_used[p], st) != cudaSuccess || cudaEventRecord(ctx->ev_out[p], st) != cudaSuccess) return FV_ERR_CUDA;
+  ctx->used_rec[p] = true;
+  if (cudaStreamWaitEvent(ctx->io_out, ctx->ev_out[p], 0) != cudaSuccess ||
+      cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, ctx->io_out) != cudaSuccess ||
+      cudaEventRecord(ctx->ev_copied[p], ctx->io_out) != cudaSuccess)
+    return FV_ERR_CUDA;
+  ctx->copied_rec[p] = true;
+  ctx->io_count += 1;
+  return FV_OK;
+}
+
+// Makes `stream` wait for every result copy fv_var_step_host has enqueued: once the stream has run, they have landed.
+fv_status fv_host_io_flush(fv_ctx* ctx, void* stream) {
+  if (!ctx) return FV_ERR_INVALID_ARG;
+  for (int p = 0; p < 2; ++p)
+    if (ctx->copied_rec[p] && cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), ctx->ev_copied[p], 0) != cudaSuccess) return FV_ERR_CUDA;
+  return FV_OK;
 }
 
 void fv_struct_sizes(size_t* sizes3_host) {

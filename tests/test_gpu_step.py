@@ -377,12 +377,19 @@ def test_step_with_host_buffers_equals_the_device_call():
     ctx = make_ctx(wl, mt)
     ref, _ = gpu_schedule(ctx, wl, xs)
     ctx.reset()
-    for i, x in enumerate(xs):
-        hin = torch.from_numpy(x).pin_memory()
-        hout = torch.empty_like(hin).pin_memory()
-        ctx.var_step_host(hin, i, wl.keep[i], hout)
+    hins = [torch.from_numpy(x).pin_memory() for x in xs]
+    houts = [torch.empty_like(h).pin_memory() for h in hins]
+    for rep in range(2):          # all steps enqueued back to back: copies and steps overlap across calls
+        ctx.reset()
+        for h in houts:
+            h.zero_()
+        for i in range(len(xs)):
+            ctx.var_step_host(hins[i], i, wl.keep[i], houts[i])
+        ctx.host_io_flush()
         torch.cuda.synchronize()
-        assert np.array_equal(hout.numpy(), ref[i])
+        for i in range(len(xs)):
+            assert np.array_equal(houts[i].numpy(), ref[i]), (rep, i)
+    hin, hout = hins[0], houts[0]
     assert ctx.device_status() == 0
     with pytest.raises(fv.FvError) as e:      # staging too small
         fv._check(fv.lib().fv_var_step_host(ctx.ctx, hin.data_ptr(), 1, 0, 1.0, hout.data_ptr(), 1024, 16, None), "fv_var_step_host")
