@@ -74,8 +74,8 @@ fv_status fv_prune_select(const float *x_dev, int32_t B, int32_t h, int32_t w, i
  *   - Inputs and outputs are still the caller's; arguments as in fv_prune_select, minus the workspace.
  *   - It allocates nothing: no cudaMalloc / cudaFree, no allocating library routine.  Shapes whose
  *     scratch need, fv_prune_select_workspace_bytes(B, h*w, C), exceeds the capacity are refused with
- *     FV_ERR_CAPACITY (e.g. B = 2, 64x64 tokens, C = 2048 needs 2.2 MiB; B = 1, 128x128, C = 2048 needs
- *     4.1 MiB; B = 4 at 128x128, C = 2048 does not fit).
+ *     FV_ERR_CAPACITY (e.g. B = 2, 64x64 tokens, C = 2048 needs 2.3 MiB; B = 1, 128x128, C = 2048 needs
+ *     4.2 MiB; B = 4 at 128x128, C = 2048 does not fit).
  *   - The first call on each device looks up the array's device address (with that device current);
  *     make that first call outside any stream capture.
  *   - All calls on a device share the one array and it keeps the previous call's contents; every

@@ -45,7 +45,7 @@ struct LaunchScope {
 
 // ---- select.cu : Pivotal Token Selection (Eq. 4-5, Algorithm 1) ---------------------------------
 constexpr int kColsumRows = 32;        // token rows folded into one chunk partial of the column sums
-constexpr int kMaxGroups = 8;          // chunk partials are folded again into at most this many group partials
+constexpr int kMaxGroups = 16;         // chunk partials are folded again into at most this many group partials
 constexpr int kTopkMaxTokens = 49152;  // scores of one image must fit the top-k CTA's shared memory
 // Scratch of the selection, carved out of one caller buffer.  Column sums of the token map are kept at
 // two levels: one partial per chunk of kColsumRows tokens, folded (by the last CTA of each group to

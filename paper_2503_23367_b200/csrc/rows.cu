@@ -12,6 +12,7 @@
 
 #include "colsum_fold.cuh"
 #include "internal.h"
+#include "sm100.cuh"
 
 namespace fv {
 
@@ -284,6 +285,103 @@ __global__ void __launch_bounds__(256) restore_rows_f32_kernel(const float4* __r
 }
 
 
+// The kept rows of a restoration (part 2) with the group fold of the column sums done inside a thread-block
+// cluster: the chunks of one group are the CTAs of one cluster, every CTA sends its chunk sums to the CTA that
+// owns the channel slice (distributed shared memory), and after one cluster barrier every CTA adds the chunks of
+// its slice in chunk order and writes the group partial.  Same values and the same order of additions as the
+// fold through global memory (chunk partial -> ticket -> last arriver), without its chain of round trips.
+// grid (group * ngroups, B), cluster (group, 1, 1), 256 threads; C8 <= 256.
+constexpr int kFoldEntries = 256 + 16;   // group * ceil(C8 / group) <= C8 + group
+__global__ void __launch_bounds__(256) restore_kept_cluster_kernel(float4* __restrict__ x, const uint4* __restrict__ y,
+                                                                   const int32_t* __restrict__ inv, const float* __restrict__ gamma,
+                                                                   int mod_stride, int n, int k, int C8, int nchunks, int group, int ngroups,
+                                                                   const float4* __restrict__ chunk_partial, float4* __restrict__ group_partial) {
+  __shared__ const uint4* s_src[kColsumRows];
+  __shared__ int s_on[kColsumRows];
+  __shared__ __align__(16) float s_fold[kFoldEntries * 8];   // [chunk of the group][channel group of this CTA's slice][8]
+  pdl_trigger();
+  pdl_wait();
+  const int b = blockIdx.y;
+  const int rank = (int)cluster_ctarank();
+  const int g = blockIdx.x / group;
+  const int chunk = blockIdx.x;                     // = g * group + rank
+  const bool valid = chunk < nchunks;
+  const int members = min(group, nchunks - g * group);
+  const int slice = (C8 + group - 1) / group;       // channel groups (of 8) per owner
+  const int t0 = chunk * kColsumRows;
+  const int rows = valid ? min(kColsumRows, n - t0) : 0;
+  if ((int)threadIdx.x < rows) {
+    const int j = __ldg(inv + (size_t)b * n + t0 + threadIdx.x);
+    s_src[threadIdx.x] = y + ((size_t)b * k + max(j, 0)) * C8;
+    s_on[threadIdx.x] = j >= 0;
+  }
+  __syncthreads();
+  const int c8 = threadIdx.x;
+  if (valid && c8 < C8) {
+    float4 g0 = make_float4(1.f, 1.f, 1.f, 1.f), g1 = g0;
+    if (gamma) {
+      const float4* gp = reinterpret_cast<const float4*>(gamma + (size_t)b * mod_stride);
+      g0 = __ldg(gp + 2 * c8); g1 = __ldg(gp + 2 * c8 + 1);
+    }
+    // continue the sums of the rows the first part updated
+    const float4* cp = chunk_partial + ((size_t)b * nchunks + chunk) * C8 * 2 + 2 * c8;
+    float4 a0 = __ldcg(cp), a1 = __ldcg(cp + 1);
+    float4* xbase = x + ((size_t)b * n + t0) * C8 * 2;
+    for (int r = 0; r < rows; r += 4) {
+      uint4 p[4];
+      float4 x0[4], x1[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (r + i < rows && s_on[r + i]) {
+          float4* xr = xbase + (size_t)(r + i) * C8 * 2 + 2 * c8;
+          x0[i] = xr[0]; x1[i] = xr[1];
+          p[i] = __ldg(s_src[r + i] + c8);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (r + i < rows && s_on[r + i]) {
+          float f[8];
+          bf16x8_to_float(p[i], f);
+          float4 u0 = x0[i], u1 = x1[i];
+          if (gamma) {
+            u0.x = fmaf(g0.x, f[0], u0.x); u0.y = fmaf(g0.y, f[1], u0.y); u0.z = fmaf(g0.z, f[2], u0.z); u0.w = fmaf(g0.w, f[3], u0.w);
+            u1.x = fmaf(g1.x, f[4], u1.x); u1.y = fmaf(g1.y, f[5], u1.y); u1.z = fmaf(g1.z, f[6], u1.z); u1.w = fmaf(g1.w, f[7], u1.w);
+          } else {
+            u0.x += f[0]; u0.y += f[1]; u0.z += f[2]; u0.w += f[3];
+            u1.x += f[4]; u1.y += f[5]; u1.z += f[6]; u1.w += f[7];
+          }
+          float4* xr = xbase + (size_t)(r + i) * C8 * 2 + 2 * c8;
+          xr[0] = u0; xr[1] = u1;
+          a0.x += u0.x; a0.y += u0.y; a0.z += u0.z; a0.w += u0.w;
+          a1.x += u1.x; a1.y += u1.y; a1.z += u1.z; a1.w += u1.w;
+        }
+      }
+    }
+    // the chunk's sums of this thread's 8 channels go to the CTA that owns the channel slice
+    const int owner = c8 / slice, local = c8 - owner * slice;
+    uint32_t dst;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(smem_u32(s_fold + ((size_t)rank * slice + local) * 8)), "r"(owner));
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(a0.x), "f"(a0.y), "f"(a0.z), "f"(a0.w) : "memory");
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + 16), "f"(a1.x), "f"(a1.y), "f"(a1.z), "f"(a1.w) : "memory");
+  }
+  cluster_sync_all();
+  // this CTA's slice of the group partial: the group's chunks in chunk order
+  const int lc = threadIdx.x;
+  const int my_c8 = rank * slice + lc;
+  if (lc < slice && my_c8 < C8) {
+    float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
+    for (int m = 0; m < members; ++m) {
+      const float4* e = reinterpret_cast<const float4*>(s_fold + ((size_t)m * slice + lc) * 8);
+      const float4 v0 = e[0], v1 = e[1];
+      s0.x += v0.x; s0.y += v0.y; s0.z += v0.z; s0.w += v0.w;
+      s1.x += v1.x; s1.y += v1.y; s1.z += v1.z; s1.w += v1.w;
+    }
+    float4* gp = group_partial + ((size_t)b * ngroups + g) * C8 * 2 + 2 * my_c8;
+    gp[0] = s0; gp[1] = s1;
+  }
+}
+
 // restore_residual_kernel with bilinear (TAPS 4) or bicubic (TAPS 16) interpolation of the cache: an unkept
 // token blends TAPS cached rows (fp32), a kept token takes its forwarded row.  Same CTA shape, row ownership
 // and column-sum handling; fewer rows in flight (two, or one with sixteen source rows).  part 2 (kept rows only) never interpolates and
@@ -471,6 +569,29 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
   const double rows_x = part == 0 ? (double)n : (part == 1 ? (double)(n - k) : (double)k);
   const double rr_bytes = (double)B * C * (8.0 * rows_x + (part != 1 ? 2.0 * k : 0.0) + (part != 2 ? 2.0 * hc * wc : 0.0));
   LaunchScope scope(KC_RESTORE, 1, rr_bytes, rr_bytes, st);
+  // kept rows + group fold inside clusters (one cluster per group of chunks) where the group fits a cluster
+  static bool cluster_fold_ok = true;
+  if (part == 2 && colsum_ws && cluster_fold_ok && ws.group >= 1 && ws.group <= 8 && C / 8 <= 256) {
+    static bool attr_set = false;
+    if (!attr_set) {
+      cluster_fold_ok = cudaFuncSetAttribute(restore_kept_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+      attr_set = true;
+    }
+    if (cluster_fold_ok) {
+      cudaLaunchConfig_t cfg{};
+      cfg.gridDim = dim3(ws.group * ws.ngroups, B); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = ws.group; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      cfg.attrs = at; cfg.numAttrs = 1;
+      const cudaError_t e = cudaLaunchKernelEx(&cfg, restore_kept_cluster_kernel, reinterpret_cast<float4*>(x), reinterpret_cast<const uint4*>(y),
+                                               inv, gamma, mod_stride, n, k, C / 8, nchunks, ws.group, ws.ngroups,
+                                               reinterpret_cast<const float4*>(ws.chunk_partial), reinterpret_cast<float4*>(ws.group_partial));
+      if (e == cudaSuccess) return e;
+      (void)cudaGetLastError();      // this cluster size cannot be scheduled here: the fold through global memory from now on
+      cluster_fold_ok = false;
+    }
+  }
   auto* kern = (interp_mode == 0 || part == 2) ? restore_residual_kernel
                : (interp_mode == 1 ? restore_residual_interp_kernel<4> : restore_residual_interp_kernel<16>);
   if (part == 0)
