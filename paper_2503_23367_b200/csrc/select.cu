@@ -223,17 +223,18 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float
   // Ordered compaction: thread t owns the contiguous tokens [t*per, (t+1)*per).
   const int per = (n + kTopkThreads - 1) / kTopkThreads;
   const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
-  uint32_t eq = 0;
-  for (int i = i0; i < i1; ++i) eq += (s_keys[KI(i)] == tau);
-  uint32_t tot;
-  uint32_t eq_before = block_exclusive_scan(eq, s_warp, &tot);
-  uint32_t kept = 0, e = eq_before;
+  // one scan for both counts a thread needs: keys above the threshold (low half) and keys equal to it (high
+  // half) among the tokens before its own; n <= 49152 keeps either total below 2^16
+  uint32_t cnt = 0;
   for (int i = i0; i < i1; ++i) {
-    uint32_t key = s_keys[KI(i)];
-    if (key > tau) ++kept;
-    else if (key == tau) { kept += (e < need_eq); ++e; }
+    const uint32_t key = s_keys[KI(i)];
+    cnt += (key > tau) + ((uint32_t)(key == tau) << 16);
   }
-  uint32_t pos = block_exclusive_scan(kept, s_warp, &tot);
+  uint32_t tot;
+  const uint32_t before = block_exclusive_scan(cnt, s_warp, &tot);
+  const uint32_t eq_before = before >> 16;
+  uint32_t pos = (before & 0xFFFFu) + min(eq_before, need_eq);   // kept tokens before this thread's first
+  uint32_t e;
   e = eq_before;
   const float tau_f = __uint_as_float(tau + kmin);
   const float band = 1e-5f * tau_f;
