@@ -1,7 +1,7 @@
 // Pivotal Token Selection (Sec. 3.3, Eq. 4-5, Algorithm 1 first routine) on sm_100a.
 //
 //   colsum_chunk_kernel : Eq. 4's sum over tokens, one partial per chunk of 32 tokens, folded into at most
-//                         8 group partials per image by the last CTA of each group (fixed order).  Skipped
+//                         16 group partials per image by the last CTA of each group (fixed order).  Skipped
 //                         when the previous restore kernel has already left the partials of its output.
 //   score_topk_kernel   : s[b,t] = sum_c (x[b,t,c] - mean[b,c])^2, one warp per token, the mean token
 //                         rebuilt from the group partials in shared memory; the last CTA of each image to
