@@ -109,8 +109,15 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
+ORACLE_MAX_REPS, ORACLE_MAX_WARMUP = 2, 1    # the one-block sample takes seconds to tens of seconds per run
+
+
 def time_oracle(wl, reps: int, warmup: int):
+    """Times the oracle's sample `reps` times after `warmup` untimed runs (both capped: the oracle is slow by
+    design and the whole leg has to stay within minutes).  `value` extrapolates the one-block time to the
+    workload's depth; `sample_seconds` is what one run of the sample really took."""
     run, tokens, desc = oracle_sample(wl)
+    reps, warmup = max(1, min(reps, ORACLE_MAX_REPS)), max(0, min(warmup, ORACLE_MAX_WARMUP))
     for _ in range(warmup):
         run()
     ts = []
@@ -118,18 +125,30 @@ def time_oracle(wl, reps: int, warmup: int):
         t0 = time.perf_counter(); run(); ts.append(time.perf_counter() - t0)
     t = statistics.mean(ts)
     return {"value": tokens / (t * wl.L), "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": desc,
-            "sample_seconds": t}
+            "sample_seconds": t, "runs": reps, "warmup_runs": warmup}
+
+
+def config_of(wl: I.Workload, world: int) -> dict:
+    """The `config` object of the JSON line, spelled the same way by both arms."""
+    return {"workload": wl.name, "B_per_gpu": wl.B, "L": wl.L, "C": wl.C, "H": wl.H, "cross_len": wl.cross_len,
+            "sides": list(wl.sides), "keep": list(wl.keep), "parallelism": f"replicas x{world} (images sharded, no collective)",
+            "cache_hygiene": "inputs larger than L2 (weights + KV + token maps of one pass >> 126 MB)",
+            "step": "one full scale schedule for one batch"}
 
 
 def reference_arm(args, wl):
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    cb = time_oracle(wl, max(1, args.steps), max(0, args.warmup))
-    ms_step = cb["sample_seconds"] * wl.L * 1e3
+    cb = time_oracle(wl, args.steps, args.warmup)
+    # one "step" of this arm = one run of the bounded sample (one transformer block of every pruned scale step);
+    # ms_per_step is the time such a run really took, the extrapolation to full depth is a key of its own
     line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "B": wl.B, "note": "CPU oracle, pruned scale steps only, depth-extrapolated"},
+            "steps": cb["runs"], "warmup": cb["warmup_runs"], "steps_requested": args.steps, "warmup_requested": args.warmup,
+            "repetition_cap": f"at most {ORACLE_MAX_REPS} timed and {ORACLE_MAX_WARMUP} warm-up runs of the sample",
+            "ms_per_step": cb["sample_seconds"] * 1e3, "ms_per_step_extrapolated_to_full_depth": cb["sample_seconds"] * wl.L * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_of(wl, args.gpus),
+            "note": "CPU oracle (numpy fp64), pruned scale steps only, one block timed and extrapolated to the workload's depth",
             "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
             "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -456,6 +475,53 @@ def ours(args, wl):
                     "speedup_pruned_steps": u_pruned / pruned_ms}
         ctx_full.close()
 
+    # ---- the 1024-pixel configuration beside it (13 scales up to 64x64, batch 2, keep 0.6 / 0.4 / 0.2): the same
+    # device-resident timing, no other legs
+    other = None
+    if not args.skip_other and wl.name == "infinity_2b_2k":
+        wl2 = I.WORKLOADS["infinity_2b_1k"]
+        if args.blocks > 0:
+            wl2 = wl2.with_depth(args.blocks)
+        del gt
+        torch.cuda.empty_cache()
+        gt2 = GpuTensors(wl2, dev, seed=wl2.seed)
+        S2 = len(wl2.sides)
+        pruned2 = [i for i in range(S2) if wl2.keep[i] < 1.0]
+        ctx2 = fv.FvContext(wl2.L, wl2.C, wl2.H, [(s_, s_) for s_ in wl2.sides], wl2.cache_step, wl2.B, sum(kept(wl2, i) for i in range(S2)),
+                            gt2, cross_len=wl2.cross_len, mlp_ratio=wl2.mlp_ratio, device=dev)
+        g2 = torch.Generator(device=dev); g2.manual_seed(R.rank_seed(wl2.seed + 77, rank))
+        xs2 = [torch.randn(wl2.B, wl2.tokens(i), wl2.C, generator=g2, device=dev, dtype=torch.float32) for i in range(S2)]
+        outs2 = [torch.empty_like(x) for x in xs2]
+
+        def schedule2(events=None):
+            ctx2.reset()
+            for i in range(S2):
+                if events is not None:
+                    events[i].record()
+                ctx2.var_step(xs2[i], i, wl2.keep[i], out=outs2[i])
+            if events is not None:
+                events[S2].record()
+
+        for _ in range(3):
+            schedule2()
+        barrier()
+        n2 = max(2, min(args.steps, 5))
+        ev2b = [[torch.cuda.Event(enable_timing=True) for _ in range(S2 + 1)] for _ in range(n2)]
+        for k in range(n2):
+            schedule2(ev2b[k])
+        barrier()
+        if ctx2.device_status() != 0:
+            raise SystemExit("a kernel reported an expired wait")
+        o_total = max_over_ranks(statistics.mean(ev2b[k][0].elapsed_time(ev2b[k][S2]) for k in range(n2)))
+        o_pruned = max_over_ranks(sum(statistics.mean(ev2b[k][i].elapsed_time(ev2b[k][i + 1]) for k in range(n2)) for i in pruned2))
+        fwd2 = sum(wl2.B * kept(wl2, i) for i in pruned2)
+        other = {"infinity_2b_1k": {"what": "the 1024-pixel configuration: 13 scales up to 64x64, batch 2, keep 0.6 / 0.4 / 0.2 on the last three",
+                                    "value": world * fwd2 / (o_pruned * 1e-3), "unit": UNIT, "ms_per_step": o_total,
+                                    "ms_per_image": o_total / wl2.B, "ms_pruned_steps": o_pruned, "config": config_of(wl2, world)}}
+        ctx2.close()
+        del ctx2, gt2, xs2, outs2
+        torch.cuda.empty_cache()
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.skip_cpu:
         cb = time_oracle(wl, reps=1, warmup=0)
@@ -469,14 +535,11 @@ def ours(args, wl):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": {"workload": wl.name, "B_per_gpu": wl.B, "L": wl.L, "C": wl.C, "H": wl.H, "cross_len": wl.cross_len,
-                       "sides": list(wl.sides), "keep": list(wl.keep), "parallelism": f"replicas x{world} (images sharded, no collective)",
-                       "cache_hygiene": "inputs larger than L2 (weights + KV + token maps of one pass >> 126 MB)",
-                       "step": "one full scale schedule for one batch"},
+            "config": config_of(wl, world),
             "ms_per_image": ms_per_step / wl.B, "ms_per_image_pruned_steps": pruned_ms / wl.B,
             "scale_step_ms": [round(t, 4) for t in step_ms], "wall_ms_per_step": t_wall * 1e3 / args.steps,
             "roofline": roofline, "kernels": kernels, "kernels_pruned_steps": kernels_pruned, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": gpu_launches,
-            "clocks": clocks, "unpruned_gpu": unpruned, "per_step_granularity": variant, "backbone_options": extras, "generation_loop": generation,
+            "clocks": clocks, "unpruned_gpu": unpruned, "per_step_granularity": variant, "backbone_options": extras, "generation_loop": generation, "other_workloads": other,
             "peaks": peaks}
     print(json.dumps(line))
 
@@ -556,7 +619,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="infinity_2b_1k", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--workload", default="infinity_2b_2k", choices=sorted(I.WORKLOADS))
     ap.add_argument("--skip-cpu", action="store_true", help="omit the CPU-oracle leg")
     ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer end-to-end leg")
     ap.add_argument("--skip-profile", action="store_true", help="omit the per-kernel-class timing passes")
@@ -564,6 +627,7 @@ def main():
     ap.add_argument("--skip-generation", action="store_true", help="omit the generation-loop (fv_generate) timing")
     ap.add_argument("--sweep", action="store_true", help="print pruning-ratio and caching-step curves instead of the bench line")
     ap.add_argument("--skip-variant", action="store_true", help="omit the per-step-granularity comparison")
+    ap.add_argument("--skip-other", action="store_true", help="omit the timing of the 1024-pixel configuration beside the default one")
     ap.add_argument("--blocks", type=int, default=0,
                     help="profiling only: run this many transformer blocks instead of the workload's depth (the line says so; not a bench number)")
     args = ap.parse_args()

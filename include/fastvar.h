@@ -249,11 +249,36 @@ fv_status fv_gather_ln(const float *x_dev, const int32_t *idx_dev, int32_t B, in
 /* Restore fused with gate and residual (Eq. 6 + the block's x += gamma * y):
  *   x[b,t,:] += gamma[b,:] * (inv[b,t] >= 0 ? y[b, inv[b,t], :] : cache[b, src(t), :]).
  * gamma_dev NULL = 1.  y, cache bf16; x fp32 in place.  C % 8 == 0.  interp_mode as for fv_restore (with 1
- * the cache term is the bilinear blend of four cached rows). */
+ * the cache term is the bilinear blend of four cached rows).
+ *   colsum_ws_dev NULL, or a selection workspace (fv_prune_select_workspace_bytes(B, h*w, C) bytes, 16-byte
+ *               aligned): the kernel then also leaves there the per-image column sums of the UPDATED map
+ *               -- Eq. 4's sum over tokens for the next sublayer's selection -- so that
+ *               fv_prune_select_after_restore can rank the map without summing it again.  They are kept as
+ *               a few partial sums per image, see fv_prune_select_workspace_layout.
+ *   part        0: every row.  1: only the rows that were NOT kept (they need the selection and the cache
+ *               alone, so inside a step they run beside the sublayer's GEMMs).  2: only the kept rows, after
+ *               part 1 on the same workspace (its sums continue part 1's and are then folded per image).
+ *               Parts 1 and 2 together give the bits of part 0 in x (the sums add the rows in another order).
+ * Errors: INVALID_ARG, CAPACITY (workspace too small), CUDA. */
 fv_status fv_restore_residual(float *x_dev, const void *y_dev, const void *cache_dev,
                               const int32_t *inv_dev, const float *gamma_dev, int32_t mod_stride,
                               int32_t B, int32_t k, int32_t h, int32_t w, int32_t hc, int32_t wc,
-                              int32_t C, int32_t interp_mode, void *stream);
+                              int32_t C, int32_t interp_mode, void *colsum_ws_dev, size_t colsum_ws_bytes,
+                              int32_t part, void *stream);
+/* Pivotal Token Selection (as fv_prune_select) of a map whose column sums fv_restore_residual has left in
+ * workspace_dev: the form every selection after the first takes inside fv_var_step. */
+fv_status fv_prune_select_after_restore(const float *x_dev, int32_t B, int32_t h, int32_t w, int32_t C,
+                                        double keep_ratio, int32_t *idx_out_dev, int32_t *inv_out_dev,
+                                        float *score_out_dev, int32_t *near_tie_dev, int32_t *k_out_host,
+                                        void *workspace_dev, size_t workspace_bytes, void *stream);
+/* Where a selection workspace keeps the column sums (for tests): they sit at byte offset *offset_host as
+ * fp32 [B, *n_partials_host, C]; the sum over the partials of image b is the column sum of its map. */
+fv_status fv_prune_select_workspace_layout(int32_t B, int32_t n_tokens, int32_t C, size_t *offset_host,
+                                           int32_t *n_partials_host);
+/* Test / profiling hook (process-wide): how the kept-row part of a restoration folds its column sums.
+ * 0 = chosen per shape (default); 1 = always through global memory (arrival counters); 2 = inside
+ * thread-block clusters wherever the shape allows it. */
+fv_status fv_restore_force_fold(int32_t mode);
 
 /* tcgen05 GEMM  out = epilogue(A[M,K] * W[N,K]^T + bias), bf16 operands, fp32 accumulation in TMEM.
  *   epilogue 0: bf16 store to out [M, N].          1: tanh-GELU then bf16 store.
@@ -287,10 +312,20 @@ fv_status fv_gemm_bf16(const void *a_dev, const void *w_dev, const void *bias_de
  *   q_dev  [B*rows, C] bf16 (image b owns rows [b*rows, (b+1)*rows)); head h = channels [h*hd, ..).
  *   k_dev  [B, kv_capacity, C] bf16;  vt_dev [B, C, kv_capacity] bf16 (V transposed).
  *   kv_len keys are attended (rows [0, kv_len) of every image).  out_dev [B*rows, C] bf16.
- *   hd = C / H in {64, 128}; kv_capacity % 8 == 0. */
+ *   hd = C / H in {64, 128}; kv_capacity % 8 == 0.
+ *   workspace_dev NULL: one CTA per (256 queries, head, image).  Else fv_attention_workspace_bytes() bytes of
+ *               scratch, 16-byte aligned, whose first 65536 bytes are zero (the kernel leaves them zero): the
+ *               (queries, head, image, key tile) work is then cut into equal pieces, one per SM, and the
+ *               pieces of one query block are merged in key order (same bits run to run).
+ *               CAPACITY if workspace_bytes is too small. */
+size_t fv_attention_workspace_bytes(void);
 fv_status fv_attention(const void *q_dev, const void *k_dev, const void *vt_dev, int32_t B,
                        int32_t rows, int32_t H, int32_t C, int32_t kv_len, int32_t kv_capacity,
-                       void *out_dev, int32_t *status_dev, void *stream);
+                       void *out_dev, int32_t *status_dev, void *workspace_dev, size_t workspace_bytes,
+                       void *stream);
+/* Test / profiling hook (process-wide): number of CTAs of a fv_attention launch that is given a workspace
+ * (0 = one per SM, the default; capped at 160 and at what the work allows). */
+fv_status fv_attention_force_ctas(int32_t ctas);
 
 /* ------------------------------------------------------------------------------------------------
  * (4) The generation loop around the scale step -- Sec. 3.1: step k turns the token map of scale k into a

@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "FV_OK", 1: "FV_ERR_INVALID_ARG", 2: "FV_ERR_BAD_STATE", 3: "
 EXPORTS = ["fv_status_string", "fv_k_for", "fv_prune_select_workspace_bytes", "fv_prune_select", "fv_restore",
            "fv_workspace_bytes", "fv_kv_bytes", "fv_cache_bytes", "fv_create", "fv_destroy", "fv_reset",
            "fv_get_state", "fv_set_state", "fv_kv_pointers", "fv_cache_pointer", "fv_prepare_text",
-           "fv_device_status", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_gemm_bf16", "fv_gemm_splitk_workspace_bytes", "fv_gemm_force_path", "fv_attention",
+           "fv_device_status", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_prune_select_after_restore",
+           "fv_prune_select_workspace_layout", "fv_restore_force_fold", "fv_gemm_bf16", "fv_gemm_splitk_workspace_bytes", "fv_gemm_force_path", "fv_attention", "fv_attention_workspace_bytes", "fv_attention_force_ctas",
            "fv_kernel_launches", "fv_profile_enable", "fv_profile_read",
            "fv_prune_select_static", "fv_prune_select_static_capacity",
            "fv_head_workspace_bytes", "fv_head_tokens", "fv_argmax_rows", "fv_residual_accumulate", "fv_next_scale_input",
@@ -88,13 +89,20 @@ def lib() -> C.CDLL:
         L.fv_var_step.restype = C.c_int; L.fv_var_step.argtypes = [vp, vp, i32, i32, dbl, vp, vp, vp, vp]
         L.fv_gather_ln.restype = C.c_int; L.fv_gather_ln.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, i32, vp, vp]
         L.fv_restore_residual.restype = C.c_int
-        L.fv_restore_residual.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp]
+        L.fv_restore_residual.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp, sz, i32, vp]
+        L.fv_prune_select_after_restore.restype = C.c_int
+        L.fv_prune_select_after_restore.argtypes = [vp, i32, i32, i32, i32, dbl, vp, vp, vp, vp, C.POINTER(i32), vp, sz, vp]
+        L.fv_prune_select_workspace_layout.restype = C.c_int
+        L.fv_prune_select_workspace_layout.argtypes = [i32, i32, i32, C.POINTER(sz), C.POINTER(i32)]
+        L.fv_restore_force_fold.restype = C.c_int; L.fv_restore_force_fold.argtypes = [i32]
         L.fv_gemm_bf16.restype = C.c_int
         L.fv_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, sz, vp]
         L.fv_gemm_splitk_workspace_bytes.restype = sz; L.fv_gemm_splitk_workspace_bytes.argtypes = []
         L.fv_gemm_force_path.restype = C.c_int; L.fv_gemm_force_path.argtypes = [i32]
         L.fv_attention.restype = C.c_int
-        L.fv_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp]
+        L.fv_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.fv_attention_workspace_bytes.restype = sz; L.fv_attention_workspace_bytes.argtypes = []
+        L.fv_attention_force_ctas.restype = C.c_int; L.fv_attention_force_ctas.argtypes = [i32]
         L.fv_prune_select_static_capacity.restype = sz; L.fv_prune_select_static_capacity.argtypes = []
         L.fv_prune_select_static.restype = C.c_int
         L.fv_prune_select_static.argtypes = [vp, i32, i32, i32, i32, dbl, vp, vp, vp, vp, C.POINTER(i32), vp]
@@ -223,11 +231,45 @@ def fv_gather_ln(x: torch.Tensor, idx: Optional[torch.Tensor], sigma: Optional[t
 
 
 def fv_restore_residual(x: torch.Tensor, y: torch.Tensor, cache: torch.Tensor, inv: torch.Tensor,
-                        gamma: Optional[torch.Tensor], mod_stride: int, h: int, w: int, hc: int, wc: int, interp_mode: int = 0) -> None:
+                        gamma: Optional[torch.Tensor], mod_stride: int, h: int, w: int, hc: int, wc: int, interp_mode: int = 0,
+                        colsum_ws: Optional[torch.Tensor] = None, part: int = 0) -> None:
+    """colsum_ws: uint8 selection workspace that receives the column sums of the updated map, or None."""
     B, n, Cw = x.shape
     k = y.shape[1]
     _check(lib().fv_restore_residual(_ptr(x), _ptr(y), _ptr(cache), _ptr(inv), _ptr(gamma), mod_stride, B, k, h, w, hc, wc,
-                                     Cw, int(interp_mode), _stream()), "fv_restore_residual")
+                                     Cw, int(interp_mode), _ptr(colsum_ws), 0 if colsum_ws is None else colsum_ws.numel(),
+                                     int(part), _stream()), "fv_restore_residual")
+
+
+def fv_prune_select_workspace(B: int, n: int, Cw: int, device) -> torch.Tensor:
+    return torch.empty(lib().fv_prune_select_workspace_bytes(B, n, Cw), dtype=torch.uint8, device=device)
+
+
+def fv_colsum_partials(workspace: torch.Tensor, B: int, n: int, Cw: int) -> torch.Tensor:
+    """fp32 view [B, partials, C] of the column sums a restoration left in a selection workspace."""
+    off, cnt = C.c_size_t(), C.c_int32()
+    _check(lib().fv_prune_select_workspace_layout(B, n, Cw, C.byref(off), C.byref(cnt)), "fv_prune_select_workspace_layout")
+    return workspace[off.value: off.value + 4 * B * cnt.value * Cw].view(torch.float32).view(B, cnt.value, Cw)
+
+
+def fv_prune_select_after_restore(x: torch.Tensor, h: int, w: int, keep_ratio: float, workspace: torch.Tensor,
+                                  want_score: bool = False, want_near_tie: bool = False):
+    """fv_prune_select of a map whose column sums fv_restore_residual left in `workspace`."""
+    B, n, Cw = x.shape
+    k = fv_k_for(keep_ratio, h, w)
+    idx = torch.empty((B, k), dtype=torch.int32, device=x.device)
+    inv = torch.empty((B, n), dtype=torch.int32, device=x.device)
+    score = torch.empty((B, n), dtype=torch.float32, device=x.device) if want_score else None
+    near = torch.empty((B,), dtype=torch.int32, device=x.device) if want_near_tie else None
+    k_out = C.c_int32(0)
+    _check(lib().fv_prune_select_after_restore(_ptr(x), B, h, w, Cw, float(keep_ratio), _ptr(idx), _ptr(inv), _ptr(score), _ptr(near),
+                                               C.byref(k_out), _ptr(workspace), workspace.numel(), _stream()),
+           "fv_prune_select_after_restore")
+    return {"idx": idx, "inv": inv, "score": score, "near_tie": near, "k": k}
+
+
+def fv_restore_force_fold(mode: int) -> None:
+    _check(lib().fv_restore_force_fold(int(mode)), "fv_restore_force_fold")
 
 
 def fv_gemm_bf16(a: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor], epilogue: int = 0,
@@ -247,14 +289,20 @@ def fv_gemm_bf16(a: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor],
     return out
 
 
+def fv_attention_workspace(device) -> torch.Tensor:
+    """Zeroed scratch for fv_attention's split over the SMs (its arrival counters must start at zero)."""
+    return torch.zeros(lib().fv_attention_workspace_bytes(), dtype=torch.uint8, device=device)
+
+
 def fv_attention(q: torch.Tensor, k_cache: torch.Tensor, vt_cache: torch.Tensor, B: int, rows: int, H: int, kv_len: int,
-                 status: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """q bf16 [B*rows, C]; k_cache bf16 [B, cap, C]; vt_cache bf16 [B, C, cap] -> bf16 [B*rows, C]."""
+                 status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """q bf16 [B*rows, C]; k_cache bf16 [B, cap, C]; vt_cache bf16 [B, C, cap] -> bf16 [B*rows, C].
+    workspace: fv_attention_workspace(...) to cut the work into one piece per SM, or None."""
     Cw = q.shape[1]
     cap = k_cache.shape[1]
     out = torch.empty_like(q)
     _check(lib().fv_attention(_ptr(q), _ptr(k_cache), _ptr(vt_cache), B, rows, H, Cw, kv_len, cap, _ptr(out), _ptr(status),
-                              _stream()), "fv_attention")
+                              _ptr(workspace), 0 if workspace is None else workspace.numel(), _stream()), "fv_attention")
     return out
 
 

@@ -31,6 +31,7 @@ struct fv_ctx {
   int32_t *idx = nullptr, *inv = nullptr;
   void* sel_ws = nullptr;
   void* splitk_ws = nullptr;
+  void* attn_ws = nullptr;
   cudaStream_t side = nullptr;           // the unkept rows of a restoration run here, beside the sublayer's branch
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   float* step_cache = nullptr;  // fp32 output map of the caching step [B_max, n_cache, C] (skipped steps; granularity 1)
@@ -57,6 +58,7 @@ cudaError_t g_init_err = cudaSuccess;
 cudaError_t ensure_init() {
   std::call_once(g_init_once, [] {
     g_init_err = select_init();
+    if (g_init_err == cudaSuccess) g_init_err = rows_init();
     if (g_init_err == cudaSuccess) g_init_err = gemm_init();
     if (g_init_err == cudaSuccess) g_init_err = attention_init();
   });
@@ -66,7 +68,7 @@ cudaError_t ensure_init() {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 struct Layout {
-  size_t status, a, q, o, y, hbuf, idx, inv, sel, splitk, xc, rope, total;
+  size_t status, a, q, o, y, hbuf, idx, inv, sel, splitk, attn, xc, rope, total;
 };
 
 int max_tokens(const fv_config* c) {
@@ -103,6 +105,7 @@ Layout workspace_layout(const fv_config* c) {
   l.inv = take(M * 4);
   l.sel = take(select_workspace_bytes(c->B_max, max_tokens(c), c->C));
   l.splitk = take(gemm_splitk_ws_bytes());
+  l.attn = take(attention_ws_bytes());
   l.xc = take(c->granularity == 1 ? M * C * 4 : 0);
   size_t rope_bytes = 0;
   if (c->rope_base > 0.f)
@@ -187,12 +190,52 @@ fv_status fv_gather_ln(const float* x_dev, const int32_t* idx_dev, int32_t B, in
 
 fv_status fv_restore_residual(float* x_dev, const void* y_dev, const void* cache_dev, const int32_t* inv_dev,
                               const float* gamma_dev, int32_t mod_stride, int32_t B, int32_t k, int32_t h, int32_t w,
-                              int32_t hc, int32_t wc, int32_t C, int32_t interp_mode, void* stream) {
-  if (interp_mode < 0 || interp_mode > 2) return FV_ERR_INVALID_ARG;
+                              int32_t hc, int32_t wc, int32_t C, int32_t interp_mode, void* colsum_ws_dev, size_t colsum_ws_bytes,
+                              int32_t part, void* stream) {
+  if (interp_mode < 0 || interp_mode > 2 || part < 0 || part > 2) return FV_ERR_INVALID_ARG;
   if (!x_dev || !y_dev || !cache_dev || !inv_dev || B <= 0 || k <= 0 || h <= 0 || w <= 0 || hc <= 0 || wc <= 0) return FV_ERR_INVALID_ARG;
   if (C <= 0 || (C % 8)) return FV_ERR_INVALID_ARG;
+  if (ensure_init() != cudaSuccess) return FV_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (colsum_ws_dev) {
+    if (!aligned16(colsum_ws_dev)) return FV_ERR_INVALID_ARG;
+    if ((long)h * w > kTopkMaxTokens) return FV_ERR_UNSUPPORTED;
+    if (colsum_ws_bytes < select_workspace_bytes(B, h * w, C)) return FV_ERR_CAPACITY;
+    // the arrival counters at the head of the workspace start at zero (the kernels leave them at zero)
+    if (part != 2 && cudaMemsetAsync(colsum_ws_dev, 0, select_ticket_bytes(B), st) != cudaSuccess) return FV_ERR_CUDA;
+  }
   return cuda_status(launch_restore_residual(x_dev, y_dev, cache_dev, inv_dev, gamma_dev, mod_stride, B, k, h, w, hc, wc, C,
-                                             nullptr, 0, interp_mode, static_cast<cudaStream_t>(stream)));
+                                             colsum_ws_dev, part, interp_mode, st));
+}
+
+fv_status fv_prune_select_after_restore(const float* x_dev, int32_t B, int32_t h, int32_t w, int32_t C, double keep_ratio,
+                                        int32_t* idx_out_dev, int32_t* inv_out_dev, float* score_out_dev, int32_t* near_tie_dev,
+                                        int32_t* k_out_host, void* workspace_dev, size_t workspace_bytes, void* stream) {
+  if (!x_dev || !idx_out_dev || !workspace_dev || B <= 0 || h <= 0 || w <= 0 || C <= 0) return FV_ERR_INVALID_ARG;
+  if (!(keep_ratio > 0.0) || keep_ratio > 1.0 || (C % 4) || !aligned16(x_dev) || !aligned16(workspace_dev)) return FV_ERR_INVALID_ARG;
+  const long n = (long)h * w;
+  if (n > kTopkMaxTokens || C > kTopkMaxTokens) return FV_ERR_UNSUPPORTED;
+  if (workspace_bytes < select_workspace_bytes(B, (int)n, C)) return FV_ERR_CAPACITY;
+  if (ensure_init() != cudaSuccess) return FV_ERR_CUDA;
+  const int k = fv_k_for(keep_ratio, h, w);
+  if (k_out_host) *k_out_host = k;
+  return cuda_status(launch_select(x_dev, B, (int)n, C, k, idx_out_dev, inv_out_dev, score_out_dev, near_tie_dev, workspace_dev, true,
+                                   static_cast<cudaStream_t>(stream)));
+}
+
+fv_status fv_prune_select_workspace_layout(int32_t B, int32_t n_tokens, int32_t C, size_t* offset_host, int32_t* n_partials_host) {
+  if (B <= 0 || n_tokens <= 0 || C <= 0 || !offset_host || !n_partials_host) return FV_ERR_INVALID_ARG;
+  static char origin[1];     // carve relative to any address; only the offset is reported
+  const SelectWs w = select_ws_carve(origin, B, n_tokens, C);
+  *offset_host = (size_t)(reinterpret_cast<char*>(w.group_partial) - origin);
+  *n_partials_host = w.ngroups;
+  return FV_OK;
+}
+
+fv_status fv_restore_force_fold(int32_t mode) {
+  if (mode < 0 || mode > 2) return FV_ERR_INVALID_ARG;
+  restore_force_fold(mode);
+  return FV_OK;
 }
 
 fv_status fv_gemm_bf16(const void* a_dev, const void* w_dev, const void* bias_dev, int32_t M, int32_t N, int32_t K,
@@ -210,11 +253,22 @@ fv_status fv_gemm_bf16(const void* a_dev, const void* w_dev, const void* bias_de
   return launch_gemm(g, static_cast<cudaStream_t>(stream));
 }
 
+size_t fv_attention_workspace_bytes(void) { return attention_ws_bytes(); }
+
+fv_status fv_attention_force_ctas(int32_t ctas) {
+  if (ctas < 0) return FV_ERR_INVALID_ARG;
+  attention_force_ctas(ctas);
+  return FV_OK;
+}
+
 fv_status fv_attention(const void* q_dev, const void* k_dev, const void* vt_dev, int32_t B, int32_t rows, int32_t H,
-                       int32_t C, int32_t kv_len, int32_t kv_capacity, void* out_dev, int32_t* status_dev, void* stream) {
+                       int32_t C, int32_t kv_len, int32_t kv_capacity, void* out_dev, int32_t* status_dev, void* workspace_dev,
+                       size_t workspace_bytes, void* stream) {
   if (ensure_init() != cudaSuccess) return FV_ERR_CUDA;
   if (!aligned16(q_dev) || !aligned16(k_dev) || !aligned16(vt_dev) || !aligned16(out_dev)) return FV_ERR_INVALID_ARG;
+  if (workspace_dev && (!aligned16(workspace_dev) || workspace_bytes < attention_ws_bytes())) return FV_ERR_CAPACITY;
   AttnArgs a{};
+  a.workspace = workspace_dev;
   a.q = q_dev; a.k = k_dev; a.vt = vt_dev; a.out = out_dev; a.B = B; a.rows = rows; a.H = H; a.C = C; a.kv_len = kv_len;
   a.kv_capacity = kv_capacity; a.status = status_dev;
   return launch_attention(a, static_cast<cudaStream_t>(stream));
@@ -308,6 +362,7 @@ fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, v
   c->inv = reinterpret_cast<int32_t*>(c->ws + lay.inv);
   c->sel_ws = c->ws + lay.sel;
   c->splitk_ws = c->ws + lay.splitk;
+  c->attn_ws = c->ws + lay.attn;
   c->xc = reinterpret_cast<float*>(c->ws + lay.xc);
   c->qk_scale = wts->qk_scale_dev;
   bool rope_ok = true;
@@ -324,6 +379,7 @@ fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, v
   if (!rope_ok || cudaMemset(kv_dev, 0, fv_kv_bytes(cfg)) != cudaSuccess || cudaMemset(c->status, 0, 256) != cudaSuccess ||
       cudaMemset(c->sel_ws, 0, select_ticket_bytes(cfg->B_max)) != cudaSuccess ||
       cudaMemset(c->splitk_ws, 0, gemm_splitk_ticket_bytes()) != cudaSuccess ||
+      cudaMemset(c->attn_ws, 0, attention_ws_ticket_bytes()) != cudaSuccess ||
       cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
@@ -550,7 +606,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         if (s != FV_OK) break;
         AttnArgs a{};
         a.q = ctx->q_buf; a.k = kbase; a.vt = kbase + ctx->k_bytes; a.out = ctx->o_buf; a.B = B; a.rows = k; a.H = c.H; a.C = C;
-        a.kv_len = ctx->kv_len + k; a.kv_capacity = c.kv_capacity; a.status = ctx->status;
+        a.kv_len = ctx->kv_len + k; a.kv_capacity = c.kv_capacity; a.status = ctx->status; a.workspace = ctx->attn_ws;
         s = launch_attention(a, st);
         if (s != FV_OK) break;
         last_in = ctx->o_buf; last_w = ctx->w_o[l]; last_b = ctx->b_o[l];
@@ -560,7 +616,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         if (s != FV_OK) break;
         AttnArgs a{};
         a.q = ctx->q_buf; a.k = text_k(ctx, l); a.vt = text_k(ctx, l) + ctx->text_k_bytes; a.out = ctx->o_buf; a.B = B; a.rows = k;
-        a.H = c.H; a.C = C; a.kv_len = c.cross_len; a.kv_capacity = c.cross_len; a.status = ctx->status;
+        a.H = c.H; a.C = C; a.kv_len = c.cross_len; a.kv_capacity = c.cross_len; a.status = ctx->status; a.workspace = ctx->attn_ws;
         s = launch_attention(a, st);
         if (s != FV_OK) break;
         last_in = ctx->o_buf; last_w = ctx->w_o_x[l]; last_b = nullptr;

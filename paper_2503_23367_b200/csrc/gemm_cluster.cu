@@ -91,6 +91,9 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // first half of the "every CTA of the cluster has started" barrier; the second half precedes the first
+  // store into another CTA's shared memory (a rank with an empty K slice gets there almost at once)
+  cluster_arrive_relaxed();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -149,6 +152,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (have && !mbar_wait(acc_full, 0)) { report(p.status, DEV_TIMEOUT_EPI); have = false; }
     have = __all_sync(0xffffffffu, have);   // the TMEM loads below are warp-wide
     tc_fence_after();
+    cluster_wait();                         // every CTA of the cluster is running: its shared memory may be written
     const uint32_t dst = map_to_cta(red + ((size_t)rank * ROWS_PER + lrow) * Cfg::kRedPitch, owner);
     const uint32_t t0 = tmem_base + (uint32_t(quarter * 32) << 16);
 #pragma unroll 1
@@ -171,6 +175,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   // Every thread of every CTA of the cluster: the partials are in place after this barrier, and no CTA is
   // written to afterwards (so each may finish and exit on its own).
   __syncwarp();
+  if (warp < 2) cluster_wait();             // completes these warps' half of the start-up barrier
   cluster_sync_all();
   if (warp >= 2) {
     const int e = threadIdx.x - 64;                        // 0..127

@@ -78,6 +78,8 @@ cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, i
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv,
                                     const float* gamma, int mod_stride, int B, int k, int h, int w, int hc, int wc,
                                     int C, void* colsum_ws, int part, int interp_mode, cudaStream_t st);
+cudaError_t rows_init();               // one-time function attributes
+void restore_force_fold(int mode);     // test hook: 0 by shape, 1 fold through global memory, 2 fold inside clusters
 // Per-step granularity: fp32 gather of the kept rows, and fp32 restoration of the step's output map.
 cudaError_t launch_gather_rows(const float* x, const int32_t* idx, int B, int n, int k, int C, float* out, cudaStream_t st);
 cudaError_t launch_restore_rows_f32(const float* cache, int hc, int wc, const float* pivots, const int32_t* inv, int B, int k,
@@ -130,8 +132,12 @@ struct AttnArgs {
   void* out;       // [B*rows, C] bf16
   int B, rows, H, C, kv_len, kv_capacity;
   int32_t* status;
+  void* workspace;   // null (one work item per CTA), or attention_ws_bytes() of scratch whose leading attention_ws_ticket_bytes() are zero
 };
 cudaError_t attention_init();
+size_t attention_ws_bytes();
+size_t attention_ws_ticket_bytes();
+void attention_force_ctas(int ctas);   // test hook: CTAs of a split launch (0 = one per SM)
 fv_status launch_attention(const AttnArgs& a, cudaStream_t st);
 
 // ---- tensor maps (gemm.cu) ------------------------------------------------------------------------

@@ -300,6 +300,7 @@ __global__ void __launch_bounds__(256) restore_kept_cluster_kernel(float4* __res
   __shared__ int s_on[kColsumRows];
   __shared__ __align__(16) float s_fold[kFoldEntries * 8];   // [chunk of the group][channel group of this CTA's slice][8]
   pdl_trigger();
+  cluster_arrive_relaxed();   // first half of the start-up barrier (completed before the remote stores below)
   pdl_wait();
   const int b = blockIdx.y;
   const int rank = (int)cluster_ctarank();
@@ -317,6 +318,7 @@ __global__ void __launch_bounds__(256) restore_kept_cluster_kernel(float4* __res
   }
   __syncthreads();
   const int c8 = threadIdx.x;
+  float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
   if (valid && c8 < C8) {
     float4 g0 = make_float4(1.f, 1.f, 1.f, 1.f), g1 = g0;
     if (gamma) {
@@ -325,7 +327,7 @@ __global__ void __launch_bounds__(256) restore_kept_cluster_kernel(float4* __res
     }
     // continue the sums of the rows the first part updated
     const float4* cp = chunk_partial + ((size_t)b * nchunks + chunk) * C8 * 2 + 2 * c8;
-    float4 a0 = __ldcg(cp), a1 = __ldcg(cp + 1);
+    a0 = __ldcg(cp); a1 = __ldcg(cp + 1);
     float4* xbase = x + ((size_t)b * n + t0) * C8 * 2;
     for (int r = 0; r < rows; r += 4) {
       uint4 p[4];
@@ -358,6 +360,9 @@ __global__ void __launch_bounds__(256) restore_kept_cluster_kernel(float4* __res
         }
       }
     }
+  }
+  cluster_wait();    // every CTA of the cluster has started: their shared memory may be written
+  if (valid && c8 < C8) {
     // the chunk's sums of this thread's 8 channels go to the CTA that owns the channel slice
     const int owner = c8 / slice, local = c8 - owner * slice;
     uint32_t dst;
@@ -550,6 +555,16 @@ __global__ void rope_table_kernel(float2* __restrict__ table, int h, int w, int 
 }
 }  // namespace
 
+// How the kept-row part of a restoration folds its column sums: 0 by shape, 1 global memory, 2 clusters.
+static int g_fold_mode = 0;
+static bool g_cluster_fold_ok = false;
+void restore_force_fold(int mode) { g_fold_mode = mode; }
+cudaError_t rows_init() {
+  g_cluster_fold_ok = cudaFuncSetAttribute(restore_kept_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+  (void)cudaGetLastError();
+  return cudaSuccess;
+}
+
 cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
                              const float* beta, int mod_stride, void* a_out, cudaStream_t st) {
   const int rows = B * k;
@@ -570,27 +585,18 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
   const double rr_bytes = (double)B * C * (8.0 * rows_x + (part != 1 ? 2.0 * k : 0.0) + (part != 2 ? 2.0 * hc * wc : 0.0));
   LaunchScope scope(KC_RESTORE, 1, rr_bytes, rr_bytes, st);
   // kept rows + group fold inside clusters (one cluster per group of chunks) where the group fits a cluster
-  static bool cluster_fold_ok = true;
-  if (part == 2 && colsum_ws && cluster_fold_ok && ws.group >= 1 && ws.group <= 8 && C / 8 <= 256) {
-    static bool attr_set = false;
-    if (!attr_set) {
-      cluster_fold_ok = cudaFuncSetAttribute(restore_kept_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
-      attr_set = true;
-    }
-    if (cluster_fold_ok) {
-      cudaLaunchConfig_t cfg{};
-      cfg.gridDim = dim3(ws.group * ws.ngroups, B); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = st;
-      cudaLaunchAttribute at[1];
-      at[0].id = cudaLaunchAttributeClusterDimension;
-      at[0].val.clusterDim.x = ws.group; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-      cfg.attrs = at; cfg.numAttrs = 1;
-      const cudaError_t e = cudaLaunchKernelEx(&cfg, restore_kept_cluster_kernel, reinterpret_cast<float4*>(x), reinterpret_cast<const uint4*>(y),
-                                               inv, gamma, mod_stride, n, k, C / 8, nchunks, ws.group, ws.ngroups,
-                                               reinterpret_cast<const float4*>(ws.chunk_partial), reinterpret_cast<float4*>(ws.group_partial));
-      if (e == cudaSuccess) return e;
-      (void)cudaGetLastError();      // this cluster size cannot be scheduled here: the fold through global memory from now on
-      cluster_fold_ok = false;
-    }
+  if (part == 2 && colsum_ws && g_cluster_fold_ok && g_fold_mode != 1 && ws.group >= 1 && ws.group <= 8 && C / 8 <= 256) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(ws.group * ws.ngroups, B); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = ws.group; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, restore_kept_cluster_kernel, reinterpret_cast<float4*>(x), reinterpret_cast<const uint4*>(y),
+                                             inv, gamma, mod_stride, n, k, C / 8, nchunks, ws.group, ws.ngroups,
+                                             reinterpret_cast<const float4*>(ws.chunk_partial), reinterpret_cast<float4*>(ws.group_partial));
+    if (e == cudaSuccess || g_fold_mode == 2) return e;
+    (void)cudaGetLastError();      // this cluster size cannot be scheduled here: the fold through global memory instead
   }
   auto* kern = (interp_mode == 0 || part == 2) ? restore_residual_kernel
                : (interp_mode == 1 ? restore_residual_interp_kernel<4> : restore_residual_interp_kernel<16>);

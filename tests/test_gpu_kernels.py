@@ -195,24 +195,106 @@ def test_restore_residual_bilinear(B, hc, wc, h, w, C, k, mode):
     np.testing.assert_allclose(xd.cpu().numpy(), ref, rtol=2e-6, atol=1e-5)      # fp32 blend of 4 / 16 rows, then one fma
 
 
-def test_restore_residual_large():
-    """The 64x64 pruned step's restore (67 MB map, 820 kept rows per image, cache of the 32x32 step), with the
-    column sums of the updated map left in a selection workspace: they must equal the map's own column sums."""
-    B, hc, wc, h, w, C, k = 2, 32, 32, 64, 64, 2048, 820
+def _restore_case(B, hc, wc, h, w, C, k, seed=54):
     n = h * w
-    x = I.normal(54, (B, n, C))
-    y = I.normal_bf16(55, (B, k, C))
-    cache = I.normal_bf16(56, (B, hc * wc, C))
-    mod = I.normal(57, (B, 6, C), 0.3)
-    idx = np.stack([np.sort(np.argsort(I.uniform01(61 + b, n))[:k]) for b in range(B)])
+    x = I.normal(seed, (B, n, C))
+    y = I.normal_bf16(seed + 1, (B, k, C))
+    cache = I.normal_bf16(seed + 2, (B, hc * wc, C))
+    mod = I.normal(seed + 3, (B, 6, C), 0.3)
+    idx = np.stack([np.sort(np.argsort(I.uniform01(seed + 7 + b, n))[:k]) for b in range(B)])
     inv = O.inverse_map(idx, n).astype(np.int32)
-    xd, modd = dev(x), dev(mod)
-    fv.fv_restore_residual(xd, bf16_dev(y), bf16_dev(cache), dev(inv), modd.data_ptr() + 2 * 4 * C, 6 * C, h, w, hc, wc)
-    torch.cuda.synchronize()
     yfull = O.cached_token_restoration(I.bf16_bits_to_f32(y).astype(np.float64), idx,
                                        I.bf16_bits_to_f32(cache).astype(np.float64), hc, wc, h, w)
     ref = x.astype(np.float64) + mod[:, 2].astype(np.float64)[:, None, :] * yfull
+    return x, y, cache, mod, inv, ref
+
+
+def test_restore_residual_large():
+    """The 64x64 pruned step's restore (67 MB map, 820 kept rows per image, cache of the 32x32 step): every element
+    of the updated map against the oracle."""
+    B, hc, wc, h, w, C, k = 2, 32, 32, 64, 64, 2048, 820
+    x, y, cache, mod, inv, ref = _restore_case(B, hc, wc, h, w, C, k)
+    xd, modd = dev(x), dev(mod)
+    fv.fv_restore_residual(xd, bf16_dev(y), bf16_dev(cache), dev(inv), modd.data_ptr() + 2 * 4 * C, 6 * C, h, w, hc, wc)
+    torch.cuda.synchronize()
     np.testing.assert_allclose(xd.cpu().numpy(), ref, rtol=1e-6, atol=2e-6)
+
+
+# Maps whose chunks of 32 tokens fold in groups of 1 / 2 / 4 / 5 / 8 (one thread-block cluster per group), with a
+# ragged last chunk (33 x 31, 50 x 50), a ragged last group (50 x 50: 79 chunks in groups of 5), and groups too
+# large for a cluster (96 x 96, 128 x 128: 18 and 32 chunks per group, folded through global memory).
+COLSUM_CASES = [  # B, hc, wc, h, w, C, k
+    (1, 10, 10, 13, 13, 256, 85), (3, 10, 10, 33, 31, 256, 205), (2, 32, 32, 40, 40, 2048, 960), (2, 32, 32, 48, 48, 2048, 922),
+    (2, 32, 32, 64, 64, 2048, 820), (1, 13, 13, 50, 50, 1920, 625), (1, 48, 48, 96, 96, 2048, 1844), (1, 48, 48, 128, 128, 2048, 3277),
+]
+
+
+@pytest.mark.parametrize("B,hc,wc,h,w,C,k", COLSUM_CASES)
+@pytest.mark.parametrize("fold", [0, 1])
+def test_restore_leaves_the_column_sums_of_the_updated_map(B, hc, wc, h, w, C, k, fold):
+    """Eq. 4 for the NEXT selection comes from the restoration: the partial sums it leaves in the selection
+    workspace, added up per image, are the column sums of the map it has just updated -- for the one-pass form
+    (part 0), for the two-pass form a scale step uses (part 1: rows that were not kept, part 2: kept rows + fold),
+    with the fold inside thread-block clusters (fold 0, where the shape allows) and through global memory (fold 1).
+    The two forms must give the same bits in the map (their sums add the rows in a different order)."""
+    n = h * w
+    x, y, cache, mod, inv, ref = _restore_case(B, hc, wc, h, w, C, k, seed=154)
+    yd, cd, invd, modd = bf16_dev(y), bf16_dev(cache), dev(inv), dev(mod)
+    gamma = modd.data_ptr() + 2 * 4 * C
+    colsum_ref = ref.sum(axis=1)                                            # fp64 [B, C]
+    scale = np.abs(ref).sum(axis=1).max()                                   # fp32 sums of n terms in a fixed order
+    fv.fv_restore_force_fold(fold)
+    try:
+        results = []
+        for parts in ((0,), (1, 2)):
+            xd = dev(x)
+            ws = fv.fv_prune_select_workspace(B, n, C, DEV)
+            ws.fill_(0xFF)                                                  # stale contents must not matter (NaN patterns)
+            for part in parts:
+                fv.fv_restore_residual(xd, yd, cd, invd, gamma, 6 * C, h, w, hc, wc, colsum_ws=ws, part=part)
+            torch.cuda.synchronize()
+            got = fv.fv_colsum_partials(ws, B, n, C).cpu().numpy().astype(np.float64).sum(axis=1)
+            assert np.abs(got - colsum_ref).max() <= 1e-5 * scale, (parts, np.abs(got - colsum_ref).max(), scale)
+            np.testing.assert_allclose(xd.cpu().numpy(), ref, rtol=1e-6, atol=2e-6)
+            results.append(xd.cpu().numpy())
+        assert np.array_equal(results[0], results[1])
+    finally:
+        fv.fv_restore_force_fold(0)
+
+
+@pytest.mark.parametrize("B,hc,wc,h,w,C,k", COLSUM_CASES)
+def test_selection_from_the_restoration_s_column_sums(B, hc, wc, h, w, C, k):
+    """The selection that follows a restoration inside a scale step: it takes Eq. 4's mean token from the sums the
+    restoration left behind instead of summing the map again.  Scores and kept set against the oracle applied to
+    the updated map, and the same kept set as the stand-alone selection of the same map up to near-ties."""
+    n = h * w
+    keep = k / n
+    assert O.kept_count(keep, h, w) == k
+    x, y, cache, mod, inv, ref = _restore_case(B, hc, wc, h, w, C, k, seed=254)
+    xd, modd = dev(x), dev(mod)
+    ws = fv.fv_prune_select_workspace(B, n, C, DEV)
+    for part in (1, 2):
+        fv.fv_restore_residual(xd, bf16_dev(y), bf16_dev(cache), dev(inv), modd.data_ptr() + 2 * 4 * C, 6 * C, h, w, hc, wc,
+                               colsum_ws=ws, part=part)
+    r = fv.fv_prune_select_after_restore(xd, h, w, keep, ws, want_score=True)
+    alone = fv.fv_prune_select(xd, h, w, keep, want_score=True)
+    torch.cuda.synchronize()
+    x_new = xd.cpu().numpy()
+    score_o = O.pts_score(x_new)                                            # oracle on the map the GPU holds
+    score_g = r["score"].cpu().numpy()
+    np.testing.assert_allclose(score_g, score_o, rtol=2e-5, atol=1e-4)
+    idx_g = r["idx"].cpu().numpy().astype(np.int64)
+    assert np.array_equal(idx_g, O.pts_topk(score_g, k))
+    assert np.array_equal(r["inv"].cpu().numpy(), O.inverse_map(idx_g, n))
+    idx_o = O.pts_topk(score_o, k)
+    for b in range(B):
+        diff = np.setxor1d(idx_g[b], idx_o[b])
+        if len(diff):
+            tau = np.sort(score_o[b])[::-1][k - 1]
+            assert np.all(np.abs(score_o[b, diff] - tau) <= 1e-5 * tau), "index mismatch away from a near-tie"
+    # the stand-alone selection sums the rows of a chunk in another order: same scores up to fp32 rounding
+    np.testing.assert_allclose(alone["score"].cpu().numpy(), score_g, rtol=2e-6, atol=1e-5)
+    assert np.array_equal(alone["idx"].cpu().numpy(), O.pts_topk(alone["score"].cpu().numpy(), k))
 
 
 # ------------------------------------------------------------------ tcgen05 GEMM
@@ -236,6 +318,22 @@ def test_gemm_bf16(M, N, K, epilogue):
     if epilogue == 1:
         ref = O.gelu_tanh(ref)
     err, cos = per_token_errors(bf16_host(out), ref)
+    assert err <= MAX_ABS and cos >= MIN_COS, (err, cos)
+
+
+@pytest.mark.parametrize("N,K", [(6144, 2048), (2048, 2048), (8192, 2048), (2048, 8192)])
+def test_gemm_bf16_at_the_2k_step_s_row_count(N, K):
+    """The four projection shapes of a block at the 128x128 zero-shot step (3277 kept rows: 25 full row tiles and a
+    ragged one of 77), bias + GELU epilogue; the oracle runs on a sample of rows that covers every row tile."""
+    M = 3277
+    a = I.normal_bf16(170, (M, K), 1.0 if K <= 2048 else 0.5); w = I.normal_bf16(171, (N, K), 0.02); b = I.normal_bf16(172, (N,), 0.02)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = fv.fv_gemm_bf16(bf16_dev(a), bf16_dev(w), bf16_dev(b), epilogue=1, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rows = np.unique(np.concatenate([np.arange(0, M, 11), np.arange(M - 80, M)]))
+    ref = O.gelu_tanh(O.linear(I.bf16_bits_to_f32(a[rows]), I.bf16_bits_to_f32(w), I.bf16_bits_to_f32(b)))
+    err, cos = per_token_errors(bf16_host(out)[rows], ref)
     assert err <= MAX_ABS and cos >= MIN_COS, (err, cos)
 
 
@@ -409,20 +507,14 @@ def test_gemm_residual_epilogue_at_step_shapes(rows, N, K):
 ATTN_CASES = [  # B, rows, H, C, kv_len, cap
     (2, 85, 4, 256, 340, 344), (1, 300, 2, 256, 1000, 1024), (2, 128, 16, 1024, 485, 488), (1, 1, 4, 256, 1, 8),
     (1, 130, 2, 256, 129, 136), (2, 820, 16, 2048, 5223, 5224), (1, 37, 30, 1920, 640, 640),
+    (1, 3277, 16, 2048, 13646, 13648),      # the 128x128 zero-shot step: 13 query-tile pairs x 107 key tiles per head
+    (1, 1280, 16, 2048, 8525, 8528), (2, 260, 4, 256, 700, 704), (1, 52, 16, 2048, 6000, 6000),
 ]
 
 
-@pytest.mark.parametrize("B,rows,H,C,kv_len,cap", ATTN_CASES)
-def test_attention_over_kv_cache(B, rows, H, C, kv_len, cap):
-    q = I.normal_bf16(90, (B * rows, C)); kk = I.normal_bf16(91, (B, cap, C)); vv = I.normal_bf16(92, (B, cap, C))
-    vt = np.ascontiguousarray(vv.transpose(0, 2, 1))
-    status = torch.zeros(1, dtype=torch.int32, device=DEV)
-    out = fv.fv_attention(bf16_dev(q), bf16_dev(kk), bf16_dev(vt), B, rows, H, kv_len, status=status)
-    torch.cuda.synchronize()
-    assert int(status.item()) == 0
+def _attention_reference_check(got, q, kk, vv, B, rows, H, C, kv_len):
     qf, kf, vf = (I.bf16_bits_to_f32(t).astype(np.float64) for t in (q, kk, vv))
-    got = bf16_host(out)
-    heads = range(H) if B * rows * kv_len * C < 3e9 else (0, H - 1)    # bound the oracle's time on the big case
+    heads = range(H) if B * rows * kv_len * C < 3e9 else (0, H - 1)    # bound the oracle's time on the big cases
     hd = C // H
     for b in range(B):
         if len(heads) == H:
@@ -435,3 +527,53 @@ def test_attention_over_kv_cache(B, rows, H, C, kv_len, cap):
                 ref = O.attention(qf[b * rows:(b + 1) * rows, sl], kf[b, :kv_len, sl], vf[b, :kv_len, sl], 1)
                 err, cos = per_token_errors(got[b * rows:(b + 1) * rows, sl], ref)
                 assert err <= MAX_ABS and cos >= MIN_COS, (err, cos)
+
+
+@pytest.mark.parametrize("B,rows,H,C,kv_len,cap", ATTN_CASES)
+def test_attention_over_kv_cache(B, rows, H, C, kv_len, cap):
+    """Without scratch (one CTA per block of 256 queries of a head) and with it (the work cut into one piece per SM,
+    the pieces of a query block merged in key order): both against the oracle, the split twice with identical bits,
+    its arrival counters left at zero."""
+    q = I.normal_bf16(90, (B * rows, C)); kk = I.normal_bf16(91, (B, cap, C)); vv = I.normal_bf16(92, (B, cap, C))
+    vt = np.ascontiguousarray(vv.transpose(0, 2, 1))
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    qd, kd, vd = bf16_dev(q), bf16_dev(kk), bf16_dev(vt)
+    out = fv.fv_attention(qd, kd, vd, B, rows, H, kv_len, status=status)
+    ws = fv.fv_attention_workspace(DEV)
+    out_s = fv.fv_attention(qd, kd, vd, B, rows, H, kv_len, status=status, workspace=ws)
+    out_s2 = fv.fv_attention(qd, kd, vd, B, rows, H, kv_len, status=status, workspace=ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(out_s, out_s2)
+    assert int(ws[:65536].view(torch.int32).abs().sum().item()) == 0
+    _attention_reference_check(bf16_host(out), q, kk, vv, B, rows, H, C, kv_len)
+    _attention_reference_check(bf16_host(out_s), q, kk, vv, B, rows, H, C, kv_len)
+
+
+@pytest.mark.parametrize("ctas", [1, 2, 3, 5, 7, 16, 37, 97, 160])
+@pytest.mark.parametrize("B,rows,H,C,kv_len,cap", [(2, 300, 2, 256, 1000, 1024), (1, 130, 2, 256, 129, 136), (2, 260, 4, 256, 700, 704),
+                                                   (1, 820, 2, 256, 2000, 2000), (3, 37, 4, 256, 333, 336), (1, 1, 4, 256, 1, 8)])
+def test_attention_split_into_any_number_of_pieces(B, rows, H, C, kv_len, cap, ctas):
+    """The split with a forced piece count: pieces that end inside a query block, that hold the end of one block, whole
+    blocks and the start of another, blocks merged from many parts, single-tile blocks, a ragged last key tile, and
+    more pieces asked for than the work allows.  Every output row against the oracle."""
+    q = I.normal_bf16(190, (B * rows, C)); kk = I.normal_bf16(191, (B, cap, C)); vv = I.normal_bf16(192, (B, cap, C))
+    vt = np.ascontiguousarray(vv.transpose(0, 2, 1))
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = fv.fv_attention_workspace(DEV)
+    assert fv.lib().fv_attention_force_ctas(ctas) == 0
+    try:
+        out = fv.fv_attention(bf16_dev(q), bf16_dev(kk), bf16_dev(vt), B, rows, H, kv_len, status=status, workspace=ws)
+        torch.cuda.synchronize()
+    finally:
+        fv.lib().fv_attention_force_ctas(0)
+    assert int(status.item()) == 0
+    assert int(ws[:65536].view(torch.int32).abs().sum().item()) == 0
+    _attention_reference_check(bf16_host(out), q, kk, vv, B, rows, H, C, kv_len)
+
+
+def test_attention_refuses_small_scratch():
+    q = torch.zeros((8, 256), dtype=torch.bfloat16, device=DEV); k = torch.zeros((1, 8, 256), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(fv.FvError) as e:
+        fv.fv_attention(q, k, k.transpose(1, 2).contiguous(), 1, 8, 4, 8, workspace=torch.zeros(4096, dtype=torch.uint8, device=DEV))
+    assert e.value.code == 3
