@@ -6,8 +6,8 @@
 // Work item = 256 queries (two tiles of 128) of one head of one image; keys are consumed in tiles of 128.
 // The kept-row counts of the pruned steps give item counts that fit the GPU badly (64, 80, 128 or 208 items
 // on 148 SMs, the last item of a head often a single, part-filled tile), so the (item, key tile) units are
-// laid out on one line, items of two tiles weighted 3 and single-tile items 2, and the line is cut into
-// equal pieces, one per CTA (one CTA per SM).  A CTA walks its piece as segments: a range of key tiles of
+// laid out on one line (a weight per item kind; both kinds cost the same per key tile as measured) and the line
+// is cut into equal pieces, one per CTA (one CTA per SM), when that beats one whole item per CTA.  A CTA walks its piece as segments: a range of key tiles of
 // one item.  A segment that covers all key tiles of its item writes the output itself; otherwise it leaves
 // its unnormalised partial (O, running maximum, row sum) in scratch, and the last part of an item to arrive
 // (arrival counter) merges the parts IN KEY ORDER, so the result does not depend on arrival order.
@@ -62,7 +62,9 @@ template <int HD> struct AttnCfg {
 constexpr int kAttnMaxItems = 16384;
 constexpr int kAttnMaxCtas = 160;
 constexpr size_t kAttnTicketBytes = (size_t)kAttnMaxItems * sizeof(unsigned int);
-constexpr int kWeightPair = 3, kWeightSingle = 2;   // cost of a key tile for an item of two query tiles / of one
+// Cost of a key tile for an item of two query tiles / of one.  Measured equal: with one tile there is nothing to
+// overlap the S -> softmax -> P V -> next S chain with, so the tile takes as long as the pair's two.
+constexpr int kWeightPair = 1, kWeightSingle = 1;
 
 struct AttnDev {
   __nv_bfloat16* out;
@@ -154,6 +156,61 @@ __device__ __noinline__ void item_parts(const AttnDev& p, int c, int nctas, int 
   *nparts = b - a + 1;
 }
 
+// Online softmax of one query row over the key tiles [ja, jb) of a segment: scores out of TMEM, probabilities
+// back into it, the O accumulator rescaled in place when the running maximum moves.  Returns false if a wait
+// expired.  `tiles` counts the score tiles this thread's query tile has consumed (the phase of the barriers).
+// Out of line so that the loop keeps the whole register file to itself (a thread holds a score row of 128 floats).
+template <int HD>
+__device__ __noinline__ bool softmax_key_tiles(const AttnDev& p, int ja, int jb, uint32_t s_addr, uint32_t o_addr, uint64_t* s_full_t,
+                                               uint64_t* p_full_t, uint64_t* o_done_t, uint32_t& tiles, float& m_out, float& l_out) {
+  float m_run = -INFINITY, l_run = 0.f;
+  uint32_t sc_cnt = tiles;
+  const float scale_log2 = p.scale_log2;
+  for (int j = ja; j < jb; ++j, ++sc_cnt) {
+    if (!mbar_wait(s_full_t, sc_cnt & 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); tiles = sc_cnt; return false; }
+    tc_fence_after();
+    const int valid = p.kv_len - j * KT;  // >= 1
+    float sc[KT];
+    if (valid < KT) tile_load_scores<true>(s_addr, valid, sc);
+    else tile_load_scores<false>(s_addr, valid, sc);
+    float mx0 = sc[0], mx1 = sc[1], mx2 = sc[2], mx3 = sc[3];
+#pragma unroll
+    for (int i = 4; i < KT; i += 4) {
+      mx0 = fmaxf(mx0, sc[i]); mx1 = fmaxf(mx1, sc[i + 1]); mx2 = fmaxf(mx2, sc[i + 2]); mx3 = fmaxf(mx3, sc[i + 3]);
+    }
+    const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale_log2;
+    // Raise the running maximum only when it would grow by more than the threshold: probabilities
+    // may then exceed 1 (by at most 2^threshold), which fp32 sums and bf16 P hold without loss.
+    float alpha = 1.f;
+    if (mx > m_run + kRescaleThreshold) {
+      alpha = fast_exp2(m_run - mx);  // 0 on the first tile (m_run = -inf)
+      m_run = mx;
+    }
+    // S_t of tile j was issued after P V of tile j-1, so O_t is at rest here.
+    if (j > ja && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+      for (int c = 0; c < HD / 32; ++c) {
+        uint32_t o[32];
+        tmem_ld32(o_addr + c * 32, o);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+        tmem_st32(o_addr + c * 32, o);
+      }
+    }
+    const float rs = tile_exp_store(sc, s_addr, scale_log2, m_run);
+    l_run = fmaf(l_run, alpha, rs);
+    tmem_wait_st();
+    tc_fence_before();
+    mbar_arrive(p_full_t);
+  }
+  tiles = sc_cnt;
+  m_out = m_run; l_out = l_run;
+  if (!mbar_wait(o_done_t, (sc_cnt - 1) & 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); return false; }
+  tc_fence_after();
+  return true;
+}
+
 // End of a segment for one softmax thread (query row r of tile t): O_t leaves tensor memory -- as the normalised
 // bf16 output when the segment covered every key tile of its item, else as this part's unnormalised partial in
 // scratch, after which the last part of the item to arrive merges all of them in key order.  Kept out of line so
@@ -240,20 +297,34 @@ __device__ __noinline__ void finish_segment(const AttnDev& p, int u0, int u_hi, 
   }
   const float inv_l = 1.f / l_star;
   __nv_bfloat16* dst = p.out + ((size_t)img * p.rows + row) * p.C + head * HD;
+  // 32 output channels at a time: the eight float4 of a part are requested together (the loop is bound by the
+  // latency of these loads, not by their bytes), parts added in key order
 #pragma unroll 1
-  for (int c8 = 0; c8 < HD / 8; ++c8) {     // 8 output channels = two float4 of every part
-    float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+  for (int c32 = 0; c32 < HD / 32; ++c32) {
+    float4 acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
     for (int q = 0; q < nparts; ++q) {
       const char* slot = part_slot(q);
+      const float4* os = reinterpret_cast<const float4*>(slot + Cfg::kPartMlBytes) + ((size_t)t * (HD / 4) + c32 * 8) * QT + r;
+      float4 v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = __ldcg(os + (size_t)i * QT);
       const float wq = fast_exp2(__ldcg(reinterpret_cast<const float2*>(slot) + t * QT + r).x - m_star) * inv_l;
-      const float4* os = reinterpret_cast<const float4*>(slot + Cfg::kPartMlBytes) + (size_t)t * (HD / 4) * QT + r;
-      const float4 v0 = __ldcg(os + (size_t)(2 * c8) * QT), v1 = __ldcg(os + (size_t)(2 * c8 + 1) * QT);
-      a0.x = fmaf(v0.x, wq, a0.x); a0.y = fmaf(v0.y, wq, a0.y); a0.z = fmaf(v0.z, wq, a0.z); a0.w = fmaf(v0.w, wq, a0.w);
-      a1.x = fmaf(v1.x, wq, a1.x); a1.y = fmaf(v1.y, wq, a1.y); a1.z = fmaf(v1.z, wq, a1.z); a1.w = fmaf(v1.w, wq, a1.w);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        acc[i].x = fmaf(v[i].x, wq, acc[i].x); acc[i].y = fmaf(v[i].y, wq, acc[i].y);
+        acc[i].z = fmaf(v[i].z, wq, acc[i].z); acc[i].w = fmaf(v[i].w, wq, acc[i].w);
+      }
     }
-    uint4 v;
-    v.x = pack_bf16x2(a0.x, a0.y); v.y = pack_bf16x2(a0.z, a0.w); v.z = pack_bf16x2(a1.x, a1.y); v.w = pack_bf16x2(a1.z, a1.w);
-    reinterpret_cast<uint4*>(dst)[c8] = v;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint4 v;
+      v.x = pack_bf16x2(acc[2 * i].x, acc[2 * i].y); v.y = pack_bf16x2(acc[2 * i].z, acc[2 * i].w);
+      v.z = pack_bf16x2(acc[2 * i + 1].x, acc[2 * i + 1].y); v.w = pack_bf16x2(acc[2 * i + 1].z, acc[2 * i + 1].w);
+      reinterpret_cast<uint4*>(dst + c32 * 32)[i] = v;
+    }
   }
 }
 
@@ -433,48 +504,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       u += sg.jb - sg.ja;
       const bool active = t < sg.ntiles;
       float m_run = -INFINITY, l_run = 0.f;
-      if (active && ok) {
-        for (int j = sg.ja; j < sg.jb; ++j, ++sc_cnt) {
-          if (!mbar_wait(&s_full[t], sc_cnt & 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); ok = false; break; }
-          tc_fence_after();
-          const int valid = p.kv_len - j * KT;  // >= 1
-          float sc[KT];
-          if (valid < KT) tile_load_scores<true>(s_addr, valid, sc);
-          else tile_load_scores<false>(s_addr, valid, sc);
-          float mx0 = sc[0], mx1 = sc[1], mx2 = sc[2], mx3 = sc[3];
-#pragma unroll
-          for (int i = 4; i < KT; i += 4) {
-            mx0 = fmaxf(mx0, sc[i]); mx1 = fmaxf(mx1, sc[i + 1]); mx2 = fmaxf(mx2, sc[i + 2]); mx3 = fmaxf(mx3, sc[i + 3]);
-          }
-          const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
-          // Raise the running maximum only when it would grow by more than the threshold: probabilities
-          // may then exceed 1 (by at most 2^threshold), which fp32 sums and bf16 P hold without loss.
-          float alpha = 1.f;
-          if (mx > m_run + kRescaleThreshold) {
-            alpha = fast_exp2(m_run - mx);  // 0 on the first tile (m_run = -inf)
-            m_run = mx;
-          }
-          // S_t of tile j was issued after P V of tile j-1, so O_t is at rest here.
-          if (j > sg.ja && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll
-            for (int c = 0; c < HD / 32; ++c) {
-              uint32_t o[32];
-              tmem_ld32(o_addr + c * 32, o);
-              tmem_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-              tmem_st32(o_addr + c * 32, o);
-            }
-          }
-          const float rs = tile_exp_store(sc, s_addr, p.scale_log2, m_run);
-          l_run = fmaf(l_run, alpha, rs);
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(&p_full[t]);
-        }
-        if (ok && !mbar_wait(&o_done[t], (sc_cnt - 1) & 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); ok = false; }
-        tc_fence_after();
-      }
+      if (active && ok) ok = softmax_key_tiles<HD>(p, sg.ja, sg.jb, s_addr, o_addr, &s_full[t], &p_full[t], &o_done[t], sc_cnt, m_run, l_run);
       finish_segment<HD>(p, u0, u_hi, t, r, o_addr, m_run, l_run, ok, &o_free[t], s_info);
     }
   }
@@ -515,13 +545,17 @@ template <int HD> fv_status launch_hd(const AttnArgs& a, cudaStream_t st) {
   long long ctas = items;
   p.split = 0;
   if (a.workspace && items <= kAttnMaxItems) {
-    // one CTA per SM, every piece at least two key tiles of a two-tile item long (so that no piece is empty and
-    // the merge of an item stays a handful of parts)
+    // One piece per SM when that beats whole items: a launch of whole items takes ceil(items / SMs) rounds of T key
+    // tiles; the pieces take items * T / SMs key tiles plus what the cuts cost (query tiles loaded again, the
+    // partials written and merged: about kSplitOverheadTiles key tiles, measured).  A forced piece count always splits.
+    constexpr long long kSplitOverheadTiles = 6;
     long long g = g_attn_force_ctas > 0 ? g_attn_force_ctas : g_attn_sms;
     if (g > kAttnMaxCtas) g = kAttnMaxCtas;
-    const long long most = p.total_cost / (2 * kWeightPair);
+    const long long most = p.total_cost / (2 * kWeightPair);   // every piece at least two key tiles long
     if (g > most) g = most;
-    if (g >= 1) {
+    const long long rounds = (items + g_attn_sms - 1) / g_attn_sms;
+    const bool pays = g >= 1 && 100 * (items * p.T / g + kSplitOverheadTiles) < 92 * rounds * p.T;
+    if (g >= 1 && (pays || g_attn_force_ctas > 0)) {
       p.split = 1;
       ctas = g;
       p.tickets = static_cast<unsigned int*>(a.workspace);
