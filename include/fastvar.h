@@ -324,7 +324,8 @@ fv_status fv_attention(const void *q_dev, const void *k_dev, const void *vt_dev,
                        void *out_dev, int32_t *status_dev, void *workspace_dev, size_t workspace_bytes,
                        void *stream);
 /* Test / profiling hook (process-wide): number of CTAs of a fv_attention launch that is given a workspace
- * (0 = one per SM, the default; capped at 160 and at what the work allows). */
+ * (0 = one per SM where that pays, the default; n > 0 = always n pieces, capped at 160 and at what the work
+ * allows; -1 = never cut the work, as if no workspace were given). */
 fv_status fv_attention_force_ctas(int32_t ctas);
 
 /* ------------------------------------------------------------------------------------------------

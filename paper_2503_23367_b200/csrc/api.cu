@@ -256,7 +256,7 @@ fv_status fv_gemm_bf16(const void* a_dev, const void* w_dev, const void* bias_de
 size_t fv_attention_workspace_bytes(void) { return attention_ws_bytes(); }
 
 fv_status fv_attention_force_ctas(int32_t ctas) {
-  if (ctas < 0) return FV_ERR_INVALID_ARG;
+  if (ctas < -1) return FV_ERR_INVALID_ARG;
   attention_force_ctas(ctas);
   return FV_OK;
 }

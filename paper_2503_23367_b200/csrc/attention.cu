@@ -544,17 +544,18 @@ template <int HD> fv_status launch_hd(const AttnArgs& a, cudaStream_t st) {
   p.total_cost = p.cost_group * a.H * a.B;
   long long ctas = items;
   p.split = 0;
-  if (a.workspace && items <= kAttnMaxItems) {
+  if (a.workspace && items <= kAttnMaxItems && g_attn_force_ctas >= 0) {
     // One piece per SM when that beats whole items: a launch of whole items takes ceil(items / SMs) rounds of T key
     // tiles; the pieces take items * T / SMs key tiles plus what the cuts cost (query tiles loaded again, the
-    // partials written and merged: about kSplitOverheadTiles key tiles, measured).  A forced piece count always splits.
-    constexpr long long kSplitOverheadTiles = 6;
+    // partials written and merged: about kSplitOverheadTiles key tiles, measured; short key ranges lose).  A forced
+    // piece count always splits.
+    constexpr long long kSplitOverheadTiles = 10;
     long long g = g_attn_force_ctas > 0 ? g_attn_force_ctas : g_attn_sms;
     if (g > kAttnMaxCtas) g = kAttnMaxCtas;
     const long long most = p.total_cost / (2 * kWeightPair);   // every piece at least two key tiles long
     if (g > most) g = most;
     const long long rounds = (items + g_attn_sms - 1) / g_attn_sms;
-    const bool pays = g >= 1 && 100 * (items * p.T / g + kSplitOverheadTiles) < 92 * rounds * p.T;
+    const bool pays = g >= 1 && p.T >= 16 && 100 * (items * p.T / g + kSplitOverheadTiles) < 92 * rounds * p.T;
     if (g >= 1 && (pays || g_attn_force_ctas > 0)) {
       p.split = 1;
       ctas = g;
