@@ -563,11 +563,12 @@ def sweep(args, wl):
     outs = [torch.empty_like(x) for x in xs]
     hw = [(s_, s_) for s_ in wl.sides]
 
-    def run(keep):
+    def run(keep, cache_step=None):
         w2 = replace(wl, keep=tuple(keep))
         pruned = [i for i in range(S) if keep[i] < 1.0]
         cap = sum(kept(w2, i) for i in range(S))
-        ctx = fv.FvContext(wl.L, wl.C, wl.H, hw, w2.cache_step, wl.B, cap, gt, cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio, device=dev)
+        ctx = fv.FvContext(wl.L, wl.C, wl.H, hw, w2.cache_step if cache_step is None else cache_step, wl.B, cap, gt,
+                           cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio, device=dev)
         ev = [[torch.cuda.Event(enable_timing=True) for _ in range(S + 1)] for _ in range(3)]
         for rep in range(5):
             ctx.reset()
@@ -610,6 +611,19 @@ def sweep(args, wl):
                      "cache_step": S - n_pruned - 1, "pruning_ratio": 0.5, "ms_per_image": total / wl.B,
                      "speedup_whole_schedule": base_total / total, "speedup_pruned_steps": sum(base_step[i] for i in pruned) / p_ms,
                      "forwarded_tokens_per_s": sum(wl.B * kept(w2, i) for i in pruned) / (p_ms * 1e-3)})
+    # the caching step of the paper's ablation: the workload's pruned steps stay as they are, the step whose layer
+    # outputs are cached moves back from K-N (the last unpruned step) to K-N-3 (smaller cached maps, upsampled further)
+    first_pruned = default_pruned[0]
+    for back in (0, 1, 2, 3):
+        cs = first_pruned - 1 - back
+        if cs < 0:
+            continue
+        total, step, pruned, w2 = run(list(wl.keep), cache_step=cs)
+        p_ms = sum(step[i] for i in pruned)
+        rows.append({"sweep": "caching step K-N-j with the workload's pruned steps fixed", "cache_step": cs, "steps_before_the_first_pruned": back + 1,
+                     "cached_side": wl.sides[cs], "ms_per_image": total / wl.B, "speedup_whole_schedule": base_total / total,
+                     "speedup_pruned_steps": sum(base_step[i] for i in pruned) / p_ms,
+                     "forwarded_tokens_per_s": sum(wl.B * kept(w2, i) for i in pruned) / (p_ms * 1e-3)})
     print(json.dumps({"sweep": rows, "workload": wl.name, "B": wl.B, "unpruned_ms_per_image": base_total / wl.B, "data": "synthetic"}))
 
 
@@ -631,6 +645,16 @@ def main():
     ap.add_argument("--blocks", type=int, default=0,
                     help="profiling only: run this many transformer blocks instead of the workload's depth (the line says so; not a bench number)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours" and not args.sweep:
+        # started plainly with --gpus N: become the launcher of N ranks, one per GPU (replicas; the process group
+        # only carries the measurement), and pass their output through
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+               "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = I.WORKLOADS[args.workload]
     if args.blocks > 0:

@@ -33,7 +33,8 @@ typedef enum {
   FV_ERR_CAPACITY = 3,    /* KV cache or workspace too small for this call                           */
   FV_ERR_UNSUPPORTED = 4, /* shape outside what the kernels cover (stated per call)                  */
   FV_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed (launch error, descriptor encoding) */
-  FV_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (see fv_device_status)               */
+  FV_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (see fv_device_status)               */
+  FV_ERR_DEVICE_DATA = 7  /* a kernel met an index outside its range and clamped it (fv_device_status) */
 } fv_status;
 
 const char *fv_status_string(fv_status s);
@@ -192,9 +193,15 @@ fv_status fv_cache_pointer(const fv_ctx *ctx, int32_t block, int32_t sublayer, v
 /* Projects the text tokens to per-block K / V^T for cross-attention (step-invariant).  Called by
  * fv_var_step at scale step 0; call it yourself after fv_set_state on a fresh context. */
 fv_status fv_prepare_text(fv_ctx *ctx, int32_t B, void *stream);
-/* Synchronises `stream` and returns FV_OK, or FV_ERR_TIMEOUT (code in *code_host) if a kernel's bounded
- * wait expired since the last call; clears the word. */
+/* Synchronises `stream` and reads the context's device status word: FV_OK, or -- with the kernel's code in
+ * *code_host -- FV_ERR_TIMEOUT if a bounded wait expired since the last call (codes 101-105: operand loads, MMA
+ * issue, epilogue, softmax, the self-test below) or FV_ERR_DEVICE_DATA if a kernel met an index outside its range
+ * and clamped it (40: a token id outside the codebook; 41: a kept-row index outside the token map).  Clears the word. */
 fv_status fv_device_status(fv_ctx *ctx, int32_t *code_host, void *stream);
+/* Self-test of the convention above (no counterpart in the paper): one warp waits, with the library's bounded
+ * wait, for limit_ns nanoseconds (at most 1e9) on a barrier that nothing ever completes, then records code 105
+ * and returns normally.  Nothing traps; the context stays usable.  fv_device_status then reports FV_ERR_TIMEOUT. */
+fv_status fv_selftest_expired_wait(fv_ctx *ctx, uint64_t limit_ns, void *stream);
 
 /* One scale step over all L blocks.
  *   tokens_dev  [B, h*w, C] fp32: residual stream entering block 0 at this scale.
@@ -241,10 +248,12 @@ fv_status fv_host_io_flush(fv_ctx *ctx, void *stream);
 /* Gather + LayerNorm + AdaLN modulate (the compaction of Algorithm 1's gather fused with the block's
  * pre-norm): a[b,j,:] = LN(x[b, idx[b,j], :]) * (1 + sigma[b,:]) + beta[b,:]  -> bf16.
  *   idx_dev NULL = all rows (k = n_tokens);  sigma_dev / beta_dev NULL = plain LayerNorm;
- *   their per-image stride is mod_stride floats.  C % 4 == 0, C <= 2048. */
+ *   their per-image stride is mod_stride floats.  C % 4 == 0, C <= 2048.
+ *   status_dev NULL, or an int32 device word: an index outside [0, n_tokens) is clamped into the map (the read
+ *   stays in bounds) and code 41 is left there. */
 fv_status fv_gather_ln(const float *x_dev, const int32_t *idx_dev, int32_t B, int32_t n_tokens,
                        int32_t k, int32_t C, const float *sigma_dev, const float *beta_dev,
-                       int32_t mod_stride, void *a_out_dev, void *stream);
+                       int32_t mod_stride, void *a_out_dev, int32_t *status_dev, void *stream);
 
 /* Restore fused with gate and residual (Eq. 6 + the block's x += gamma * y):
  *   x[b,t,:] += gamma[b,:] * (inv[b,t] >= 0 ? y[b, inv[b,t], :] : cache[b, src(t), :]).
@@ -395,7 +404,8 @@ typedef struct {
  *   ids_out_dev int32 [B * sum_k h_k*w_k]: step k's ids [B, h_k*w_k] start at B * sum_{j<k} h_j*w_j.
  *   r_out_dev fp32 [B, h_K*w_K, d]: the final prediction r_K.
  *   workspace_dev: fv_generate_workspace_bytes(ctx, gen) bytes, 1024-byte aligned.
- * Errors: those of the calls it makes. */
+ * Device-side codes of every stage (an expired wait in the head GEMM, a token id outside the codebook) land in
+ * the context's status word: read them with fv_device_status.  Errors: those of the calls it makes. */
 size_t fv_generate_workspace_bytes(const fv_ctx *ctx, const fv_generator *gen);
 fv_status fv_generate(fv_ctx *ctx, const fv_generator *gen, const float *start_dev, int32_t B,
                       const double *keep_host, const float *const *noise_host, int32_t *ids_out_dev,

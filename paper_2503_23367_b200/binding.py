@@ -17,12 +17,12 @@ LIB_PATH = os.path.join(_HERE, "libfastvar.so")
 
 FV_OK = 0
 STATUS_NAMES = {0: "FV_OK", 1: "FV_ERR_INVALID_ARG", 2: "FV_ERR_BAD_STATE", 3: "FV_ERR_CAPACITY",
-                4: "FV_ERR_UNSUPPORTED", 5: "FV_ERR_CUDA", 6: "FV_ERR_TIMEOUT"}
+                4: "FV_ERR_UNSUPPORTED", 5: "FV_ERR_CUDA", 6: "FV_ERR_TIMEOUT", 7: "FV_ERR_DEVICE_DATA"}
 
 EXPORTS = ["fv_status_string", "fv_k_for", "fv_prune_select_workspace_bytes", "fv_prune_select", "fv_restore",
            "fv_workspace_bytes", "fv_kv_bytes", "fv_cache_bytes", "fv_create", "fv_destroy", "fv_reset",
            "fv_get_state", "fv_set_state", "fv_kv_pointers", "fv_cache_pointer", "fv_prepare_text",
-           "fv_device_status", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_prune_select_after_restore",
+           "fv_device_status", "fv_selftest_expired_wait", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_prune_select_after_restore",
            "fv_prune_select_workspace_layout", "fv_restore_force_fold", "fv_gemm_bf16", "fv_gemm_splitk_workspace_bytes", "fv_gemm_force_path", "fv_attention", "fv_attention_workspace_bytes", "fv_attention_force_ctas",
            "fv_kernel_launches", "fv_profile_enable", "fv_profile_read",
            "fv_prune_select_static", "fv_prune_select_static_capacity",
@@ -87,7 +87,8 @@ def lib() -> C.CDLL:
         L.fv_prepare_text.restype = C.c_int; L.fv_prepare_text.argtypes = [vp, i32, vp]
         L.fv_device_status.restype = C.c_int; L.fv_device_status.argtypes = [vp, C.POINTER(i32), vp]
         L.fv_var_step.restype = C.c_int; L.fv_var_step.argtypes = [vp, vp, i32, i32, dbl, vp, vp, vp, vp]
-        L.fv_gather_ln.restype = C.c_int; L.fv_gather_ln.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, i32, vp, vp]
+        L.fv_gather_ln.restype = C.c_int; L.fv_gather_ln.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, i32, vp, vp, vp]
+        L.fv_selftest_expired_wait.restype = C.c_int; L.fv_selftest_expired_wait.argtypes = [vp, C.c_uint64, vp]
         L.fv_restore_residual.restype = C.c_int
         L.fv_restore_residual.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp, sz, i32, vp]
         L.fv_prune_select_after_restore.restype = C.c_int
@@ -221,11 +222,11 @@ def fv_restore(cache_prev: torch.Tensor, hc: int, wc: int, pivots: torch.Tensor,
 
 
 def fv_gather_ln(x: torch.Tensor, idx: Optional[torch.Tensor], sigma: Optional[torch.Tensor],
-                 beta: Optional[torch.Tensor], mod_stride: int = 0) -> torch.Tensor:
+                 beta: Optional[torch.Tensor], mod_stride: int = 0, status: Optional[torch.Tensor] = None) -> torch.Tensor:
     B, n, Cw = x.shape
     k = n if idx is None else idx.shape[1]
     out = torch.empty((B, k, Cw), dtype=torch.bfloat16, device=x.device)
-    _check(lib().fv_gather_ln(_ptr(x), _ptr(idx), B, n, k, Cw, _ptr(sigma), _ptr(beta), mod_stride, _ptr(out), _stream()),
+    _check(lib().fv_gather_ln(_ptr(x), _ptr(idx), B, n, k, Cw, _ptr(sigma), _ptr(beta), mod_stride, _ptr(out), _ptr(status), _stream()),
            "fv_gather_ln")
     return out
 
@@ -477,11 +478,19 @@ class FvContext:
         _check(lib().fv_prepare_text(self.ctx, B, _stream()), "fv_prepare_text")
 
     def device_status(self) -> int:
+        """The kernels' status code since the last call (0 = fine); the word is cleared."""
+        return self.device_status_pair()[1]
+
+    def device_status_pair(self):
+        """(fv_status, code): (0, 0), (FV_ERR_TIMEOUT, 101..105) or (FV_ERR_DEVICE_DATA, 40 / 41)."""
         code = C.c_int32()
         rc = lib().fv_device_status(self.ctx, C.byref(code), _stream())
-        if rc not in (0, 6):
+        if rc not in (0, 6, 7):
             raise FvError(rc, "fv_device_status")
-        return code.value
+        return rc, code.value
+
+    def selftest_expired_wait(self, limit_ns: int) -> None:
+        _check(lib().fv_selftest_expired_wait(self.ctx, int(limit_ns), _stream()), "fv_selftest_expired_wait")
 
     def kv_views(self, block: int):
         """(K [B_max, cap, C], V^T [B_max, C, cap]) bf16 views of one block's KV cache."""

@@ -48,6 +48,7 @@ struct fv_ctx {
 
 namespace fv {
 const fv_config* ctx_config(const fv_ctx* ctx) { return &ctx->cfg; }
+int32_t* ctx_status_word(const fv_ctx* ctx) { return ctx->status; }
 }  // namespace fv
 
 namespace {
@@ -130,6 +131,7 @@ const char* fv_status_string(fv_status s) {
     case FV_ERR_UNSUPPORTED: return "unsupported shape";
     case FV_ERR_CUDA: return "CUDA error";
     case FV_ERR_TIMEOUT: return "device-side wait expired";
+    case FV_ERR_DEVICE_DATA: return "a kernel met an index outside its range";
   }
   return "unknown";
 }
@@ -179,12 +181,13 @@ fv_status fv_restore(const void* cache_prev_dev, int32_t hc, int32_t wc, const v
 }
 
 fv_status fv_gather_ln(const float* x_dev, const int32_t* idx_dev, int32_t B, int32_t n_tokens, int32_t k, int32_t C,
-                       const float* sigma_dev, const float* beta_dev, int32_t mod_stride, void* a_out_dev, void* stream) {
+                       const float* sigma_dev, const float* beta_dev, int32_t mod_stride, void* a_out_dev, int32_t* status_dev,
+                       void* stream) {
   if (!x_dev || !a_out_dev || B <= 0 || n_tokens <= 0 || k <= 0 || k > n_tokens || C <= 0 || (C % 4)) return FV_ERR_INVALID_ARG;
   if ((sigma_dev == nullptr) != (beta_dev == nullptr)) return FV_ERR_INVALID_ARG;
   if (C > 2048) return FV_ERR_UNSUPPORTED;
   if (!idx_dev && k != n_tokens) return FV_ERR_INVALID_ARG;
-  return cuda_status(launch_gather_ln(x_dev, idx_dev, B, n_tokens, k, C, sigma_dev, beta_dev, mod_stride, a_out_dev,
+  return cuda_status(launch_gather_ln(x_dev, idx_dev, B, n_tokens, k, C, sigma_dev, beta_dev, mod_stride, a_out_dev, status_dev,
                                       static_cast<cudaStream_t>(stream)));
 }
 
@@ -473,9 +476,14 @@ fv_status fv_device_status(fv_ctx* ctx, int32_t* code_host, void* stream) {
   if (code != 0) {
     cudaMemsetAsync(ctx->status, 0, 4, st);
     cudaStreamSynchronize(st);
-    return FV_ERR_TIMEOUT;
+    return code >= 100 ? FV_ERR_TIMEOUT : FV_ERR_DEVICE_DATA;
   }
   return FV_OK;
+}
+
+fv_status fv_selftest_expired_wait(fv_ctx* ctx, uint64_t limit_ns, void* stream) {
+  if (!ctx || limit_ns == 0 || limit_ns > 1000000000ull) return FV_ERR_INVALID_ARG;
+  return cuda_status(launch_expired_wait(ctx->status, limit_ns, static_cast<cudaStream_t>(stream)));
 }
 
 fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t scale_idx, double keep_ratio, float* out_dev,
@@ -540,7 +548,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
     }
     if (e != cudaSuccess) return FV_ERR_CUDA;
     if (idx_trace_dev && cudaMemcpyAsync(idx_trace_dev, idx, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return FV_ERR_CUDA;
-    if (launch_gather_rows(tokens_dev, idx, B, n, k, C, ctx->xc, st) != cudaSuccess) return FV_ERR_CUDA;
+    if (launch_gather_rows(tokens_dev, idx, B, n, k, C, ctx->xc, ctx->status, st) != cudaSuccess) return FV_ERR_CUDA;
     xr = ctx->xc;
     nr = k;
     step_idx = idx;
@@ -550,6 +558,14 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   bool have_partials = false;
   const bool selecting = sub_pruned && !forced_idx_dev;
   if (selecting && cudaMemsetAsync(ctx->sel_ws, 0, select_ticket_bytes(B), st) != cudaSuccess) return FV_ERR_CUDA;
+
+  // A failed launch between the fork to the side stream and the join must not leave the side stream's part of the
+  // restoration unordered against whatever the caller does next with x, the selection scratch or the context.
+  bool forked = false;
+  struct JoinGuard {
+    cudaStream_t st; cudaEvent_t ev; const bool& forked;
+    ~JoinGuard() { if (forked) cudaStreamWaitEvent(st, ev, 0); }
+  } join_guard{st, ctx->ev_join, forked};
 
   for (int l = 0; l < c.L && s == FV_OK; ++l) {
     const float* mod = ctx->mod + (size_t)l * c.B_max * 6 * C;
@@ -585,9 +601,11 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
         e = launch_restore_residual(x, ctx->y_buf, cache_sub, ctx->inv, gamma, mod_stride, B, k, h, w, hc, wc, C,
                                     more ? ctx->sel_ws : nullptr, 1, c.interp_mode, ctx->side);
-        if (e != cudaSuccess || cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) { s = FV_ERR_CUDA; break; }
+        const cudaError_t e_join = cudaEventRecord(ctx->ev_join, ctx->side);   // recorded even if the launch failed
+        forked = e_join == cudaSuccess;
+        if (e != cudaSuccess || e_join != cudaSuccess) { s = FV_ERR_CUDA; break; }
       }
-      e = launch_gather_ln(xr, idx, B, nr, k, C, sigma, beta, mod_stride, ctx->a_buf, st);
+      e = launch_gather_ln(xr, idx, B, nr, k, C, sigma, beta, mod_stride, ctx->a_buf, ctx->status, st);
       if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
       // ---- branch on the compact rows
       GemmArgs g{};
@@ -636,6 +654,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         s = launch_gemm(o, st);
         if (s != FV_OK) break;
         if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
+        forked = false;
         e = launch_restore_residual(x, ctx->y_buf, cache_sub, ctx->inv, gamma, mod_stride, B, k, h, w, hc, wc, C,
                                     more ? ctx->sel_ws : nullptr, 2, c.interp_mode, st);
         if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }

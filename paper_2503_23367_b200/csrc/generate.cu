@@ -10,11 +10,10 @@
 #include <vector>
 
 #include "internal.h"
+#include "sm100.cuh"   // the device status codes
 
 namespace fv {
 namespace {
-
-constexpr int DEV_BAD_TOKEN_ID = 40;   // status code: a token id outside [0, V)
 
 // ---- ids[r] = argmax_v (logits[r, v] + tau * noise[r, v]), lowest v on ties; one warp per row ----
 __global__ void __launch_bounds__(256) argmax_rows_kernel(const float4* __restrict__ logits, const float4* __restrict__ noise, float tau,
@@ -234,7 +233,7 @@ fv_status fv_head_tokens(const float* y_dev, int32_t B, int32_t n, int32_t C, co
   float* logits = logits_out_dev ? logits_out_dev : reinterpret_cast<float*>(ws + l.logits);
   // the K-split arrival counters must start at zero (the GEMM leaves them zero)
   if (cudaMemsetAsync(ws + l.splitk, 0, gemm_splitk_ticket_bytes(), st) != cudaSuccess) return FV_ERR_CUDA;
-  fv_status s = fv_gather_ln(y_dev, nullptr, B, n, n, C, mod_head_dev, mod_head_dev + C, 2 * C, ws + l.a, stream);
+  fv_status s = fv_gather_ln(y_dev, nullptr, B, n, n, C, mod_head_dev, mod_head_dev + C, 2 * C, ws + l.a, status_dev, stream);
   if (s != FV_OK) return s;
   s = fv_gemm_bf16(ws + l.a, w_head_dev, b_head_dev, rows, V, C, EPI_F32, logits, nullptr, nullptr, 0, n, status_dev, ws + l.splitk,
                    gemm_splitk_ws_bytes(), stream);
@@ -294,14 +293,15 @@ fv_status fv_generate(fv_ctx* ctx, const fv_generator* gen, const float* start_d
   if (workspace_bytes < l.total) return FV_ERR_CAPACITY;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* ws = static_cast<char*>(workspace_dev);
-  int32_t* status = reinterpret_cast<int32_t*>(ws + l.status);
+  // the head GEMM and Eq. 2 report into the context's own status word, which fv_device_status reads
+  int32_t* status = ctx_status_word(ctx);
   float* x = reinterpret_cast<float*>(ws + l.x);
   float* y = reinterpret_cast<float*>(ws + l.y);
   float* r[2] = {reinterpret_cast<float*>(ws + l.r0), reinterpret_cast<float*>(ws + l.r1)};
   const size_t head_bytes = l.total - l.head;
   fv_status s = fv_reset(ctx);
   if (s != FV_OK) return s;
-  if (cudaMemsetAsync(status, 0, 256, st) != cudaSuccess) return FV_ERR_CUDA;
+  (void)st;
   const int K = c.n_steps;
   size_t id_off = 0;
   for (int k = 0; k < K; ++k) {

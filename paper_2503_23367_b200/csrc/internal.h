@@ -70,8 +70,12 @@ cudaError_t launch_inv_fill(int B, int n, int32_t* inv, cudaStream_t st);  // ev
 cudaError_t select_init();  // one-time function attributes
 
 // ---- rows.cu : gather + LayerNorm + modulate, restore (+ gate and residual) ----------------------
+// status (all gathers): device status word that receives DEV_BAD_ROW_INDEX when an index lies outside [0, n) (the
+// index is clamped, so the read stays inside the map), or null.
 cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
-                             const float* beta, int mod_stride, void* a_out, cudaStream_t st);
+                             const float* beta, int mod_stride, void* a_out, int32_t* status, cudaStream_t st);
+// A wait nobody ends: one warp waits on an mbarrier without arrivals for limit_ns, then writes DEV_TIMEOUT_SELFTEST.
+cudaError_t launch_expired_wait(int32_t* status, unsigned long long limit_ns, cudaStream_t st);
 // colsum_ws: null, or the selection workspace that receives the column sums of the updated x.
 // part: 0 = every row; 1 = the rows that were not kept; 2 = the kept rows (and the fold of the column sums).
 // interp_mode (all restore launchers): 0 nearest, 1 bilinear with half-pixel centres.
@@ -81,7 +85,7 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
 cudaError_t rows_init();               // one-time function attributes
 void restore_force_fold(int mode);     // test hook: 0 by shape, 1 fold through global memory, 2 fold inside clusters
 // Per-step granularity: fp32 gather of the kept rows, and fp32 restoration of the step's output map.
-cudaError_t launch_gather_rows(const float* x, const int32_t* idx, int B, int n, int k, int C, float* out, cudaStream_t st);
+cudaError_t launch_gather_rows(const float* x, const int32_t* idx, int B, int n, int k, int C, float* out, int32_t* status, cudaStream_t st);
 cudaError_t launch_restore_rows_f32(const float* cache, int hc, int wc, const float* pivots, const int32_t* inv, int B, int k,
                                     int h, int w, int C, float* out, int interp_mode, cudaStream_t st);
 cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* pivots, const int32_t* inv, int B,
@@ -149,4 +153,5 @@ bool make_tmap_bf16_2d(void* tmap_out, const void* base, uint64_t rows, uint64_t
 struct fv_ctx;
 namespace fv {
 const fv_config* ctx_config(const fv_ctx* ctx);
+int32_t* ctx_status_word(const fv_ctx* ctx);   // the device status word in the context's workspace
 }  // namespace fv

@@ -25,14 +25,18 @@ constexpr int kMaxVec = 16;  // float4 per lane -> C <= 2048
 __global__ void __launch_bounds__(256) gather_ln_kernel(const float4* __restrict__ x, const int32_t* __restrict__ idx, int n,
                                                         int k, int C4, const float* __restrict__ sigma,
                                                         const float* __restrict__ beta, int mod_stride,
-                                                        uint2* __restrict__ a_out) {
+                                                        uint2* __restrict__ a_out, int32_t* status) {
   extern __shared__ float4 s_mod[];  // sigma [C4] then beta [C4]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.y, j = blockIdx.x * 8 + warp;
   const bool live = j < k;
   pdl_trigger();
   pdl_wait();
-  const int t = live ? (idx ? __ldg(idx + (size_t)b * k + j) : j) : 0;
+  int t = live ? (idx ? __ldg(idx + (size_t)b * k + j) : j) : 0;
+  if (t < 0 || t >= n) {   // a caller's index outside the map: stay inside it and say so
+    if (status && lane == 0) atomicCAS(status, 0, DEV_BAD_ROW_INDEX);
+    t = min(max(t, 0), n - 1);
+  }
   if (sigma) {
     const float4* sg = reinterpret_cast<const float4*>(sigma + (size_t)b * mod_stride);
     const float4* bt = reinterpret_cast<const float4*>(beta + (size_t)b * mod_stride);
@@ -254,13 +258,17 @@ __global__ void __launch_bounds__(256) restore_bf16_kernel(const uint4* __restri
 // Per-step granularity: compact copy of the kept rows of the fp32 token map (Algorithm 1's gather).
 // grid (ceil(k / 8), B): one warp per kept row.
 __global__ void __launch_bounds__(256) gather_rows_kernel(const float4* __restrict__ x, const int32_t* __restrict__ idx, int n,
-                                                          int k, int C4, float4* __restrict__ out) {
+                                                          int k, int C4, float4* __restrict__ out, int32_t* status) {
   pdl_trigger();
   pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.y, j = blockIdx.x * 8 + warp;
   if (j >= k) return;
-  const int t = __ldg(idx + (size_t)b * k + j);
+  int t = __ldg(idx + (size_t)b * k + j);
+  if (t < 0 || t >= n) {
+    if (status && lane == 0) atomicCAS(status, 0, DEV_BAD_ROW_INDEX);
+    t = min(max(t, 0), n - 1);
+  }
   const float4* src = x + ((size_t)b * n + t) * C4;
   float4* dst = out + ((size_t)b * k + j) * C4;
   for (int c4 = lane; c4 < C4; c4 += 32) dst[c4] = __ldg(src + c4);
@@ -553,7 +561,19 @@ __global__ void rope_table_kernel(float2* __restrict__ table, int h, int w, int 
     table[i] = make_float2((float)cs, (float)sn);
   }
 }
+// One warp waits on an mbarrier that nothing arrives at: the wait expires after limit_ns and the code is recorded.
+__global__ void expired_wait_kernel(int32_t* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+  __syncwarp();
+  if (threadIdx.x == 0 && !mbar_wait(&bar, 0, limit_ns)) atomicCAS(status, 0, DEV_TIMEOUT_SELFTEST);
+}
 }  // namespace
+
+cudaError_t launch_expired_wait(int32_t* status, unsigned long long limit_ns, cudaStream_t st) {
+  expired_wait_kernel<<<1, 32, 0, st>>>(status, limit_ns);
+  return cudaGetLastError();
+}
 
 // How the kept-row part of a restoration folds its column sums: 0 by shape, 1 global memory, 2 clusters.
 static int g_fold_mode = 0;
@@ -566,11 +586,11 @@ cudaError_t rows_init() {
 }
 
 cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
-                             const float* beta, int mod_stride, void* a_out, cudaStream_t st) {
+                             const float* beta, int mod_stride, void* a_out, int32_t* status, cudaStream_t st) {
   const int rows = B * k;
   LaunchScope scope(KC_GATHER_LN, 1, (double)rows * C * 6.0, (double)rows * C * 6.0, st);
   return launch_pdl(gather_ln_kernel, dim3((k + 7) / 8, B), dim3(256), sigma ? (size_t)C * 8 : 0, st, reinterpret_cast<const float4*>(x),
-                    idx, n, k, C / 4, sigma, beta, mod_stride, reinterpret_cast<uint2*>(a_out));
+                    idx, n, k, C / 4, sigma, beta, mod_stride, reinterpret_cast<uint2*>(a_out), status);
 }
 
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv, const float* gamma,
@@ -623,10 +643,10 @@ cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* p
                     reinterpret_cast<const uint4*>(pivots), inv, h * w, k, h, w, C / 8, reinterpret_cast<uint4*>(out), rows);
 }
 
-cudaError_t launch_gather_rows(const float* x, const int32_t* idx, int B, int n, int k, int C, float* out, cudaStream_t st) {
+cudaError_t launch_gather_rows(const float* x, const int32_t* idx, int B, int n, int k, int C, float* out, int32_t* status, cudaStream_t st) {
   LaunchScope scope(KC_GATHER_LN, 1, (double)B * k * C * 8.0, (double)B * k * C * 8.0, st);
   return launch_pdl(gather_rows_kernel, dim3((k + 7) / 8, B), dim3(256), 0, st, reinterpret_cast<const float4*>(x), idx, n, k, C / 4,
-                    reinterpret_cast<float4*>(out));
+                    reinterpret_cast<float4*>(out), status);
 }
 
 cudaError_t launch_restore_rows_f32(const float* cache, int hc, int wc, const float* pivots, const int32_t* inv, int B, int k,

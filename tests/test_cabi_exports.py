@@ -47,7 +47,7 @@ def test_argument_validation_happens_before_any_launch(lib):
     # NULL pointers and bad sizes are rejected on the host (no CUDA call is made)
     assert lib.fv_prune_select(None, 1, 2, 2, 8, 0.5, None, None, None, None, None, None, 0, None) == 1
     assert lib.fv_restore(None, 1, 1, None, None, 1, 1, 1, 1, 8, None, None, 0, None) == 1
-    assert lib.fv_gather_ln(None, None, 1, 4, 4, 8, None, None, 0, None, None) == 1
+    assert lib.fv_gather_ln(None, None, 1, 4, 4, 8, None, None, 0, None, None, None) == 1
     assert lib.fv_var_step(None, None, 1, 0, 1.0, None, None, None, None) == 1
     assert lib.fv_reset(None) == 1
     cfg = fv.fv_config(2, 256, 4, 4, 0, 1, 0, None, None, -1, 64)

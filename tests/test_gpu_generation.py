@@ -61,7 +61,7 @@ def test_residual_accumulate_flags_bad_ids():
     st = torch.zeros(1, dtype=torch.int32, device=DEV)
     ids = torch.tensor([[0, 9, -1, 7]], dtype=torch.int32, device=DEV)
     out = fv.fv_residual_accumulate(ids, 2, 2, cb, status=st).cpu().numpy()
-    assert int(st.item()) != 0
+    assert int(st.item()) == 40
     np.testing.assert_array_equal(out[0, 1], cb[7].cpu().numpy())   # clamped, not read out of bounds
     np.testing.assert_array_equal(out[0, 2], cb[0].cpu().numpy())
 

@@ -459,6 +459,48 @@ def test_state_and_argument_errors():
     ctx.close()
 
 
+def test_an_expired_device_wait_is_reported_not_fatal():
+    """The library's kernels never wait without a limit: a wait that nothing ends gives up after its limit, leaves a
+    code in the context's status word and the kernel returns normally.  The self-test kernel waits 50 microseconds
+    on a barrier nobody completes; fv_device_status must report FV_ERR_TIMEOUT with its code, clear the word, and
+    the context must go on working (a full schedule afterwards still matches the run before it)."""
+    wl = I.WORKLOADS["tiny"]
+    mt = I.model_tensors(wl)
+    xs = [I.step_input(wl, i) for i in range(len(wl.sides))]
+    ctx = make_ctx(wl, mt)
+    before, _ = gpu_schedule(ctx, wl, xs)
+    ctx.selftest_expired_wait(50_000)
+    assert ctx.device_status_pair() == (6, 105)          # FV_ERR_TIMEOUT, the self-test's code
+    assert ctx.device_status_pair() == (0, 0)            # cleared by the read
+    with pytest.raises(fv.FvError) as e:
+        ctx.selftest_expired_wait(0)                     # a limit is mandatory
+    assert e.value.code == 1
+    after, _ = gpu_schedule(ctx, wl, xs)
+    for a, b in zip(before, after):
+        assert np.array_equal(a, b)
+    ctx.close()
+
+
+def test_an_index_outside_the_map_is_clamped_and_reported():
+    """A kept-row index outside [0, n) (a caller's mistake in forced-index mode) must not become a read outside the
+    token map: the gather clamps it into the map and leaves code 41 in the status word."""
+    B, n, C, k = 2, 50, 256, 4
+    x = I.normal(321, (B, n, C))
+    idx = np.array([[0, 7, 49, 50], [-3, 2, 10, 4999]], dtype=np.int32)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    got = fv.fv_gather_ln(torch.from_numpy(x).to(DEV), torch.from_numpy(idx).to(DEV), None, None, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 41
+    clamped = np.clip(idx, 0, n - 1).astype(np.int64)
+    ref = O.layernorm(O.pts_gather(x.astype(np.float64), clamped))
+    err, cos = per_token_errors(got.float().cpu().numpy(), ref)
+    assert err <= MAX_ABS and cos >= MIN_COS
+    status.zero_()
+    fv.fv_gather_ln(torch.from_numpy(x).to(DEV), torch.from_numpy(clamped.astype(np.int32)).to(DEV), None, None, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+
+
 def test_step_with_host_buffers_equals_the_device_call():
     """fv_var_step_host (pinned host token maps in, host result out) gives the bits of fv_var_step."""
     wl = I.WORKLOADS["tiny"]

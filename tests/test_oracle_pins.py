@@ -13,6 +13,7 @@ import torch.nn.functional as F
 
 from oracle import fastvar_oracle as O
 from paper_2503_23367_b200 import inputs as I
+from tests.helpers import oracle_weights
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 rng = np.random.default_rng(1234)
@@ -267,15 +268,6 @@ def _tiny_model(L=2, C=32, H=4, B=2, sides=(1, 2, 3, 4, 6), cross_len=0, seed=7)
                     cross_len=cross_len, seed=seed)
     mt = I.model_tensors(wl, w_std=0.15)
     return wl, mt, oracle_weights(mt)
-
-
-def oracle_weights(mt):
-    f = lambda lst: [I.bf16_bits_to_f32(a).astype(np.float64) for a in lst]
-    w = {k: f(getattr(mt, k)) for k in ("w_qkv", "b_qkv", "w_o", "b_o", "w_fc1", "b_fc1", "w_fc2", "b_fc2",
-                                          "w_q_x", "w_kv_x", "w_o_x")}
-    w["mod"] = mt.mod.astype(np.float64)
-    w["text"] = None if mt.text is None else I.bf16_bits_to_f32(mt.text).astype(np.float64)
-    return w
 
 
 def _torch_block_causal_forward(wl, w, xs):

@@ -66,3 +66,28 @@ def test_two_gloo_ranks_report_the_slowest_time_and_all_tokens():
         assert abs(rate - 820.0 * 5 / 0.5) < 1e-9               # all ranks' tokens over the slowest time
         assert owned == [1, 1, 1, 1, 1]                         # each image owned exactly once
     assert got[0][4] != got[1][4]
+
+
+def test_bench_started_plainly_with_gpus_n_launches_n_ranks(monkeypatch):
+    """`python bench.py --gpus N` (no launcher around it) must itself start N ranks, one per GPU, on 127.0.0.1 and
+    hand them its own arguments; under a launcher (WORLD_SIZE set) it must not."""
+    import importlib
+    import subprocess
+    import sys
+
+    bench = importlib.import_module("bench")
+    seen = {}
+
+    def fake_call(cmd, *a, **k):
+        seen["cmd"] = cmd
+        return 0
+
+    monkeypatch.setattr(subprocess, "call", fake_call)
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4", "--steps", "2", "--warmup", "3"])
+    with pytest.raises(SystemExit) as e:
+        bench.main()
+    assert e.value.code == 0
+    cmd = seen["cmd"]
+    assert "torch.distributed.run" in cmd and "--nproc-per-node=4" in cmd and "127.0.0.1" in cmd
+    assert cmd[-6:] == ["--gpus", "4", "--steps", "2", "--warmup", "3"] and cmd[-7].endswith("bench.py")
