@@ -29,7 +29,10 @@ struct fv_ctx {
   int32_t* status = nullptr;
   char *a_buf = nullptr, *q_buf = nullptr, *o_buf = nullptr, *y_buf = nullptr, *h_buf = nullptr;
   int32_t *idx = nullptr, *inv = nullptr;
+  int32_t *idx2 = nullptr, *inv2 = nullptr;   // second set: the fused selection reads the previous sublayer's indices while it writes the next
   void* sel_ws = nullptr;
+  void* fsel_ws = nullptr;                    // scratch of the fused selection (arrival counts, kept-row partial sums)
+  unsigned int fsel_done = 0, fsel_epoch = 0; // what its grid-wide waits compare against (grow with every launch)
   void* splitk_ws = nullptr;
   void* attn_ws = nullptr;
   cudaStream_t side = nullptr;           // the unkept rows of a restoration run here, beside the sublayer's branch
@@ -53,6 +56,8 @@ int32_t* ctx_status_word(const fv_ctx* ctx) { return ctx->status; }
 
 namespace {
 
+bool g_step_fused = true;   // test / profiling hook: false = one launch each for selection, gather and kept-row restoration
+
 std::once_flag g_init_once;
 cudaError_t g_init_err = cudaSuccess;
 
@@ -69,7 +74,7 @@ cudaError_t ensure_init() {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 struct Layout {
-  size_t status, a, q, o, y, hbuf, idx, inv, sel, splitk, attn, xc, rope, total;
+  size_t status, a, q, o, y, hbuf, idx, inv, idx2, inv2, sel, fsel, splitk, attn, xc, rope, total;
 };
 
 int max_tokens(const fv_config* c) {
@@ -104,7 +109,10 @@ Layout workspace_layout(const fv_config* c) {
   l.hbuf = take(M * F * 2);
   l.idx = take(M * 4);
   l.inv = take(M * 4);
+  l.idx2 = take(M * 4);
+  l.inv2 = take(M * 4);
   l.sel = take(select_workspace_bytes(c->B_max, max_tokens(c), c->C));
+  l.fsel = take(select_fused_ws_bytes(c->B_max, c->C));
   l.splitk = take(gemm_splitk_ws_bytes());
   l.attn = take(attention_ws_bytes());
   l.xc = take(c->granularity == 1 ? M * C * 4 : 0);
@@ -232,6 +240,11 @@ fv_status fv_prune_select_workspace_layout(int32_t B, int32_t n_tokens, int32_t 
   const SelectWs w = select_ws_carve(origin, B, n_tokens, C);
   *offset_host = (size_t)(reinterpret_cast<char*>(w.group_partial) - origin);
   *n_partials_host = w.ngroups;
+  return FV_OK;
+}
+
+fv_status fv_step_force_unfused(int32_t on) {
+  g_step_fused = on == 0;
   return FV_OK;
 }
 
@@ -363,7 +376,10 @@ fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, v
   c->h_buf = c->ws + lay.hbuf;
   c->idx = reinterpret_cast<int32_t*>(c->ws + lay.idx);
   c->inv = reinterpret_cast<int32_t*>(c->ws + lay.inv);
+  c->idx2 = reinterpret_cast<int32_t*>(c->ws + lay.idx2);
+  c->inv2 = reinterpret_cast<int32_t*>(c->ws + lay.inv2);
   c->sel_ws = c->ws + lay.sel;
+  c->fsel_ws = c->ws + lay.fsel;
   c->splitk_ws = c->ws + lay.splitk;
   c->attn_ws = c->ws + lay.attn;
   c->xc = reinterpret_cast<float*>(c->ws + lay.xc);
@@ -381,6 +397,7 @@ fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, v
   // Never-written KV rows must read as zeros (they meet zero probabilities in P*V).
   if (!rope_ok || cudaMemset(kv_dev, 0, fv_kv_bytes(cfg)) != cudaSuccess || cudaMemset(c->status, 0, 256) != cudaSuccess ||
       cudaMemset(c->sel_ws, 0, select_ticket_bytes(cfg->B_max)) != cudaSuccess ||
+      cudaMemset(c->fsel_ws, 0, select_fused_sync_bytes(cfg->B_max)) != cudaSuccess ||
       cudaMemset(c->splitk_ws, 0, gemm_splitk_ticket_bytes()) != cudaSuccess ||
       cudaMemset(c->attn_ws, 0, attention_ws_ticket_bytes()) != cudaSuccess ||
       cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
@@ -475,6 +492,12 @@ fv_status fv_device_status(fv_ctx* ctx, int32_t* code_host, void* stream) {
   if (code_host) *code_host = code;
   if (code != 0) {
     cudaMemsetAsync(ctx->status, 0, 4, st);
+    // a kernel that gave up may have left arrival counts half-way: every counter starts afresh
+    cudaMemsetAsync(ctx->sel_ws, 0, select_ticket_bytes(ctx->cfg.B_max), st);
+    cudaMemsetAsync(ctx->fsel_ws, 0, select_fused_sync_bytes(ctx->cfg.B_max), st);
+    cudaMemsetAsync(ctx->splitk_ws, 0, gemm_splitk_ticket_bytes(), st);
+    cudaMemsetAsync(ctx->attn_ws, 0, attention_ws_ticket_bytes(), st);
+    ctx->fsel_done = 0; ctx->fsel_epoch = 0;
     cudaStreamSynchronize(st);
     return code >= 100 ? FV_ERR_TIMEOUT : FV_ERR_DEVICE_DATA;
   }
@@ -558,6 +581,13 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   bool have_partials = false;
   const bool selecting = sub_pruned && !forced_idx_dev;
   if (selecting && cudaMemsetAsync(ctx->sel_ws, 0, select_ticket_bytes(B), st) != cudaSuccess) return FV_ERR_CUDA;
+  // Free-running selections take one launch each: the previous sublayer's kept-row restoration, the selection and the
+  // gather + LayerNorm of the newly kept rows (select_fused_kernel).  The kept rows of a sublayer are then restored
+  // by the NEXT sublayer's launch; only the last sublayer of the step restores its own.
+  const bool fused = selecting && g_step_fused && select_fused_supported(B, n, C);
+  bool pending = false;                 // a kept-row restoration waits for the next fused selection
+  const float* pending_gamma = nullptr;
+  int flip = 0;
 
   // A failed launch between the fork to the side stream and the join must not leave the side stream's part of the
   // restoration unordered against whatever the caller does next with x, the selection scratch or the context.
@@ -580,12 +610,12 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         if (forced_idx_dev) {
           idx = forced_idx_dev + trace_off;
           e = launch_inv_from_idx(idx, B, k, n, ctx->inv, st);
-        } else {
+        } else if (!fused) {
           idx = ctx->idx;
           e = launch_select(x, B, n, C, k, ctx->idx, ctx->inv, nullptr, nullptr, ctx->sel_ws, have_partials, st);
         }
         if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
-        if (idx_trace_dev && cudaMemcpyAsync(idx_trace_dev + trace_off, idx, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+        if (!fused && idx_trace_dev && cudaMemcpyAsync(idx_trace_dev + trace_off, idx, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
           s = FV_ERR_CUDA; break;
         }
       }
@@ -594,19 +624,46 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
       const float* beta = kind == 0 ? mod + C : (kind == 2 ? mod + 4 * C : nullptr);
       const float* gamma = kind == 0 ? mod + 2 * C : (kind == 2 ? mod + 5 * C : nullptr);
       const bool more = selecting && !(l == c.L - 1 && sub == ctx->n_sub - 1);
+      int32_t* inv_cur = ctx->inv;
+      if (fused) {
+        int32_t* idx_cur = flip ? ctx->idx2 : ctx->idx;
+        inv_cur = flip ? ctx->inv2 : ctx->inv;
+        FusedSelect f{};
+        f.x = x; f.B = B; f.n = n; f.C = C; f.k = k; f.mod_stride = mod_stride;
+        f.sel_ws = ctx->sel_ws; f.fused_ws = ctx->fsel_ws; f.idx = idx_cur; f.inv = inv_cur;
+        f.sigma = sigma; f.beta = beta; f.a_out = ctx->a_buf; f.status = ctx->status;
+        f.done_total = &ctx->fsel_done; f.epoch = &ctx->fsel_epoch;
+        if (pending) {
+          // the rows of the previous sublayer that were not kept (side stream) must be in x, and their sums folded
+          if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
+          forked = false;
+          f.y = ctx->y_buf; f.idx_prev = flip ? ctx->idx : ctx->idx2; f.gamma_prev = pending_gamma;
+        } else if (launch_colsum(x, B, n, C, ctx->sel_ws, st) != cudaSuccess) {   // first sublayer of the step: sum the map itself
+          s = FV_ERR_CUDA; break;
+        }
+        if (launch_select_fused(f, st) != cudaSuccess) { s = FV_ERR_CUDA; break; }
+        pending = false;
+        idx = idx_cur;
+        flip ^= 1;
+        if (idx_trace_dev && cudaMemcpyAsync(idx_trace_dev + trace_off, idx, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+          s = FV_ERR_CUDA; break;
+        }
+      }
       if (sub_pruned) {
         // Cached Token Restoration of the rows that were NOT kept needs only the selection and the cache:
         // it runs on the side stream while the gather and the branch below work on the kept rows (the two
         // touch disjoint rows of x).
         if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
-        e = launch_restore_residual(x, ctx->y_buf, cache_sub, ctx->inv, gamma, mod_stride, B, k, h, w, hc, wc, C,
-                                    more ? ctx->sel_ws : nullptr, 1, c.interp_mode, ctx->side);
+        e = launch_restore_residual(x, ctx->y_buf, cache_sub, inv_cur, gamma, mod_stride, B, k, h, w, hc, wc, C,
+                                    more ? ctx->sel_ws : nullptr, (fused && more) ? 3 : 1, c.interp_mode, ctx->side);
         const cudaError_t e_join = cudaEventRecord(ctx->ev_join, ctx->side);   // recorded even if the launch failed
         forked = e_join == cudaSuccess;
         if (e != cudaSuccess || e_join != cudaSuccess) { s = FV_ERR_CUDA; break; }
       }
-      e = launch_gather_ln(xr, idx, B, nr, k, C, sigma, beta, mod_stride, ctx->a_buf, ctx->status, st);
-      if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
+      if (!fused) {
+        e = launch_gather_ln(xr, idx, B, nr, k, C, sigma, beta, mod_stride, ctx->a_buf, ctx->status, st);
+        if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
+      }
       // ---- branch on the compact rows
       GemmArgs g{};
       g.status = ctx->status; g.rows_per_image = k; g.mod_stride = mod_stride; g.splitk_ws = ctx->splitk_ws;
@@ -653,9 +710,14 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         o.epilogue = EPI_BF16; o.out = ctx->y_buf;
         s = launch_gemm(o, st);
         if (s != FV_OK) break;
+        if (fused && more) {     // the next sublayer's launch restores these kept rows
+          pending = true;
+          pending_gamma = gamma;
+          continue;
+        }
         if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
         forked = false;
-        e = launch_restore_residual(x, ctx->y_buf, cache_sub, ctx->inv, gamma, mod_stride, B, k, h, w, hc, wc, C,
+        e = launch_restore_residual(x, ctx->y_buf, cache_sub, inv_cur, gamma, mod_stride, B, k, h, w, hc, wc, C,
                                     more ? ctx->sel_ws : nullptr, 2, c.interp_mode, st);
         if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
         have_partials = more;

@@ -11,8 +11,8 @@
 namespace fv {
 
 // Called by ALL threads of the CTA after they have stored their part of chunk partial (b, chunk).
-// Returns with the group partial written if this CTA was the last of its group.
-__device__ __forceinline__ void fold_group_partials(int b, int chunk, int nchunks, int group, int ngroups, int C4,
+// Returns true, with the group partial written, if this CTA was the last of its group.
+__device__ __forceinline__ bool fold_group_partials(int b, int chunk, int nchunks, int group, int ngroups, int C4,
                                                     const float4* __restrict__ chunk_partial,
                                                     float4* __restrict__ group_partial, unsigned int* tickets) {
   __shared__ int s_last;
@@ -28,7 +28,7 @@ __device__ __forceinline__ void fold_group_partials(int b, int chunk, int nchunk
     if (s_last) *t = 0u;  // every member has arrived: leave the counter ready for the next launch
   }
   __syncthreads();
-  if (!s_last) return;
+  if (!s_last) return false;
   __threadfence();
   const int first = g * group;
   const int last = min(nchunks, first + group);
@@ -49,6 +49,7 @@ __device__ __forceinline__ void fold_group_partials(int b, int chunk, int nchunk
     }
     group_partial[((size_t)b * ngroups + g) * C4 + c4] = acc;
   }
+  return true;
 }
 
 }  // namespace fv

@@ -65,6 +65,24 @@ SelectWs select_ws_carve(void* workspace, int B, int n, int C);
 // launch_restore_residual), so the column-sum pass is skipped.
 cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* idx, int32_t* inv, float* score,
                           int32_t* near_tie, void* workspace, bool have_partials, cudaStream_t st);
+// The selection of a wrapped sublayer inside a scale step, in one launch with what surrounds it on the kept rows:
+// the previous sublayer's kept-row restoration before it (y != null) and the gather + LayerNorm + modulation of the
+// newly kept rows after it.  sel_ws holds the column sums of the rows the kernel does not update itself (left there
+// by the restoration of the rows that were not kept, or by launch_colsum for a map nothing has restored yet).
+struct FusedSelect {
+  float* x; int B, n, C, k;
+  const void* y; const int32_t* idx_prev; const float* gamma_prev; int mod_stride;   // y null: no kept rows to restore
+  void* sel_ws; void* fused_ws;
+  int32_t* idx; int32_t* inv;
+  const float* sigma; const float* beta; void* a_out;
+  int32_t* status;
+  unsigned int* done_total; unsigned int* epoch;   // host counters of the context: what the kernel's waits compare against
+};
+size_t select_fused_ws_bytes(int B, int C);
+size_t select_fused_sync_bytes(int B);            // leading bytes of fused_ws that must be zero before first use
+bool select_fused_supported(int B, int n, int C);
+cudaError_t launch_select_fused(const FusedSelect& f, cudaStream_t st);
+cudaError_t launch_colsum(const float* x, int B, int n, int C, void* workspace, cudaStream_t st);   // column sums of a map -> sel_ws
 cudaError_t launch_inv_from_idx(const int32_t* idx, int B, int k, int n, int32_t* inv, cudaStream_t st);
 cudaError_t launch_inv_fill(int B, int n, int32_t* inv, cudaStream_t st);  // every token unkept (-1)
 cudaError_t select_init();  // one-time function attributes
@@ -77,7 +95,8 @@ cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, i
 // A wait nobody ends: one warp waits on an mbarrier without arrivals for limit_ns, then writes DEV_TIMEOUT_SELFTEST.
 cudaError_t launch_expired_wait(int32_t* status, unsigned long long limit_ns, cudaStream_t st);
 // colsum_ws: null, or the selection workspace that receives the column sums of the updated x.
-// part: 0 = every row; 1 = the rows that were not kept; 2 = the kept rows (and the fold of the column sums).
+// part: 0 = every row; 1 = the rows that were not kept; 2 = the kept rows (and the fold of the column sums);
+// 3 = the rows that were not kept, their column sums folded (the kept rows are left to the next fused selection).
 // interp_mode (all restore launchers): 0 nearest, 1 bilinear with half-pixel centres.
 cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv,
                                     const float* gamma, int mod_stride, int B, int k, int h, int w, int hc, int wc,

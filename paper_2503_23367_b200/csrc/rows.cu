@@ -164,7 +164,9 @@ __device__ __forceinline__ void bf16x8_to_float(const uint4& p, float (&f)[8]) {
 // `part` splits the work so that the bulk of it can run beside the sublayer's GEMMs and attention:
 //   0 : every row;  1 : only the rows that were NOT kept (they depend on the selection and the cache alone:
 //   column sums start at zero and are left as the chunk partial);  2 : only the kept rows (after the
-//   branch has produced y: column sums continue from the chunk partial of part 1, then the group fold).
+//   branch has produced y: column sums continue from the chunk partial of part 1, then the group fold);
+//   3 : as 1, but the sums of the rows that were not kept are folded here (the kept rows are then restored, and
+//   summed, by the next selection's kernel).
 __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restrict__ x, const uint4* __restrict__ y,
                                                                const uint4* __restrict__ cache, const int32_t* __restrict__ inv,
                                                                const float* __restrict__ gamma, int mod_stride, int n, int k,
@@ -184,7 +186,7 @@ __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restric
     const int j = __ldg(inv + (size_t)b * n + t);
     s_src[threadIdx.x] = (j >= 0) ? y + ((size_t)b * k + j) * C8
                                   : cache + ((size_t)b * hc * wc + nearest_src(t, h, w, hc, wc)) * C8;
-    s_on[threadIdx.x] = part == 0 || (part == 1) == (j < 0);
+    s_on[threadIdx.x] = part == 0 || (part == 1 || part == 3) == (j < 0);
   }
   __syncthreads();
   float4* xbase = x + ((size_t)b * n + t0) * C8 * 2;
@@ -425,7 +427,7 @@ __global__ void __launch_bounds__(256) restore_residual_interp_kernel(float4* __
       const InterpTaps<TAPS> bt = interp_taps<TAPS>(t, h, w, hc, wc);
       for (int q = 0; q < TAPS; ++q) { s_src[threadIdx.x][q] = cache + ((size_t)b * hc * wc + bt.src[q]) * C8; s_wt[threadIdx.x][q] = bt.wt[q]; }
     }
-    s_on[threadIdx.x] = part == 0 || (part == 1) == (j < 0);
+    s_on[threadIdx.x] = part == 0 || (part == 1 || part == 3) == (j < 0);
   }
   __syncthreads();
   float4* xbase = x + ((size_t)b * n + t0) * C8 * 2;
@@ -601,8 +603,9 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
   if (colsum_ws) ws = select_ws_carve(colsum_ws, B, n, C);
   const int nchunks = (n + kColsumRows - 1) / kColsumRows;
   // algorithmic bytes of the part: x read + written for its rows, its source rows
-  const double rows_x = part == 0 ? (double)n : (part == 1 ? (double)(n - k) : (double)k);
-  const double rr_bytes = (double)B * C * (8.0 * rows_x + (part != 1 ? 2.0 * k : 0.0) + (part != 2 ? 2.0 * hc * wc : 0.0));
+  const bool unkept_only = part == 1 || part == 3;
+  const double rows_x = part == 0 ? (double)n : (unkept_only ? (double)(n - k) : (double)k);
+  const double rr_bytes = (double)B * C * (8.0 * rows_x + (!unkept_only ? 2.0 * k : 0.0) + (part != 2 ? 2.0 * hc * wc : 0.0));
   LaunchScope scope(KC_RESTORE, 1, rr_bytes, rr_bytes, st);
   // kept rows + group fold inside clusters (one cluster per group of chunks) where the group fits a cluster
   if (part == 2 && colsum_ws && g_cluster_fold_ok && g_fold_mode != 1 && ws.group >= 1 && ws.group <= 8 && C / 8 <= 256) {

@@ -11,8 +11,11 @@
 // Few launches and short chains of dependent loads matter more here than peak bandwidth: the maps are
 // tens of MB, and every dependent global access costs about a microsecond.  All HBM access is 128-bit
 // and coalesced; no float atomics anywhere (bit-reproducible).
+#include <cuda_bf16.h>
+
 #include "colsum_fold.cuh"
 #include "internal.h"
+#include "sm100.cuh"
 
 namespace fv {
 
@@ -78,57 +81,56 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
   return warp_excl + inc - v;
 }
 
-// grid (CTAs per image, B), 512 threads, sized to be resident all at once (two CTAs per SM); the warps of
-// an image stride over its token rows.  Dynamic shared memory max(C, n + n/32) * 4 bytes (mean token, then keys).
-__global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float4* __restrict__ x,
-                                                                  const float4* __restrict__ group_partial, int ngroups, int n,
-                                                                  int C4, int k, float* __restrict__ score,
-                                                                  unsigned int* img_tickets, int32_t* __restrict__ idx,
-                                                                  int32_t* __restrict__ inv, int32_t* __restrict__ near_tie) {
-  extern __shared__ float4 s_dyn[];
-  float4* s_mean = s_dyn;
-  uint32_t* s_keys = reinterpret_cast<uint32_t*>(s_dyn);  // reused once the scores are out
-  __shared__ uint32_t s_hist[256];
-  __shared__ uint32_t s_warp[32];
-  __shared__ uint32_t s_prefix, s_remaining, s_near;
-  __shared__ int s_last;
-  const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  pdl_trigger();
-  pdl_wait();
-
-  // ---- Eq. 4: the mean token of image b from the group partials (fixed order)
-  {
-    const float4* gp = group_partial + (size_t)b * ngroups * C4;
-    const float fn = (float)n;
-    for (int c4 = tid; c4 < C4; c4 += kTopkThreads) {
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int g = 0; g < ngroups; ++g) {
-        const float4 v = __ldcg(gp + (size_t)g * C4 + c4);
-        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-      }
-      s_mean[c4] = make_float4(acc.x / fn, acc.y / fn, acc.z / fn, acc.w / fn);
-    }
+// ---- Eq. 4: the mean token of image b from up to two sets of at most kMaxGroups partial column sums, added in a
+// fixed order (set a, then set b).  The loads are requested eight at a time before the first of them is used.
+__device__ __forceinline__ void add_partials(float4& acc, const float4* __restrict__ gp, int ng, int C4, int c4) {
+#pragma unroll
+  for (int g0 = 0; g0 < kMaxGroups; g0 += 8) {
+    if (g0 >= ng) break;
+    float4 v[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g)
+      if (g0 + g < ng) v[g] = __ldcg(gp + (size_t)(g0 + g) * C4 + c4);
+#pragma unroll
+    for (int g = 0; g < 8; ++g)
+      if (g0 + g < ng) { acc.x += v[g].x; acc.y += v[g].y; acc.z += v[g].z; acc.w += v[g].w; }
   }
-  __syncthreads();
+}
+__device__ __forceinline__ void mean_from_partials(float4* s_mean, const float4* __restrict__ gp_a, int nga,
+                                                   const float4* __restrict__ gp_b, int ngb, int C4, int n) {
+  const float fn = (float)n;
+  for (int c4 = threadIdx.x; c4 < C4; c4 += kTopkThreads) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    add_partials(acc, gp_a, nga, C4, c4);
+    if (ngb > 0) add_partials(acc, gp_b, ngb, C4, c4);
+    s_mean[c4] = make_float4(acc.x / fn, acc.y / fn, acc.z / fn, acc.w / fn);
+  }
+}
 
-  // ---- Eq. 5 / Algorithm 1: squared deviation from the mean, one warp per token row
+// ---- Eq. 5 / Algorithm 1: squared deviation from the mean, one warp per token row; the warps of an image stride
+// over its rows.  NC: the map was not written by this kernel, so its rows may take the read-only path; the fused
+// kernel, whose other CTAs have just updated rows of it, reads them through L2.
+// BATCH: 16-byte loads a lane requests together (8 with 64 registers per thread, 16 with 128).
+template <bool NC, int BATCH>
+__device__ __forceinline__ void score_rows(const float4* x, const float4* s_mean, int b, int n, int C4, float* __restrict__ score) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int r = blockIdx.x * kTopkWarps + warp; r < n; r += gridDim.x * kTopkWarps) {
     const float4* row = x + ((size_t)b * n + r) * C4;
     float acc = 0.f;
     int c4 = lane;
-    for (; c4 + 32 * 7 < C4; c4 += 32 * 8) {
-      float4 v[8];
+    for (; c4 + 32 * (BATCH - 1) < C4; c4 += 32 * BATCH) {
+      float4 v[BATCH];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) v[i] = __ldg(row + c4 + 32 * i);
+      for (int i = 0; i < BATCH; ++i) v[i] = NC ? __ldg(row + c4 + 32 * i) : __ldcg(row + c4 + 32 * i);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < BATCH; ++i) {
         const float4 m = s_mean[c4 + 32 * i];
         const float dx = v[i].x - m.x, dy = v[i].y - m.y, dz = v[i].z - m.z, dw = v[i].w - m.w;
         acc += dx * dx; acc += dy * dy; acc += dz * dz; acc += dw * dw;
       }
     }
     for (; c4 < C4; c4 += 32) {
-      const float4 v = __ldg(row + c4);
+      const float4 v = NC ? __ldg(row + c4) : __ldcg(row + c4);
       const float4 m = s_mean[c4];
       const float dx = v.x - m.x, dy = v.y - m.y, dz = v.z - m.z, dw = v.w - m.w;
       acc += dx * dx; acc += dy * dy; acc += dz * dz; acc += dw * dw;
@@ -137,24 +139,23 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     if (lane == 0) score[(size_t)b * n + r] = acc;
   }
-  __threadfence();  // this thread's scores are visible device-wide before the CTA takes its ticket
+}
 
-  // ---- the last CTA of this image to get here ranks the image
-  __syncthreads();
-  if (tid == 0) {
-    const unsigned int prev = atomicAdd(img_tickets + b, 1u);
-    s_last = (prev == gridDim.x - 1);
-    if (s_last) img_tickets[b] = 0u;
-    s_prefix = 0u; s_remaining = (uint32_t)k; s_near = 0u;
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
+// Scratch of the top-k in static shared memory.
+struct TopkShared {
+  uint32_t hist[256];
+  uint32_t warp[32];
+  uint32_t prefix, remaining, near;
+};
 
-  // Keys = fp32 bit patterns of the scores (s >= 0, so they order like the values) taken relative to the
-  // smallest key of the image: the scores of one map share their leading bits, and ranking only the
-  // bits that differ both skips passes and spreads the keys over the histogram bins.
-  const float* sc = score + (size_t)b * n;
+// ---- exact top-k of one image by one CTA (all kTopkThreads threads): radix select on the fp32 bit patterns of the
+// scores (s >= 0, so they order like the values), ties to the lowest index, ascending output, inverse map.
+__device__ __forceinline__ void topk_image(const float* __restrict__ sc, int n, int k, uint32_t* s_keys, TopkShared& sh,
+                                           int32_t* __restrict__ idx_b, int32_t* __restrict__ inv_b, int32_t* near_tie_b) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) { sh.prefix = 0u; sh.remaining = (uint32_t)k; sh.near = 0u; }
+  // Keys are taken relative to the smallest key of the image: the scores of one map share their leading bits, and
+  // ranking only the bits that differ both skips passes and spreads the keys over the histogram bins.
   uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
   for (int i = tid; i < n; i += kTopkThreads) {
     const uint32_t key = __float_as_uint(__ldcg(sc + i)) & 0x7FFFFFFFu;  // drops the sign of -0
@@ -163,10 +164,10 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float
   }
   kmin = __reduce_min_sync(0xffffffffu, kmin);
   kmax = __reduce_max_sync(0xffffffffu, kmax);
-  if (lane == 0) { s_warp[warp] = kmin; s_hist[warp] = kmax; }
+  if (lane == 0) { sh.warp[warp] = kmin; sh.hist[warp] = kmax; }
   __syncthreads();
-  kmin = s_warp[lane < kTopkWarps ? lane : 0];
-  kmax = s_hist[lane < kTopkWarps ? lane : 0];
+  kmin = sh.warp[lane < kTopkWarps ? lane : 0];
+  kmax = sh.hist[lane < kTopkWarps ? lane : 0];
   kmin = __reduce_min_sync(0xffffffffu, kmin);
   kmax = __reduce_max_sync(0xffffffffu, kmax);
   __syncthreads();
@@ -174,32 +175,32 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float
   const uint32_t range = kmax - kmin;
   const int npass = range ? (32 - __clz(range) + 7) / 8 : 0;
 
-  // Radix select, most significant byte first: after the passes s_prefix is the k-th largest key and
-  // s_remaining how many keys equal to it belong to the kept set.
+  // Radix select, most significant byte first: after the passes sh.prefix is the k-th largest key and
+  // sh.remaining how many keys equal to it belong to the kept set.
   for (int pass = 0; pass < npass; ++pass) {
     const int shift = 8 * (npass - 1 - pass);
     const uint32_t hi_mask = shift + 8 >= 32 ? 0u : (0xFFFFFFFFu << (shift + 8));
-    if (tid < 256) s_hist[tid] = 0u;
+    if (tid < 256) sh.hist[tid] = 0u;
     __syncthreads();
-    const uint32_t prefix = s_prefix;
+    const uint32_t prefix = sh.prefix;
     for (int i = tid; i < n; i += kTopkThreads) {
       const uint32_t key = s_keys[KI(i)];
-      if ((key & hi_mask) == prefix) atomicAdd(&s_hist[(key >> shift) & 255u], 1u);
+      if ((key & hi_mask) == prefix) atomicAdd(&sh.hist[(key >> shift) & 255u], 1u);
     }
     __syncthreads();
     if (tid < 32) {
       // lane l owns bins 255-8l .. 248-8l (descending); find the bin where the running count from the
-      // top reaches s_remaining.
+      // top reaches sh.remaining.
       uint32_t local[8], sum = 0;
 #pragma unroll
-      for (int j = 0; j < 8; ++j) { local[j] = s_hist[255 - 8 * lane - j]; sum += local[j]; }
+      for (int j = 0; j < 8; ++j) { local[j] = sh.hist[255 - 8 * lane - j]; sum += local[j]; }
       uint32_t inc = sum;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
         uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
         if (lane >= o) inc += t;
       }
-      const uint32_t rem = s_remaining;
+      const uint32_t rem = sh.remaining;
       const uint32_t excl = inc - sum;
       const bool mine = (excl < rem) && (inc >= rem);  // exactly one lane
       if (mine) {
@@ -207,8 +208,8 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           if (cum + local[j] >= rem) {
-            s_prefix = prefix | ((uint32_t)(255 - 8 * lane - j) << shift);
-            s_remaining = rem - cum;
+            sh.prefix = prefix | ((uint32_t)(255 - 8 * lane - j) << shift);
+            sh.remaining = rem - cum;
             break;
           }
           cum += local[j];
@@ -217,8 +218,9 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float
     }
     __syncthreads();
   }
-  const uint32_t tau = s_prefix;  // relative to kmin
-  const uint32_t need_eq = s_remaining;
+  __syncthreads();
+  const uint32_t tau = sh.prefix;  // relative to kmin
+  const uint32_t need_eq = sh.remaining;
 
   // Ordered compaction: thread t owns the contiguous tokens [t*per, (t+1)*per).
   const int per = (n + kTopkThreads - 1) / kTopkThreads;
@@ -231,11 +233,10 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float
     cnt += (key > tau) + ((uint32_t)(key == tau) << 16);
   }
   uint32_t tot;
-  const uint32_t before = block_exclusive_scan(cnt, s_warp, &tot);
+  const uint32_t before = block_exclusive_scan(cnt, sh.warp, &tot);
   const uint32_t eq_before = before >> 16;
   uint32_t pos = (before & 0xFFFFu) + min(eq_before, need_eq);   // kept tokens before this thread's first
-  uint32_t e;
-  e = eq_before;
+  uint32_t e = eq_before;
   const float tau_f = __uint_as_float(tau + kmin);
   const float band = 1e-5f * tau_f;
   uint32_t near = 0;
@@ -243,19 +244,316 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float
     uint32_t key = s_keys[KI(i)];
     bool take = key > tau;
     if (key == tau) { take = (e < need_eq); ++e; }
-    if (take) idx[(size_t)b * k + pos] = i;
-    if (inv) inv[(size_t)b * n + i] = take ? (int32_t)pos : -1;
+    if (take) idx_b[pos] = i;
+    if (inv_b) inv_b[i] = take ? (int32_t)pos : -1;
     pos += take;
     near += (fabsf(__uint_as_float(key + kmin) - tau_f) <= band);
   }
-  if (near_tie) {
+  if (near_tie_b) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) near += __shfl_xor_sync(0xffffffffu, near, o);
-    if (lane == 0) atomicAdd(&s_near, near);
+    if (lane == 0) atomicAdd(&sh.near, near);
     __syncthreads();
-    if (tid == 0) near_tie[b] = (int32_t)s_near;
+    if (tid == 0) *near_tie_b = (int32_t)sh.near;
   }
 }
+
+// grid (CTAs per image, B), 512 threads, sized to be resident all at once (two CTAs per SM); the warps of
+// an image stride over its token rows.  Dynamic shared memory max(C, n + n/32) * 4 bytes (mean token, then keys).
+__global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float4* __restrict__ x,
+                                                                  const float4* __restrict__ group_partial, int ngroups, int n,
+                                                                  int C4, int k, float* __restrict__ score,
+                                                                  unsigned int* img_tickets, int32_t* __restrict__ idx,
+                                                                  int32_t* __restrict__ inv, int32_t* __restrict__ near_tie) {
+  extern __shared__ float4 s_dyn[];
+  float4* s_mean = s_dyn;
+  uint32_t* s_keys = reinterpret_cast<uint32_t*>(s_dyn);  // reused once the scores are out
+  __shared__ TopkShared sh;
+  __shared__ int s_last;
+  const int b = blockIdx.y, tid = threadIdx.x;
+  pdl_trigger();
+  pdl_wait();
+  mean_from_partials(s_mean, group_partial + (size_t)b * ngroups * C4, ngroups, nullptr, 0, C4, n);
+  __syncthreads();
+  score_rows<true, 8>(x, s_mean, b, n, C4, score);
+  __threadfence();  // this thread's scores are visible device-wide before the CTA takes its ticket
+
+  // ---- the last CTA of this image to get here ranks the image
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned int prev = atomicAdd(img_tickets + b, 1u);
+    s_last = (prev == gridDim.x - 1);
+    if (s_last) img_tickets[b] = 0u;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  topk_image(score + (size_t)b * n, n, k, s_keys, sh, idx + (size_t)b * k, inv ? inv + (size_t)b * n : nullptr, near_tie ? near_tie + b : nullptr);
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// The selection of a wrapped sublayer inside a scale step, fused with what surrounds it on the kept rows:
+//   phase 0  Cached Token Restoration of the PREVIOUS sublayer's kept rows (Eq. 6's scatter of the forwarded rows,
+//            with gate and residual): x[idx_prev[j]] += gamma * y[j].  (The rows that were not kept were restored
+//            from the cache by the restore kernel on the side stream, which also left their column sums.)  The
+//            column sums of the rows updated here are folded CTA -> group of CTAs -> image, in a fixed order.
+//   barrier  every CTA waits until all groups are folded (an arrival count in global memory; bounded wait).
+//   phase 1  Eq. 4's mean token from the two sets of sums, Eq. 5's scores, and -- by the last CTA of an image to
+//            finish -- the exact top-k (kept indices ascending, inverse map).
+//   flag     the other CTAs of the image wait for its top-k (bounded).
+//   phase 2  Algorithm 1's gather of the kept rows fused with LayerNorm and AdaLN modulation -> bf16 A operand.
+// The grid never exceeds what the GPU holds at once (the launcher asks the occupancy calculator), so the waits
+// cannot starve a CTA that has not started.  A wait that expires leaves a code in the status word and the CTA
+// returns; nothing spins without a limit.
+struct FusedSelectArgs {
+  float4* x; int n, C4, k;
+  // phase 0 (y == nullptr: no kept rows to restore; the given sums then cover the whole map)
+  const uint4* y; const int32_t* idx_prev; const float* gamma_prev; int mod_stride; int k_prev;
+  float4* kept_cta_partial; float4* kept_group; unsigned int* kept_tickets; int gs, ngk;
+  unsigned int* done; unsigned int done_target;
+  // phase 1
+  const float4* group_partial; int ngroups;
+  float* score; unsigned int* img_tickets; int32_t* idx; int32_t* inv;
+  unsigned int* ready; unsigned int epoch;
+  // phase 2
+  const float* sigma; const float* beta; uint2* a_out;
+  int32_t* status;
+};
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+// Waits until the counter at `w` has reached `target` (counters only grow; compared as a wrapping difference), for
+// at most two seconds.
+__device__ __forceinline__ bool wait_counter(const unsigned int* w, unsigned int target) {
+  unsigned long long t0 = 0;
+  for (unsigned int spins = 0;; ++spins) {
+    if ((int)(ld_acquire_u32(w) - target) >= 0) return true;
+    if (spins == 64) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    if (spins > 64 && (spins & 63u) == 0) {
+      unsigned long long t1;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+      if (t1 - t0 > 2000000000ull) return false;
+    }
+    if (spins > 16) __nanosleep(64);
+  }
+}
+
+// LayerNorm (+ modulation) of one token row by one warp, the row held in registers (C <= 2048); same arithmetic and
+// order of sums as the stand-alone gather kernel.  Rows of the map may have been updated by other CTAs of this
+// kernel (before the grid-wide wait), so they are read through L2, not through the read-only path.
+__device__ __forceinline__ void gather_ln_row(const float4* row, int C4, const float4* s_sigma, const float4* s_beta,
+                                              uint2* __restrict__ dst) {
+  constexpr int kVec = 16;
+  const int lane = threadIdx.x & 31;
+  float4 v[kVec];
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) {
+    const int c4 = lane + 32 * i;
+    if (c4 < C4) v[i] = __ldcg(row + c4);
+  }
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) {
+    const int c4 = lane + 32 * i;
+    if (c4 < C4) sum += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  const float inv_c = 1.0f / (float)(C4 * 4);
+  const float mu = sum * inv_c;
+  float var = 0.f;
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) {
+    const int c4 = lane + 32 * i;
+    if (c4 < C4) {
+      const float dx = v[i].x - mu, dy = v[i].y - mu, dz = v[i].z - mu, dw = v[i].w - mu;
+      var += (dx * dx + dy * dy) + (dz * dz + dw * dw);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) var += __shfl_xor_sync(0xffffffffu, var, o);
+  const float rstd = rsqrtf(var * inv_c + 1e-6f);
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) {
+    const int c4 = lane + 32 * i;
+    if (c4 < C4) {
+      float4 a;
+      a.x = (v[i].x - mu) * rstd; a.y = (v[i].y - mu) * rstd; a.z = (v[i].z - mu) * rstd; a.w = (v[i].w - mu) * rstd;
+      if (s_sigma) {
+        const float4 sg = s_sigma[c4], bb = s_beta[c4];
+        a.x = fmaf(a.x, 1.f + sg.x, bb.x); a.y = fmaf(a.y, 1.f + sg.y, bb.y);
+        a.z = fmaf(a.z, 1.f + sg.z, bb.z); a.w = fmaf(a.w, 1.f + sg.w, bb.w);
+      }
+      __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
+      uint2 o;
+      o.x = *reinterpret_cast<uint32_t*>(&lo);
+      o.y = *reinterpret_cast<uint32_t*>(&hi);
+      dst[c4] = o;
+    }
+  }
+}
+
+__device__ __forceinline__ void bf16x8_widen(const uint4& p, float (&f)[8]) {
+  const uint32_t u[4] = {p.x, p.y, p.z, p.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(u[i] << 16); f[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u); }
+}
+
+// grid (CTAs per image, B), kTopkThreads threads, one CTA per SM (a thread may hold a token row's sixteen 16-byte
+// words).  Dynamic shared memory: the largest of the mean token, the keys of the top-k, the row-parallel copies of
+// phase 0's sums and the modulation vectors of phase 2.
+__global__ void __launch_bounds__(kTopkThreads, 1) select_fused_kernel(const FusedSelectArgs a) {
+  extern __shared__ float4 s_dyn[];
+  __shared__ TopkShared sh;
+  __shared__ int s_flag;
+  const int b = blockIdx.y, cta = blockIdx.x, G = gridDim.x, tid = threadIdx.x;
+  const int n = a.n, C4 = a.C4;
+  pdl_trigger();
+  pdl_wait();
+  bool ok = true;
+
+  // ---- phase 0: the previous sublayer's kept rows
+  if (a.y) {
+    const int C8 = C4 / 2;
+    const int rows_par = kTopkThreads / C8;       // rows a CTA updates side by side (>= 2: C <= 2048)
+    const int c8 = tid % C8, rp = tid / C8;
+    float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+    if (rp < rows_par) {
+      float4 g0 = make_float4(1.f, 1.f, 1.f, 1.f), g1 = g0;
+      if (a.gamma_prev) {
+        const float4* g = reinterpret_cast<const float4*>(a.gamma_prev + (size_t)b * a.mod_stride);
+        g0 = __ldg(g + 2 * c8); g1 = __ldg(g + 2 * c8 + 1);
+      }
+      const int stride = G * rows_par;
+      const int32_t* ip = a.idx_prev + (size_t)b * a.k_prev;
+      const uint4* yb = a.y + (size_t)b * a.k_prev * C8;
+      float4* xb = a.x + (size_t)b * n * C4;
+      for (int j = cta + G * rp; j < a.k_prev; j += 2 * stride) {     // two rows in flight
+        const int j2 = j + stride;
+        const bool two = j2 < a.k_prev;
+        const int t1 = min(max(__ldg(ip + j), 0), n - 1);
+        const int t2 = two ? min(max(__ldg(ip + j2), 0), n - 1) : t1;
+        float4* xr1 = xb + (size_t)t1 * C4 + 2 * c8;
+        float4* xr2 = xb + (size_t)t2 * C4 + 2 * c8;
+        float4 u0 = xr1[0], u1 = xr1[1];
+        const uint4 p1 = __ldg(yb + (size_t)j * C8 + c8);
+        float4 w0 = u0, w1 = u1;
+        uint4 p2 = p1;
+        if (two) { w0 = xr2[0]; w1 = xr2[1]; p2 = __ldg(yb + (size_t)j2 * C8 + c8); }
+        float f[8];
+        bf16x8_widen(p1, f);
+        if (a.gamma_prev) {
+          u0.x = fmaf(g0.x, f[0], u0.x); u0.y = fmaf(g0.y, f[1], u0.y); u0.z = fmaf(g0.z, f[2], u0.z); u0.w = fmaf(g0.w, f[3], u0.w);
+          u1.x = fmaf(g1.x, f[4], u1.x); u1.y = fmaf(g1.y, f[5], u1.y); u1.z = fmaf(g1.z, f[6], u1.z); u1.w = fmaf(g1.w, f[7], u1.w);
+        } else {
+          u0.x += f[0]; u0.y += f[1]; u0.z += f[2]; u0.w += f[3];
+          u1.x += f[4]; u1.y += f[5]; u1.z += f[6]; u1.w += f[7];
+        }
+        xr1[0] = u0; xr1[1] = u1;
+        a0.x += u0.x; a0.y += u0.y; a0.z += u0.z; a0.w += u0.w;
+        a1.x += u1.x; a1.y += u1.y; a1.z += u1.z; a1.w += u1.w;
+        if (two) {
+          bf16x8_widen(p2, f);
+          if (a.gamma_prev) {
+            w0.x = fmaf(g0.x, f[0], w0.x); w0.y = fmaf(g0.y, f[1], w0.y); w0.z = fmaf(g0.z, f[2], w0.z); w0.w = fmaf(g0.w, f[3], w0.w);
+            w1.x = fmaf(g1.x, f[4], w1.x); w1.y = fmaf(g1.y, f[5], w1.y); w1.z = fmaf(g1.z, f[6], w1.z); w1.w = fmaf(g1.w, f[7], w1.w);
+          } else {
+            w0.x += f[0]; w0.y += f[1]; w0.z += f[2]; w0.w += f[3];
+            w1.x += f[4]; w1.y += f[5]; w1.z += f[6]; w1.w += f[7];
+          }
+          xr2[0] = w0; xr2[1] = w1;
+          a0.x += w0.x; a0.y += w0.y; a0.z += w0.z; a0.w += w0.w;
+          a1.x += w1.x; a1.y += w1.y; a1.z += w1.z; a1.w += w1.w;
+        }
+      }
+    }
+    // the row-parallel copies of the sums, added in a fixed order -> this CTA's partial
+    if (rp > 0 && rp < rows_par) { s_dyn[((size_t)(rp - 1) * C8 + c8) * 2] = a0; s_dyn[((size_t)(rp - 1) * C8 + c8) * 2 + 1] = a1; }
+    __syncthreads();
+    if (rp == 0) {
+      for (int r = 1; r < rows_par; ++r) {
+        const float4 v0 = s_dyn[((size_t)(r - 1) * C8 + c8) * 2], v1 = s_dyn[((size_t)(r - 1) * C8 + c8) * 2 + 1];
+        a0.x += v0.x; a0.y += v0.y; a0.z += v0.z; a0.w += v0.w;
+        a1.x += v1.x; a1.y += v1.y; a1.z += v1.z; a1.w += v1.w;
+      }
+      float4* cp = a.kept_cta_partial + ((size_t)b * G + cta) * C4 + 2 * c8;
+      cp[0] = a0; cp[1] = a1;
+    }
+    const bool folded = fold_group_partials(b, cta, G, a.gs, a.ngk, C4, a.kept_cta_partial, a.kept_group, a.kept_tickets);
+    if (folded) {      // uniform over the CTA
+      __threadfence();
+      __syncthreads();
+      if (tid == 0) atomicAdd(a.done, 1u);
+    }
+    // ---- every group of every image folded?
+    if (tid == 0) {
+      const bool w = wait_counter(a.done, a.done_target);
+      if (!w && a.status) atomicCAS(a.status, 0, DEV_TIMEOUT_GRID);
+      s_flag = w;
+    }
+    __syncthreads();
+    ok = s_flag != 0;
+    __syncthreads();      // s_flag is reused below
+    __threadfence();
+  }
+  if (!ok) return;
+
+  // ---- phase 1: mean token, scores, top-k
+  mean_from_partials(s_dyn, a.group_partial + (size_t)b * a.ngroups * C4, a.ngroups,
+                     a.y ? a.kept_group + (size_t)b * a.ngk * C4 : nullptr, a.y ? a.ngk : 0, C4, n);
+  __syncthreads();
+  score_rows<false, 16>(a.x, s_dyn, b, n, C4, a.score);
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned int prev = atomicAdd(a.img_tickets + b, 1u);
+    const int last = (prev == (unsigned int)G - 1u);
+    if (last) a.img_tickets[b] = 0u;
+    s_flag = last;
+  }
+  __syncthreads();
+  const bool last = s_flag != 0;
+  float4* s_sigma = nullptr;
+  float4* s_beta = nullptr;
+  if (last) {
+    __threadfence();
+    topk_image(a.score + (size_t)b * n, n, a.k, reinterpret_cast<uint32_t*>(s_dyn), sh, a.idx + (size_t)b * a.k, a.inv + (size_t)b * n, nullptr);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.ready + b), "r"(a.epoch) : "memory");
+  }
+  // the modulation vectors of the image (they do not depend on the selection: fetched before the wait)
+  if (a.sigma) {
+    s_sigma = s_dyn; s_beta = s_dyn + C4;
+    const float4* sg = reinterpret_cast<const float4*>(a.sigma + (size_t)b * a.mod_stride);
+    const float4* bt = reinterpret_cast<const float4*>(a.beta + (size_t)b * a.mod_stride);
+    for (int i = tid; i < C4; i += kTopkThreads) { s_sigma[i] = __ldg(sg + i); s_beta[i] = __ldg(bt + i); }
+  }
+  if (!last) {
+    if (tid == 0) {
+      const bool w = wait_counter(a.ready + b, a.epoch);
+      if (!w && a.status) atomicCAS(a.status, 0, DEV_TIMEOUT_GRID);
+      s_flag = w;
+    }
+    __syncthreads();
+    if (s_flag == 0) return;
+    __threadfence();
+  } else {
+    __syncthreads();
+  }
+
+  // ---- phase 2: gather + LayerNorm + modulation of the kept rows, one warp per row
+  const int warp = tid >> 5;
+  const int32_t* ib = a.idx + (size_t)b * a.k;
+  for (int j = cta * kTopkWarps + warp; j < a.k; j += G * kTopkWarps) {
+    const int t = min(max(__ldcg(ib + j), 0), n - 1);
+    gather_ln_row(a.x + ((size_t)b * n + t) * C4, C4, s_sigma, s_beta, a.a_out + ((size_t)b * a.k + j) * C4);
+  }
+}
+
 __global__ void inv_fill_kernel(int32_t* inv, size_t total) {
   pdl_trigger();
   pdl_wait();
@@ -313,7 +611,9 @@ cudaError_t select_init() {
   cudaError_t e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(score_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkMaxSmem);
+  e = cudaFuncSetAttribute(score_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkMaxSmem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(select_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkMaxSmem);
 }
 
 cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* idx, int32_t* inv, float* score,
@@ -338,6 +638,79 @@ cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* i
              reinterpret_cast<const float4*>(w.group_partial), w.ngroups, n, C4, k, sc, w.tickets + (size_t)B * kMaxGroups, idx, inv,
              near_tie);
   return cudaGetLastError();
+}
+
+// ---- the fused selection of a scale step
+constexpr int kFusedMaxCtas = 320;     // CTAs per image the kept-row partials have room for
+size_t select_fused_sync_bytes(int B) { return align_up((size_t)B * (kMaxGroups + 1) * sizeof(unsigned int) + 64, 256); }
+size_t select_fused_ws_bytes(int B, int C) {
+  return select_fused_sync_bytes(B) + align_up((size_t)B * kFusedMaxCtas * C * sizeof(float), 256) +
+         align_up((size_t)B * kMaxGroups * C * sizeof(float), 256);
+}
+
+static size_t fused_smem_bytes(int n, int C) {
+  const size_t keys = ((size_t)n + n / 32 + 1) * 4;
+  const size_t vec = (size_t)C * 4;                       // the mean token
+  const int rows_par = kTopkThreads / (C / 8);
+  const size_t comb = (size_t)(rows_par > 1 ? rows_par - 1 : 0) * C * 4;
+  size_t m = keys > 2 * vec ? keys : 2 * vec;             // keys | sigma + beta
+  return m > comb ? m : comb;
+}
+
+// CTAs per image of the fused kernel: never more than the GPU holds at once (its CTAs wait on one another), never
+// more than one warp per token row.  0: the shape cannot take the fused path.
+static int fused_ctas_per_image(int B, int n, int C) {
+  if (C % 8 || C / 8 > kTopkThreads / 2 || C > 2048 || n > kTopkMaxTokens) return 0;
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_fused_kernel, kTopkThreads, fused_smem_bytes(n, C)) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return 0;
+  }
+  long g = (long)per_sm * g_num_sms / B;
+  const long need = (n + kTopkWarps - 1) / kTopkWarps;
+  if (g > need) g = need;
+  if (g > kFusedMaxCtas) g = kFusedMaxCtas;
+  return (int)g;
+}
+bool select_fused_supported(int B, int n, int C) { return fused_ctas_per_image(B, n, C) >= 1; }
+
+cudaError_t launch_select_fused(const FusedSelect& f, cudaStream_t st) {
+  const int G = fused_ctas_per_image(f.B, f.n, f.C);
+  if (G < 1) return cudaErrorInvalidConfiguration;
+  const SelectWs w = select_ws_carve(f.sel_ws, f.B, f.n, f.C);
+  char* fw = static_cast<char*>(f.fused_ws);
+  FusedSelectArgs a{};
+  a.x = reinterpret_cast<float4*>(f.x); a.n = f.n; a.C4 = f.C / 4; a.k = f.k;
+  a.y = reinterpret_cast<const uint4*>(f.y); a.idx_prev = f.idx_prev; a.gamma_prev = f.gamma_prev; a.mod_stride = f.mod_stride; a.k_prev = f.k;
+  a.kept_tickets = reinterpret_cast<unsigned int*>(fw);
+  a.done = a.kept_tickets + (size_t)f.B * kMaxGroups;
+  a.ready = a.done + 16;                                   // one word per image
+  a.kept_cta_partial = reinterpret_cast<float4*>(fw + select_fused_sync_bytes(f.B));
+  a.kept_group = reinterpret_cast<float4*>(fw + select_fused_sync_bytes(f.B) + align_up((size_t)f.B * kFusedMaxCtas * f.C * sizeof(float), 256));
+  a.gs = (G + kMaxGroups - 1) / kMaxGroups;
+  a.ngk = (G + a.gs - 1) / a.gs;
+  if (f.y) *f.done_total += (unsigned int)(f.B * a.ngk);
+  a.done_target = *f.done_total;
+  a.epoch = ++*f.epoch;
+  a.group_partial = reinterpret_cast<const float4*>(w.group_partial); a.ngroups = w.ngroups;
+  a.score = w.score; a.img_tickets = w.tickets + (size_t)f.B * kMaxGroups; a.idx = f.idx; a.inv = f.inv;
+  a.sigma = f.sigma; a.beta = f.beta; a.a_out = reinterpret_cast<uint2*>(f.a_out);
+  a.status = f.status;
+  // algorithmic bytes: the selection (x once, scores, indices), the gather (kept rows in, bf16 out) and, when it
+  // carries the previous sublayer's kept rows, their restoration (x read + written, y read)
+  const double rows = (double)f.B * f.k;
+  const double sel_bytes = (double)f.B * f.n * f.C * 4.0 + 4.0 * f.B * f.n + 4.0 * f.B * ((double)f.k + f.n);
+  const double gat_bytes = rows * f.C * 6.0;
+  const double res_bytes = f.y ? rows * f.C * 10.0 : 0.0;
+  LaunchScope scope(KC_SELECT, 1, sel_bytes + gat_bytes + res_bytes, sel_bytes + gat_bytes + res_bytes, st);
+  return launch_pdl(select_fused_kernel, dim3(G, f.B), dim3(kTopkThreads), fused_smem_bytes(f.n, f.C), st, a);
+}
+
+cudaError_t launch_colsum(const float* x, int B, int n, int C, void* workspace, cudaStream_t st) {
+  const SelectWs w = select_ws_carve(workspace, B, n, C);
+  LaunchScope scope(KC_SELECT, 1, (double)B * n * C * 4.0, (double)B * n * C * 4.0, st);
+  return launch_pdl(colsum_chunk_kernel, dim3(w.nchunks, B), dim3(256), 0, st, reinterpret_cast<const float4*>(x), n, C / 4, w.nchunks, w.group,
+                    w.ngroups, reinterpret_cast<float4*>(w.chunk_partial), reinterpret_cast<float4*>(w.group_partial), w.tickets);
 }
 
 cudaError_t launch_inv_fill(int B, int n, int32_t* inv, cudaStream_t st) {

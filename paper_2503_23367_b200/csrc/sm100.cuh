@@ -12,7 +12,7 @@ namespace fv {
 // Error codes a kernel may leave in the device status word (0 = fine).
 // Codes below 100: a kernel met bad data (an index outside its range) and clamped it.  100 and above: a bounded wait expired.
 enum : int { DEV_OK = 0, DEV_BAD_TOKEN_ID = 40, DEV_BAD_ROW_INDEX = 41,
-             DEV_TIMEOUT_TMA = 101, DEV_TIMEOUT_MMA = 102, DEV_TIMEOUT_EPI = 103, DEV_TIMEOUT_SOFTMAX = 104, DEV_TIMEOUT_SELFTEST = 105 };
+             DEV_TIMEOUT_TMA = 101, DEV_TIMEOUT_MMA = 102, DEV_TIMEOUT_EPI = 103, DEV_TIMEOUT_SOFTMAX = 104, DEV_TIMEOUT_SELFTEST = 105, DEV_TIMEOUT_GRID = 106 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));

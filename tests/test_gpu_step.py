@@ -196,14 +196,19 @@ ZERO_BRANCH_CASES = [  # h, w, hc, wc, C, H, B, B_max, keep, kind, oracle_runs_t
 ]
 
 
+@pytest.mark.parametrize("unfused", [0, 1])
 @pytest.mark.parametrize("h,w,hc,wc,C,H,B,B_max,keep,kind,full_oracle", ZERO_BRANCH_CASES)
-def test_every_selection_of_a_step_on_bit_identical_input(h, w, hc, wc, C, H, B, B_max, keep, kind, full_oracle):
+def test_every_selection_of_a_step_on_bit_identical_input(h, w, hc, wc, C, H, B, B_max, keep, kind, full_oracle, unfused):
     """Inside fv_var_step only the first selection sums the token map itself; every later one takes Eq. 4's column
     sums from the restoration before it (rows that were not kept on a side stream, kept rows + fold after the last
     GEMM).  With every branch ending in a zero projection and zero sublayer caches, each restoration adds exactly 0,
     so x entering EVERY sublayer is bit-identical on both sides and each of the 2 blocks x 3 selections must keep
     the oracle's set (any difference on a near-tie at the threshold, within 1e-5 relative).  Runs at the bench
-    shapes' maps, at ragged chunk / group counts and with a partial batch."""
+    shapes' maps, at ragged chunk / group counts and with a partial batch, in both forms the step has: one fused
+    launch per selection (kept rows of the previous sublayer restored and summed inside it, grid-wide wait, gather
+    of the new rows) and the separate kernels."""
+    if full_oracle and unfused:
+        full_oracle = False          # the oracle's own step was run in the fused case
     wl = I.Workload("zero-branch", L=2, C=C, H=H, B=B_max, sides=(hc, h), keep=(1.0, keep), cross_len=64, mlp_ratio=1, seed=811)
     mt = _zero_branch_tensors(wl)
     n, k = h * w, O.kept_count(keep, h, w)
@@ -216,7 +221,11 @@ def test_every_selection_of_a_step_on_bit_identical_input(h, w, hc, wc, C, H, B,
     ctx.prepare_text(B)
     trace = torch.full((wl.L, 3, B, k), -1, dtype=torch.int32, device=DEV)
     xd = torch.from_numpy(x).to(DEV)
-    got = ctx.var_step(xd, 1, keep, idx_trace=trace).cpu().numpy()
+    assert fv.lib().fv_step_force_unfused(unfused) == 0
+    try:
+        got = ctx.var_step(xd, 1, keep, idx_trace=trace).cpu().numpy()
+    finally:
+        fv.lib().fv_step_force_unfused(0)
     assert ctx.device_status() == 0 and ctx.state() == (2, k)
     assert np.array_equal(got, x), "a zero branch changed the residual stream"
     # the oracle's selection of this (unchanged) map: one score vector serves all six sublayers
