@@ -509,6 +509,7 @@ ATTN_CASES = [  # B, rows, H, C, kv_len, cap
     (1, 130, 2, 256, 129, 136), (2, 820, 16, 2048, 5223, 5224), (1, 37, 30, 1920, 640, 640),
     (1, 3277, 16, 2048, 13646, 13648),      # the 128x128 zero-shot step: 13 query-tile pairs x 107 key tiles per head
     (1, 1280, 16, 2048, 8525, 8528), (2, 260, 4, 256, 700, 704), (1, 52, 16, 2048, 6000, 6000),
+    (1, 820, 16, 2048, 7245, 7248),         # the 64x64 step of the 2K workload: 64 query blocks, cut into one piece per SM
 ]
 
 
