@@ -284,13 +284,14 @@ fv_status fv_prune_select_after_restore(const float *x_dev, int32_t B, int32_t h
  * fp32 [B, *n_partials_host, C]; the sum over the partials of image b is the column sum of its map. */
 fv_status fv_prune_select_workspace_layout(int32_t B, int32_t n_tokens, int32_t C, size_t *offset_host,
                                            int32_t *n_partials_host);
-/* Test / profiling hook (process-wide).  Inside fv_var_step a free-running selection is one launch that also
- * restores the previous sublayer's kept rows before it and gathers + normalises the newly kept rows after it;
- * on != 0 makes the step take the separate kernels instead (selection, gather + LayerNorm, kept-row restoration),
- * which forced-index steps always do.  The two add Eq. 4's column sums in a different order, so their scores
- * agree to fp32 rounding and a near-tie at the threshold may fall the other way; given the kept sets the token maps
- * are the same bit for bit. */
-fv_status fv_step_force_unfused(int32_t on);
+/* Test / profiling hook (process-wide).  on != 0: inside fv_var_step every free-running selection becomes ONE launch
+ * that also restores the previous sublayer's kept rows before it and gathers + normalises the newly kept rows after
+ * it (its CTAs wait on one another with bounded waits; the grid never exceeds what the GPU holds at once).  Off by
+ * default: measured on B200 the separate kernels (selection, gather + LayerNorm, kept-row restoration), whose launch
+ * gaps programmatic dependent launch already hides, are as fast or faster.  The two forms add Eq. 4's column sums in
+ * a different order, so their scores agree to fp32 rounding and a near-tie at the threshold may fall the other way;
+ * given the kept sets the token maps are the same bit for bit.  Forced-index steps always take the separate kernels. */
+fv_status fv_step_fused_selection(int32_t on);
 /* Test / profiling hook (process-wide): how the kept-row part of a restoration folds its column sums.
  * 0 = chosen per shape (default); 1 = always through global memory (arrival counters); 2 = inside
  * thread-block clusters wherever the shape allows it. */

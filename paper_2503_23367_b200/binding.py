@@ -23,7 +23,7 @@ EXPORTS = ["fv_status_string", "fv_k_for", "fv_prune_select_workspace_bytes", "f
            "fv_workspace_bytes", "fv_kv_bytes", "fv_cache_bytes", "fv_create", "fv_destroy", "fv_reset",
            "fv_get_state", "fv_set_state", "fv_kv_pointers", "fv_cache_pointer", "fv_prepare_text",
            "fv_device_status", "fv_selftest_expired_wait", "fv_var_step", "fv_gather_ln", "fv_restore_residual", "fv_prune_select_after_restore",
-           "fv_prune_select_workspace_layout", "fv_restore_force_fold", "fv_step_force_unfused", "fv_gemm_bf16", "fv_gemm_splitk_workspace_bytes", "fv_gemm_force_path", "fv_attention", "fv_attention_workspace_bytes", "fv_attention_force_ctas",
+           "fv_prune_select_workspace_layout", "fv_restore_force_fold", "fv_step_fused_selection", "fv_gemm_bf16", "fv_gemm_splitk_workspace_bytes", "fv_gemm_force_path", "fv_attention", "fv_attention_workspace_bytes", "fv_attention_force_ctas",
            "fv_kernel_launches", "fv_profile_enable", "fv_profile_read",
            "fv_prune_select_static", "fv_prune_select_static_capacity",
            "fv_head_workspace_bytes", "fv_head_tokens", "fv_argmax_rows", "fv_residual_accumulate", "fv_next_scale_input",
@@ -96,7 +96,7 @@ def lib() -> C.CDLL:
         L.fv_prune_select_workspace_layout.restype = C.c_int
         L.fv_prune_select_workspace_layout.argtypes = [i32, i32, i32, C.POINTER(sz), C.POINTER(i32)]
         L.fv_restore_force_fold.restype = C.c_int; L.fv_restore_force_fold.argtypes = [i32]
-        L.fv_step_force_unfused.restype = C.c_int; L.fv_step_force_unfused.argtypes = [i32]
+        L.fv_step_fused_selection.restype = C.c_int; L.fv_step_fused_selection.argtypes = [i32]
         L.fv_gemm_bf16.restype = C.c_int
         L.fv_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, sz, vp]
         L.fv_gemm_splitk_workspace_bytes.restype = sz; L.fv_gemm_splitk_workspace_bytes.argtypes = []

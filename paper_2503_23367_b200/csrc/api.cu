@@ -56,7 +56,11 @@ int32_t* ctx_status_word(const fv_ctx* ctx) { return ctx->status; }
 
 namespace {
 
-bool g_step_fused = true;   // test / profiling hook: false = one launch each for selection, gather and kept-row restoration
+// Test / profiling hook.  true: a free-running selection is one launch that also restores the previous sublayer's kept
+// rows and gathers the new ones (select_fused_kernel).  Measured on B200 it does not pay: with programmatic dependent
+// launch the separate kernels already overlap their launch gaps, while the fused kernel runs one CTA per SM and waits
+// twice grid-wide (pruned steps of the 1024-pixel workload 3 % slower, of the 2K workload equal), so it is off.
+bool g_step_fused = false;
 
 std::once_flag g_init_once;
 cudaError_t g_init_err = cudaSuccess;
@@ -243,8 +247,8 @@ fv_status fv_prune_select_workspace_layout(int32_t B, int32_t n_tokens, int32_t 
   return FV_OK;
 }
 
-fv_status fv_step_force_unfused(int32_t on) {
-  g_step_fused = on == 0;
+fv_status fv_step_fused_selection(int32_t on) {
+  g_step_fused = on != 0;
   return FV_OK;
 }
 
@@ -581,9 +585,10 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   bool have_partials = false;
   const bool selecting = sub_pruned && !forced_idx_dev;
   if (selecting && cudaMemsetAsync(ctx->sel_ws, 0, select_ticket_bytes(B), st) != cudaSuccess) return FV_ERR_CUDA;
-  // Free-running selections take one launch each: the previous sublayer's kept-row restoration, the selection and the
-  // gather + LayerNorm of the newly kept rows (select_fused_kernel).  The kept rows of a sublayer are then restored
-  // by the NEXT sublayer's launch; only the last sublayer of the step restores its own.
+  // Optional (fv_step_fused_selection): free-running selections take one launch each -- the previous sublayer's
+  // kept-row restoration, the selection and the gather + LayerNorm of the newly kept rows (select_fused_kernel).  The
+  // kept rows of a sublayer are then restored by the NEXT sublayer's launch; only the last sublayer of the step
+  // restores its own.
   const bool fused = selecting && g_step_fused && select_fused_supported(B, n, C);
   bool pending = false;                 // a kept-row restoration waits for the next fused selection
   const float* pending_gamma = nullptr;

@@ -516,6 +516,214 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   }
 }
 
+// ---- One whole work item per CTA: grid (query blocks, heads, images).  The launcher takes this kernel whenever it does
+// not cut the work into pieces: it is the kernel above without the segment bookkeeping, and its leaner loops hand
+// the tiles between the softmax warpgroups and the MMA thread measurably faster (15 % per key tile).
+struct WholeDev {
+  __nv_bfloat16* out;
+  int rows, C, kv_len, kv_capacity;
+  float scale_log2;  // log2(e) / sqrt(hd)
+  int32_t* status;
+};
+
+template <int HD>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attention_whole_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                 const __grid_constant__ CUtensorMap tmV, const WholeDev p) {
+  using Cfg = AttnCfg<HD>;
+  constexpr int NS = Cfg::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* q_s = smem;                          // two query tiles
+  uint8_t* k_s = q_s + 2 * Cfg::kQBytes;
+  uint8_t* v_s = k_s + NS * Cfg::kKBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(v_s + NS * Cfg::kVBytes);
+  uint64_t* q_full = bars;
+  uint64_t* k_full = bars + 1;
+  uint64_t* k_empty = k_full + NS;
+  uint64_t* v_full = k_empty + NS;
+  uint64_t* v_empty = v_full + NS;
+  uint64_t* s_full = v_empty + NS;   // [2] scores of query tile t are in TMEM
+  uint64_t* p_full = s_full + 2;     // [2] probabilities of query tile t are in TMEM (128 arrivals)
+  uint64_t* o_done = p_full + 2;     // [2] the latest P V of query tile t has completed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_done + 2);
+
+  pdl_trigger();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q0 = blockIdx.x * (2 * QT), head = blockIdx.y, img = blockIdx.z;
+  const int T = (p.kv_len + KT - 1) / KT;
+  const int ntiles = (p.rows - q0 > QT) ? 2 : 1;
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int s = 0; s < NS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); }
+    for (int t = 0; t < 2; ++t) { mbar_init(&s_full[t], 1); mbar_init(&p_full[t], QT); mbar_init(&o_done[t], 1); }
+    mbar_fence_init();
+    tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+  }
+  if (warp == 9) { tmem_alloc(tmem_slot, Cfg::kTmemCols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();  // set-up above overlaps the previous kernel; Q / K / V and the output are touched only from here
+
+  // A softmax thread holds a whole score row (128 fp32) in registers, so the register file is re-divided
+  // between the warpgroups: 2 x 128 x 216 + 128 x 40 <= 64 K registers.
+  if (warp >= 8) {
+   asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+   if (warp == 8) {
+    if (lane == 0) {
+      mbar_expect_tx(q_full, ntiles * Cfg::kQBytes);
+      for (int t = 0; t < ntiles; ++t)
+        for (int a = 0; a < HD / 64; ++a)
+          tma_load_2d(q_s + t * Cfg::kQBytes + a * (QT * 128), &tmQ, head * HD + a * 64, img * p.rows + q0 + t * QT, q_full);
+      for (int j = 0; j < T; ++j) {
+        const int s = j % NS;
+        const uint32_t ph = (j / NS) & 1;
+        if (!mbar_wait(&k_empty[s], ph ^ 1)) { report(p.status, DEV_TIMEOUT_TMA); break; }
+        mbar_expect_tx(&k_full[s], Cfg::kKBytes);
+        for (int a = 0; a < HD / 64; ++a)
+          tma_load_2d(k_s + s * Cfg::kKBytes + a * (KT * 128), &tmK, head * HD + a * 64, img * p.kv_capacity + j * KT, &k_full[s]);
+        if (!mbar_wait(&v_empty[s], ph ^ 1)) { report(p.status, DEV_TIMEOUT_TMA); break; }
+        mbar_expect_tx(&v_full[s], Cfg::kVBytes);
+        for (int a = 0; a < KT / 64; ++a)
+          tma_load_2d(v_s + s * Cfg::kVBytes + a * (HD * 128), &tmV, j * KT + a * 64, img * p.C + head * HD, &v_full[s]);
+      }
+    }
+  } else if (warp == 9) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = umma_idesc_bf16(QT, KT);
+      constexpr uint32_t idesc_pv = umma_idesc_bf16(QT, HD);
+      const uint32_t q_addr = smem_u32(q_s);
+      // S_t = Q_t K^T for the key tile in stage s
+      auto issue_qk = [&](int t, int s) {
+        const uint32_t k_addr = smem_u32(k_s + s * Cfg::kKBytes);
+        const uint32_t qa = q_addr + t * Cfg::kQBytes;
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * (QT * 128) + (kk & 3) * 32;
+          umma_bf16(tmem_base + t * KT, umma_desc_k_sw128(qa + off), umma_desc_k_sw128(k_addr + off), idesc_qk, kk != 0);
+        }
+        umma_commit(&s_full[t]);
+      };
+      bool ok = mbar_wait(q_full, 0) && mbar_wait(&k_full[0], 0);
+      if (!ok) report(p.status, DEV_TIMEOUT_MMA);
+      if (ok) {
+        tc_fence_after();
+        for (int t = 0; t < ntiles; ++t) issue_qk(t, 0);
+        umma_commit(&k_empty[0]);
+      }
+      for (int j = 0; ok && j < T; ++j) {
+        const int s = j % NS, sn = (j + 1) % NS;
+        const bool more = j + 1 < T;
+        if (!mbar_wait(&v_full[s], (j / NS) & 1) || (more && !mbar_wait(&k_full[sn], ((j + 1) / NS) & 1))) {
+          report(p.status, DEV_TIMEOUT_MMA); ok = false; break;
+        }
+        const uint32_t v_addr = smem_u32(v_s + s * Cfg::kVBytes);
+        for (int t = 0; t < ntiles; ++t) {
+          if (!mbar_wait(&p_full[t], j & 1)) { report(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
+          tc_fence_after();
+          const uint32_t p_tmem = tmem_base + t * KT;              // P_t over the first 64 columns of S_t
+          const uint32_t o_tmem = tmem_base + 256 + t * 128;
+#pragma unroll
+          for (int kk = 0; kk < KT / 16; ++kk) {
+            const uint32_t b_off = (kk >> 2) * (HD * 128) + (kk & 3) * 32;
+            umma_bf16_ts(o_tmem, p_tmem + kk * 8, umma_desc_k_sw128(v_addr + b_off), idesc_pv, (j | kk) != 0);
+          }
+          umma_commit(&o_done[t]);
+          if (more) issue_qk(t, sn);
+        }
+        if (!ok) break;
+        umma_commit(&v_empty[s]);
+        if (more) umma_commit(&k_empty[sn]);
+      }
+    }
+   }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    // ---- softmax + output: thread = one query row of tile t ----
+    const int t = warp >> 2;
+    const int quarter = warp & 3;                 // the TMEM lanes this warp may touch
+    const int r = quarter * 32 + lane;
+    const uint32_t lane_off = uint32_t(quarter * 32) << 16;
+    const uint32_t s_addr = tmem_base + lane_off + t * KT;
+    const uint32_t o_addr = tmem_base + lane_off + 256 + t * 128;
+    if (t < ntiles) {
+      float m_run = -INFINITY, l_run = 0.f;
+      bool ok = true;
+      for (int j = 0; j < T; ++j) {
+        if (!mbar_wait(&s_full[t], j & 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); ok = false; break; }
+        tc_fence_after();
+        const int valid = p.kv_len - j * KT;  // >= 1
+        float sc[KT];
+        if (valid < KT) tile_load_scores<true>(s_addr, valid, sc);
+        else tile_load_scores<false>(s_addr, valid, sc);
+        float mx0 = sc[0], mx1 = sc[1], mx2 = sc[2], mx3 = sc[3];
+#pragma unroll
+        for (int i = 4; i < KT; i += 4) {
+          mx0 = fmaxf(mx0, sc[i]); mx1 = fmaxf(mx1, sc[i + 1]); mx2 = fmaxf(mx2, sc[i + 2]); mx3 = fmaxf(mx3, sc[i + 3]);
+        }
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+        // Raise the running maximum only when it would grow by more than the threshold: probabilities
+        // may then exceed 1 (by at most 2^threshold), which fp32 sums and bf16 P hold without loss.
+        float alpha = 1.f;
+        if (mx > m_run + kRescaleThreshold) {
+          alpha = fast_exp2(m_run - mx);  // 0 on the first tile (m_run = -inf)
+          m_run = mx;
+        }
+        // S_t of tile j was issued after P V of tile j-1, so O_t is at rest here.
+        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+          for (int c = 0; c < HD / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(o_addr + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+            tmem_st32(o_addr + c * 32, o);
+          }
+        }
+        const float rs = tile_exp_store(sc, s_addr, p.scale_log2, m_run);
+        l_run = fmaf(l_run, alpha, rs);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&p_full[t]);
+      }
+      if (ok && !mbar_wait(&o_done[t], (T - 1) & 1)) { report(p.status, DEV_TIMEOUT_SOFTMAX); ok = false; }
+      tc_fence_after();
+      if (ok) {
+        const float inv_l = 1.f / l_run;
+        const int row = q0 + t * QT + r;
+        __nv_bfloat16* dst = p.out + ((size_t)img * p.rows + row) * p.C + head * HD;
+#pragma unroll
+        for (int c = 0; c < HD / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(o_addr + c * 32, o);
+          tmem_wait_ld();
+          if (row < p.rows) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint4 v;
+              v.x = pack_bf16x2(__uint_as_float(o[8 * g + 0]) * inv_l, __uint_as_float(o[8 * g + 1]) * inv_l);
+              v.y = pack_bf16x2(__uint_as_float(o[8 * g + 2]) * inv_l, __uint_as_float(o[8 * g + 3]) * inv_l);
+              v.z = pack_bf16x2(__uint_as_float(o[8 * g + 4]) * inv_l, __uint_as_float(o[8 * g + 5]) * inv_l);
+              v.w = pack_bf16x2(__uint_as_float(o[8 * g + 6]) * inv_l, __uint_as_float(o[8 * g + 7]) * inv_l);
+              reinterpret_cast<uint4*>(dst + c * 32)[g] = v;
+            }
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+}
+
 bool make_tmap_rows(void* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
   return make_tmap_bf16_2d(out, base, rows, cols, box_rows);
 }
@@ -555,7 +763,8 @@ template <int HD> fv_status launch_hd(const AttnArgs& a, cudaStream_t st) {
     const long long most = p.total_cost / (2 * kWeightPair);   // every piece at least two key tiles long
     if (g > most) g = most;
     const long long rounds = (items + g_attn_sms - 1) / g_attn_sms;
-    const bool pays = g >= 1 && p.T >= 16 && 100 * (items * p.T / g + kSplitOverheadTiles) < 92 * rounds * p.T;
+    // (the kernel that walks pieces also takes about 15 % longer per key tile than the one that runs whole items)
+    const bool pays = g >= 1 && p.T >= 16 && 115 * (items * p.T / g + kSplitOverheadTiles) < 100 * rounds * p.T;
     if (g >= 1 && (pays || g_attn_force_ctas > 0)) {
       p.split = 1;
       ctas = g;
@@ -563,9 +772,16 @@ template <int HD> fv_status launch_hd(const AttnArgs& a, cudaStream_t st) {
       p.parts = static_cast<char*>(a.workspace) + kAttnTicketBytes;
     }
   }
-  dim3 grid((unsigned)ctas);
   LaunchScope scope(KC_ATTENTION, 1, 4.0 * a.B * (double)a.rows * a.kv_len * a.C,
                     2.0 * a.B * a.C * (2.0 * a.rows + 2.0 * a.kv_len), st);  // Q in, O out, K and V^T once
+  if (!p.split) {
+    WholeDev w;
+    w.out = p.out; w.rows = p.rows; w.C = p.C; w.kv_len = p.kv_len; w.kv_capacity = p.kv_capacity; w.scale_log2 = p.scale_log2; w.status = p.status;
+    dim3 grid3((a.rows + 2 * QT - 1) / (2 * QT), a.H, a.B);
+    return launch_pdl(attention_whole_kernel<HD>, grid3, dim3(kAttnThreads), AttnCfg<HD>::kSmemBytes, st, tmQ, tmK, tmV, w) == cudaSuccess
+               ? FV_OK : FV_ERR_CUDA;
+  }
+  dim3 grid((unsigned)ctas);
   return launch_pdl(attention_kernel<HD>, grid, dim3(kAttnThreads), AttnCfg<HD>::kSmemBytes, st, tmQ, tmK, tmV, p) == cudaSuccess
              ? FV_OK : FV_ERR_CUDA;
 }
@@ -582,6 +798,8 @@ cudaError_t attention_init() {
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_attn_sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<64>::kSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attention_whole_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<64>::kSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attention_whole_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<128>::kSmemBytes);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<128>::kSmemBytes);
 }

@@ -16,6 +16,43 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // launched this way executes pdl_wait() before its first access to global memory that an earlier
 // kernel may write or read.
 #ifdef __CUDACC__
+}  // namespace fv
+#include <cuda_bf16.h>
+namespace fv {
+// Four / eight consecutive elements of the residual stream, fp32 or bf16, as floats.  NC: read-only path, else through L2.
+template <bool NC> __device__ __forceinline__ float4 x_load4(const float* p) {
+  return NC ? __ldg(reinterpret_cast<const float4*>(p)) : __ldcg(reinterpret_cast<const float4*>(p));
+}
+template <bool NC> __device__ __forceinline__ float4 x_load4(const __nv_bfloat16* p) {
+  const uint2 u = NC ? __ldg(reinterpret_cast<const uint2*>(p)) : __ldcg(reinterpret_cast<const uint2*>(p));
+  return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u), __uint_as_float(u.y << 16), __uint_as_float(u.y & 0xFFFF0000u));
+}
+__device__ __forceinline__ void x_load8(const float* p, float (&f)[8]) {
+  const float4 a = reinterpret_cast<const float4*>(p)[0], b = reinterpret_cast<const float4*>(p)[1];
+  f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+}
+__device__ __forceinline__ void x_load8(const __nv_bfloat16* p, float (&f)[8]) {
+  const uint4 v = *reinterpret_cast<const uint4*>(p);
+  const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(u[i] << 16); f[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u); }
+}
+__device__ __forceinline__ void x_store8(float* p, const float (&f)[8]) {
+  reinterpret_cast<float4*>(p)[0] = make_float4(f[0], f[1], f[2], f[3]);
+  reinterpret_cast<float4*>(p)[1] = make_float4(f[4], f[5], f[6], f[7]);
+}
+// bf16 stream: the updated values are rounded to nearest even once, and those rounded values are what is stored,
+// summed and scored from then on (f is overwritten with them).
+__device__ __forceinline__ void x_store8(__nv_bfloat16* p, float (&f)[8]) {
+  uint32_t u[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    u[i] = *reinterpret_cast<const uint32_t*>(&v);
+    f[2 * i] = __uint_as_float(u[i] << 16); f[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
+  }
+  *reinterpret_cast<uint4*>(p) = make_uint4(u[0], u[1], u[2], u[3]);
+}
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 template <typename... KArgs, typename... Args>
@@ -63,8 +100,9 @@ SelectWs select_ws_carve(void* workspace, int B, int n, int C);
 // Scores [B,n] (fp32), then exact per-image top-k -> idx [B,k] ascending, inv [B,n].  have_partials:
 // the group partials in the workspace already hold the column sums of x (left there by
 // launch_restore_residual), so the column-sum pass is skipped.
-cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* idx, int32_t* inv, float* score,
-                          int32_t* near_tie, void* workspace, bool have_partials, cudaStream_t st);
+// x_bf16 (select, gather, restore launchers): the residual stream is bf16 instead of fp32 (fv_config.resid_dtype).
+cudaError_t launch_select(const void* x, int B, int n, int C, int k, int32_t* idx, int32_t* inv, float* score,
+                          int32_t* near_tie, void* workspace, bool have_partials, cudaStream_t st, bool x_bf16 = false);
 // The selection of a wrapped sublayer inside a scale step, in one launch with what surrounds it on the kept rows:
 // the previous sublayer's kept-row restoration before it (y != null) and the gather + LayerNorm + modulation of the
 // newly kept rows after it.  sel_ws holds the column sums of the rows the kernel does not update itself (left there
@@ -90,17 +128,17 @@ cudaError_t select_init();  // one-time function attributes
 // ---- rows.cu : gather + LayerNorm + modulate, restore (+ gate and residual) ----------------------
 // status (all gathers): device status word that receives DEV_BAD_ROW_INDEX when an index lies outside [0, n) (the
 // index is clamped, so the read stays inside the map), or null.
-cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
-                             const float* beta, int mod_stride, void* a_out, int32_t* status, cudaStream_t st);
+cudaError_t launch_gather_ln(const void* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
+                             const float* beta, int mod_stride, void* a_out, int32_t* status, cudaStream_t st, bool x_bf16 = false);
 // A wait nobody ends: one warp waits on an mbarrier without arrivals for limit_ns, then writes DEV_TIMEOUT_SELFTEST.
 cudaError_t launch_expired_wait(int32_t* status, unsigned long long limit_ns, cudaStream_t st);
 // colsum_ws: null, or the selection workspace that receives the column sums of the updated x.
 // part: 0 = every row; 1 = the rows that were not kept; 2 = the kept rows (and the fold of the column sums);
 // 3 = the rows that were not kept, their column sums folded (the kept rows are left to the next fused selection).
 // interp_mode (all restore launchers): 0 nearest, 1 bilinear with half-pixel centres.
-cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv,
+cudaError_t launch_restore_residual(void* x, const void* y, const void* cache, const int32_t* inv,
                                     const float* gamma, int mod_stride, int B, int k, int h, int w, int hc, int wc,
-                                    int C, void* colsum_ws, int part, int interp_mode, cudaStream_t st);
+                                    int C, void* colsum_ws, int part, int interp_mode, cudaStream_t st, bool x_bf16 = false);
 cudaError_t rows_init();               // one-time function attributes
 void restore_force_fold(int mode);     // test hook: 0 by shape, 1 fold through global memory, 2 fold inside clusters
 // Per-step granularity: fp32 gather of the kept rows, and fp32 restoration of the step's output map.
@@ -111,7 +149,8 @@ cudaError_t launch_restore_bf16(const void* cache, int hc, int wc, const void* p
                                 int k, int h, int w, int C, void* out, int interp_mode, cudaStream_t st);
 
 // ---- gemm.cu : tcgen05 GEMM with fused epilogues -----------------------------------------------
-enum GemmEpilogue : int { EPI_BF16 = 0, EPI_GELU_BF16 = 1, EPI_RESIDUAL = 2, EPI_QKV_SPLIT = 3, EPI_F32 = 4 };
+enum GemmEpilogue : int { EPI_BF16 = 0, EPI_GELU_BF16 = 1, EPI_RESIDUAL = 2, EPI_QKV_SPLIT = 3, EPI_F32 = 4,
+                          EPI_RESIDUAL_XBF16 = 5 /* as EPI_RESIDUAL with a bf16 residual stream: out bf16 [M,N] in place */ };
 struct GemmArgs {
   const void* a;     // [M,K] bf16
   const void* w;     // [N,K] bf16

@@ -22,7 +22,8 @@ constexpr int kMaxVec = 16;  // float4 per lane -> C <= 2048
 
 // grid (ceil(k / 8), B): one warp per kept row; sigma / beta of the image staged in shared memory while
 // the row index and the row itself are in flight.
-__global__ void __launch_bounds__(256) gather_ln_kernel(const float4* __restrict__ x, const int32_t* __restrict__ idx, int n,
+template <typename XT>
+__global__ void __launch_bounds__(256) gather_ln_kernel(const XT* __restrict__ x, const int32_t* __restrict__ idx, int n,
                                                         int k, int C4, const float* __restrict__ sigma,
                                                         const float* __restrict__ beta, int mod_stride,
                                                         uint2* __restrict__ a_out, int32_t* status) {
@@ -42,14 +43,14 @@ __global__ void __launch_bounds__(256) gather_ln_kernel(const float4* __restrict
     const float4* bt = reinterpret_cast<const float4*>(beta + (size_t)b * mod_stride);
     for (int i = threadIdx.x; i < C4; i += 256) { s_mod[i] = __ldg(sg + i); s_mod[C4 + i] = __ldg(bt + i); }
   }
-  const float4* row = x + ((size_t)b * n + t) * C4;
+  const XT* row = x + ((size_t)b * n + t) * C4 * 4;
   float4 v[kMaxVec];
   float sum = 0.f;
   if (live) {
 #pragma unroll
     for (int i = 0; i < kMaxVec; ++i) {
       const int c4 = lane + 32 * i;
-      if (c4 < C4) v[i] = __ldg(row + c4);
+      if (c4 < C4) v[i] = x_load4<true>(row + (size_t)c4 * 4);
     }
 #pragma unroll
     for (int i = 0; i < kMaxVec; ++i) {
@@ -167,7 +168,8 @@ __device__ __forceinline__ void bf16x8_to_float(const uint4& p, float (&f)[8]) {
 //   branch has produced y: column sums continue from the chunk partial of part 1, then the group fold);
 //   3 : as 1, but the sums of the rows that were not kept are folded here (the kept rows are then restored, and
 //   summed, by the next selection's kernel).
-__global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restrict__ x, const uint4* __restrict__ y,
+template <typename XT>
+__global__ void __launch_bounds__(256) restore_residual_kernel(XT* __restrict__ x, const uint4* __restrict__ y,
                                                                const uint4* __restrict__ cache, const int32_t* __restrict__ inv,
                                                                const float* __restrict__ gamma, int mod_stride, int n, int k,
                                                                int h, int w, int hc, int wc, int C8, int nchunks, int group,
@@ -189,7 +191,7 @@ __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restric
     s_on[threadIdx.x] = part == 0 || (part == 1 || part == 3) == (j < 0);
   }
   __syncthreads();
-  float4* xbase = x + ((size_t)b * n + t0) * C8 * 2;
+  XT* xbase = x + ((size_t)b * n + t0) * C8 * 8;
   for (int c8 = threadIdx.x; c8 < C8; c8 += 256) {
     float4 g0 = make_float4(1.f, 1.f, 1.f, 1.f), g1 = g0;
     if (gamma) {
@@ -203,12 +205,11 @@ __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restric
     }
     for (int r = 0; r < rows; r += 4) {
       uint4 p[4];
-      float4 x0[4], x1[4];
+      float xv[4][8];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         if (r + i < rows && s_on[r + i]) {
-          float4* xr = xbase + (size_t)(r + i) * C8 * 2 + 2 * c8;
-          x0[i] = xr[0]; x1[i] = xr[1];
+          x_load8(xbase + ((size_t)(r + i) * C8 + c8) * 8, xv[i]);
           p[i] = __ldg(s_src[r + i] + c8);
         }
       }
@@ -217,18 +218,17 @@ __global__ void __launch_bounds__(256) restore_residual_kernel(float4* __restric
         if (r + i < rows && s_on[r + i]) {
           float f[8];
           bf16x8_to_float(p[i], f);
-          float4 u0 = x0[i], u1 = x1[i];
+          float (&u)[8] = xv[i];
           if (gamma) {
-            u0.x = fmaf(g0.x, f[0], u0.x); u0.y = fmaf(g0.y, f[1], u0.y); u0.z = fmaf(g0.z, f[2], u0.z); u0.w = fmaf(g0.w, f[3], u0.w);
-            u1.x = fmaf(g1.x, f[4], u1.x); u1.y = fmaf(g1.y, f[5], u1.y); u1.z = fmaf(g1.z, f[6], u1.z); u1.w = fmaf(g1.w, f[7], u1.w);
+            u[0] = fmaf(g0.x, f[0], u[0]); u[1] = fmaf(g0.y, f[1], u[1]); u[2] = fmaf(g0.z, f[2], u[2]); u[3] = fmaf(g0.w, f[3], u[3]);
+            u[4] = fmaf(g1.x, f[4], u[4]); u[5] = fmaf(g1.y, f[5], u[5]); u[6] = fmaf(g1.z, f[6], u[6]); u[7] = fmaf(g1.w, f[7], u[7]);
           } else {
-            u0.x += f[0]; u0.y += f[1]; u0.z += f[2]; u0.w += f[3];
-            u1.x += f[4]; u1.y += f[5]; u1.z += f[6]; u1.w += f[7];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) u[e] += f[e];
           }
-          float4* xr = xbase + (size_t)(r + i) * C8 * 2 + 2 * c8;
-          xr[0] = u0; xr[1] = u1;
-          a0.x += u0.x; a0.y += u0.y; a0.z += u0.z; a0.w += u0.w;
-          a1.x += u1.x; a1.y += u1.y; a1.z += u1.z; a1.w += u1.w;
+          x_store8(xbase + ((size_t)(r + i) * C8 + c8) * 8, u);     // a bf16 stream: u now holds the stored (rounded) values
+          a0.x += u[0]; a0.y += u[1]; a0.z += u[2]; a0.w += u[3];
+          a1.x += u[4]; a1.y += u[5]; a1.z += u[6]; a1.w += u[7];
         }
       }
     }
@@ -402,7 +402,7 @@ __global__ void __launch_bounds__(256) restore_kept_cluster_kernel(float4* __res
 // and column-sum handling; fewer rows in flight (two, or one with sixteen source rows).  part 2 (kept rows only) never interpolates and
 // runs the kernel above.
 template <int TAPS>
-__global__ void __launch_bounds__(256) restore_residual_interp_kernel(float4* __restrict__ x, const uint4* __restrict__ y,
+__global__ void __launch_bounds__(256) restore_residual_interp_kernel(float* __restrict__ xf, const uint4* __restrict__ y,
                                                                         const uint4* __restrict__ cache, const int32_t* __restrict__ inv,
                                                                         const float* __restrict__ gamma, int mod_stride, int n, int k,
                                                                         int h, int w, int hc, int wc, int C8, int nchunks, int group,
@@ -410,6 +410,7 @@ __global__ void __launch_bounds__(256) restore_residual_interp_kernel(float4* __
                                                                         float4* __restrict__ group_partial, unsigned int* tickets,
                                                                         int part) {
   constexpr int ROWS = TAPS == 4 ? 2 : 1;   // rows in flight per thread
+  float4* x = reinterpret_cast<float4*>(xf);
   __shared__ const uint4* s_src[kColsumRows][TAPS];
   __shared__ float s_wt[kColsumRows][TAPS];
   __shared__ int s_on[kColsumRows];
@@ -587,17 +588,21 @@ cudaError_t rows_init() {
   return cudaSuccess;
 }
 
-cudaError_t launch_gather_ln(const float* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
-                             const float* beta, int mod_stride, void* a_out, int32_t* status, cudaStream_t st) {
+cudaError_t launch_gather_ln(const void* x, const int32_t* idx, int B, int n, int k, int C, const float* sigma,
+                             const float* beta, int mod_stride, void* a_out, int32_t* status, cudaStream_t st, bool x_bf16) {
   const int rows = B * k;
-  LaunchScope scope(KC_GATHER_LN, 1, (double)rows * C * 6.0, (double)rows * C * 6.0, st);
-  return launch_pdl(gather_ln_kernel, dim3((k + 7) / 8, B), dim3(256), sigma ? (size_t)C * 8 : 0, st, reinterpret_cast<const float4*>(x),
+  const double bytes = (double)rows * C * (x_bf16 ? 4.0 : 6.0);
+  LaunchScope scope(KC_GATHER_LN, 1, bytes, bytes, st);
+  if (x_bf16)
+    return launch_pdl(gather_ln_kernel<__nv_bfloat16>, dim3((k + 7) / 8, B), dim3(256), sigma ? (size_t)C * 8 : 0, st,
+                      static_cast<const __nv_bfloat16*>(x), idx, n, k, C / 4, sigma, beta, mod_stride, reinterpret_cast<uint2*>(a_out), status);
+  return launch_pdl(gather_ln_kernel<float>, dim3((k + 7) / 8, B), dim3(256), sigma ? (size_t)C * 8 : 0, st, static_cast<const float*>(x),
                     idx, n, k, C / 4, sigma, beta, mod_stride, reinterpret_cast<uint2*>(a_out), status);
 }
 
-cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, const int32_t* inv, const float* gamma,
+cudaError_t launch_restore_residual(void* x, const void* y, const void* cache, const int32_t* inv, const float* gamma,
                                     int mod_stride, int B, int k, int h, int w, int hc, int wc, int C, void* colsum_ws,
-                                    int part, int interp_mode, cudaStream_t st) {
+                                    int part, int interp_mode, cudaStream_t st, bool x_bf16) {
   const int n = h * w;
   SelectWs ws{};
   if (colsum_ws) ws = select_ws_carve(colsum_ws, B, n, C);
@@ -605,8 +610,16 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
   // algorithmic bytes of the part: x read + written for its rows, its source rows
   const bool unkept_only = part == 1 || part == 3;
   const double rows_x = part == 0 ? (double)n : (unkept_only ? (double)(n - k) : (double)k);
-  const double rr_bytes = (double)B * C * (8.0 * rows_x + (!unkept_only ? 2.0 * k : 0.0) + (part != 2 ? 2.0 * hc * wc : 0.0));
+  const double rr_bytes = (double)B * C * ((x_bf16 ? 4.0 : 8.0) * rows_x + (!unkept_only ? 2.0 * k : 0.0) + (part != 2 ? 2.0 * hc * wc : 0.0));
   LaunchScope scope(KC_RESTORE, 1, rr_bytes, rr_bytes, st);
+  if (x_bf16) {   // bf16 residual stream: the generic kernel (nearest interpolation, fold through global memory)
+    if (interp_mode != 0) return cudaErrorNotSupported;
+    restore_residual_kernel<__nv_bfloat16><<<dim3(nchunks, B), 256, 0, st>>>(
+        static_cast<__nv_bfloat16*>(x), reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h, w,
+        hc, wc, C / 8, nchunks, ws.group, ws.ngroups, reinterpret_cast<float4*>(ws.chunk_partial), reinterpret_cast<float4*>(ws.group_partial),
+        ws.tickets, part);
+    return cudaGetLastError();
+  }
   // kept rows + group fold inside clusters (one cluster per group of chunks) where the group fits a cluster
   if (part == 2 && colsum_ws && g_cluster_fold_ok && g_fold_mode != 1 && ws.group >= 1 && ws.group <= 8 && C / 8 <= 256) {
     cudaLaunchConfig_t cfg{};
@@ -621,16 +634,16 @@ cudaError_t launch_restore_residual(float* x, const void* y, const void* cache, 
     if (e == cudaSuccess || g_fold_mode == 2) return e;
     (void)cudaGetLastError();      // this cluster size cannot be scheduled here: the fold through global memory instead
   }
-  auto* kern = (interp_mode == 0 || part == 2) ? restore_residual_kernel
+  auto* kern = (interp_mode == 0 || part == 2) ? restore_residual_kernel<float>
                : (interp_mode == 1 ? restore_residual_interp_kernel<4> : restore_residual_interp_kernel<16>);
   if (part == 0)
-    return launch_pdl(kern, dim3(nchunks, B), dim3(256), 0, st, reinterpret_cast<float4*>(x),
+    return launch_pdl(kern, dim3(nchunks, B), dim3(256), 0, st, static_cast<float*>(x),
                       reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h, w, hc, wc,
                       C / 8, nchunks, ws.group, ws.ngroups, reinterpret_cast<float4*>(ws.chunk_partial),
                       reinterpret_cast<float4*>(ws.group_partial), ws.tickets, part);
   // The two halves of a split restoration are ordered against another stream by events: they are
   // launched as ordinary stream work, not as programmatic dependents.
-  kern<<<dim3(nchunks, B), 256, 0, st>>>(reinterpret_cast<float4*>(x), reinterpret_cast<const uint4*>(y),
+  kern<<<dim3(nchunks, B), 256, 0, st>>>(static_cast<float*>(x), reinterpret_cast<const uint4*>(y),
                                          reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h, w, hc, wc, C / 8, nchunks,
                                          ws.group, ws.ngroups, reinterpret_cast<float4*>(ws.chunk_partial),
                                          reinterpret_cast<float4*>(ws.group_partial), ws.tickets, part);

@@ -28,7 +28,8 @@ constexpr int kTopkWarps = kTopkThreads / 32;
 __device__ __forceinline__ int KI(int i) { return i + (i >> 5); }
 constexpr size_t kTopkMaxSmem = ((size_t)kTopkMaxTokens + kTopkMaxTokens / 32 + 1) * 4;
 
-__global__ void __launch_bounds__(256) colsum_chunk_kernel(const float4* __restrict__ x, int n, int C4, int nchunks, int group,
+template <typename XT>
+__global__ void __launch_bounds__(256) colsum_chunk_kernel(const XT* __restrict__ x, int n, int C4, int nchunks, int group,
                                                            int ngroups, float4* __restrict__ chunk_partial,
                                                            float4* __restrict__ group_partial, unsigned int* tickets) {
   pdl_trigger();
@@ -36,19 +37,19 @@ __global__ void __launch_bounds__(256) colsum_chunk_kernel(const float4* __restr
   const int b = blockIdx.y, chunk = blockIdx.x;
   const int r0 = chunk * kColsumRows;
   const int r1 = min(n, r0 + kColsumRows);
-  const float4* base = x + (size_t)b * n * C4;
+  const XT* base = x + (size_t)b * n * C4 * 4;
   for (int c4 = threadIdx.x; c4 < C4; c4 += blockDim.x) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     int r = r0;
     for (; r + 8 <= r1; r += 8) {
       float4 v[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) v[i] = __ldg(base + (size_t)(r + i) * C4 + c4);
+      for (int i = 0; i < 8; ++i) v[i] = x_load4<true>(base + ((size_t)(r + i) * C4 + c4) * 4);
 #pragma unroll
       for (int i = 0; i < 8; ++i) { acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w; }
     }
     for (; r < r1; ++r) {
-      const float4 v = __ldg(base + (size_t)r * C4 + c4);
+      const float4 v = x_load4<true>(base + ((size_t)r * C4 + c4) * 4);
       acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
     }
     chunk_partial[((size_t)b * nchunks + chunk) * C4 + c4] = acc;
@@ -111,17 +112,17 @@ __device__ __forceinline__ void mean_from_partials(float4* s_mean, const float4*
 // over its rows.  NC: the map was not written by this kernel, so its rows may take the read-only path; the fused
 // kernel, whose other CTAs have just updated rows of it, reads them through L2.
 // BATCH: 16-byte loads a lane requests together (8 with 64 registers per thread, 16 with 128).
-template <bool NC, int BATCH>
-__device__ __forceinline__ void score_rows(const float4* x, const float4* s_mean, int b, int n, int C4, float* __restrict__ score) {
+template <bool NC, int BATCH, typename XT>
+__device__ __forceinline__ void score_rows(const XT* x, const float4* s_mean, int b, int n, int C4, float* __restrict__ score) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int r = blockIdx.x * kTopkWarps + warp; r < n; r += gridDim.x * kTopkWarps) {
-    const float4* row = x + ((size_t)b * n + r) * C4;
+    const XT* row = x + ((size_t)b * n + r) * C4 * 4;
     float acc = 0.f;
     int c4 = lane;
     for (; c4 + 32 * (BATCH - 1) < C4; c4 += 32 * BATCH) {
       float4 v[BATCH];
 #pragma unroll
-      for (int i = 0; i < BATCH; ++i) v[i] = NC ? __ldg(row + c4 + 32 * i) : __ldcg(row + c4 + 32 * i);
+      for (int i = 0; i < BATCH; ++i) v[i] = x_load4<NC>(row + (size_t)(c4 + 32 * i) * 4);
 #pragma unroll
       for (int i = 0; i < BATCH; ++i) {
         const float4 m = s_mean[c4 + 32 * i];
@@ -130,7 +131,7 @@ __device__ __forceinline__ void score_rows(const float4* x, const float4* s_mean
       }
     }
     for (; c4 < C4; c4 += 32) {
-      const float4 v = NC ? __ldg(row + c4) : __ldcg(row + c4);
+      const float4 v = x_load4<NC>(row + (size_t)c4 * 4);
       const float4 m = s_mean[c4];
       const float dx = v.x - m.x, dy = v.y - m.y, dz = v.z - m.z, dw = v.w - m.w;
       acc += dx * dx; acc += dy * dy; acc += dz * dz; acc += dw * dw;
@@ -157,11 +158,34 @@ __device__ __forceinline__ void topk_image(const float* __restrict__ sc, int n, 
   // Keys are taken relative to the smallest key of the image: the scores of one map share their leading bits, and
   // ranking only the bits that differ both skips passes and spreads the keys over the histogram bins.
   uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-  for (int i = tid; i < n; i += kTopkThreads) {
-    const uint32_t key = __float_as_uint(__ldcg(sc + i)) & 0x7FFFFFFFu;  // drops the sign of -0
+  // the scores come from L2: up to eight 16-byte loads per thread are requested before the first is used (one CTA
+  // fetching them one dependent load at a time took longer than the ranking itself)
+  const int n4 = (n % 4 == 0 && (reinterpret_cast<uintptr_t>(sc) & 15u) == 0) ? n / 4 : 0;
+  for (int i0 = tid; i0 < n4; i0 += kTopkThreads * 8) {
+    float4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (i0 + u * kTopkThreads < n4) v[u] = __ldcg(reinterpret_cast<const float4*>(sc) + i0 + u * kTopkThreads);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i4 = i0 + u * kTopkThreads;
+      if (i4 < n4) {
+        const float f[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const uint32_t key = __float_as_uint(f[e]) & 0x7FFFFFFFu;  // drops the sign of -0
+          s_keys[KI(4 * i4 + e)] = key;
+          kmin = min(kmin, key); kmax = max(kmax, key);
+        }
+      }
+    }
+  }
+  for (int i = 4 * n4 + tid; i < n; i += kTopkThreads) {
+    const uint32_t key = __float_as_uint(__ldcg(sc + i)) & 0x7FFFFFFFu;
     s_keys[KI(i)] = key;
     kmin = min(kmin, key); kmax = max(kmax, key);
   }
+  __syncthreads();   // a thread's keys were written by other threads
   kmin = __reduce_min_sync(0xffffffffu, kmin);
   kmax = __reduce_max_sync(0xffffffffu, kmax);
   if (lane == 0) { sh.warp[warp] = kmin; sh.hist[warp] = kmax; }
@@ -260,7 +284,8 @@ __device__ __forceinline__ void topk_image(const float* __restrict__ sc, int n, 
 
 // grid (CTAs per image, B), 512 threads, sized to be resident all at once (two CTAs per SM); the warps of
 // an image stride over its token rows.  Dynamic shared memory max(C, n + n/32) * 4 bytes (mean token, then keys).
-__global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float4* __restrict__ x,
+template <typename XT>
+__global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const XT* __restrict__ x,
                                                                   const float4* __restrict__ group_partial, int ngroups, int n,
                                                                   int C4, int k, float* __restrict__ score,
                                                                   unsigned int* img_tickets, int32_t* __restrict__ idx,
@@ -275,7 +300,7 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const float
   pdl_wait();
   mean_from_partials(s_mean, group_partial + (size_t)b * ngroups * C4, ngroups, nullptr, 0, C4, n);
   __syncthreads();
-  score_rows<true, 8>(x, s_mean, b, n, C4, score);
+  score_rows<true, 8, XT>(x, s_mean, b, n, C4, score);
   __threadfence();  // this thread's scores are visible device-wide before the CTA takes its ticket
 
   // ---- the last CTA of this image to get here ranks the image
@@ -505,7 +530,7 @@ __global__ void __launch_bounds__(kTopkThreads, 1) select_fused_kernel(const Fus
   mean_from_partials(s_dyn, a.group_partial + (size_t)b * a.ngroups * C4, a.ngroups,
                      a.y ? a.kept_group + (size_t)b * a.ngk * C4 : nullptr, a.y ? a.ngk : 0, C4, n);
   __syncthreads();
-  score_rows<false, 16>(a.x, s_dyn, b, n, C4, a.score);
+  score_rows<false, 16, float>(reinterpret_cast<const float*>(a.x), s_dyn, b, n, C4, a.score);
   __threadfence();
   __syncthreads();
   if (tid == 0) {
@@ -604,6 +629,7 @@ SelectWs select_ws_carve(void* workspace, int B, int n, int C) {
   return w;
 }
 
+
 static int g_num_sms = 148;
 
 cudaError_t select_init() {
@@ -611,21 +637,18 @@ cudaError_t select_init() {
   cudaError_t e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(score_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkMaxSmem);
+  e = cudaFuncSetAttribute(score_topk_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkMaxSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(score_topk_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkMaxSmem);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(select_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkMaxSmem);
 }
 
-cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* idx, int32_t* inv, float* score,
-                          int32_t* near_tie, void* workspace, bool have_partials, cudaStream_t st) {
+template <typename XT>
+static cudaError_t launch_select_t(const XT* x, int B, int n, int C, int k, int32_t* idx, int32_t* inv, float* sc, int32_t* near_tie,
+                                   const SelectWs& w, bool have_partials, cudaStream_t st) {
   const int C4 = C / 4;
-  const SelectWs w = select_ws_carve(workspace, B, n, C);
-  float* sc = score ? score : w.score;
-  const double sel_bytes = (double)B * n * C * 4.0 + 4.0 * B * n + 4.0 * B * ((double)k + n);
-  // the stand-alone column-sum pass reads the map a second time
-  LaunchScope scope(KC_SELECT, have_partials ? 1 : 2, sel_bytes, sel_bytes + (have_partials ? 0.0 : (double)B * n * C * 4.0), st);
   if (!have_partials)
-    launch_pdl(colsum_chunk_kernel, dim3(w.nchunks, B), dim3(256), 0, st, reinterpret_cast<const float4*>(x), n, C4, w.nchunks, w.group,
+    launch_pdl(colsum_chunk_kernel<XT>, dim3(w.nchunks, B), dim3(256), 0, st, x, n, C4, w.nchunks, w.group,
                w.ngroups, reinterpret_cast<float4*>(w.chunk_partial), reinterpret_cast<float4*>(w.group_partial), w.tickets);
   const size_t keys_smem = ((size_t)n + n / 32 + 1) * 4;
   const size_t smem = keys_smem > (size_t)C * 4 ? keys_smem : (size_t)C * 4;
@@ -634,10 +657,22 @@ cudaError_t launch_select(const float* x, int B, int n, int C, int k, int32_t* i
   const int need = (n + kTopkWarps - 1) / kTopkWarps;
   if (per_image > need) per_image = need;
   if (per_image < 1) per_image = 1;
-  launch_pdl(score_topk_kernel, dim3(per_image, B), dim3(kTopkThreads), smem, st, reinterpret_cast<const float4*>(x),
+  launch_pdl(score_topk_kernel<XT>, dim3(per_image, B), dim3(kTopkThreads), smem, st, x,
              reinterpret_cast<const float4*>(w.group_partial), w.ngroups, n, C4, k, sc, w.tickets + (size_t)B * kMaxGroups, idx, inv,
              near_tie);
   return cudaGetLastError();
+}
+
+cudaError_t launch_select(const void* x, int B, int n, int C, int k, int32_t* idx, int32_t* inv, float* score,
+                          int32_t* near_tie, void* workspace, bool have_partials, cudaStream_t st, bool x_bf16) {
+  const SelectWs w = select_ws_carve(workspace, B, n, C);
+  float* sc = score ? score : w.score;
+  const double es = x_bf16 ? 2.0 : 4.0;
+  const double sel_bytes = (double)B * n * C * es + 4.0 * B * n + 4.0 * B * ((double)k + n);
+  // the stand-alone column-sum pass reads the map a second time
+  LaunchScope scope(KC_SELECT, have_partials ? 1 : 2, sel_bytes, sel_bytes + (have_partials ? 0.0 : (double)B * n * C * es), st);
+  if (x_bf16) return launch_select_t(static_cast<const __nv_bfloat16*>(x), B, n, C, k, idx, inv, sc, near_tie, w, have_partials, st);
+  return launch_select_t(static_cast<const float*>(x), B, n, C, k, idx, inv, sc, near_tie, w, have_partials, st);
 }
 
 // ---- the fused selection of a scale step
@@ -709,7 +744,7 @@ cudaError_t launch_select_fused(const FusedSelect& f, cudaStream_t st) {
 cudaError_t launch_colsum(const float* x, int B, int n, int C, void* workspace, cudaStream_t st) {
   const SelectWs w = select_ws_carve(workspace, B, n, C);
   LaunchScope scope(KC_SELECT, 1, (double)B * n * C * 4.0, (double)B * n * C * 4.0, st);
-  return launch_pdl(colsum_chunk_kernel, dim3(w.nchunks, B), dim3(256), 0, st, reinterpret_cast<const float4*>(x), n, C / 4, w.nchunks, w.group,
+  return launch_pdl(colsum_chunk_kernel<float>, dim3(w.nchunks, B), dim3(256), 0, st, x, n, C / 4, w.nchunks, w.group,
                     w.ngroups, reinterpret_cast<float4*>(w.chunk_partial), reinterpret_cast<float4*>(w.group_partial), w.tickets);
 }
 

@@ -196,19 +196,19 @@ ZERO_BRANCH_CASES = [  # h, w, hc, wc, C, H, B, B_max, keep, kind, oracle_runs_t
 ]
 
 
-@pytest.mark.parametrize("unfused", [0, 1])
+@pytest.mark.parametrize("fused", [0, 1])
 @pytest.mark.parametrize("h,w,hc,wc,C,H,B,B_max,keep,kind,full_oracle", ZERO_BRANCH_CASES)
-def test_every_selection_of_a_step_on_bit_identical_input(h, w, hc, wc, C, H, B, B_max, keep, kind, full_oracle, unfused):
+def test_every_selection_of_a_step_on_bit_identical_input(h, w, hc, wc, C, H, B, B_max, keep, kind, full_oracle, fused):
     """Inside fv_var_step only the first selection sums the token map itself; every later one takes Eq. 4's column
     sums from the restoration before it (rows that were not kept on a side stream, kept rows + fold after the last
     GEMM).  With every branch ending in a zero projection and zero sublayer caches, each restoration adds exactly 0,
     so x entering EVERY sublayer is bit-identical on both sides and each of the 2 blocks x 3 selections must keep
     the oracle's set (any difference on a near-tie at the threshold, within 1e-5 relative).  Runs at the bench
-    shapes' maps, at ragged chunk / group counts and with a partial batch, in both forms the step has: one fused
-    launch per selection (kept rows of the previous sublayer restored and summed inside it, grid-wide wait, gather
-    of the new rows) and the separate kernels."""
-    if full_oracle and unfused:
-        full_oracle = False          # the oracle's own step was run in the fused case
+    shapes' maps, at ragged chunk / group counts and with a partial batch, in both forms the step has: the separate
+    kernels (the default) and one fused launch per selection (kept rows of the previous sublayer restored and
+    summed inside it, grid-wide wait, gather of the new rows)."""
+    if full_oracle and fused:
+        full_oracle = False          # the oracle's own step is run once, in the default form
     wl = I.Workload("zero-branch", L=2, C=C, H=H, B=B_max, sides=(hc, h), keep=(1.0, keep), cross_len=64, mlp_ratio=1, seed=811)
     mt = _zero_branch_tensors(wl)
     n, k = h * w, O.kept_count(keep, h, w)
@@ -221,11 +221,11 @@ def test_every_selection_of_a_step_on_bit_identical_input(h, w, hc, wc, C, H, B,
     ctx.prepare_text(B)
     trace = torch.full((wl.L, 3, B, k), -1, dtype=torch.int32, device=DEV)
     xd = torch.from_numpy(x).to(DEV)
-    assert fv.lib().fv_step_force_unfused(unfused) == 0
+    assert fv.lib().fv_step_fused_selection(fused) == 0
     try:
         got = ctx.var_step(xd, 1, keep, idx_trace=trace).cpu().numpy()
     finally:
-        fv.lib().fv_step_force_unfused(0)
+        fv.lib().fv_step_fused_selection(0)
     assert ctx.device_status() == 0 and ctx.state() == (2, k)
     assert np.array_equal(got, x), "a zero branch changed the residual stream"
     # the oracle's selection of this (unchanged) map: one score vector serves all six sublayers
@@ -297,6 +297,37 @@ def test_free_running_selection_matches_oracle_on_identical_input():
         assert np.array_equal(got[i], again[i])
         if traces[i] is not None:
             assert np.array_equal(traces[i], traces2[i])
+    ctx.close()
+
+
+def test_fused_selection_follows_the_separate_kernels_through_a_schedule():
+    """The optional one-launch form of the in-step selection over a whole free-running schedule (two pruned steps,
+    two blocks): given the same kept sets it must give the token maps of the separate kernels bit for bit (their
+    arithmetic on x is identical; only the column sums are added in another order), and twice in a row the same bits."""
+    wl = I.WORKLOADS["tiny"]
+    mt = I.model_tensors(wl)
+    xs = [I.step_input(wl, i, "structured") for i in range(len(wl.sides))]
+    ctx = make_ctx(wl, mt)
+    ref, tr_ref = gpu_schedule(ctx, wl, xs, trace=True)
+    assert fv.lib().fv_step_fused_selection(1) == 0
+    try:
+        got, tr = gpu_schedule(ctx, wl, xs, trace=True)
+        again, tr2 = gpu_schedule(ctx, wl, xs, trace=True)
+    finally:
+        fv.lib().fv_step_fused_selection(0)
+    same_sets = True
+    for i in range(len(xs)):
+        assert np.array_equal(got[i], again[i])
+        if tr[i] is not None:
+            assert np.array_equal(tr[i], tr2[i])
+            g, r = tr[i].astype(np.int64), tr_ref[i].astype(np.int64)
+            assert np.all(np.diff(g, axis=-1) > 0) and g.min() >= 0 and g.max() < wl.tokens(i)
+            same_sets = same_sets and np.array_equal(g, r)
+        if same_sets:
+            assert np.array_equal(got[i], ref[i]), i
+        else:
+            err, cos = per_token_errors(got[i], ref[i])
+            assert err <= MAX_ABS and cos >= MIN_COS
     ctx.close()
 
 
