@@ -456,6 +456,43 @@ def ours(args, wl):
         del ctx_x
         torch.cuda.empty_cache()
 
+    # ---- the residual stream (token maps) in bf16 instead of fp32 (fv_config.resid_dtype = 1): every pass over the
+    # stream moves half the bytes, every update rounds it to bf16 once
+    bf16_stream = None
+    if not args.skip_variant:
+        ctx_b = fv.FvContext(wl.L, wl.C, wl.H, hw, wl.cache_step, wl.B, cap, gt, cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio,
+                             device=dev, resid_dtype=1)
+        xs_b = [x.to(torch.bfloat16) for x in xs]
+        outs_b = [torch.empty_like(x) for x in xs_b]
+
+        def schedule_b(events=None):
+            ctx_b.reset()
+            for i in range(S):
+                if events is not None:
+                    events[i].record()
+                ctx_b.var_step(xs_b[i], i, wl.keep[i], out=outs_b[i])
+            if events is not None:
+                events[S].record()
+
+        for _ in range(3):
+            schedule_b()
+        barrier()
+        nb = max(2, min(args.steps, 5))
+        evb = [[torch.cuda.Event(enable_timing=True) for _ in range(S + 1)] for _ in range(nb)]
+        for k in range(nb):
+            schedule_b(evb[k])
+        barrier()
+        if ctx_b.device_status() != 0:
+            raise SystemExit("a kernel reported an expired wait")
+        b_total = max_over_ranks(statistics.mean(evb[k][0].elapsed_time(evb[k][S]) for k in range(nb)))
+        b_pruned = max_over_ranks(sum(statistics.mean(evb[k][i].elapsed_time(evb[k][i + 1]) for k in range(nb)) for i in pruned_steps))
+        bf16_stream = {"what": "same schedule with the residual stream (token maps in and out of every step) in bf16; arithmetic stays fp32",
+                       "value": world * fwd_tokens / (b_pruned * 1e-3), "unit": UNIT, "ms_per_step": b_total, "ms_per_image": b_total / wl.B,
+                       "ms_pruned_steps": b_pruned}
+        ctx_b.close()
+        del ctx_b, xs_b, outs_b
+        torch.cuda.empty_cache()
+
     # ---- the unpruned GPU step beside it (same kernels, keep_ratio = 1 everywhere)
     unpruned = None
     if not args.skip_unpruned:
@@ -539,7 +576,7 @@ def ours(args, wl):
             "ms_per_image": ms_per_step / wl.B, "ms_per_image_pruned_steps": pruned_ms / wl.B,
             "scale_step_ms": [round(t, 4) for t in step_ms], "wall_ms_per_step": t_wall * 1e3 / args.steps,
             "roofline": roofline, "kernels": kernels, "kernels_pruned_steps": kernels_pruned, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": gpu_launches,
-            "clocks": clocks, "unpruned_gpu": unpruned, "per_step_granularity": variant, "backbone_options": extras, "generation_loop": generation, "other_workloads": other,
+            "clocks": clocks, "unpruned_gpu": unpruned, "per_step_granularity": variant, "backbone_options": extras, "bf16_residual_stream": bf16_stream, "generation_loop": generation, "other_workloads": other,
             "peaks": peaks}
     print(json.dumps(line))
 

@@ -149,6 +149,11 @@ typedef struct {
   int32_t interp_mode;/* interpolate(.) of Eq. 6: 0 nearest (src = floor(dst*in/out)); 1 bilinear with
                          half-pixel centres (src = (dst+0.5)*in/out - 0.5, clamped); 2 bicubic (cubic
                          convolution, a = -0.75, 4 x 4 cached tokens, tap indices clamped to the map)     */
+  int32_t resid_dtype;/* residual stream (the token maps of fv_var_step) in 0: fp32 (default); 1: bf16.  The paper
+                         fixes no precision.  With 1 every read of the stream -- Eq. 4's sums, Eq. 5's scores, the
+                         gather, the restoration -- moves half the bytes, and every update rounds the stream to bf16
+                         once (the arithmetic stays fp32).  Supported with granularity 0, interp_mode 0, keep ratios
+                         in (0, 1]; fv_generate and skipped steps need the fp32 stream (UNSUPPORTED otherwise)    */
 } fv_config;
 
 typedef struct { /* HOST arrays of length L holding DEVICE pointers; bf16 unless noted; borrowed   */
@@ -204,8 +209,8 @@ fv_status fv_device_status(fv_ctx *ctx, int32_t *code_host, void *stream);
 fv_status fv_selftest_expired_wait(fv_ctx *ctx, uint64_t limit_ns, void *stream);
 
 /* One scale step over all L blocks.
- *   tokens_dev  [B, h*w, C] fp32: residual stream entering block 0 at this scale.
- *   out_dev     [B, h*w, C] fp32: residual stream after block L-1 (may alias tokens_dev).
+ *   tokens_dev  [B, h*w, C] fp32 (bf16 with resid_dtype 1): residual stream entering block 0 at this scale.
+ *   out_dev     [B, h*w, C] same type: residual stream after block L-1 (may alias tokens_dev).
  *   scale_idx   must equal the context's next step (steps are taken in order).
  *   keep_ratio  1.0 = unpruned path (no select / gather / restore work at all); in (0, 1) = FastVAR;
  *               0.0 = the step is skipped (the paper's 100 % pruning ratio, Sec. 4.1): out_dev is the output
@@ -222,8 +227,8 @@ fv_status fv_selftest_expired_wait(fv_ctx *ctx, uint64_t limit_ns, void *stream)
  * cache buffer then holds, fv_cache_pointer(ctx, 0, 0)).  forced_idx_dev / idx_trace_dev are int32 [B, k].
  * Errors: INVALID_ARG, BAD_STATE (wrong scale_idx; pruned step before the cache step),
  *         CAPACITY (kv_len + k > kv_capacity), CUDA. */
-fv_status fv_var_step(fv_ctx *ctx, const float *tokens_dev, int32_t B, int32_t scale_idx,
-                      double keep_ratio, float *out_dev, const int32_t *forced_idx_dev,
+fv_status fv_var_step(fv_ctx *ctx, const void *tokens_dev, int32_t B, int32_t scale_idx,
+                      double keep_ratio, void *out_dev, const int32_t *forced_idx_dev,
                       int32_t *idx_trace_dev, void *stream);
 
 /* fv_var_step with the token maps in HOST memory (pinned memory makes the copies asynchronous).  Enqueues the
@@ -237,8 +242,8 @@ fv_status fv_var_step(fv_ctx *ctx, const float *tokens_dev, int32_t B, int32_t s
  *   two output maps at their largest).  No forced indices / trace.  Errors: those of fv_var_step, CAPACITY.
  * fv_host_io_flush makes `stream` wait for every result copy enqueued so far. */
 size_t fv_var_step_host_staging_bytes(const fv_config *cfg);
-fv_status fv_var_step_host(fv_ctx *ctx, const float *tokens_host, int32_t B, int32_t scale_idx,
-                           double keep_ratio, float *out_host, void *staging_dev, size_t staging_bytes,
+fv_status fv_var_step_host(fv_ctx *ctx, const void *tokens_host, int32_t B, int32_t scale_idx,
+                           double keep_ratio, void *out_host, void *staging_dev, size_t staging_bytes,
                            void *stream);
 fv_status fv_host_io_flush(fv_ctx *ctx, void *stream);
 
@@ -302,6 +307,7 @@ fv_status fv_restore_force_fold(int32_t mode);
  *   epilogue 2: fp32 residual: out[m,n] += gamma[m / rows_per_image, n] * (acc + bias)  (out fp32;
  *               gamma NULL = 1; if aux_dev != NULL the bf16 value of acc+bias is also stored there).
  *   epilogue 4: fp32 store of acc + bias to out [M, N] (aux_dev, gamma_dev ignored).  3 is not a public value.
+ *   epilogue 5: as 2 for a bf16 residual stream: out bf16 [M, N] in place, out = bf16(float(out) + gamma * (acc + bias)).
  *   K % 8 == 0, N % 8 == 0, all pointers 16-byte aligned.  bias_dev may be NULL.
  *   W is treated as a constant of the stream: its first tiles are requested as soon as the kernel starts,
  *   which (programmatic dependent launch) can be while the kernel enqueued just before it is still

@@ -41,7 +41,7 @@ class fv_config(C.Structure):
                 ("cross_len", C.c_int32), ("B_max", C.c_int32), ("n_steps", C.c_int32),
                 ("h", C.POINTER(C.c_int32)), ("w", C.POINTER(C.c_int32)),
                 ("cache_step", C.c_int32), ("kv_capacity", C.c_int32), ("granularity", C.c_int32),
-                ("rope_base", C.c_float), ("interp_mode", C.c_int32)]
+                ("rope_base", C.c_float), ("interp_mode", C.c_int32), ("resid_dtype", C.c_int32)]
 
 
 class fv_weights(C.Structure):
@@ -399,7 +399,7 @@ class FvContext:
 
     def __init__(self, L: int, Cw: int, H: int, sides_hw: Sequence[Sequence[int]], cache_step: int, B_max: int,
                  kv_capacity: int, tensors, cross_len: int = 0, mlp_ratio: int = 4, device="cuda:0", granularity: int = 0,
-                 rope_base: float = 0.0, interp_mode: int = 0, qk_scale=None):
+                 rope_base: float = 0.0, interp_mode: int = 0, qk_scale=None, resid_dtype: int = 0):
         self.dev = torch.device(device)
         self.L, self.C, self.H, self.B_max, self.cross_len = L, Cw, H, B_max, cross_len
         self.n_sub = 3 if cross_len else 2
@@ -409,7 +409,8 @@ class FvContext:
         self._w = (C.c_int32 * len(self.hw))(*[s[1] for s in self.hw])
         self.granularity = granularity
         self.cfg = fv_config(L, Cw, H, mlp_ratio, cross_len, B_max, len(self.hw), self._h, self._w, cache_step,
-                             self.kv_capacity, granularity, float(rope_base), int(interp_mode))
+                             self.kv_capacity, granularity, float(rope_base), int(interp_mode), int(resid_dtype))
+        self.x_dtype = torch.bfloat16 if resid_dtype == 1 else torch.float32
         self._keep: List[torch.Tensor] = []
 
         def dev_bf16(a):
@@ -517,7 +518,7 @@ class FvContext:
     def var_step_host(self, tokens_host: torch.Tensor, scale_idx: int, keep_ratio: float, out_host: torch.Tensor) -> torch.Tensor:
         """fv_var_step_host: token maps in (pinned) host memory; the step runs on the current stream, the copies on the
         context's own streams.  Call host_io_flush() and synchronise before reading out_host."""
-        assert not tokens_host.is_cuda and not out_host.is_cuda and tokens_host.dtype == torch.float32
+        assert not tokens_host.is_cuda and not out_host.is_cuda and tokens_host.dtype == self.x_dtype and out_host.dtype == self.x_dtype
         assert tokens_host.is_contiguous() and out_host.is_contiguous()
         if getattr(self, "_staging", None) is None:
             nbytes = lib().fv_var_step_host_staging_bytes(C.byref(self.cfg))
@@ -533,7 +534,7 @@ class FvContext:
 
     def var_step(self, tokens: torch.Tensor, scale_idx: int, keep_ratio: float, out: Optional[torch.Tensor] = None,
                  forced_idx: Optional[torch.Tensor] = None, idx_trace: Optional[torch.Tensor] = None) -> torch.Tensor:
-        assert tokens.dtype == torch.float32
+        assert tokens.dtype == self.x_dtype, "token maps take the context's residual-stream type"
         B = tokens.shape[0]
         if out is None:
             out = torch.empty_like(tokens)

@@ -95,6 +95,7 @@ bool config_ok(const fv_config* c) {
   if (c->cache_step >= c->n_steps) return false;
   if (c->granularity != 0 && c->granularity != 1) return false;
   if (c->interp_mode < 0 || c->interp_mode > 2) return false;
+  if (c->resid_dtype != 0 && c->resid_dtype != 1) return false;
   if (!(c->rope_base >= 0.f)) return false;
   return true;
 }
@@ -261,7 +262,7 @@ fv_status fv_restore_force_fold(int32_t mode) {
 fv_status fv_gemm_bf16(const void* a_dev, const void* w_dev, const void* bias_dev, int32_t M, int32_t N, int32_t K,
                        int32_t epilogue, void* out_dev, void* aux_dev, const float* gamma_dev, int32_t mod_stride,
                        int32_t rows_per_image, int32_t* status_dev, void* splitk_ws_dev, size_t splitk_ws_bytes, void* stream) {
-  if (!a_dev || !w_dev || !out_dev || epilogue < 0 || epilogue > 4 || epilogue == EPI_QKV_SPLIT) return FV_ERR_INVALID_ARG;
+  if (!a_dev || !w_dev || !out_dev || epilogue < 0 || epilogue > 5 || epilogue == EPI_QKV_SPLIT) return FV_ERR_INVALID_ARG;
   if (splitk_ws_dev && (splitk_ws_bytes < gemm_splitk_ws_bytes() || !aligned16(splitk_ws_dev))) return FV_ERR_CAPACITY;
   if (!aligned16(a_dev) || !aligned16(w_dev) || !aligned16(out_dev) || (bias_dev && !aligned16(bias_dev))) return FV_ERR_INVALID_ARG;
   if (ensure_init() != cudaSuccess) return FV_ERR_CUDA;
@@ -336,6 +337,7 @@ fv_status fv_create(const fv_config* cfg, const fv_weights* wts, void* kv_dev, v
   const int hd = cfg->C / cfg->H;
   if ((hd != 64 && hd != 128) || cfg->C > 2048 || cfg->C % 128) return FV_ERR_UNSUPPORTED;
   if (max_tokens(cfg) > kTopkMaxTokens) return FV_ERR_UNSUPPORTED;
+  if (cfg->resid_dtype == 1 && (cfg->granularity != 0 || cfg->interp_mode != 0)) return FV_ERR_UNSUPPORTED;
   if (!wts->w_qkv || !wts->b_qkv || !wts->w_o || !wts->b_o || !wts->w_fc1 || !wts->b_fc1 || !wts->w_fc2 || !wts->b_fc2 || !wts->mod_dev)
     return FV_ERR_INVALID_ARG;
   if (cfg->cross_len && (!wts->w_q_x || !wts->w_kv_x || !wts->w_o_x || !wts->text_dev)) return FV_ERR_INVALID_ARG;
@@ -513,14 +515,17 @@ fv_status fv_selftest_expired_wait(fv_ctx* ctx, uint64_t limit_ns, void* stream)
   return cuda_status(launch_expired_wait(ctx->status, limit_ns, static_cast<cudaStream_t>(stream)));
 }
 
-fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t scale_idx, double keep_ratio, float* out_dev,
+fv_status fv_var_step(fv_ctx* ctx, const void* tokens_dev, int32_t B, int32_t scale_idx, double keep_ratio, void* out_dev,
                       const int32_t* forced_idx_dev, int32_t* idx_trace_dev, void* stream) {
   if (!ctx || !tokens_dev || !out_dev || B <= 0 || B > ctx->cfg.B_max) return FV_ERR_INVALID_ARG;
   if (!(keep_ratio >= 0.0) || keep_ratio > 1.0 || !aligned16(tokens_dev) || !aligned16(out_dev)) return FV_ERR_INVALID_ARG;
   const fv_config& c = ctx->cfg;
   if (scale_idx < 0 || scale_idx >= c.n_steps) return FV_ERR_INVALID_ARG;
   if (scale_idx != ctx->next_step) return FV_ERR_BAD_STATE;
+  const bool xb = c.resid_dtype == 1;          // bf16 residual stream
+  const size_t xes = xb ? 2 : 4;
   if (keep_ratio == 0.0) {
+    if (xb) return FV_ERR_UNSUPPORTED;
     // Skipped step (the paper's 100 % pruning ratio, Sec. 4.1): no token is forwarded, nothing enters the
     // KV cache; the output is the caching step's output map interpolated to this scale.
     if (c.cache_step < 0 || scale_idx <= c.cache_step) return FV_ERR_BAD_STATE;
@@ -529,7 +534,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
     const int h0 = c.h[scale_idx], w0 = c.w[scale_idx];
     if (launch_inv_fill(B, h0 * w0, ctx->inv, st0) != cudaSuccess) return FV_ERR_CUDA;
     if (launch_restore_rows_f32(ctx->step_cache, c.h[c.cache_step], c.w[c.cache_step], ctx->step_cache, ctx->inv, B, 0, h0, w0, c.C,
-                                out_dev, c.interp_mode, st0) != cudaSuccess)
+                                static_cast<float*>(out_dev), c.interp_mode, st0) != cudaSuccess)
       return FV_ERR_CUDA;
     ctx->next_step += 1;
     return FV_OK;
@@ -543,10 +548,10 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   if (ctx->kv_len + k > c.kv_capacity) return FV_ERR_CAPACITY;
   if (c.cross_len && scale_idx > 0 && !ctx->text_ready) return FV_ERR_BAD_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  float* x = out_dev;
+  void* x = out_dev;
   // (per-step granularity, pruned step: the output map is written whole by the final restoration)
   if (out_dev != tokens_dev && !(pruned && c.granularity == 1) &&
-      cudaMemcpyAsync(out_dev, tokens_dev, (size_t)B * n * C * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      cudaMemcpyAsync(out_dev, tokens_dev, (size_t)B * n * C * xes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
     return FV_ERR_CUDA;
   if (c.cross_len && scale_idx == 0) {
     fv_status s = fv_prepare_text(ctx, B, stream);
@@ -561,7 +566,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   // Per sublayer (the paper): every sublayer selects from the full map x and restores into it.
   // Per step: one selection here, the blocks then run on the compact rows xr = ctx->xc as if unpruned.
   const bool sub_pruned = pruned && !whole_step;
-  float* xr = x;        // residual stream the blocks update
+  void* xr = x;         // residual stream the blocks update
   int nr = n;           // its rows per image
   const int32_t* step_idx = nullptr;   // per-step granularity: the kept indices of the whole step
   if (pruned && whole_step) {
@@ -575,7 +580,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
     }
     if (e != cudaSuccess) return FV_ERR_CUDA;
     if (idx_trace_dev && cudaMemcpyAsync(idx_trace_dev, idx, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return FV_ERR_CUDA;
-    if (launch_gather_rows(tokens_dev, idx, B, n, k, C, ctx->xc, ctx->status, st) != cudaSuccess) return FV_ERR_CUDA;
+    if (launch_gather_rows(static_cast<const float*>(tokens_dev), idx, B, n, k, C, ctx->xc, ctx->status, st) != cudaSuccess) return FV_ERR_CUDA;
     xr = ctx->xc;
     nr = k;
     step_idx = idx;
@@ -589,7 +594,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
   // kept-row restoration, the selection and the gather + LayerNorm of the newly kept rows (select_fused_kernel).  The
   // kept rows of a sublayer are then restored by the NEXT sublayer's launch; only the last sublayer of the step
   // restores its own.
-  const bool fused = selecting && g_step_fused && select_fused_supported(B, n, C);
+  const bool fused = selecting && g_step_fused && !xb && select_fused_supported(B, n, C);
   bool pending = false;                 // a kept-row restoration waits for the next fused selection
   const float* pending_gamma = nullptr;
   int flip = 0;
@@ -617,7 +622,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
           e = launch_inv_from_idx(idx, B, k, n, ctx->inv, st);
         } else if (!fused) {
           idx = ctx->idx;
-          e = launch_select(x, B, n, C, k, ctx->idx, ctx->inv, nullptr, nullptr, ctx->sel_ws, have_partials, st);
+          e = launch_select(x, B, n, C, k, ctx->idx, ctx->inv, nullptr, nullptr, ctx->sel_ws, have_partials, st, xb);
         }
         if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
         if (!fused && idx_trace_dev && cudaMemcpyAsync(idx_trace_dev + trace_off, idx, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
@@ -634,7 +639,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         int32_t* idx_cur = flip ? ctx->idx2 : ctx->idx;
         inv_cur = flip ? ctx->inv2 : ctx->inv;
         FusedSelect f{};
-        f.x = x; f.B = B; f.n = n; f.C = C; f.k = k; f.mod_stride = mod_stride;
+        f.x = static_cast<float*>(x); f.B = B; f.n = n; f.C = C; f.k = k; f.mod_stride = mod_stride;
         f.sel_ws = ctx->sel_ws; f.fused_ws = ctx->fsel_ws; f.idx = idx_cur; f.inv = inv_cur;
         f.sigma = sigma; f.beta = beta; f.a_out = ctx->a_buf; f.status = ctx->status;
         f.done_total = &ctx->fsel_done; f.epoch = &ctx->fsel_epoch;
@@ -643,7 +648,7 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
           if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
           forked = false;
           f.y = ctx->y_buf; f.idx_prev = flip ? ctx->idx : ctx->idx2; f.gamma_prev = pending_gamma;
-        } else if (launch_colsum(x, B, n, C, ctx->sel_ws, st) != cudaSuccess) {   // first sublayer of the step: sum the map itself
+        } else if (launch_colsum(static_cast<const float*>(x), B, n, C, ctx->sel_ws, st) != cudaSuccess) {   // first sublayer of the step: sum the map itself
           s = FV_ERR_CUDA; break;
         }
         if (launch_select_fused(f, st) != cudaSuccess) { s = FV_ERR_CUDA; break; }
@@ -660,13 +665,13 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         // touch disjoint rows of x).
         if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
         e = launch_restore_residual(x, ctx->y_buf, cache_sub, inv_cur, gamma, mod_stride, B, k, h, w, hc, wc, C,
-                                    more ? ctx->sel_ws : nullptr, (fused && more) ? 3 : 1, c.interp_mode, ctx->side);
+                                    more ? ctx->sel_ws : nullptr, (fused && more) ? 3 : 1, c.interp_mode, ctx->side, xb);
         const cudaError_t e_join = cudaEventRecord(ctx->ev_join, ctx->side);   // recorded even if the launch failed
         forked = e_join == cudaSuccess;
         if (e != cudaSuccess || e_join != cudaSuccess) { s = FV_ERR_CUDA; break; }
       }
       if (!fused) {
-        e = launch_gather_ln(xr, idx, B, nr, k, C, sigma, beta, mod_stride, ctx->a_buf, ctx->status, st);
+        e = launch_gather_ln(xr, idx, B, nr, k, C, sigma, beta, mod_stride, ctx->a_buf, ctx->status, st, xb);
         if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
       }
       // ---- branch on the compact rows
@@ -723,22 +728,22 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
         if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
         forked = false;
         e = launch_restore_residual(x, ctx->y_buf, cache_sub, inv_cur, gamma, mod_stride, B, k, h, w, hc, wc, C,
-                                    more ? ctx->sel_ws : nullptr, 2, c.interp_mode, st);
+                                    more ? ctx->sel_ws : nullptr, 2, c.interp_mode, st, xb);
         if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
         have_partials = more;
       } else {
-        o.epilogue = EPI_RESIDUAL; o.out = xr; o.gamma = gamma; o.aux = (write_cache && !whole_step) ? cache_sub : nullptr;
+        o.epilogue = xb ? EPI_RESIDUAL_XBF16 : EPI_RESIDUAL; o.out = xr; o.gamma = gamma; o.aux = (write_cache && !whole_step) ? cache_sub : nullptr;
         s = launch_gemm(o, st);
         if (s != FV_OK) break;
       }
     }
   }
   if (s != FV_OK) return s;
-  if (write_cache &&
+  if (write_cache && !xb &&   // (a bf16 stream has no skipped steps and no per-step granularity: nothing reads this copy)
       cudaMemcpyAsync(ctx->step_cache, x, (size_t)B * n * C * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
     return FV_ERR_CUDA;  // the step-level cache: this step's output map (image stride n*C == n_cache*C here)
   if (whole_step && pruned &&
-      launch_restore_rows_f32(ctx->step_cache, hc, wc, ctx->xc, ctx->inv, B, k, h, w, C, out_dev, c.interp_mode, st) != cudaSuccess)
+      launch_restore_rows_f32(ctx->step_cache, hc, wc, ctx->xc, ctx->inv, B, k, h, w, C, static_cast<float*>(out_dev), c.interp_mode, st) != cudaSuccess)
     return FV_ERR_CUDA;
   if (s != FV_OK) return s;
   ctx->kv_len += k;
@@ -751,10 +756,10 @@ fv_status fv_var_step(fv_ctx* ctx, const float* tokens_dev, int32_t B, int32_t s
 // the input of call i+1 travels while call i computes, and the result of call i travels while call i+1 computes.
 size_t fv_var_step_host_staging_bytes(const fv_config* cfg) {
   if (!config_ok(cfg)) return 0;
-  return 4 * align_up((size_t)cfg->B_max * max_tokens(cfg) * cfg->C * sizeof(float), 1024);
+  return 4 * align_up((size_t)cfg->B_max * max_tokens(cfg) * cfg->C * (cfg->resid_dtype == 1 ? 2 : 4), 1024);
 }
 
-fv_status fv_var_step_host(fv_ctx* ctx, const float* tokens_host, int32_t B, int32_t scale_idx, double keep_ratio, float* out_host,
+fv_status fv_var_step_host(fv_ctx* ctx, const void* tokens_host, int32_t B, int32_t scale_idx, double keep_ratio, void* out_host,
                            void* staging_dev, size_t staging_bytes, void* stream) {
   if (!ctx || !tokens_host || !out_host || !staging_dev || B <= 0 || B > ctx->cfg.B_max) return FV_ERR_INVALID_ARG;
   if (scale_idx < 0 || scale_idx >= ctx->cfg.n_steps || (reinterpret_cast<uintptr_t>(staging_dev) & 1023u)) return FV_ERR_INVALID_ARG;
@@ -769,10 +774,10 @@ fv_status fv_var_step_host(fv_ctx* ctx, const float* tokens_host, int32_t B, int
   }
   const fv_config& c = ctx->cfg;
   const size_t half = fv_var_step_host_staging_bytes(&c) / 4;
-  const size_t bytes = (size_t)B * c.h[scale_idx] * c.w[scale_idx] * c.C * sizeof(float);
+  const size_t bytes = (size_t)B * c.h[scale_idx] * c.w[scale_idx] * c.C * (c.resid_dtype == 1 ? 2 : 4);
   const int p = (int)(ctx->io_count & 1u);
-  float* in_dev = reinterpret_cast<float*>(static_cast<char*>(staging_dev) + (size_t)p * half);
-  float* out_dev = reinterpret_cast<float*>(static_cast<char*>(staging_dev) + (size_t)(2 + p) * half);
+  void* in_dev = static_cast<char*>(staging_dev) + (size_t)p * half;
+  void* out_dev = static_cast<char*>(staging_dev) + (size_t)(2 + p) * half;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // in: this buffer's previous reader (the step two calls ago) must be done
   if (ctx->used_rec[p] && cudaStreamWaitEvent(ctx->io_in, ctx->ev_used[p], 0) != cudaSuccess) return FV_ERR_CUDA;

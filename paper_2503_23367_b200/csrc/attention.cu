@@ -389,9 +389,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   };
 
   // A softmax thread holds a whole score row (128 fp32) in registers, so the register file is re-divided
-  // between the warpgroups: 2 x 128 x 216 + 128 x 72 = 384 x 168, what the CTA was launched with (a larger request would wait forever).
+  // between the warpgroups: 2 x 128 x 208 + 128 x 88 = 384 x 168, what the CTA was launched with (a larger request would
+  // wait forever); 88 rather than fewer for the producer / MMA warps measured 3 % faster here.
   if (warp >= 8) {
-   asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+   asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
    if (warp == 8) {
     if (lane == 0) {
       uint32_t kt = 0;      // key tiles loaded so far: ring position of the K and V^T stages
@@ -488,7 +489,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
    }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
     // ---- softmax + output: thread = one query row of tile t ----
     const int t = warp >> 2;
     const int quarter = warp & 3;                 // the TMEM lanes this warp may touch

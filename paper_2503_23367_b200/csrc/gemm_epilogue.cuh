@@ -220,6 +220,38 @@ __device__ __forceinline__ void store_chunk(const GemmDev& p, const float (&v)[3
         }
       }
     }
+  } else if (p.epilogue == EPI_RESIDUAL_XBF16) {
+    // gate + residual into a bf16 residual stream: out = bf16(float(out) + gamma * v), rounded once (+ bf16 copy of v)
+    uint4* xr = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + (size_t)row * p.N + col);
+    const float4* gp = p.gamma ? reinterpret_cast<const float4*>(p.gamma + (size_t)img * p.mod_stride + col) : nullptr;
+    uint4* ap = p.aux ? reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.aux) + (size_t)row * p.N + col) : nullptr;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      if (col + 8 * g < p.N) {
+        const uint4 xo = xr[g];
+        const uint32_t u[4] = {xo.x, xo.y, xo.z, xo.w};
+        float xv[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { xv[2 * i] = __uint_as_float(u[i] << 16); xv[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u); }
+        if (gp) {
+          const float4 ga = __ldg(gp + 2 * g), gb = __ldg(gp + 2 * g + 1);
+          xv[0] = fmaf(ga.x, v[8 * g + 0], xv[0]); xv[1] = fmaf(ga.y, v[8 * g + 1], xv[1]); xv[2] = fmaf(ga.z, v[8 * g + 2], xv[2]); xv[3] = fmaf(ga.w, v[8 * g + 3], xv[3]);
+          xv[4] = fmaf(gb.x, v[8 * g + 4], xv[4]); xv[5] = fmaf(gb.y, v[8 * g + 5], xv[5]); xv[6] = fmaf(gb.z, v[8 * g + 6], xv[6]); xv[7] = fmaf(gb.w, v[8 * g + 7], xv[7]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) xv[i] += v[8 * g + i];
+        }
+        uint4 o;
+        o.x = pack_bf16x2(xv[0], xv[1]); o.y = pack_bf16x2(xv[2], xv[3]); o.z = pack_bf16x2(xv[4], xv[5]); o.w = pack_bf16x2(xv[6], xv[7]);
+        xr[g] = o;
+        if (ap) {
+          uint4 c;
+          c.x = pack_bf16x2(v[8 * g + 0], v[8 * g + 1]); c.y = pack_bf16x2(v[8 * g + 2], v[8 * g + 3]);
+          c.z = pack_bf16x2(v[8 * g + 4], v[8 * g + 5]); c.w = pack_bf16x2(v[8 * g + 6], v[8 * g + 7]);
+          ap[g] = c;
+        }
+      }
+    }
   } else {  // EPI_QKV_SPLIT, K or V part
     const int kc = col - p.q_cols;
     const size_t krow = (size_t)img * p.kv_capacity + p.kv_offset + jrow;

@@ -289,6 +289,7 @@ fv_status fv_generate(fv_ctx* ctx, const fv_generator* gen, const float* start_d
   if (!gen->codebook_dev || !gen->w_head_dev || !gen->mod_head_dev || !gen->w_in_dev) return FV_ERR_INVALID_ARG;
   const fv_config& c = *ctx_config(ctx);
   if (B <= 0 || B > c.B_max || (reinterpret_cast<uintptr_t>(workspace_dev) & 1023u)) return FV_ERR_INVALID_ARG;
+  if (c.resid_dtype != 0) return FV_ERR_UNSUPPORTED;   // the head reads an fp32 token map
   const GenLayout l = gen_layout(c, *gen);
   if (workspace_bytes < l.total) return FV_ERR_CAPACITY;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -19,11 +19,11 @@ DEV = "cuda:0"
 MAX_ABS, MIN_COS = 3e-2, 0.999
 
 
-def make_ctx(wl: I.Workload, mt: I.ModelTensors, unpruned=False, granularity=0) -> fv.FvContext:
+def make_ctx(wl: I.Workload, mt: I.ModelTensors, unpruned=False, granularity=0, resid_dtype=0) -> fv.FvContext:
     cap = sum(wl.tokens(i) if (unpruned or wl.keep[i] >= 1.0) else O.kept_count(wl.keep[i], wl.sides[i], wl.sides[i])
               for i in range(len(wl.sides)))
     return fv.FvContext(wl.L, wl.C, wl.H, [(s, s) for s in wl.sides], wl.cache_step, wl.B, cap, mt,
-                        cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio, device=DEV, granularity=granularity)
+                        cross_len=wl.cross_len, mlp_ratio=wl.mlp_ratio, device=DEV, granularity=granularity, resid_dtype=resid_dtype)
 
 
 def gpu_schedule(ctx, wl, xs, forced=None, trace=False):
@@ -328,6 +328,93 @@ def test_fused_selection_follows_the_separate_kernels_through_a_schedule():
         else:
             err, cos = per_token_errors(got[i], ref[i])
             assert err <= MAX_ABS and cos >= MIN_COS
+    ctx.close()
+
+
+# ------------------------------------------------------------------ bf16 residual stream (fv_config.resid_dtype = 1)
+def _bf16_round(a):
+    return I.bf16_bits_to_f32(I.to_bf16_bits(a))
+
+
+def test_bf16_residual_stream_schedule_against_the_oracle():
+    """The token maps of fv_var_step in bf16: every kernel that touches the stream (column sums, scores, gather,
+    restoration, the residual epilogue of the unpruned steps) reads and writes bf16 and computes in fp32.  Inputs are
+    bf16-representable on both sides; the oracle stays fp64.  Each of the U updates of a step rounds the stream once
+    (<= 2^-9 relative), so the bound is the usual 3e-2 of the branch arithmetic plus U * 2^-9 * max|x|; the first
+    selection of every pruned step sees identical input and must keep the oracle's set."""
+    wl = I.WORKLOADS["tiny"]
+    mt = I.model_tensors(wl)
+    xs = [_bf16_round(I.step_input(wl, i, "structured")) for i in range(len(wl.sides))]
+    orc, ref, tr = run_oracle(wl, mt, xs)
+    forced = [trace_to_index_tensor(wl, tr[i]) if wl.keep[i] < 1.0 else None for i in range(len(xs))]
+    ctx = make_ctx(wl, mt, resid_dtype=1)
+    updates = wl.L * wl.n_sub
+    worst = 0.0
+    for mode in ("forced", "free"):
+        ctx.reset()
+        for i, x in enumerate(xs):
+            xd = torch.from_numpy(x).to(DEV).to(torch.bfloat16)
+            f = t = None
+            if wl.keep[i] < 1.0:
+                if mode == "forced":
+                    f = torch.from_numpy(forced[i]).to(DEV)
+                else:
+                    t = torch.zeros((wl.L, wl.n_sub, wl.B, forced[i].shape[-1]), dtype=torch.int32, device=DEV)
+            got = ctx.var_step(xd, i, wl.keep[i], forced_idx=f, idx_trace=t)
+            assert got.dtype == torch.bfloat16
+            got = got.float().cpu().numpy()
+            if mode == "forced":
+                err, cos = per_token_errors(got, ref[i])
+                bound = MAX_ABS + updates * 2.0 ** -9 * np.abs(ref[i]).max()
+                worst = max(worst, err)
+                assert err <= bound and cos >= MIN_COS, (i, err, bound, cos)
+            elif t is not None:
+                idx_g = t[0, 0].cpu().numpy().astype(np.int64)
+                idx_o, s_o = tr[i][(0, "attn")]["idx"], tr[i][(0, "attn")]["score"]
+                for b in range(wl.B):
+                    diff = np.setxor1d(idx_g[b], idx_o[b])
+                    tau = np.sort(s_o[b])[::-1][idx_o.shape[1] - 1]
+                    assert np.all(np.abs(s_o[b, diff] - tau) <= 1e-5 * tau)
+        assert ctx.device_status() == 0 and ctx.state() == (len(xs), orc.kv_len)
+    print(f"bf16 residual stream, tiny schedule: worst max-abs error {worst:.4g}")
+    # what the bf16 stream does not take
+    with pytest.raises(fv.FvError) as e:
+        fv.FvContext(wl.L, wl.C, wl.H, [(s, s) for s in wl.sides], wl.cache_step, wl.B, 64, mt, device=DEV, granularity=1, resid_dtype=1)
+    assert e.value.code == 4
+    ctx.close()
+
+
+@pytest.mark.parametrize("h,w,hc,wc,C,H,B,B_max,keep", [(64, 64, 32, 32, 2048, 16, 2, 2, 0.2), (33, 31, 10, 10, 256, 4, 3, 4, 0.5),
+                                                      (128, 128, 48, 48, 2048, 16, 1, 1, 0.2)])
+def test_bf16_residual_stream_every_selection_on_bit_identical_input(h, w, hc, wc, C, H, B, B_max, keep):
+    """The zero-branch step (see test_every_selection_of_a_step_on_bit_identical_input) with a bf16 stream: x + 0 is
+    exact in bf16 too, so every one of the six selections -- five of them from the column sums the bf16 restoration
+    left -- must keep the oracle's set of the (bf16-representable) map."""
+    wl = I.Workload("zero-branch", L=2, C=C, H=H, B=B_max, sides=(hc, h), keep=(1.0, keep), cross_len=64, mlp_ratio=1, seed=811)
+    mt = _zero_branch_tensors(wl)
+    n, k = h * w, O.kept_count(keep, h, w)
+    x = _bf16_round(I.token_map(900 + h, B, h, w, C, "structured"))
+    ctx = fv.FvContext(wl.L, C, H, [(hc, wc), (h, w)], 0, B_max, k, mt, cross_len=64, mlp_ratio=1, device=DEV, resid_dtype=1)
+    for l in range(wl.L):
+        for si in range(3):
+            ctx.cache_view(l, si).zero_()
+    ctx.set_state(1, 0)
+    ctx.prepare_text(B)
+    trace = torch.full((wl.L, 3, B, k), -1, dtype=torch.int32, device=DEV)
+    got = ctx.var_step(torch.from_numpy(x).to(DEV).to(torch.bfloat16), 1, keep, idx_trace=trace).float().cpu().numpy()
+    assert ctx.device_status() == 0
+    assert np.array_equal(got, x)
+    score_o = O.pts_score(x)
+    idx_o = O.pts_topk(score_o, k)
+    tau = np.sort(score_o, axis=1)[:, ::-1][:, k - 1]
+    idx_g = trace.cpu().numpy().astype(np.int64)
+    for l in range(wl.L):
+        for si in range(3):
+            for b in range(B):
+                g = idx_g[l, si, b]
+                assert np.all(np.diff(g) > 0) and g[0] >= 0 and g[-1] < n
+                diff = np.setxor1d(g, idx_o[b])
+                assert np.all(np.abs(score_o[b, diff] - tau[b]) <= 1e-5 * tau[b]), (l, si, b)
     ctx.close()
 
 
