@@ -226,3 +226,33 @@ def test_head_tokens_at_the_last_scale_of_the_bench_workload_sampled_rows():
     np.testing.assert_array_equal(ids[:, rows][clear], ref_ids[clear])
     # every id (all 8192 rows) is the exact argmax of the GPU's own fp32 logits
     np.testing.assert_array_equal(ids, lg.argmax(-1))
+
+
+def test_head_tokens_of_the_bench_s_own_head_within_one_bf16_rounding():
+    """The head bench.py times (generation_tensors' default: weights of std 0.08, logits of +-15), at full size.  Its
+    logits are too large for the absolute 3e-2 bar, so the bound is the arithmetic's own: the normalised, modulated
+    activations are rounded to bf16 once before the tensor-core GEMM (<= 2^-9 relative per element, fp32 accumulation),
+    hence |logit - oracle| <= 2^-9 * sum_c |a_c * w_vc| (+ 1e-4 for the fp32 sums) for every sampled logit; ids may
+    differ from the oracle's only where its margin is inside twice that bound."""
+    B, n, C, V = 2, 4096, 2048, 4096
+    y = I.normal(61, (B, n, C), 1.5) + 0.3
+    wl = I.Workload("h", L=1, C=C, H=16, B=B, sides=(1,), keep=(1.0,), cross_len=0, seed=19)
+    gt = I.generation_tensors(wl, V=V, d=32)                          # the bench's head
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ids, logits = fv.fv_head_tokens(T(y), T(gt.mod_head), BF(gt.w_head), BF(gt.b_head), want_logits=True, status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    ids = ids.cpu().numpy(); lg = logits.cpu().numpy().reshape(B, n, V)
+    rows = np.unique(np.concatenate([(I.uniform01(63, 64) * n).astype(np.int64), [0, 127, 128, n - 1]]))
+    wh, bh = I.bf16_bits_to_f32(gt.w_head).astype(np.float64), I.bf16_bits_to_f32(gt.b_head).astype(np.float64)
+    ref = G.head_logits(y[:, rows], gt.mod_head[:, 0], gt.mod_head[:, 1], wh, bh)
+    a = O.modulate(O.layernorm(y[:, rows].astype(np.float64)), gt.mod_head[:, 0].astype(np.float64), gt.mod_head[:, 1].astype(np.float64))
+    bound = 2.0 ** -9 * (np.abs(a) @ np.abs(wh).T) + 1e-4             # [B, rows, V]
+    err = np.abs(lg[:, rows] - ref)
+    assert np.all(err <= bound), float((err / bound).max())
+    assert np.abs(ref).max() > 7.0                                     # the case the absolute bar does not cover
+    ref_ids, margin = G.choose_tokens(ref)
+    clear = margin > 2 * bound.max(axis=-1)
+    assert clear.mean() > 0.5
+    np.testing.assert_array_equal(ids[:, rows][clear], ref_ids[clear])
+    np.testing.assert_array_equal(ids, lg.argmax(-1))
