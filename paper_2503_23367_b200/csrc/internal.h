@@ -88,7 +88,7 @@ constexpr int kTopkMaxTokens = 49152;  // scores of one image must fit the top-k
 // two levels: one partial per chunk of kColsumRows tokens, folded (by the last CTA of each group to
 // finish) into <= kMaxGroups group partials per image, which the scoring kernel adds up itself.
 struct SelectWs {
-  unsigned int* tickets;  // [B, kMaxGroups] group arrival counters, then [B] image counters; zero between launches
+  unsigned int* tickets;  // [B, kMaxGroups] group arrival counters, [B] image counters, [B, 2] score range words; zero between launches
   float* chunk_partial;   // [B, nchunks, C]
   float* group_partial;   // [B, ngroups, C]
   float* score;           // [B, n]

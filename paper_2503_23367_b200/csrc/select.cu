@@ -21,12 +21,11 @@ namespace fv {
 
 namespace {
 
-constexpr int kTopkThreads = 512;
+constexpr int kSelectThreads = 1024;   // the stand-alone score + top-k kernel: one CTA per SM
+constexpr int kSelectWarps = kSelectThreads / 32;
+constexpr int kTopkThreads = 512;      // the fused kernel of a scale step (a thread may hold a whole row slice)
 constexpr int kTopkWarps = kTopkThreads / 32;
-// Keys sit in shared memory with one pad word per 32, so that both access patterns of the top-k are
-// free of bank conflicts: consecutive lanes on consecutive tokens, and each lane on its own contiguous run.
-__device__ __forceinline__ int KI(int i) { return i + (i >> 5); }
-constexpr size_t kTopkMaxSmem = ((size_t)kTopkMaxTokens + kTopkMaxTokens / 32 + 1) * 4;
+constexpr size_t kTopkMaxSmem = (size_t)kTopkMaxTokens * 4;   // one key per token (consecutive lanes on consecutive tokens)
 
 template <typename XT>
 __global__ void __launch_bounds__(256) colsum_chunk_kernel(const XT* __restrict__ x, int n, int C4, int nchunks, int group,
@@ -57,8 +56,9 @@ __global__ void __launch_bounds__(256) colsum_chunk_kernel(const XT* __restrict_
   fold_group_partials(b, chunk, nchunks, group, ngroups, C4, chunk_partial, group_partial, tickets);
 }
 
-// Exclusive prefix sum of one value per thread over the whole CTA (kTopkThreads threads); returns the
+// Exclusive prefix sum of one value per thread over the whole CTA (T threads, the template argument); returns the
 // exclusive prefix and, through `total`, the CTA-wide sum.  s_warp is 32 words of scratch.
+template <int T>
 __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s_warp, uint32_t* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t inc = v;
@@ -70,7 +70,7 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
   __syncthreads();  // s_warp may still be read from a previous scan
   if (lane == 31) s_warp[warp] = inc;
   __syncthreads();
-  uint32_t wv = lane < kTopkWarps ? s_warp[lane] : 0u;
+  uint32_t wv = lane < (T / 32) ? s_warp[lane] : 0u;
   uint32_t winc = wv;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -97,10 +97,11 @@ __device__ __forceinline__ void add_partials(float4& acc, const float4* __restri
       if (g0 + g < ng) { acc.x += v[g].x; acc.y += v[g].y; acc.z += v[g].z; acc.w += v[g].w; }
   }
 }
+template <int T>
 __device__ __forceinline__ void mean_from_partials(float4* s_mean, const float4* __restrict__ gp_a, int nga,
                                                    const float4* __restrict__ gp_b, int ngb, int C4, int n) {
   const float fn = (float)n;
-  for (int c4 = threadIdx.x; c4 < C4; c4 += kTopkThreads) {
+  for (int c4 = threadIdx.x; c4 < C4; c4 += T) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     add_partials(acc, gp_a, nga, C4, c4);
     if (ngb > 0) add_partials(acc, gp_b, ngb, C4, c4);
@@ -108,14 +109,56 @@ __device__ __forceinline__ void mean_from_partials(float4* s_mean, const float4*
   }
 }
 
+// The same sums in the same order by twice as many threads: the upper half of the CTA fetches the partials of the
+// groups from 8 on into shared memory while the lower half adds the first 8; the lower half then continues with the
+// staged values.  One round trip to L2 instead of two.  stage: 8 * C4 float4 words.
+template <int T>
+__device__ __forceinline__ void mean_from_partials_halves(float4* s_mean, float4* stage, const float4* __restrict__ gp, int ng, int C4, int n) {
+  constexpr int H = T / 2;
+  const int tid = threadIdx.x, half = tid / H, t = tid - half * H;
+  const float fn = (float)n;
+  for (int c0 = 0; c0 < C4; c0 += H) {
+    const int c4 = c0 + t;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c4 < C4) {
+      float4 v[8];
+      const int g_lo = half * 8;
+#pragma unroll
+      for (int g = 0; g < 8; ++g)
+        if (g_lo + g < ng) v[g] = __ldcg(gp + (size_t)(g_lo + g) * C4 + c4);
+      if (half == 0) {
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+          if (g < ng) { acc.x += v[g].x; acc.y += v[g].y; acc.z += v[g].z; acc.w += v[g].w; }
+      } else {
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+          if (8 + g < ng) stage[(size_t)g * C4 + c4] = v[g];
+      }
+    }
+    __syncthreads();
+    if (half == 0 && c4 < C4) {
+#pragma unroll
+      for (int g = 0; g < 8; ++g)
+        if (8 + g < ng) { const float4 u = stage[(size_t)g * C4 + c4]; acc.x += u.x; acc.y += u.y; acc.z += u.z; acc.w += u.w; }
+      s_mean[c4] = make_float4(acc.x / fn, acc.y / fn, acc.z / fn, acc.w / fn);
+    }
+  }
+}
+static_assert(kMaxGroups == 16, "mean_from_partials_halves splits the groups 8 + 8");
+
 // ---- Eq. 5 / Algorithm 1: squared deviation from the mean, one warp per token row; the warps of an image stride
 // over its rows.  NC: the map was not written by this kernel, so its rows may take the read-only path; the fused
 // kernel, whose other CTAs have just updated rows of it, reads them through L2.
 // BATCH: 16-byte loads a lane requests together (8 with 64 registers per thread, 16 with 128).
-template <bool NC, int BATCH, typename XT>
-__device__ __forceinline__ void score_rows(const XT* x, const float4* s_mean, int b, int n, int C4, float* __restrict__ score) {
+// lo / hi: running smallest / largest score key (the bit pattern without its sign) of the rows this warp has scored.
+// inv (may be null): the inverse map of the image is set to "not kept" for every row scored here, so that the CTA
+// that ranks the image only has to write the entries of the kept rows (one SM stores slowly).
+template <int T, bool NC, int BATCH, typename XT>
+__device__ __forceinline__ void score_rows(const XT* x, const float4* s_mean, int b, int n, int C4, float* __restrict__ score,
+                                           int32_t* __restrict__ inv, uint32_t& lo, uint32_t& hi) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int r = blockIdx.x * kTopkWarps + warp; r < n; r += gridDim.x * kTopkWarps) {
+  for (int r = blockIdx.x * (T / 32) + warp; r < n; r += gridDim.x * (T / 32)) {
     const XT* row = x + ((size_t)b * n + r) * C4 * 4;
     float acc = 0.f;
     int c4 = lane;
@@ -138,140 +181,261 @@ __device__ __forceinline__ void score_rows(const XT* x, const float4* s_mean, in
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) score[(size_t)b * n + r] = acc;
+    if (lane == 0) {
+      score[(size_t)b * n + r] = acc;
+      if (inv) inv[(size_t)b * n + r] = -1;
+    }
+    const uint32_t key = __float_as_uint(acc) & 0x7FFFFFFFu;
+    lo = min(lo, key); hi = max(hi, key);
   }
 }
 
 // Scratch of the top-k in static shared memory.
+constexpr int kFirstDigitBits = 11;                 // the first radix digit: up to 2048 bins
+constexpr int kHistBins = 1 << kFirstDigitBits;
+constexpr int kCandMax = 1024;                      // longest candidate list kept beside the keys
+constexpr int kCountMax = 128;                      // a list this short is finished by counting
 struct TopkShared {
-  uint32_t hist[256];
+  uint32_t hist[kHistBins];      // radix histogram; afterwards the kept / equal counts per 128 tokens of the compaction
+  uint32_t cand[2][kCandMax];    // keys that still share the threshold's leading digits
   uint32_t warp[32];
-  uint32_t prefix, remaining, near;
+  uint32_t range[64];
+  uint32_t prefix, remaining, nbin, near, ncand[2];
 };
+static_assert(kTopkMaxTokens / 128 <= 512 && kTopkMaxTokens % 4 == 0, "one count per 128 tokens and thread; keys in 16-byte words");
 
-// ---- exact top-k of one image by one CTA (all kTopkThreads threads): radix select on the fp32 bit patterns of the
+// Smallest and largest score key of the image, gathered while the scores are computed: every CTA folds the keys of
+// its rows and adds them to two words per image with integer atomics (order-independent); the words hold ~min and
+// max so that zero means "nothing yet", and the CTA that ranks the image zeroes them again.
+template <int T>
+__device__ __forceinline__ void publish_range(uint32_t lo, uint32_t hi, TopkShared& sh, unsigned int* range_b) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) { sh.range[warp] = lo; sh.range[32 + warp] = hi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (T / 32); ++w) { lo = min(lo, sh.range[w]); hi = max(hi, sh.range[32 + w]); }
+    if (lo <= hi) { atomicMax(range_b, ~lo); atomicMax(range_b + 1, hi); }
+  }
+}
+
+// The bin, counted from the top, in which the running count reaches sh.remaining: its index is added to sh.prefix at
+// `shift`, sh.remaining becomes the rank inside the bin and sh.nbin the bin's count.  All threads; ends with a barrier.
+template <int T>
+__device__ __forceinline__ void threshold_bin(TopkShared& sh, int nbins, int shift) {
+  const int tid = threadIdx.x;
+  uint32_t local[4], sum = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int bin = nbins - 1 - 4 * tid - j;
+    local[j] = bin >= 0 ? sh.hist[bin] : 0u;
+    sum += local[j];
+  }
+  const uint32_t rem = sh.remaining;   // read before the barriers of the scan, rewritten after them
+  uint32_t tot;
+  const uint32_t excl = block_exclusive_scan<T>(sum, sh.warp, &tot);
+  if (excl < rem && excl + sum >= rem) {   // exactly one thread
+    uint32_t cum = excl;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (cum + local[j] >= rem) {
+        sh.prefix |= (uint32_t)(nbins - 1 - 4 * tid - j) << shift;
+        sh.remaining = rem - cum;
+        sh.nbin = local[j];
+        break;
+      }
+      cum += local[j];
+    }
+  }
+  __syncthreads();
+}
+
+// ---- exact top-k of one image by one CTA (all T threads): radix select on the fp32 bit patterns of the
 // scores (s >= 0, so they order like the values), ties to the lowest index, ascending output, inverse map.
+// range_b: the image's two range words (see publish_range), complete when this is called.
+//   1. one sweep brings the scores from L2 into shared memory as keys relative to the smallest, and counts the first
+//      digit -- the top 11 bits of the range the keys really span, so that the counts spread over the bins;
+//   2. the keys inside the threshold's bin (a few dozen on a map of distinct scores) are copied to a list, which
+//      is finished by counting when it is short and by 8-bit digits otherwise; a bin too full for the list (many
+//      equal scores) is refined with 8-bit digits over all keys until it fits;
+//   3. ordered compaction: counts per 128 tokens, one scan over them, then every lane knows the output slots of its
+//      four tokens.
+// One SM does all of this while the others idle, and its instruction issue is what the sweeps wait for: they take
+// four keys per lane and 16-byte shared-memory accesses.
+template <int T>
 __device__ __forceinline__ void topk_image(const float* __restrict__ sc, int n, int k, uint32_t* s_keys, TopkShared& sh,
-                                           int32_t* __restrict__ idx_b, int32_t* __restrict__ inv_b, int32_t* near_tie_b) {
+                                           int32_t* __restrict__ idx_b, int32_t* __restrict__ inv_b, int32_t* near_tie_b,
+                                           unsigned int* range_b) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) { sh.prefix = 0u; sh.remaining = (uint32_t)k; sh.near = 0u; }
-  // Keys are taken relative to the smallest key of the image: the scores of one map share their leading bits, and
-  // ranking only the bits that differ both skips passes and spreads the keys over the histogram bins.
-  uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-  // the scores come from L2: up to eight 16-byte loads per thread are requested before the first is used (one CTA
-  // fetching them one dependent load at a time took longer than the ranking itself)
+  const uint32_t kmin = ~__ldcg(range_b), kmax = __ldcg(range_b + 1);
+  const uint32_t range = kmax >= kmin ? kmax - kmin : 0u;
+  const int bits = range ? 32 - __clz(range) : 0;
+  int width = min(bits, kFirstDigitBits);
+  int shift = bits - width;
+#pragma unroll
+  for (int j = 0; j < kHistBins / T; ++j) sh.hist[tid + j * T] = 0u;
+  if (tid == 0) { sh.prefix = 0u; sh.remaining = (uint32_t)k; sh.near = 0u; sh.ncand[0] = 0u; sh.ncand[1] = 0u; }
+  __syncthreads();
+  if (tid == 0) { range_b[0] = 0u; range_b[1] = 0u; }   // every thread has read them
+
+  // ---- 1. scores -> keys, first digit counted on the way.  Up to eight 16-byte loads per thread are requested
+  // before the first is used (one CTA fetching them one dependent load at a time took longer than the ranking).
   const int n4 = (n % 4 == 0 && (reinterpret_cast<uintptr_t>(sc) & 15u) == 0) ? n / 4 : 0;
-  for (int i0 = tid; i0 < n4; i0 += kTopkThreads * 8) {
+  const uint32_t top = (1u << width) - 1u;
+  for (int i0 = tid; i0 < n4; i0 += T * 8) {
     float4 v[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u)
-      if (i0 + u * kTopkThreads < n4) v[u] = __ldcg(reinterpret_cast<const float4*>(sc) + i0 + u * kTopkThreads);
+      if (i0 + u * T < n4) v[u] = __ldcg(reinterpret_cast<const float4*>(sc) + i0 + u * T);
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const int i4 = i0 + u * kTopkThreads;
+      const int i4 = i0 + u * T;
       if (i4 < n4) {
-        const float f[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const uint32_t key = __float_as_uint(f[e]) & 0x7FFFFFFFu;  // drops the sign of -0
-          s_keys[KI(4 * i4 + e)] = key;
-          kmin = min(kmin, key); kmax = max(kmax, key);
-        }
+        uint4 key;
+        key.x = (__float_as_uint(v[u].x) & 0x7FFFFFFFu) - kmin;   // the mask drops the sign of -0
+        key.y = (__float_as_uint(v[u].y) & 0x7FFFFFFFu) - kmin;
+        key.z = (__float_as_uint(v[u].z) & 0x7FFFFFFFu) - kmin;
+        key.w = (__float_as_uint(v[u].w) & 0x7FFFFFFFu) - kmin;
+        reinterpret_cast<uint4*>(s_keys)[i4] = key;
+        // (the clamp only matters if the range words were damaged, e.g. by two launches sharing one workspace)
+        atomicAdd(&sh.hist[min(key.x >> shift, top)], 1u); atomicAdd(&sh.hist[min(key.y >> shift, top)], 1u);
+        atomicAdd(&sh.hist[min(key.z >> shift, top)], 1u); atomicAdd(&sh.hist[min(key.w >> shift, top)], 1u);
       }
     }
   }
-  for (int i = 4 * n4 + tid; i < n; i += kTopkThreads) {
-    const uint32_t key = __float_as_uint(__ldcg(sc + i)) & 0x7FFFFFFFu;
-    s_keys[KI(i)] = key;
-    kmin = min(kmin, key); kmax = max(kmax, key);
+  for (int i = 4 * n4 + tid; i < n; i += T) {
+    const uint32_t key = (__float_as_uint(__ldcg(sc + i)) & 0x7FFFFFFFu) - kmin;
+    s_keys[i] = key;
+    atomicAdd(&sh.hist[min(key >> shift, top)], 1u);
   }
-  __syncthreads();   // a thread's keys were written by other threads
-  kmin = __reduce_min_sync(0xffffffffu, kmin);
-  kmax = __reduce_max_sync(0xffffffffu, kmax);
-  if (lane == 0) { sh.warp[warp] = kmin; sh.hist[warp] = kmax; }
   __syncthreads();
-  kmin = sh.warp[lane < kTopkWarps ? lane : 0];
-  kmax = sh.hist[lane < kTopkWarps ? lane : 0];
-  kmin = __reduce_min_sync(0xffffffffu, kmin);
-  kmax = __reduce_max_sync(0xffffffffu, kmax);
-  __syncthreads();
-  for (int i = tid; i < n; i += kTopkThreads) s_keys[KI(i)] -= kmin;  // each thread rewrites its own keys
-  const uint32_t range = kmax - kmin;
-  const int npass = range ? (32 - __clz(range) + 7) / 8 : 0;
 
-  // Radix select, most significant byte first: after the passes sh.prefix is the k-th largest key and
-  // sh.remaining how many keys equal to it belong to the kept set.
-  for (int pass = 0; pass < npass; ++pass) {
-    const int shift = 8 * (npass - 1 - pass);
-    const uint32_t hi_mask = shift + 8 >= 32 ? 0u : (0xFFFFFFFFu << (shift + 8));
-    if (tid < 256) sh.hist[tid] = 0u;
-    __syncthreads();
-    const uint32_t prefix = sh.prefix;
-    for (int i = tid; i < n; i += kTopkThreads) {
-      const uint32_t key = s_keys[KI(i)];
-      if ((key & hi_mask) == prefix) atomicAdd(&sh.hist[(key >> shift) & 255u], 1u);
-    }
-    __syncthreads();
-    if (tid < 32) {
-      // lane l owns bins 255-8l .. 248-8l (descending); find the bin where the running count from the
-      // top reaches sh.remaining.
-      uint32_t local[8], sum = 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) { local[j] = sh.hist[255 - 8 * lane - j]; sum += local[j]; }
-      uint32_t inc = sum;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += t;
-      }
-      const uint32_t rem = sh.remaining;
-      const uint32_t excl = inc - sum;
-      const bool mine = (excl < rem) && (inc >= rem);  // exactly one lane
-      if (mine) {
-        uint32_t cum = excl;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (cum + local[j] >= rem) {
-            sh.prefix = prefix | ((uint32_t)(255 - 8 * lane - j) << shift);
-            sh.remaining = rem - cum;
-            break;
-          }
-          cum += local[j];
+  // ---- 2. the k-th largest key: after this sh.prefix is that key (relative to kmin) and sh.remaining how many of
+  // the keys equal to it belong to the kept set.
+  bool listed = false;
+  int cur = 0;
+  uint32_t nlist = 0;
+  for (;;) {
+    threshold_bin<T>(sh, 1 << width, shift);
+    if (shift == 0) break;                        // every bit of the range is decided
+    const uint32_t prefix = sh.prefix, nbin = sh.nbin;
+    if (listed || nbin <= (uint32_t)kCandMax) {   // the keys of the threshold's bin, in any order
+      const int nxt = listed ? cur ^ 1 : 0;
+      if (listed) {
+        for (uint32_t i = tid; i < nlist; i += T) {
+          const uint32_t key = sh.cand[cur][i];
+          if ((key >> shift) == (prefix >> shift)) sh.cand[nxt][atomicAdd(&sh.ncand[nxt], 1u)] = key;
         }
+      } else {
+        for (int i0 = tid * 4; i0 < n; i0 += T * 4) {
+          const uint4 v = reinterpret_cast<const uint4*>(s_keys)[i0 >> 2];
+          const uint32_t key[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            if (i0 + e < n && (key[e] >> shift) == (prefix >> shift)) sh.cand[nxt][atomicAdd(&sh.ncand[nxt], 1u)] = key[e];
+        }
+      }
+      listed = true; cur = nxt; nlist = nbin;
+      __syncthreads();
+      if (nlist <= (uint32_t)kCountMax) {         // finish by counting: the key with fewer than `remaining` keys above
+        const uint32_t rem = sh.remaining;        // it and at least `remaining` keys not below it
+        __syncthreads();
+        if ((uint32_t)tid < nlist) {
+          const uint32_t key = sh.cand[cur][tid];
+          uint32_t gt = 0, eq = 0;
+          for (uint32_t j = 0; j < nlist; ++j) { const uint32_t c = sh.cand[cur][j]; gt += c > key; eq += c == key; }
+          if (gt < rem && rem <= gt + eq) { sh.prefix = key; sh.remaining = rem - gt; }   // equal keys write the same
+        }
+        __syncthreads();
+        break;
+      }
+    }
+    // the next 8-bit digit of the keys that share the prefix
+    width = min(shift, 8);
+    shift -= width;
+    if (tid < 256) sh.hist[tid] = 0u;
+    if (tid == 0 && listed) sh.ncand[cur ^ 1] = 0u;
+    __syncthreads();
+    const uint32_t dmask = (1u << width) - 1u;
+    if (listed) {
+      for (uint32_t i = tid; i < nlist; i += T) atomicAdd(&sh.hist[(sh.cand[cur][i] >> shift) & dmask], 1u);
+    } else {
+      const int up = shift + width;               // <= 20: the first digit took at least one bit above it
+      for (int i0 = tid * 4; i0 < n; i0 += T * 4) {
+        const uint4 v = reinterpret_cast<const uint4*>(s_keys)[i0 >> 2];
+        const uint32_t key[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (i0 + e < n && (key[e] >> up) == (prefix >> up)) atomicAdd(&sh.hist[(key[e] >> shift) & dmask], 1u);
       }
     }
     __syncthreads();
   }
-  __syncthreads();
   const uint32_t tau = sh.prefix;  // relative to kmin
   const uint32_t need_eq = sh.remaining;
+  __syncthreads();                 // the histogram is reused below
 
-  // Ordered compaction: thread t owns the contiguous tokens [t*per, (t+1)*per).
-  const int per = (n + kTopkThreads - 1) / kTopkThreads;
-  const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
-  // one scan for both counts a thread needs: keys above the threshold (low half) and keys equal to it (high
-  // half) among the tokens before its own; n <= 49152 keeps either total below 2^16
-  uint32_t cnt = 0;
-  for (int i = i0; i < i1; ++i) {
-    const uint32_t key = s_keys[KI(i)];
-    cnt += (key > tau) + ((uint32_t)(key == tau) << 16);
+  // ---- 3. ordered compaction, 128 consecutive tokens per warp step (four per lane).  Counts per 128 tokens of the
+  // keys above the threshold (low half) and equal to it (high half; n <= 49152 keeps either total below 2^16), one
+  // scan over them, then every lane knows the output slots of its tokens.
+  uint32_t* seg = sh.hist;
+  const int nchunk = (n + 127) / 128;      // <= 384: one per thread in the scan
+  const uint4* s_keys4 = reinterpret_cast<const uint4*>(s_keys);   // the allocation is padded to whole 16-byte words
+  for (int c = warp; c < nchunk; c += (T / 32)) {
+    const int i0 = c * 128 + lane * 4;
+    uint32_t p = 0;
+    if (i0 < n) {
+      const uint4 v = s_keys4[i0 >> 2];
+      const uint32_t key[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (i0 + e < n) p += (uint32_t)(key[e] > tau) + ((uint32_t)(key[e] == tau) << 16);
+    }
+    p = __reduce_add_sync(0xffffffffu, p);
+    if (lane == 0) seg[c] = p;
   }
-  uint32_t tot;
-  const uint32_t before = block_exclusive_scan(cnt, sh.warp, &tot);
-  const uint32_t eq_before = before >> 16;
-  uint32_t pos = (before & 0xFFFFu) + min(eq_before, need_eq);   // kept tokens before this thread's first
-  uint32_t e = eq_before;
+  __syncthreads();
+  {
+    const uint32_t mine = tid < nchunk ? seg[tid] : 0u;
+    uint32_t tot;
+    const uint32_t before = block_exclusive_scan<T>(mine, sh.warp, &tot);
+    if (tid < nchunk) seg[tid] = before;
+  }
+  __syncthreads();
   const float tau_f = __uint_as_float(tau + kmin);
   const float band = 1e-5f * tau_f;
   uint32_t near = 0;
-  for (int i = i0; i < i1; ++i) {
-    uint32_t key = s_keys[KI(i)];
-    bool take = key > tau;
-    if (key == tau) { take = (e < need_eq); ++e; }
-    if (take) idx_b[pos] = i;
-    if (inv_b) inv_b[i] = take ? (int32_t)pos : -1;
-    pos += take;
-    near += (fabsf(__uint_as_float(key + kmin) - tau_f) <= band);
+  for (int c = warp; c < nchunk; c += (T / 32)) {
+    const int i0 = c * 128 + lane * 4;
+    uint32_t key[4] = {0u, 0u, 0u, 0u};
+    uint32_t p = 0;
+    if (i0 < n) {
+      const uint4 v = s_keys4[i0 >> 2];
+      key[0] = v.x; key[1] = v.y; key[2] = v.z; key[3] = v.w;
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (i0 + e < n) p += (uint32_t)(key[e] > tau) + ((uint32_t)(key[e] == tau) << 16);
+    }
+    uint32_t inc = p;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    const uint32_t base = seg[c] + inc - p;
+    uint32_t gt_before = base & 0xFFFFu, eq_before = base >> 16;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (i0 + e < n) {
+        const bool is_gt = key[e] > tau, is_eq = key[e] == tau;
+        if (is_gt || (is_eq && eq_before < need_eq)) {          // equal keys: the lowest indices
+          const uint32_t pos = gt_before + min(eq_before, need_eq);   // kept tokens before this one
+          idx_b[pos] = i0 + e;
+          if (inv_b) inv_b[i0 + e] = (int32_t)pos;   // the other entries were set to -1 when the rows were scored
+        }
+        gt_before += is_gt; eq_before += is_eq;
+        if (near_tie_b) near += (fabsf(__uint_as_float(key[e] + kmin) - tau_f) <= band);
+      }
+    }
   }
   if (near_tie_b) {
 #pragma unroll
@@ -282,13 +446,14 @@ __device__ __forceinline__ void topk_image(const float* __restrict__ sc, int n, 
   }
 }
 
-// grid (CTAs per image, B), 512 threads, sized to be resident all at once (two CTAs per SM); the warps of
-// an image stride over its token rows.  Dynamic shared memory max(C, n + n/32) * 4 bytes (mean token, then keys).
+// grid (CTAs per image, B), 1024 threads, one CTA per SM (the CTA that ranks an image then has 32 warps to hide the
+// latencies of its sweeps with); the warps of an image stride over its token rows.  Dynamic shared memory
+// max(9 C, n) * 4 bytes (mean token and staged partial sums, then keys).
 template <typename XT>
-__global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const XT* __restrict__ x,
+__global__ void __launch_bounds__(kSelectThreads, 1) score_topk_kernel(const XT* __restrict__ x,
                                                                   const float4* __restrict__ group_partial, int ngroups, int n,
-                                                                  int C4, int k, float* __restrict__ score,
-                                                                  unsigned int* img_tickets, int32_t* __restrict__ idx,
+                                                                  int C4, int k, int staged, float* __restrict__ score,
+                                                                  unsigned int* img_tickets, unsigned int* img_range, int32_t* __restrict__ idx,
                                                                   int32_t* __restrict__ inv, int32_t* __restrict__ near_tie) {
   extern __shared__ float4 s_dyn[];
   float4* s_mean = s_dyn;
@@ -298,10 +463,13 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const XT* _
   const int b = blockIdx.y, tid = threadIdx.x;
   pdl_trigger();
   pdl_wait();
-  mean_from_partials(s_mean, group_partial + (size_t)b * ngroups * C4, ngroups, nullptr, 0, C4, n);
+  if (staged) mean_from_partials_halves<kSelectThreads>(s_mean, s_mean + C4, group_partial + (size_t)b * ngroups * C4, ngroups, C4, n);
+  else mean_from_partials<kSelectThreads>(s_mean, group_partial + (size_t)b * ngroups * C4, ngroups, nullptr, 0, C4, n);   // very wide maps
   __syncthreads();
-  score_rows<true, 8, XT>(x, s_mean, b, n, C4, score);
-  __threadfence();  // this thread's scores are visible device-wide before the CTA takes its ticket
+  uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+  score_rows<kSelectThreads, true, 8, XT>(x, s_mean, b, n, C4, score, inv, lo, hi);
+  publish_range<kSelectThreads>(lo, hi, sh, img_range + 2 * b);
+  __threadfence();  // this thread's scores (and range) are visible device-wide before the CTA takes its ticket
 
   // ---- the last CTA of this image to get here ranks the image
   __syncthreads();
@@ -313,7 +481,8 @@ __global__ void __launch_bounds__(kTopkThreads, 2) score_topk_kernel(const XT* _
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  topk_image(score + (size_t)b * n, n, k, s_keys, sh, idx + (size_t)b * k, inv ? inv + (size_t)b * n : nullptr, near_tie ? near_tie + b : nullptr);
+  topk_image<kSelectThreads>(score + (size_t)b * n, n, k, s_keys, sh, idx + (size_t)b * k, inv ? inv + (size_t)b * n : nullptr, near_tie ? near_tie + b : nullptr,
+             img_range + 2 * b);
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -338,7 +507,7 @@ struct FusedSelectArgs {
   unsigned int* done; unsigned int done_target;
   // phase 1
   const float4* group_partial; int ngroups;
-  float* score; unsigned int* img_tickets; int32_t* idx; int32_t* inv;
+  float* score; unsigned int* img_tickets; unsigned int* img_range; int32_t* idx; int32_t* inv;
   unsigned int* ready; unsigned int epoch;
   // phase 2
   const float* sigma; const float* beta; uint2* a_out;
@@ -527,10 +696,12 @@ __global__ void __launch_bounds__(kTopkThreads, 1) select_fused_kernel(const Fus
   if (!ok) return;
 
   // ---- phase 1: mean token, scores, top-k
-  mean_from_partials(s_dyn, a.group_partial + (size_t)b * a.ngroups * C4, a.ngroups,
+  mean_from_partials<kTopkThreads>(s_dyn, a.group_partial + (size_t)b * a.ngroups * C4, a.ngroups,
                      a.y ? a.kept_group + (size_t)b * a.ngk * C4 : nullptr, a.y ? a.ngk : 0, C4, n);
   __syncthreads();
-  score_rows<false, 16, float>(reinterpret_cast<const float*>(a.x), s_dyn, b, n, C4, a.score);
+  uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+  score_rows<kTopkThreads, false, 16, float>(reinterpret_cast<const float*>(a.x), s_dyn, b, n, C4, a.score, a.inv, lo, hi);
+  publish_range<kTopkThreads>(lo, hi, sh, a.img_range + 2 * b);
   __threadfence();
   __syncthreads();
   if (tid == 0) {
@@ -545,7 +716,8 @@ __global__ void __launch_bounds__(kTopkThreads, 1) select_fused_kernel(const Fus
   float4* s_beta = nullptr;
   if (last) {
     __threadfence();
-    topk_image(a.score + (size_t)b * n, n, a.k, reinterpret_cast<uint32_t*>(s_dyn), sh, a.idx + (size_t)b * a.k, a.inv + (size_t)b * n, nullptr);
+    topk_image<kTopkThreads>(a.score + (size_t)b * n, n, a.k, reinterpret_cast<uint32_t*>(s_dyn), sh, a.idx + (size_t)b * a.k, a.inv + (size_t)b * n, nullptr,
+               a.img_range + 2 * b);
     __threadfence();
     __syncthreads();
     if (tid == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.ready + b), "r"(a.epoch) : "memory");
@@ -597,7 +769,8 @@ __global__ void inv_scatter_kernel(const int32_t* __restrict__ idx, int B, int k
 
 }  // namespace
 
-size_t select_ticket_bytes(int B) { return align_up((size_t)B * (kMaxGroups + 1) * sizeof(unsigned int), 256); }
+// group arrival counters [B, kMaxGroups], image arrival counters [B], score range words [B, 2]
+size_t select_ticket_bytes(int B) { return align_up((size_t)B * (kMaxGroups + 3) * sizeof(unsigned int), 256); }
 
 static void chunking(int n, int* nchunks, int* group, int* ngroups) {
   *nchunks = (n + kColsumRows - 1) / kColsumRows;
@@ -650,16 +823,20 @@ static cudaError_t launch_select_t(const XT* x, int B, int n, int C, int k, int3
   if (!have_partials)
     launch_pdl(colsum_chunk_kernel<XT>, dim3(w.nchunks, B), dim3(256), 0, st, x, n, C4, w.nchunks, w.group,
                w.ngroups, reinterpret_cast<float4*>(w.chunk_partial), reinterpret_cast<float4*>(w.group_partial), w.tickets);
-  const size_t keys_smem = ((size_t)n + n / 32 + 1) * 4;
-  const size_t smem = keys_smem > (size_t)C * 4 ? keys_smem : (size_t)C * 4;
-  // all CTAs resident at once: two per SM over the B images, never more than one warp per token row
-  int per_image = (2 * g_num_sms + B - 1) / B;
-  const int need = (n + kTopkWarps - 1) / kTopkWarps;
+  const size_t keys_smem = ((size_t)n + 3) / 4 * 16;   // whole 16-byte words
+  const int staged = (size_t)C * 4 * 9 <= kTopkMaxSmem;  // room for the mean token and eight staged partial sums
+  const size_t mean_smem = (size_t)C * 4 * (staged ? 9 : 1);
+  const size_t smem = keys_smem > mean_smem ? keys_smem : mean_smem;
+  // one CTA per SM over the B images, never more than one warp per token row
+  int per_image = g_num_sms / B;
+  const int need = (n + kSelectWarps - 1) / kSelectWarps;
   if (per_image > need) per_image = need;
   if (per_image < 1) per_image = 1;
-  launch_pdl(score_topk_kernel<XT>, dim3(per_image, B), dim3(kTopkThreads), smem, st, x,
-             reinterpret_cast<const float4*>(w.group_partial), w.ngroups, n, C4, k, sc, w.tickets + (size_t)B * kMaxGroups, idx, inv,
-             near_tie);
+  unsigned int* img_tickets = w.tickets + (size_t)B * kMaxGroups;
+  unsigned int* img_range = w.tickets + (size_t)B * (kMaxGroups + 1);
+  const float4* gp = reinterpret_cast<const float4*>(w.group_partial);
+  launch_pdl(score_topk_kernel<XT>, dim3(per_image, B), dim3(kSelectThreads), smem, st, x, gp, w.ngroups, n, C4, k, staged, sc, img_tickets,
+             img_range, idx, inv, near_tie);
   return cudaGetLastError();
 }
 
@@ -684,7 +861,7 @@ size_t select_fused_ws_bytes(int B, int C) {
 }
 
 static size_t fused_smem_bytes(int n, int C) {
-  const size_t keys = ((size_t)n + n / 32 + 1) * 4;
+  const size_t keys = ((size_t)n + 3) / 4 * 16;
   const size_t vec = (size_t)C * 4;                       // the mean token
   const int rows_par = kTopkThreads / (C / 8);
   const size_t comb = (size_t)(rows_par > 1 ? rows_par - 1 : 0) * C * 4;
@@ -728,7 +905,8 @@ cudaError_t launch_select_fused(const FusedSelect& f, cudaStream_t st) {
   a.done_target = *f.done_total;
   a.epoch = ++*f.epoch;
   a.group_partial = reinterpret_cast<const float4*>(w.group_partial); a.ngroups = w.ngroups;
-  a.score = w.score; a.img_tickets = w.tickets + (size_t)f.B * kMaxGroups; a.idx = f.idx; a.inv = f.inv;
+  a.score = w.score; a.img_tickets = w.tickets + (size_t)f.B * kMaxGroups;
+  a.img_range = w.tickets + (size_t)f.B * (kMaxGroups + 1); a.idx = f.idx; a.inv = f.inv;
   a.sigma = f.sigma; a.beta = f.beta; a.a_out = reinterpret_cast<uint2*>(f.a_out);
   a.status = f.status;
   // algorithmic bytes: the selection (x once, scores, indices), the gather (kept rows in, bf16 out) and, when it

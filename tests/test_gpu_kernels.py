@@ -82,6 +82,36 @@ def test_prune_select_ties_go_to_lowest_index():
     assert (r["near_tie"].cpu().numpy() > 1).all()
 
 
+@pytest.mark.parametrize("crowd,levels,keep", [(3000, 3000, 0.3), (3000, 300, 0.3), (600, 600, 0.1), (200, 40, 0.02),
+                                               (4000, 1, 0.5), (1100, 1100, 0.2)])
+def test_prune_select_scores_crowded_at_the_threshold(crowd, levels, keep):
+    """A few far outliers stretch the range of the scores while `crowd` tokens sit within a few hundred ulps of one
+    another (on `levels` distinct values) right where the k-th largest falls: the threshold's first-digit bin holds
+    the whole crowd, so the ranking has to refine it with further digits -- over all keys while the bin is too full
+    for the candidate list, over the list afterwards -- before it can finish by counting.  Exact given the scores."""
+    B, h, w, C = 2, 64, 64, 8
+    n = h * w
+    k = O.kept_count(keep, h, w)
+    above = max(2, k - crowd // 2)             # tokens far above the crowd: the k-th largest falls inside the crowd
+    assert above < k <= above + crowd <= n
+    a = np.zeros((B, n), dtype=np.float64)
+    for b in range(B):
+        perm = np.argsort(I.uniform01(90 + b, n), kind="stable")
+        a[b, perm[:crowd]] = 1.0 + (np.arange(crowd) % levels) * 2.0 ** -22 * (1 + b)
+        a[b, perm[crowd:crowd + above]] = 2.0 + 30.0 * I.uniform01(290 + b, above)
+        a[b, perm[crowd + above:]] = 0.25 + 0.5 * I.uniform01(190 + b, n - crowd - above)
+    x = np.zeros((B, n, C), dtype=np.float32)
+    x[:, :, 0] = a
+    x[:, 1::2, 0] *= -1.0                      # alternating signs keep the mean token near zero
+    r = fv.fv_prune_select(dev(x), h, w, keep, want_inv=True, want_score=True, want_near_tie=True)
+    torch.cuda.synchronize()
+    score_g = r["score"].cpu().numpy()
+    np.testing.assert_allclose(score_g, O.pts_score(x), rtol=2e-5, atol=1e-6)
+    idx_g = r["idx"].cpu().numpy().astype(np.int64)
+    assert np.array_equal(idx_g, O.pts_topk(score_g, k))
+    assert np.array_equal(r["inv"].cpu().numpy().astype(np.int64), O.inverse_map(idx_g, n))
+
+
 def test_prune_select_argument_errors():
     big = torch.zeros((1, 193 * 256, 8), device=DEV)                      # one row of tokens beyond the largest map
     with pytest.raises(fv.FvError) as e:
