@@ -31,11 +31,13 @@ from paper_2503_23367_b200 import inputs as I  # noqa: E402
 # the library per launch), averaged over the launches of the dominant class; the notes say what an ncu
 # capture of the same kernel measured against that count (summaries under profiles/).
 NCU_TRAFFIC_NOTE = {
-    "gemm": "A + W + out bytes per launch, mean over the pruned steps' launches; ncu on M1640 N6144 K2048: dram read 31.95 MB = A + W "
-            "(31.9 MB), out (20 MB) still in L2 at kernel end; CTA-pair kernel M1844 N2048 K8192: read 63.8 MB = A + W, write 3.8 of 7.6 MB",
-    "attention": "Q + O + K + V^T bytes per launch; ncu on q820 kv5223 H16 hd128 B2: dram read 92.7 MB (K, V^T, Q = 92.3 MB), write 3.6 of 6.7 MB",
-    "restore": "x read + written, y, cache; ncu on B2 64x64 C2048 k820: read 82.3 MB + write 11.8 MB of 149 MB (x written stays in L2)",
-    "select": "x once + scores + indices; ncu on B2 64x64 C2048: score+top-k kernel reads 67.3 MB (x = 67.1 MB)",
+    "gemm": "A + W + out bytes per launch (the library's count), mean over the pruned steps' launches; ncu at the 128x128 step's shapes: "
+            "QKV M3277 N6144 K2048 (CTA-pair kernel) dram read 38.7 MB = A + W (38.6 MB), out (40 MB) still in L2 at kernel end; second MLP "
+            "GEMM M3277 N2048 K8192 (128x192 tiles) read 130.9 MB against A + W = 87.3 MB: its second round of tiles re-reads A",
+    "attention": "Q + O + K + V^T bytes per launch; ncu on q820 kv5223 H16 hd128 B2 (whole work items): dram read 92.6 MB (K, V^T, Q = 92.3 MB), "
+                 "write 3.8 of 6.7 MB; on q820 kv7245 B1 cut into 148 pieces: read 63.7 MB (62.7 MB), partial results stay in L2",
+    "restore": "x read + written, y, cache; ncu on B2 64x64 C2048 k820: read 82.3 MB + write 14.2 MB of 149 MB (x written stays in L2)",
+    "select": "x once + scores + indices; ncu on B2 64x64 C2048: score+top-k kernel reads 67.4 MB (x = 67.1 MB); on B1 128x128: 134.4 MB (134.2 MB)",
     "gather_ln": "kept rows in, bf16 rows out; ncu on B2 k820 C2048: read 13.5 MB (rows = 13.4 MB), output left in L2",
 }
 
