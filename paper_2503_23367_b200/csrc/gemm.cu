@@ -38,10 +38,16 @@ constexpr int BK = 64;
 constexpr int kGemmThreads = 192;
 constexpr int kATileBytes = BM * BK * 2;  // 16 KB
 
+// kKps: k-blocks per pipeline stage.  The MMA-issuing thread pays a fixed price per stage (the wait on the full barrier
+// and the commit that frees the stage: about 0.2 us of dependent instructions), which for tiles of up to 128 columns
+// exceeds the time of the stage's MMAs; with two k-blocks behind one barrier it is paid half as often.  The wider
+// tiles keep one k-block per stage: their MMAs take that long anyway, and two k-blocks would leave two stages.
 template <int BN> struct GemmCfg {
+  static constexpr int kKps = (BN <= 128) ? 2 : 1;
   static constexpr int kBTileBytes = BN * BK * 2;
-  static constexpr int kStageBytes = kATileBytes + kBTileBytes;
-  static constexpr int kStages = (BN == 256) ? 4 : (BN == 192 ? 5 : (BN == 128 ? 6 : 8));
+  static constexpr int kSubBytes = kATileBytes + kBTileBytes;   // one k-block: A tile, then W tile
+  static constexpr int kStageBytes = kKps * kSubBytes;
+  static constexpr int kStages = (BN == 256) ? 4 : (BN == 192 ? 5 : (BN == 128 ? 3 : 4));
   static constexpr int kTmemCols = (BN <= 64) ? 128 : ((BN == 128) ? 256 : 512);  // two accumulators, power of two
   static constexpr int kAccStride = (BN <= 64) ? 64 : ((BN == 128) ? 128 : 256);  // column offset of the second accumulator
   // operand stages | per-warp bias slices | barriers | (residual-epilogue kernels only) one turning tile per warp
@@ -58,6 +64,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
   using Cfg = GemmCfg<BN>;
   constexpr int STAGES = Cfg::kStages;
+  constexpr int KPS = Cfg::kKps;
   constexpr bool RESID = KIND == 1;   // KIND 2: the QKV projection with cosine attention / rotary positions on Q and K
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -104,10 +111,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int tile = (int)blockIdx.x / splits, slice = (int)blockIdx.x - tile * splits;
         const int n0 = (tile / tiles_m) * BN;
         const int kb0 = slice * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
-        pre = min(STAGES, kb1 - kb0);
+        pre = min(STAGES, (kb1 - kb0 + KPS - 1) / KPS);
         for (int i = 0; i < pre; ++i) {
           mbar_expect_tx(&full_bar[i], Cfg::kStageBytes);
-          tma_load_2d(smem + i * Cfg::kStageBytes + kATileBytes, &tmB, (kb0 + i) * BK, n0, &full_bar[i]);
+          for (int u = 0; u < KPS; ++u)   // (a k-block beyond K reads zeros)
+            tma_load_2d(smem + i * Cfg::kStageBytes + u * Cfg::kSubBytes + kATileBytes, &tmB, (kb0 + KPS * i + u) * BK, n0, &full_bar[i]);
         }
       }
       pdl_wait();
@@ -115,18 +123,20 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int tile = item / splits, slice = item - tile * splits;
         const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
         const int kb0 = slice * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; kb += KPS, ++it) {   // one stage: KPS k-blocks of this work item
           const int s = it % STAGES;
           uint8_t* a_s = smem + s * Cfg::kStageBytes;
-          if ((int)it < pre) {  // W tile requested before the wait: only the activations are missing
-            tma_load_2d(a_s, &tmA, kb * BK, m0, &full_bar[s]);
+          if ((int)it < pre) {  // W tiles requested before the wait: only the activations are missing
+            for (int u = 0; u < KPS; ++u) tma_load_2d(a_s + u * Cfg::kSubBytes, &tmA, (kb + u) * BK, m0, &full_bar[s]);
             continue;
           }
           const uint32_t ph = (it / STAGES) & 1;
           if (!mbar_wait(&empty_bar[s], ph ^ 1)) { report(p.status, DEV_TIMEOUT_TMA); ok = false; break; }
           mbar_expect_tx(&full_bar[s], Cfg::kStageBytes);
-          tma_load_2d(a_s, &tmA, kb * BK, m0, &full_bar[s]);
-          tma_load_2d(a_s + kATileBytes, &tmB, kb * BK, n0, &full_bar[s]);
+          for (int u = 0; u < KPS; ++u) {
+            tma_load_2d(a_s + u * Cfg::kSubBytes, &tmA, (kb + u) * BK, m0, &full_bar[s]);
+            tma_load_2d(a_s + u * Cfg::kSubBytes + kATileBytes, &tmB, (kb + u) * BK, n0, &full_bar[s]);
+          }
         }
       }
     }
@@ -143,17 +153,20 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint32_t d = tmem_base + buf * Cfg::kAccStride;
         const int slice = item % splits;
         const int kb0 = slice * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; kb += KPS, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           if (!mbar_wait(&full_bar[s], ph)) { report(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(smem + s * Cfg::kStageBytes);
-          const uint64_t adesc = umma_desc_k_sw128(a_addr);
-          const uint64_t bdesc = umma_desc_k_sw128(a_addr + kATileBytes);
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk)
-            umma_bf16(d, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb > kb0) || kk != 0);
+          for (int u = 0; u < KPS; ++u) {
+            const uint64_t adesc = umma_desc_k_sw128(a_addr + u * Cfg::kSubBytes);
+            const uint64_t bdesc = umma_desc_k_sw128(a_addr + u * Cfg::kSubBytes + kATileBytes);
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; ++kk)
+              umma_bf16(d, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb > kb0) || (u | kk) != 0);
+          }
           umma_commit(&empty_bar[s]);
         }
         if (ok) umma_commit(&acc_full[buf]);
@@ -374,16 +387,19 @@ cudaError_t gemm_init() {
   return cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
 }
 
-// Kernel and tile width for a shape.  Measured on B200, one launch costs about
-//     fixed + rounds x k-blocks x per_kblock
-// where rounds = ceil(tiles / resident CTAs or pairs): the operand pipeline is bound by the latency of
-// its loads (all of shared memory is in flight), so a k-block costs about the same whatever the tile
-// width, and wider tiles / CTA pairs win by needing fewer rounds and less L2 traffic per flop.
+// Kernel and tile width for a shape.  Measured on B200 (launches replayed from a CUDA graph, so that the host does
+// not pace them), one launch costs about
+//     fixed + rounds x (per_round + k-blocks x per_kblock)
+// where rounds = ceil(tiles / resident CTAs or pairs).  A k-block of a 128-wide tile is paced by the thread that
+// issues its MMAs (two k-blocks per pipeline stage there), the wider tiles by the MMAs themselves and the operand
+// loads; wider tiles and CTA pairs win by needing fewer rounds and less L2 traffic per flop.
 struct TileChoice { int bn; bool pair; };
 static TileChoice pick_tile(int M, int N, int K, int sms) {
   const int num_kb = (K + BK - 1) / BK;
-  struct Cand { int bn; bool pair; double fixed_us, kb_us; };
-  const Cand cand[4] = {{128, false, 8.5, 0.271}, {192, false, 10.4, 0.278}, {256, false, 10.1, 0.361}, {256, true, 14.0, 0.297}};
+  struct Cand { int bn; bool pair; double fixed_us, round_us, kb_us; };
+  // least-squares fit over M 256 ... 3277 x the four projection shapes of a 2048-wide block, every candidate forced
+  const Cand cand[5] = {{128, false, 2.23, 0.98, 0.235}, {192, false, 2.16, 2.19, 0.292}, {256, false, 1.17, 3.01, 0.349},
+                        {256, true, 3.99, 2.30, 0.316}, {64, false, 2.9, 0.5, 0.21}};
   TileChoice best{128, false};
   double best_cost = 1e30;
   for (const Cand& c : cand) {
@@ -392,7 +408,7 @@ static TileChoice pick_tile(int M, int N, int K, int sms) {
     const int slots = c.pair ? sms / 2 : sms;
     const long tiles = (long)((M + rows - 1) / rows) * ((N + c.bn - 1) / c.bn);
     const long rounds = (tiles + slots - 1) / slots;
-    const double cost = c.fixed_us + (double)rounds * num_kb * c.kb_us;
+    const double cost = c.fixed_us + (double)rounds * (c.round_us + num_kb * c.kb_us);
     if (cost < best_cost - 1e-9) { best_cost = cost; best = TileChoice{c.bn, c.pair}; }
   }
   return best;
@@ -485,8 +501,9 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
     const int sp = pick_splits(tiles128, g.M, num_kb, g_num_sms);
     if (sp > 1 && tiles128 * sp <= g_num_sms && tiles128 * sp <= kSplitMaxItems && tiles128 * sizeof(unsigned int) <= kSplitTicketBytes) {
       bn = bn_split;
-      p.splits = sp;
       p.kb_per_split = (num_kb + sp - 1) / sp;
+      p.kb_per_split += p.kb_per_split & 1;   // even: a pipeline stage may hold two k-blocks of ONE slice
+      p.splits = (num_kb + p.kb_per_split - 1) / p.kb_per_split;   // no empty slice
       p.sk_tickets = static_cast<unsigned int*>(g.splitk_ws);
       p.sk_partial = reinterpret_cast<float*>(static_cast<char*>(g.splitk_ws) + kSplitTicketBytes);
     }
@@ -511,10 +528,13 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
   if (g_force_path == 0 && !qk_extras) {
     const int num_kb = (g.K + BK - 1) / BK;
     const long t128 = (long)tiles_m * ((g.N + 127) / 128), t64 = (long)tiles_m * ((g.N + 63) / 64);
+    // (re-measured GPU-bound after the narrow tiles took two k-blocks per pipeline stage: with more than 32 rows the
+    // 128-wide x 2 cluster, whose ring has no room for that, only wins on a long K; 64-wide x 2 wins on a short one)
     if (num_kb >= 8) {
       if (g.M > 16 && t64 * 4 <= g_num_sms) { cluster_bn = 64; cluster_slices = 4; }
+      else if (g.M > 16 && t64 * 2 <= g_num_sms && num_kb < 64) { cluster_bn = 64; cluster_slices = 2; }
       else if (t128 * 4 <= g_num_sms) { cluster_bn = 128; cluster_slices = 4; }
-      else if (t128 * 2 <= g_num_sms) { cluster_bn = 128; cluster_slices = 2; }
+      else if (t128 * 2 <= g_num_sms && (g.M <= 32 || num_kb >= 64)) { cluster_bn = 128; cluster_slices = 2; }
     }
   }
   if (g_force_path >= 8 && g_force_path <= 11 && !qk_extras) {   // 8: 128 wide x 4 slices, 9: 128 x 2, 10: 64 x 4, 11: 64 x 2
@@ -525,6 +545,7 @@ fv_status launch_gemm(const GemmArgs& g, cudaStream_t st) {
     const int num_kb = (g.K + BK - 1) / BK;
     p.splits = 1; p.sk_partial = nullptr; p.sk_tickets = nullptr;
     p.kb_per_split = (num_kb + cluster_slices - 1) / cluster_slices;
+    p.kb_per_split += p.kb_per_split & 1;   // even: a pipeline stage of the cluster kernel may hold two k-blocks of ONE slice
   }
   LaunchScope scope(KC_GEMM, 1, 2.0 * g.M * (double)g.N * g.K, 2.0 * ((double)g.M * g.K + (double)g.N * g.K + (double)g.M * g.N), st);
   if (cluster_slices) return launch_gemm_cluster(g, p, cluster_bn, cluster_slices, st) == cudaSuccess ? FV_OK : FV_ERR_CUDA;

@@ -30,13 +30,21 @@ constexpr int kThreads = 192;
 // MMA always reads a 128-row A tile from shared memory; with AROWS = 32 the rows beyond the 4 KB that were
 // loaded are whatever follows in shared memory (the stage's own W tile, the next stage, the buffers behind the
 // ring -- all inside the allocation).  They only feed accumulator rows >= 32, which belong to no row of the
-// output and are neither reduced nor stored.  The 12 KB saved per stage buy a deeper ring: more weight bytes
-// in flight per SM, which is what bounds these launches.
+// output and are neither reduced nor stored.  The 12 KB saved per k-block buy a deeper ring.
+//
+// kKps: k-blocks per pipeline stage.  The thread that issues the MMAs is a chain of dependent instructions: per stage
+// it spends about 0.16 us between its commit and seeing the next full barrier, 0.06 us on the commit and 0.03 us per
+// MMA, so with one k-block per stage a k-block costs 0.34 us whatever its bytes (measured with device timestamps: no
+// change without the A loads, with one MMA of four, with the weights resident in L2, with another weight pitch).
+// Two k-blocks behind one barrier halve the per-stage part: 0.24 us per k-block.  Where the ring would shrink to two
+// stages (128 rows of A against 128-wide tiles) one k-block per stage stays.
 template <int BN, int AROWS> struct ClusterCfg {
+  static constexpr int kKps = (AROWS == 128 && BN == 128) ? 1 : 2;
   static constexpr int kATile = AROWS * BK * 2;
   static constexpr int kBTileBytes = BN * BK * 2;
-  static constexpr int kStageBytes = kATile + kBTileBytes;
-  static constexpr int kStages = AROWS == 32 ? ((BN == 128) ? 7 : 10) : ((BN == 128) ? 4 : 6);
+  static constexpr int kSubBytes = kATile + kBTileBytes;       // one k-block: A tile, then W tile
+  static constexpr int kStageBytes = kKps * kSubBytes;
+  static constexpr int kStages = AROWS == 32 ? ((BN == 128) ? 3 : 5) : ((BN == 128) ? 4 : 3);
   static constexpr int kTmemCols = BN;                      // one accumulator (64 or 128: powers of two)
   static constexpr int kRedPitch = BN + 4;                  // floats per row of the reduce buffer (bank spread)
   static constexpr int kRedBytes = BM * kRedPitch * 4;      // [S sources][128/S rows][pitch] = 128 rows in all
@@ -59,6 +67,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   using Cfg = ClusterCfg<BN, AROWS>;
   constexpr int kATileBytes = Cfg::kATile;
   constexpr int STAGES = Cfg::kStages;
+  constexpr int KPS = Cfg::kKps;
   constexpr int ROWS_PER = BM / S;        // rows of the tile each CTA finishes
   constexpr int CHUNKS = BN / 32;         // 32-column chunks per row
   extern __shared__ uint8_t smem_raw[];
@@ -98,44 +107,51 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   if (warp == 0) {
     if (lane == 0) {
       // the weight tiles (never written by a kernel of the step) are requested before the dependency wait
-      const int pre = min(STAGES, kb1 - kb0);
+      const int nst = (kb1 - kb0 + KPS - 1) / KPS;    // stages of KPS k-blocks; a k-block beyond K reads zeros
+      const int pre = min(STAGES, nst);
       for (int i = 0; i < pre; ++i) {
         mbar_expect_tx(&full_bar[i], Cfg::kStageBytes);
-        tma_load_2d(smem + i * Cfg::kStageBytes + kATileBytes, &tmB, (kb0 + i) * BK, n0, &full_bar[i]);
+        for (int u = 0; u < KPS; ++u)
+          tma_load_2d(smem + i * Cfg::kStageBytes + u * Cfg::kSubBytes + kATileBytes, &tmB, (kb0 + KPS * i + u) * BK, n0, &full_bar[i]);
       }
       pdl_wait();
-      uint32_t it = 0;
-      for (int kb = kb0; kb < kb1; ++kb, ++it) {
+      for (int it = 0; it < nst; ++it) {
         const int s = it % STAGES;
+        const int kb = kb0 + KPS * it;
         uint8_t* a_s = smem + s * Cfg::kStageBytes;
-        if ((int)it < pre) {
-          tma_load_2d(a_s, &tmA, kb * BK, m0, &full_bar[s]);
+        if (it < pre) {
+          for (int u = 0; u < KPS; ++u) tma_load_2d(a_s + u * Cfg::kSubBytes, &tmA, (kb + u) * BK, m0, &full_bar[s]);
           continue;
         }
         const uint32_t ph = (it / STAGES) & 1;
         if (!mbar_wait(&empty_bar[s], ph ^ 1)) { report(p.status, DEV_TIMEOUT_TMA); break; }
         mbar_expect_tx(&full_bar[s], Cfg::kStageBytes);
-        tma_load_2d(a_s, &tmA, kb * BK, m0, &full_bar[s]);
-        tma_load_2d(a_s + kATileBytes, &tmB, kb * BK, n0, &full_bar[s]);
+        for (int u = 0; u < KPS; ++u) {
+          tma_load_2d(a_s + u * Cfg::kSubBytes, &tmA, (kb + u) * BK, m0, &full_bar[s]);
+          tma_load_2d(a_s + u * Cfg::kSubBytes + kATileBytes, &tmB, (kb + u) * BK, n0, &full_bar[s]);
+        }
       }
     }
   } else if (warp == 1) {
     pdl_wait();
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
-      uint32_t it = 0;
       bool ok = true;
-      for (int kb = kb0; kb < kb1; ++kb, ++it) {
+      const int nst = (kb1 - kb0 + KPS - 1) / KPS;
+      for (int it = 0; it < nst; ++it) {
         const int s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1;
         if (!mbar_wait(&full_bar[s], ph)) { report(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
         tc_fence_after();
         const uint32_t a_addr = smem_u32(smem + s * Cfg::kStageBytes);
-        const uint64_t adesc = umma_desc_k_sw128(a_addr);
-        const uint64_t bdesc = umma_desc_k_sw128(a_addr + kATileBytes);
 #pragma unroll
-        for (int kk = 0; kk < BK / 16; ++kk)
-          umma_bf16(tmem_base, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb > kb0) || kk != 0);
+        for (int u = 0; u < KPS; ++u) {
+          const uint64_t adesc = umma_desc_k_sw128(a_addr + u * Cfg::kSubBytes);
+          const uint64_t bdesc = umma_desc_k_sw128(a_addr + u * Cfg::kSubBytes + kATileBytes);
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk)
+            umma_bf16(tmem_base, adesc + 2 * kk, bdesc + 2 * kk, idesc, (it | u | kk) != 0);
+        }
         umma_commit(&empty_bar[s]);
       }
       if (ok && kb1 > kb0) umma_commit(acc_full);
