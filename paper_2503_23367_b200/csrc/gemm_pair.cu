@@ -32,9 +32,11 @@ constexpr int kThreads = 192;
 constexpr int kATileBytes = BM * BK * 2;  // 16 KB
 
 template <int BN> struct PairCfg {
+  static constexpr int kKps = 2;                                // k-blocks per pipeline stage (one barrier round trip for both)
   static constexpr int kBHalfBytes = (BN / 2) * BK * 2;
-  static constexpr int kStageBytes = kATileBytes + kBHalfBytes;
-  static constexpr int kStages = (BN == 256) ? 6 : 7;
+  static constexpr int kSubBytes = kATileBytes + kBHalfBytes;   // one k-block: this CTA's A tile, then its half of the W tile
+  static constexpr int kStageBytes = kKps * kSubBytes;
+  static constexpr int kStages = (BN == 256) ? 3 : 4;
   static constexpr int kTmemCols = 512;    // two accumulators, 256 columns apart
   static constexpr int kAccStride = 256;
   // operand stages | per-warp bias slices | barriers | (residual-epilogue kernels only) one turning tile per warp
@@ -49,6 +51,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev p) {
   using Cfg = PairCfg<BN>;
   constexpr int STAGES = Cfg::kStages;
+  constexpr int KPS = Cfg::kKps;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint4* bias_s = reinterpret_cast<uint4*>(smem + STAGES * Cfg::kStageBytes);   // per-warp bias slice of the tile
@@ -91,28 +94,31 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int pre = 0;  // stages of the first tile whose W half-tile is already on its way
       if (pair < total_tiles) {
         const int n0 = (pair / tiles_m) * BN + (int)rank * (BN / 2);
-        pre = min(STAGES, num_kb);
+        pre = min(STAGES, (num_kb + KPS - 1) / KPS);
         for (int i = 0; i < pre; ++i) {
           if (rank == 0) mbar_expect_tx(&full_bar[i], 2 * Cfg::kStageBytes);
-          tma_load_2d_pair(smem + i * Cfg::kStageBytes + kATileBytes, &tmB, i * BK, n0, &full_bar[i]);
+          for (int u = 0; u < KPS; ++u)   // (a k-block beyond K reads zeros)
+            tma_load_2d_pair(smem + i * Cfg::kStageBytes + u * Cfg::kSubBytes + kATileBytes, &tmB, (KPS * i + u) * BK, n0, &full_bar[i]);
         }
       }
       pdl_wait();
       for (int tile = pair; ok && tile < total_tiles; tile += npairs) {
         const int m0 = (tile % tiles_m) * (2 * BM) + (int)rank * BM;
         const int n0 = (tile / tiles_m) * BN + (int)rank * (BN / 2);
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        for (int kb = 0; kb < num_kb; kb += KPS, ++it) {
           const int s = it % STAGES;
           uint8_t* a_s = smem + s * Cfg::kStageBytes;
-          if ((int)it < pre) {  // W half-tile requested before the wait: only the activations are missing
-            tma_load_2d_pair(a_s, &tmA, kb * BK, m0, &full_bar[s]);
+          if ((int)it < pre) {  // W half-tiles requested before the wait: only the activations are missing
+            for (int u = 0; u < KPS; ++u) tma_load_2d_pair(a_s + u * Cfg::kSubBytes, &tmA, (kb + u) * BK, m0, &full_bar[s]);
             continue;
           }
           const uint32_t ph = (it / STAGES) & 1;
           if (!mbar_wait(&empty_bar[s], ph ^ 1)) { report(p.status, DEV_TIMEOUT_TMA); ok = false; break; }
           if (rank == 0) mbar_expect_tx(&full_bar[s], 2 * Cfg::kStageBytes);
-          tma_load_2d_pair(a_s, &tmA, kb * BK, m0, &full_bar[s]);
-          tma_load_2d_pair(a_s + kATileBytes, &tmB, kb * BK, n0, &full_bar[s]);
+          for (int u = 0; u < KPS; ++u) {
+            tma_load_2d_pair(a_s + u * Cfg::kSubBytes, &tmA, (kb + u) * BK, m0, &full_bar[s]);
+            tma_load_2d_pair(a_s + u * Cfg::kSubBytes + kATileBytes, &tmB, (kb + u) * BK, n0, &full_bar[s]);
+          }
         }
       }
     }
@@ -127,17 +133,20 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (!mbar_wait(&acc_empty[buf], ((lt >> 1) & 1) ^ 1)) { report(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
         tc_fence_after();
         const uint32_t d = tmem_base + buf * Cfg::kAccStride;
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        for (int kb = 0; kb < num_kb; kb += KPS, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           if (!mbar_wait(&full_bar[s], ph)) { report(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(smem + s * Cfg::kStageBytes);
-          const uint64_t adesc = umma_desc_k_sw128(a_addr);
-          const uint64_t bdesc = umma_desc_k_sw128(a_addr + kATileBytes);
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk)
-            umma_bf16_pair(d, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0);
+          for (int u = 0; u < KPS; ++u) {
+            const uint64_t adesc = umma_desc_k_sw128(a_addr + u * Cfg::kSubBytes);
+            const uint64_t bdesc = umma_desc_k_sw128(a_addr + u * Cfg::kSubBytes + kATileBytes);
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; ++kk)
+              umma_bf16_pair(d, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | u | kk) != 0);
+          }
           umma_commit_pair(&empty_bar[s]);
         }
         if (ok) umma_commit_pair(&acc_full[buf]);
