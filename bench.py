@@ -33,7 +33,7 @@ from paper_2503_23367_b200 import inputs as I  # noqa: E402
 NCU_TRAFFIC_NOTE = {
     "gemm": "A + W + out bytes per launch (the library's count), mean over the pruned steps' launches; ncu at the 128x128 step's shapes: "
             "QKV M3277 N6144 K2048 (CTA-pair kernel) dram read 38.7 MB = A + W (38.6 MB), out (40 MB) still in L2 at kernel end; second MLP "
-            "GEMM M3277 N2048 K8192 (128x192 tiles) read 130.9 MB against A + W = 87.3 MB: its second round of tiles re-reads A",
+            "GEMM M3277 N2048 K8192 (128x192 tiles) read 129.2 MB against A + W = 87.3 MB: its second round of tiles re-reads A",
     "attention": "Q + O + K + V^T bytes per launch; ncu on q820 kv5223 H16 hd128 B2 (whole work items): dram read 92.6 MB (K, V^T, Q = 92.3 MB), "
                  "write 3.8 of 6.7 MB; on q820 kv7245 B1 cut into 148 pieces: read 63.7 MB (62.7 MB), partial results stay in L2",
     "restore": "x read + written, y, cache; ncu on B2 64x64 C2048 k820: read 82.3 MB + write 14.2 MB of 149 MB (x written stays in L2)",
