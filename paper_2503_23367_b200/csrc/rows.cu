@@ -168,8 +168,9 @@ __device__ __forceinline__ void bf16x8_to_float(const uint4& p, float (&f)[8]) {
 //   branch has produced y: column sums continue from the chunk partial of part 1, then the group fold);
 //   3 : as 1, but the sums of the rows that were not kept are folded here (the kept rows are then restored, and
 //   summed, by the next selection's kernel).
-template <typename XT>
-__global__ void __launch_bounds__(256) restore_residual_kernel(XT* __restrict__ x, const uint4* __restrict__ y,
+// RF: rows in flight per thread (4, or 2 in the build that fits four CTAs per SM: 64 registers).
+template <typename XT, int RF>
+__global__ void __launch_bounds__(256, RF == 2 ? 4 : 3) restore_residual_kernel(XT* __restrict__ x, const uint4* __restrict__ y,
                                                                const uint4* __restrict__ cache, const int32_t* __restrict__ inv,
                                                                const float* __restrict__ gamma, int mod_stride, int n, int k,
                                                                int h, int w, int hc, int wc, int C8, int nchunks, int group,
@@ -203,18 +204,18 @@ __global__ void __launch_bounds__(256) restore_residual_kernel(XT* __restrict__ 
       const float4* cp = chunk_partial + ((size_t)b * nchunks + chunk) * C8 * 2 + 2 * c8;
       a0 = __ldcg(cp); a1 = __ldcg(cp + 1);
     }
-    for (int r = 0; r < rows; r += 4) {
-      uint4 p[4];
-      float xv[4][8];
+    for (int r = 0; r < rows; r += RF) {
+      uint4 p[RF];
+      float xv[RF][8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < RF; ++i) {
         if (r + i < rows && s_on[r + i]) {
           x_load8(xbase + ((size_t)(r + i) * C8 + c8) * 8, xv[i]);
           p[i] = __ldg(s_src[r + i] + c8);
         }
       }
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < RF; ++i) {
         if (r + i < rows && s_on[r + i]) {
           float f[8];
           bf16x8_to_float(p[i], f);
@@ -581,10 +582,13 @@ cudaError_t launch_expired_wait(int32_t* status, unsigned long long limit_ns, cu
 // How the kept-row part of a restoration folds its column sums: 0 by shape, 1 global memory, 2 clusters.
 static int g_fold_mode = 0;
 static bool g_cluster_fold_ok = false;
+static int g_rows_sms = 148;
 void restore_force_fold(int mode) { g_fold_mode = mode; }
 cudaError_t rows_init() {
   g_cluster_fold_ok = cudaFuncSetAttribute(restore_kept_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
   (void)cudaGetLastError();
+  int dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) (void)cudaDeviceGetAttribute(&g_rows_sms, cudaDevAttrMultiProcessorCount, dev);
   return cudaSuccess;
 }
 
@@ -614,7 +618,7 @@ cudaError_t launch_restore_residual(void* x, const void* y, const void* cache, c
   LaunchScope scope(KC_RESTORE, 1, rr_bytes, rr_bytes, st);
   if (x_bf16) {   // bf16 residual stream: the generic kernel (nearest interpolation, fold through global memory)
     if (interp_mode != 0) return cudaErrorNotSupported;
-    restore_residual_kernel<__nv_bfloat16><<<dim3(nchunks, B), 256, 0, st>>>(
+    restore_residual_kernel<__nv_bfloat16, 4><<<dim3(nchunks, B), 256, 0, st>>>(
         static_cast<__nv_bfloat16*>(x), reinterpret_cast<const uint4*>(y), reinterpret_cast<const uint4*>(cache), inv, gamma, mod_stride, n, k, h, w,
         hc, wc, C / 8, nchunks, ws.group, ws.ngroups, reinterpret_cast<float4*>(ws.chunk_partial), reinterpret_cast<float4*>(ws.group_partial),
         ws.tickets, part);
@@ -634,7 +638,9 @@ cudaError_t launch_restore_residual(void* x, const void* y, const void* cache, c
     if (e == cudaSuccess || g_fold_mode == 2) return e;
     (void)cudaGetLastError();      // this cluster size cannot be scheduled here: the fold through global memory instead
   }
-  auto* kern = (interp_mode == 0 || part == 2) ? restore_residual_kernel<float>
+  // more chunks than three CTAs per SM hold at once (the 128 x 128 map): the kept-row part takes the build that fits four
+  const bool small_build = part == 2 && (long)nchunks * B > 3L * g_rows_sms && (long)nchunks * B <= 4L * g_rows_sms;
+  auto* kern = (interp_mode == 0 || part == 2) ? (small_build ? restore_residual_kernel<float, 2> : restore_residual_kernel<float, 4>)
                : (interp_mode == 1 ? restore_residual_interp_kernel<4> : restore_residual_interp_kernel<16>);
   if (part == 0)
     return launch_pdl(kern, dim3(nchunks, B), dim3(256), 0, st, static_cast<float*>(x),
