@@ -639,7 +639,7 @@ cudaError_t launch_restore_residual(void* x, const void* y, const void* cache, c
     (void)cudaGetLastError();      // this cluster size cannot be scheduled here: the fold through global memory instead
   }
   // more chunks than three CTAs per SM hold at once (the 128 x 128 map): the kept-row part takes the build that fits four
-  const bool small_build = part == 2 && (long)nchunks * B > 3L * g_rows_sms && (long)nchunks * B <= 4L * g_rows_sms;
+  const bool small_build = part != 0 && (long)nchunks * B > 3L * g_rows_sms && (long)nchunks * B <= 4L * g_rows_sms;
   auto* kern = (interp_mode == 0 || part == 2) ? (small_build ? restore_residual_kernel<float, 2> : restore_residual_kernel<float, 4>)
                : (interp_mode == 1 ? restore_residual_interp_kernel<4> : restore_residual_interp_kernel<16>);
   if (part == 0)
