@@ -52,10 +52,12 @@ unkept tokens take the previous scale's output, interpolated, instead of accumul
 outputs); it is not the paper's configuration and is pinned only by its own invariants.
 
 Parity pins: every function here is pinned by tests/test_oracle_pins.py (closed forms, brute force,
-invariants, library special cases).  The end-to-end activation values of a whole step have no
-printed example in the paper: "parity unpinned" for `VarOracle.var_step` as a whole beyond the
-invariants tested there (keep_ratio = 1 equals the unpruned forward, token-count invariance,
-restore equals the cache outside the pivot slots, KV length bookkeeping).
+invariants, library special cases).  The paper prints no worked example of a whole step, so
+`VarOracle.var_step` is pinned by what the method fixes: the unpruned schedule equals a library block-causal
+forward over the whole sequence; a pruned step whose sublayers all keep one given set equals that library
+forward over [earlier scales ; kept tokens] on the kept rows and the gated sum of the cached sublayer outputs
+on the others; a free-running pruned step replays from its trace with a brute-force ranking of the current
+stream at every sublayer; keep_ratio -> 1 equals the unpruned forward; KV length, order and image invariance.
 """
 from __future__ import annotations
 

@@ -17,10 +17,12 @@ so this file takes the plain construction of VAR-style models, stated here as re
   * the token map entering step k+1 is  interpolate(r_k, (h_{k+1}, w_{k+1})) @ W_in^T + b_in + pos_{k+1}.
 
 Everything is numpy float64, each function the definition written out.  Shares no code with the CUDA
-path.  Pins: tests/test_oracle_pins.py (Eq. 2 against Eq. 3 on nested scales, brute-force argmax with
+path.  Pins: tests/test_generation_oracle_pins.py (Eq. 2 against Eq. 3 on nested scales, brute-force argmax with
 ties, the Gumbel-max identity on a small alphabet, identity / constant special cases of the head and of
-the next-input map).  The loop as a whole has no printed example in the paper: "parity unpinned" beyond
-those invariants.
+the next-input map), and the loop itself by its records: each obeys Eq. 2 against the one before, each
+step is fed the map built from the previous record, and with keep ratio 1 the transformer outputs equal a
+plain run of the same inputs.  The paper prints no worked example of
+the loop.
 """
 from __future__ import annotations
 

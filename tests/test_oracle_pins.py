@@ -380,6 +380,75 @@ def test_emission_order_of_the_index_set_does_not_matter():
     np.testing.assert_allclose(got[4], ref[4], rtol=1e-10, atol=1e-11)
 
 
+@pytest.mark.parametrize("cross_len", [0, 4])
+def test_pruned_steps_with_one_kept_set_equal_a_sequence_forward_over_the_kept_tokens(cross_len):
+    """With the same kept set at every sublayer of a pruned step the kept tokens never meet the others: they
+    see the keys of the earlier scales (at a pruned earlier step: of its kept tokens only, Sec. 3.3) and their
+    own, so their outputs are those of a library block-causal forward over the sequence
+    [x_1 ... x_{K-N} ; kept tokens of every pruned step].  Every other token moves by the gated sum of the
+    cached sublayer outputs of its source token (Eq. 6)."""
+    wl, mt, w = _tiny_model(cross_len=cross_len)
+    xs = [I.step_input(wl, s) for s in range(len(wl.sides))]
+    keep = [1.0, 1.0, 1.0, 0.5, 0.25]
+    orc = O.VarOracle(wl.L, wl.C, wl.H, [(s, s) for s in wl.sides], cache_step=2, weights=w, B=wl.B,
+                      cross_len=cross_len)
+    pick = np.random.default_rng(77)
+    kept, outs = {}, []
+    for i, x in enumerate(xs):
+        if keep[i] < 1:
+            n = wl.sides[i] ** 2
+            k = O.kept_count(keep[i], wl.sides[i], wl.sides[i])
+            kept[i] = np.stack([np.sort(pick.choice(n, size=k, replace=False)) for _ in range(wl.B)])
+            outs.append(orc.var_step(x, i, keep[i], forced_idx={(l, sub): kept[i] for l in range(wl.L) for sub in orc.subs}))
+        else:
+            outs.append(orc.var_step(x, i, 1.0))
+    compact = [x if i not in kept else np.stack([x[b, kept[i][b]] for b in range(wl.B)]) for i, x in enumerate(xs)]
+    ref = _torch_block_causal_forward(wl, w, compact)
+    gate = {"attn": 2, "ffn": 5}
+    for i in kept:
+        side, side_c = wl.sides[i], wl.sides[2]
+        src = O.nearest_source(side, side, side_c, side_c)
+        for b in range(wl.B):
+            np.testing.assert_allclose(outs[i][b, kept[i][b]], ref[i][b], rtol=1e-9, atol=1e-10)
+            rest = np.setdiff1d(np.arange(side * side), kept[i][b])
+            want = xs[i][b, rest].astype(np.float64)
+            for l in range(wl.L):
+                for sub in orc.subs:
+                    g = w["mod"][l][b, gate[sub]] if sub in gate else 1.0
+                    want = want + g * orc.cache[l][sub][b, src[rest]]
+            np.testing.assert_allclose(outs[i][b, rest], want, rtol=1e-12, atol=1e-12)
+    assert orc.kv_len == 1 + 4 + 9 + kept[3].shape[1] + kept[4].shape[1]
+
+
+def test_free_running_selections_are_taken_on_the_current_stream():
+    """Every wrapped sublayer selects on the token map as the sublayers before it left it (Sec. 3.3
+    "Implementation"): replaying the trace -- brute-force ranking of the deviation from the mean token by a
+    stable sort, the branch output scattered over the interpolated cache -- reproduces each recorded kept set
+    and the step's output."""
+    wl, mt, w = _tiny_model(L=2, cross_len=3)
+    xs = [I.step_input(wl, s) for s in range(len(wl.sides))]
+    keep = [1.0, 1.0, 1.0, 0.5, 0.25]
+    orc, outs, tr = _run(wl, w, xs, keep, cache_step=2)
+    gate = {"attn": 2, "ffn": 5}
+    for i in (3, 4):
+        side, side_c = wl.sides[i], wl.sides[2]
+        k = O.kept_count(keep[i], side, side)
+        src = O.nearest_source(side, side, side_c, side_c)
+        x = xs[i].astype(np.float64).copy()
+        for l in range(wl.L):
+            for sub in orc.subs:
+                t = tr[i][(l, sub)]
+                for b in range(wl.B):
+                    dev = x[b] - x[b].sum(axis=0) / x.shape[1]
+                    order = sorted(range(x.shape[1]), key=lambda j: -float((dev[j] * dev[j]).sum()))   # stable: ties keep index order
+                    assert sorted(order[:k]) == list(t["idx"][b])
+                    full = orc.cache[l][sub][b, src].copy()
+                    full[t["idx"][b]] = t["y"][b]
+                    g = w["mod"][l][b, gate[sub]] if sub in gate else 1.0
+                    x[b] = x[b] + g * full
+        np.testing.assert_allclose(outs[i], x, rtol=1e-12, atol=1e-12)
+
+
 def test_images_are_independent():
     wl, mt, w = _tiny_model(L=1, B=2)
     xs = [I.step_input(wl, s) for s in range(len(wl.sides))]
