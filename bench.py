@@ -267,15 +267,24 @@ def ours(args, wl):
     for _ in range(args.warmup):
         schedule(ctx, wl.keep)
     barrier()
-    fv.fv_profile_read()                                   # zero the launch counters
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(S + 1)] for _ in range(args.steps)]
-    sampler = ClockSampler(local) if rank == 0 else None
-    t_wall = time.perf_counter()
-    for k in range(args.steps):
-        schedule(ctx, wl.keep, evs[k])
-    barrier()
-    t_wall = time.perf_counter() - t_wall
-    clocks = sampler.stop() if sampler else None
+    # A timed region during which the GPU reported a thermal or hardware slowdown is taken once more (the power cap
+    # alone is normal under load and kept).
+    for attempt in range(2):
+        fv.fv_profile_read()                                   # zero the launch counters
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(S + 1)] for _ in range(args.steps)]
+        sampler = ClockSampler(local) if rank == 0 else None
+        t_wall = time.perf_counter()
+        for k in range(args.steps):
+            schedule(ctx, wl.keep, evs[k])
+        barrier()
+        t_wall = time.perf_counter() - t_wall
+        clocks = sampler.stop() if sampler else None
+        slowed = 1.0 if clocks and any(r in ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown") for r in clocks["reasons"]) else 0.0
+        if attempt == 1 or max_over_ranks(slowed) == 0.0:      # rank 0 samples; every rank follows its verdict
+            if clocks is not None and attempt == 1:
+                clocks["remeasured"] = True
+            break
+        barrier()
     launches = fv.fv_profile_read()
     gpu_launches = sum(v["launches"] for v in launches.values())
     if ctx.device_status() != 0:
