@@ -659,21 +659,20 @@ fv_status fv_var_step(fv_ctx* ctx, const void* tokens_dev, int32_t B, int32_t sc
           s = FV_ERR_CUDA; break;
         }
       }
-      if (!fused) {
-        e = launch_gather_ln(xr, idx, B, nr, k, C, sigma, beta, mod_stride, ctx->a_buf, ctx->status, st, xb);
-        if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
-      }
       if (sub_pruned) {
         // Cached Token Restoration of the rows that were NOT kept needs only the selection and the cache:
-        // it runs on the side stream while the branch below works on the kept rows (the two touch disjoint
-        // rows of x).  It is forked behind the gather, which is short and on the critical path: started before
-        // it, the side stream's traffic made the gather up to twice as long.
+        // it runs on the side stream while the gather and the branch below work on the kept rows (the two
+        // touch disjoint rows of x).
         if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess) { s = FV_ERR_CUDA; break; }
         e = launch_restore_residual(x, ctx->y_buf, cache_sub, inv_cur, gamma, mod_stride, B, k, h, w, hc, wc, C,
                                     more ? ctx->sel_ws : nullptr, (fused && more) ? 3 : 1, c.interp_mode, ctx->side, xb);
         const cudaError_t e_join = cudaEventRecord(ctx->ev_join, ctx->side);   // recorded even if the launch failed
         forked = e_join == cudaSuccess;
         if (e != cudaSuccess || e_join != cudaSuccess) { s = FV_ERR_CUDA; break; }
+      }
+      if (!fused) {
+        e = launch_gather_ln(xr, idx, B, nr, k, C, sigma, beta, mod_stride, ctx->a_buf, ctx->status, st, xb);
+        if (e != cudaSuccess) { s = FV_ERR_CUDA; break; }
       }
       // ---- branch on the compact rows
       GemmArgs g{};
