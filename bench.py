@@ -217,6 +217,52 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def gemm_back_to_back(fv, wl, dev, steps_rows, sustained_tflops):
+    """The GEMMs of one transformer block alone, at the row count of every pruned scale step: each of the block's
+    projections as a chain of 16 launches (four rotating weight sets) captured in a CUDA graph and replayed, so that
+    neither the host's enqueue time nor the side stream's restoration is in the figure.  bf16-store epilogues."""
+    C, F = wl.C, int(round(wl.C * wl.mlp_ratio))
+    shapes = [(3 * C, C, 0), (C, C, 0)] + ([(C, C, 0), (C, C, 0)] if wl.cross_len else []) + [(F, C, 1), (C, F, 0)]
+    g = torch.Generator(device=dev); g.manual_seed(9)
+    rn = lambda *sh, std=1.0: (torch.randn(*sh, generator=g, device=dev) * std).to(torch.bfloat16)
+    skws = torch.zeros(fv.lib().fv_gemm_splitk_workspace_bytes(), dtype=torch.uint8, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    nchain = 16
+    by_rows, tot_fl, tot_us = {}, 0.0, 0.0
+    for M in steps_rows:
+        fl_m = us_m = 0.0
+        for (N, K, epi) in shapes:
+            a, b = rn(M, K), rn(N, std=0.02)
+            ws = [rn(N, K, std=0.02) for _ in range(4)]
+            out = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+            for j in range(3):
+                fv.fv_gemm_bf16(a, ws[j % 4], b, epilogue=epi, out=out, status=st, splitk_ws=skws)
+            torch.cuda.synchronize()
+            side = torch.cuda.Stream()
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(gr, stream=side):
+                    for j in range(nchain):
+                        fv.fv_gemm_bf16(a, ws[j % 4], b, epilogue=epi, out=out, status=st, splitk_ws=skws)
+            ts = []
+            for _ in range(5):
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); gr.replay(); e1.record(); torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1) * 1e3 / nchain)
+            us_m += statistics.median(ts)
+            fl_m += 2.0 * M * N * K
+            del gr, a, b, ws, out
+        by_rows[str(M)] = fl_m / us_m * 1e-6
+        tot_fl += fl_m; tot_us += us_m
+    if int(st.item()) != 0:
+        raise SystemExit("a GEMM reported an expired wait")
+    mix = tot_fl / tot_us * 1e-6
+    return {"what": "the projections of one block alone at the pruned steps' row counts: chains of 16 launches replayed from a CUDA graph, "
+                    "four rotating weight sets (they stay in L2; inside a step the weights come from HBM and the unkept-row restoration runs beside the GEMMs)",
+            "tflops_by_rows": by_rows, "mix_tflops": mix, "peak": sustained_tflops, "frac": mix / sustained_tflops if sustained_tflops else None}
+
+
 def ours(args, wl):
     from paper_2503_23367_b200 import binding as fv
     from paper_2503_23367_b200 import build as fv_build
@@ -570,6 +616,10 @@ def ours(args, wl):
         del ctx2, gt2, xs2, outs2
         torch.cuda.empty_cache()
 
+    b2b = None
+    if rank == 0 and not args.skip_b2b:
+        b2b = gemm_back_to_back(fv, wl, dev, [wl.B * kept(wl, i) for i in pruned_steps], peaks.get("bf16_tflops_sustained"))
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.skip_cpu:
         cb = time_oracle(wl, reps=1, warmup=0)
@@ -588,7 +638,7 @@ def ours(args, wl):
             "scale_step_ms": [round(t, 4) for t in step_ms], "wall_ms_per_step": t_wall * 1e3 / args.steps,
             "roofline": roofline, "kernels": kernels, "kernels_pruned_steps": kernels_pruned, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": gpu_launches,
             "clocks": clocks, "unpruned_gpu": unpruned, "per_step_granularity": variant, "backbone_options": extras, "bf16_residual_stream": bf16_stream, "generation_loop": generation, "other_workloads": other,
-            "peaks": peaks}
+            "gemm_back_to_back": b2b, "peaks": peaks}
     print(json.dumps(line))
 
 
@@ -690,6 +740,7 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="print pruning-ratio and caching-step curves instead of the bench line")
     ap.add_argument("--skip-variant", action="store_true", help="omit the per-step-granularity comparison")
     ap.add_argument("--skip-other", action="store_true", help="omit the timing of the 1024-pixel configuration beside the default one")
+    ap.add_argument("--skip-b2b", action="store_true", help="omit the back-to-back timing of a block's GEMMs")
     ap.add_argument("--blocks", type=int, default=0,
                     help="profiling only: run this many transformer blocks instead of the workload's depth (the line says so; not a bench number)")
     args = ap.parse_args()
